@@ -1,0 +1,597 @@
+// Host side of the C ABI declared in include/tt_emb.h: handle, workspace plan, call orchestration.
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+static thread_local int g_last_cuda_error = 0;
+
+#define TT_CUDA(x)                                   \
+    do {                                             \
+        cudaError_t _e = (x);                        \
+        if (_e != cudaSuccess) {                     \
+            g_last_cuda_error = (int)_e;             \
+            return TT_EMB_ERR_CUDA;                  \
+        }                                            \
+    } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int device_ok(int* sm_count)
+{
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return 0; }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+    int major = 0, sms = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sm_count) *sm_count = sms;
+    return major == 10;
+}
+
+extern "C" const char* tt_emb_strerror(int code)
+{
+    switch (code) {
+        case TT_EMB_OK: return "ok";
+        case TT_EMB_ERR_ARG: return "invalid argument or limit exceeded";
+        case TT_EMB_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case TT_EMB_ERR_ARCH: return "no CUDA device of compute capability 10.x (B200) available";
+        case TT_EMB_ERR_STATE: return "call order violated (bind before forward, forward before backward, enable_backward)";
+        case TT_EMB_ERR_CUDA: return "CUDA runtime error (see tt_emb_last_cuda_error)";
+        default: return "unknown error code";
+    }
+}
+
+extern "C" int tt_emb_last_cuda_error(void) { return g_last_cuda_error; }
+
+// ------------------------------------------------------------------------------------------------ create
+
+extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
+{
+    if (!cfg || !out_handle) return TT_EMB_ERR_ARG;
+    *out_handle = nullptr;
+    const int T = cfg->num_tables, K = cfg->num_cores;
+    if (T < 1 || K < 2 || K > TT_MAXK) return TT_EMB_ERR_ARG;
+    if (!cfg->num_rows || !cfg->row_factors || !cfg->dim_factors || !cfg->ranks) return TT_EMB_ERR_ARG;
+    if (cfg->max_batch < 1 || cfg->max_lookups < 0 || cfg->max_lookups >= (1LL << 31)) return TT_EMB_ERR_ARG;
+    if ((int64_t)T * cfg->max_batch >= (1LL << 31)) return TT_EMB_ERR_ARG;
+
+    tt_emb* h = new (std::nothrow) tt_emb();
+    if (!h) return TT_EMB_ERR_ARG;
+    memset(h, 0, sizeof(*h));
+    h->tab = (TableDesc*)calloc((size_t)T, sizeof(TableDesc));
+    if (!h->tab) { delete h; return TT_EMB_ERR_ARG; }
+    auto fail = [&](int code) { free(h->tab); delete h; return code; };
+
+    h->T = T; h->K = K;
+    h->max_batch = cfg->max_batch; h->max_lookups = cfg->max_lookups;
+    h->enable_backward = cfg->enable_backward ? 1 : 0;
+    h->sm_count = 148;
+    { int sms = 0; if (device_ok(&sms) && sms > 0) h->sm_count = sms; }
+
+    int D = -1;
+    int64_t sumN = 0;
+    uint64_t words = 0;
+    uint64_t twords[TT_MAXK] = {0, 0, 0, 0};
+    uint64_t level_space[TT_MAXK + 1] = {0, 0, 0, 0, 0};
+    int stride[TT_MAXK + 1] = {0, 0, 0, 0, 0};
+    uint64_t c_mid_max = 0, c_last_max = 0;
+    int max_pl = 1, max_c = 1;
+    for (int t = 0; t < T; ++t) {
+        TableDesc& td = h->tab[t];
+        td.N = cfg->num_rows[t];
+        if (td.N < 1 || td.N >= (1LL << 31)) return fail(TT_EMB_ERR_ARG);
+        int64_t prodn = 1;
+        int prodd = 1;
+        td.P[0] = 1;
+        for (int k = 0; k < K; ++k) {
+            td.n[k] = cfg->row_factors[t * K + k];
+            td.d[k] = cfg->dim_factors[t * K + k];
+            if (td.n[k] < 1 || td.d[k] < 1) return fail(TT_EMB_ERR_ARG);
+            prodn *= td.n[k];
+            if (prodn >= (1LL << 31)) return fail(TT_EMB_ERR_ARG);
+            prodd *= td.d[k];
+            if (prodd > 1024) return fail(TT_EMB_ERR_ARG);
+            td.P[k + 1] = prodd;
+            td.prefix_space[k + 1] = (uint32_t)prodn;
+        }
+        td.prefix_space[0] = 1;
+        if (prodn < td.N) return fail(TT_EMB_ERR_ARG);
+        for (int k = 0; k <= K; ++k) {
+            td.r[k] = cfg->ranks[t * (K + 1) + k];
+            if (td.r[k] < 1 || td.r[k] > 128) return fail(TT_EMB_ERR_ARG);
+        }
+        if (td.r[0] != 1 || td.r[K] != 1) return fail(TT_EMB_ERR_ARG);
+        if (D < 0) D = prodd; else if (D != prodd) return fail(TT_EMB_ERR_ARG);
+        for (int k = 0; k < K; ++k) {
+            td.slice_floats[k] = td.r[k] * td.d[k] * td.r[k + 1];
+            td.core_floats[k] = (int64_t)td.n[k] * td.slice_floats[k];
+            if (td.P[k + 1] * td.r[k + 1] > 4096) return fail(TT_EMB_ERR_ARG);
+            if (td.P[k + 1] * td.r[k + 1] > stride[k + 1]) stride[k + 1] = td.P[k + 1] * td.r[k + 1];
+        }
+        sumN += td.N;
+        td.word_base = (uint32_t)words;
+        uint64_t nw = align_up((size_t)((td.N + 31) / 32), TT_SCAN_TILE);
+        td.num_words = (uint32_t)nw;
+        words += nw;
+        if (words >= (1ULL << 32)) return fail(TT_EMB_ERR_ARG);
+        for (int k = 1; k <= K; ++k) level_space[k] += td.prefix_space[k];
+        for (int k = 2; k <= K - 1; ++k) {
+            td.tword_base[k] = (uint32_t)twords[k];
+            td.tnum_words[k] = td.prefix_space[k] / 32 + 1;
+            twords[k] += td.tnum_words[k];
+        }
+        uint64_t c_last = (uint64_t)td.P[K - 1] * td.r[K - 1] * td.d[K - 1];
+        uint64_t c_mid = K >= 3 ? (uint64_t)td.P[K - 2] * td.r[K - 2] * td.d[K - 2] * td.r[K - 1] : 0;
+        if (c_last > c_last_max) c_last_max = c_last;
+        if (c_mid > c_mid_max) c_mid_max = c_mid;
+        for (int k = 1; k < K; ++k) {
+            int f = td.P[k] * td.r[k];
+            if (k <= K - 2 && f > max_pl) max_pl = f;
+            if (k == K - 1 && f > max_c) max_c = f;
+        }
+    }
+    h->D = D;
+    int64_t bound = cfg->max_lookups < sumN ? cfg->max_lookups : sumN;
+    if (bound < 1) bound = 1;
+    h->capU = (cfg->max_unique_rows > 0 && cfg->max_unique_rows < bound) ? cfg->max_unique_rows : bound;
+
+    // work units: every table is cut into `units` equal-cost slices, one CTA each
+    int Q = (4 * h->sm_count + T - 1) / T;
+    if (Q < 4) Q = 4;
+    if (Q > 1024) Q = 1024;
+    int unit_base = 0;
+    const int priv_budget = (227 * 1024 - 1024) / 4 - (max_pl + 2 * max_c + 8 * D);
+    int64_t gpart = 0;
+    h->max_priv_floats = 0;
+    for (int t = 0; t < T; ++t) {
+        TableDesc& td = h->tab[t];
+        td.units = Q;
+        td.unit_base = unit_base;
+        unit_base += Q;
+        td.priv_ok = (td.core_floats[K - 1] <= priv_budget) ? 1 : 0;
+        td.gpart_off = gpart;
+        if (td.priv_ok) {
+            gpart += (int64_t)Q * td.core_floats[K - 1];
+            if (td.core_floats[K - 1] > h->max_priv_floats) h->max_priv_floats = (int)td.core_floats[K - 1];
+        }
+    }
+    h->units_total = unit_base;
+    h->gpart_floats = gpart;
+
+    WsView& v = h->v;
+    v.T = T; v.K = K; v.D = D;
+    v.capU = h->capU;
+    for (int k = 1; k <= K; ++k) {
+        uint64_t c = level_space[k] < (uint64_t)h->capU ? level_space[k] : (uint64_t)h->capU;
+        v.cap[k] = (uint32_t)c;
+        v.stride[k] = stride[k];
+    }
+    v.cap[K] = (uint32_t)h->capU;
+    v.total_words = (uint32_t)words;
+    for (int k = 2; k <= K - 1; ++k) v.ttotal_words[k] = (uint32_t)twords[k];
+
+    // cost unit 2^shift FMAs such that the largest possible total stays below 2^31
+    int shift = 0;
+    for (;; ++shift) {
+        unsigned __int128 tot = ((unsigned __int128)v.cap[K - 1] * c_mid_max + (unsigned __int128)v.cap[K] * c_last_max) >> shift;
+        tot += v.cap[K - 1];
+        if (tot < ((unsigned __int128)1 << 31)) break;
+    }
+    h->cost_shift = shift;
+
+    // ---- workspace plan
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    h->off_status = take((16 + 64) * sizeof(uint32_t));
+    h->off_counters = h->off_status + 16 * sizeof(uint32_t);
+    h->off_tdesc = take((size_t)T * sizeof(TableDesc));
+    h->off_tlstart = take((size_t)(T + 1) * sizeof(int64_t));
+    h->off_bm = take((size_t)words * sizeof(uint2));
+    uint64_t scan_max = words;
+    for (int k = 1; k <= K; ++k) if (v.cap[k] > scan_max) scan_max = v.cap[k];
+    for (int k = 2; k <= K - 1; ++k) if (twords[k] > scan_max) scan_max = twords[k];
+    h->scan_tmp_elems = (size_t)(scan_max / TT_SCAN_TILE + 4);
+    h->off_scan = take(h->scan_tmp_elems * sizeof(uint32_t));
+    for (int k = 1; k <= K; ++k) {
+        h->off_val[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+        h->off_tb[k] = take((size_t)(T + 1) * sizeof(uint32_t));
+        if (k < K) h->off_cstart[k] = take(((size_t)v.cap[k] + 1) * sizeof(uint32_t));
+        if (k >= 2) h->off_parent[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+    }
+    h->off_cost = take(((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
+    for (int k = 2; k <= K - 2; ++k) h->off_pbuf[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
+    h->off_E = take((size_t)h->capU * D * sizeof(float));
+    if (h->enable_backward) {
+        h->off_cnt = take(((size_t)h->capU + 1) * sizeof(uint32_t));
+        h->off_cursor = take((size_t)h->capU * sizeof(uint32_t));
+        h->off_pairs = take((size_t)2 * (size_t)(h->max_lookups + 1) * sizeof(uint2));
+        for (int k = 2; k <= K - 1; ++k) {
+            h->off_dP[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
+            h->off_tbm[k] = take((size_t)twords[k] * sizeof(uint2));
+            h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+        }
+        h->off_carry = take(((size_t)(h->max_lookups / TT_DE_CHUNK) + 2) * 2 * D * sizeof(float));
+        h->off_gpart = take((size_t)(gpart > 0 ? gpart : 1) * sizeof(float));
+    }
+    h->ws_bytes = off;
+    *out_handle = h;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_destroy(tt_emb_t h)
+{
+    if (!h) return TT_EMB_ERR_ARG;
+    if (h->ev_created)
+        for (int i = 0; i < TT_NUM_STAGES; ++i) { cudaEventDestroy(h->ev[i][0]); cudaEventDestroy(h->ev[i][1]); }
+    free(h->tab);
+    delete h;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_workspace_bytes(tt_emb_t h, size_t* bytes)
+{
+    if (!h || !bytes) return TT_EMB_ERR_ARG;
+    *bytes = h->ws_bytes;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_core_floats(tt_emb_t h, int32_t table, int32_t core, int64_t* count)
+{
+    if (!h || !count || table < 0 || table >= h->T || core < 0 || core >= h->K) return TT_EMB_ERR_ARG;
+    *count = h->tab[table].core_floats[core];
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_dim(tt_emb_t h, int32_t* D)
+{
+    if (!h || !D) return TT_EMB_ERR_ARG;
+    *D = h->D;
+    return TT_EMB_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ bind
+
+extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace, size_t workspace_bytes,
+                           tt_emb_stream_t stream)
+{
+    if (!h || !core_ptrs) return TT_EMB_ERR_ARG;
+    if (!workspace || workspace_bytes < h->ws_bytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return TT_EMB_ERR_WORKSPACE;
+    int sms = 0;
+    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int T = h->T, K = h->K;
+    for (int t = 0; t < T; ++t)
+        for (int k = 0; k < K; ++k) {
+            float* p = core_ptrs[t * K + k];
+            if (!p || (reinterpret_cast<uintptr_t>(p) & 15)) return TT_EMB_ERR_ARG;
+            h->tab[t].core[k] = p;
+            h->tab[t].grad[k] = nullptr;
+        }
+    char* base = (char*)workspace;
+    WsView& v = h->v;
+    v.status = (int32_t*)(base + h->off_status);
+    v.counters = (uint32_t*)(base + h->off_counters);
+    v.tdesc = (TableDesc*)(base + h->off_tdesc);
+    v.tl_start = (int64_t*)(base + h->off_tlstart);
+    v.bm = (uint2*)(base + h->off_bm);
+    v.scan_tmp = (uint32_t*)(base + h->off_scan);
+    for (int k = 1; k <= K; ++k) {
+        v.val[k] = (uint32_t*)(base + h->off_val[k]);
+        v.tb[k] = (uint32_t*)(base + h->off_tb[k]);
+        v.cstart[k] = k < K ? (uint32_t*)(base + h->off_cstart[k]) : nullptr;
+        v.parent[k] = k >= 2 ? (uint32_t*)(base + h->off_parent[k]) : nullptr;
+    }
+    v.cost = (uint32_t*)(base + h->off_cost);
+    for (int k = 2; k <= K - 2; ++k) v.pbuf[k] = (float*)(base + h->off_pbuf[k]);
+    v.E = (float*)(base + h->off_E);
+    v.upairs = nullptr;
+    if (h->enable_backward) {
+        v.cnt = (uint32_t*)(base + h->off_cnt);
+        v.cursor = (uint32_t*)(base + h->off_cursor);
+        v.pairs = (uint2*)(base + h->off_pairs);
+        v.upairs = v.pairs + (h->max_lookups + 1);
+        for (int k = 2; k <= K - 1; ++k) {
+            v.dP[k] = (float*)(base + h->off_dP[k]);
+            v.tbm[k] = (uint2*)(base + h->off_tbm[k]);
+            v.tnode[k] = (uint32_t*)(base + h->off_tnode[k]);
+        }
+        v.carry = (float*)(base + h->off_carry);
+        v.gpart = (float*)(base + h->off_gpart);
+    }
+    // pageable source: the runtime stages it before returning, so h->tab may change afterwards
+    TT_CUDA(cudaMemcpyAsync(v.tdesc, h->tab, (size_t)T * sizeof(TableDesc), cudaMemcpyHostToDevice, s));
+    TT_CUDA(cudaMemsetAsync(v.status, 0, (16 + 64) * sizeof(uint32_t), s));
+    h->bound = true;
+    h->have_forward = false;
+    return TT_EMB_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ timing helpers
+
+static int stage_begin(tt_emb* h, int stage, cudaStream_t s)
+{
+    if (!h->timing) return TT_EMB_OK;
+    if (!h->ev_created) {
+        for (int i = 0; i < TT_NUM_STAGES; ++i) { TT_CUDA(cudaEventCreate(&h->ev[i][0])); TT_CUDA(cudaEventCreate(&h->ev[i][1])); }
+        h->ev_created = true;
+    }
+    TT_CUDA(cudaEventRecord(h->ev[stage][0], s));
+    return TT_EMB_OK;
+}
+
+static int stage_end(tt_emb* h, int stage, cudaStream_t s)
+{
+    if (!h->timing) return TT_EMB_OK;
+    TT_CUDA(cudaEventRecord(h->ev[stage][1], s));
+    h->ev_valid[stage] = true;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_enable_timing(tt_emb_t h, int32_t on)
+{
+    if (!h) return TT_EMB_ERR_ARG;
+    h->timing = on != 0;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_stage_ms(tt_emb_t h, int32_t stage, float* ms)
+{
+    if (!h || !ms || stage < 0 || stage >= TT_NUM_STAGES) return TT_EMB_ERR_ARG;
+    if (!h->ev_created || !h->ev_valid[stage]) return TT_EMB_ERR_STATE;
+    TT_CUDA(cudaEventSynchronize(h->ev[stage][1]));
+    TT_CUDA(cudaEventElapsedTime(ms, h->ev[stage][0], h->ev[stage][1]));
+    return TT_EMB_OK;
+}
+
+#define TT_STAGE(h, id, s, call)                                 \
+    do {                                                         \
+        int _r = stage_begin(h, id, s);                          \
+        if (_r) return _r;                                       \
+        TT_CUDA(call);                                           \
+        _r = stage_end(h, id, s);                                \
+        if (_r) return _r;                                       \
+    } while (0)
+
+// ------------------------------------------------------------------------------------------------ forward / backward / sgd
+
+extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                              int64_t num_lookups, float* out, tt_emb_stream_t stream)
+{
+    if (!h || !offsets || !out || (!indices && num_lookups > 0)) return TT_EMB_ERR_ARG;
+    if (!h->bound) return TT_EMB_ERR_STATE;
+    if (batch < 1 || batch > h->max_batch || num_lookups < 0 || num_lookups > h->max_lookups) return TT_EMB_ERR_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    WsView& v = h->v;
+    v.B = batch; v.L = num_lookups;
+    v.indices = indices; v.offsets = offsets;
+    h->have_forward = false;
+    for (int i = 0; i < 4; ++i) h->ev_valid[i] = false;
+    TT_STAGE(h, 0, s, tt_launch_grouping(h, s));
+    TT_STAGE(h, 1, s, tt_launch_schedule(h, s));
+    TT_STAGE(h, 2, s, tt_launch_contraction(h, s));
+    TT_STAGE(h, 3, s, tt_launch_pooling(h, out, s));
+    h->have_forward = true;
+    return TT_EMB_OK;
+}
+
+static int upload_grads(tt_emb* h, float* const* core_grads, cudaStream_t s)
+{
+    const int T = h->T, K = h->K;
+    for (int t = 0; t < T; ++t)
+        for (int k = 0; k < K; ++k) {
+            float* p = core_grads[t * K + k];
+            if (!p || (reinterpret_cast<uintptr_t>(p) & 15)) return TT_EMB_ERR_ARG;
+            h->tab[t].grad[k] = p;
+        }
+    TT_CUDA(cudaMemcpyAsync(h->v.tdesc, h->tab, (size_t)T * sizeof(TableDesc), cudaMemcpyHostToDevice, s));
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads, tt_emb_stream_t stream)
+{
+    if (!h || !grad_out || !core_grads) return TT_EMB_ERR_ARG;
+    if (!h->bound || !h->have_forward || !h->enable_backward) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    int r = upload_grads(h, core_grads, s);
+    if (r) return r;
+    for (int i = 4; i < 8; ++i) h->ev_valid[i] = false;
+    TT_STAGE(h, 4, s, tt_launch_bwd_sort(h, s));
+    TT_STAGE(h, 5, s, tt_launch_bwd_dE(h, grad_out, s));
+    TT_STAGE(h, 6, s, tt_launch_bwd_contraction(h, s));
+    TT_STAGE(h, 7, s, tt_launch_bwd_middle(h, s));
+    h->have_forward = false;  // dE overwrote the rows; a second backward needs a new forward
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_sgd_step(tt_emb_t h, float* const* core_grads, float lr, tt_emb_stream_t stream)
+{
+    if (!h || !core_grads) return TT_EMB_ERR_ARG;
+    if (!h->bound) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    int r = upload_grads(h, core_grads, s);
+    if (r) return r;
+    h->ev_valid[8] = false;
+    TT_STAGE(h, 8, s, tt_launch_sgd(h, lr, s));
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_status(tt_emb_t h, int32_t* status_host, tt_emb_stream_t stream)
+{
+    if (!h || !status_host) return TT_EMB_ERR_ARG;
+    if (!h->bound) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    TT_CUDA(cudaMemcpyAsync(status_host, h->v.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    TT_CUDA(cudaStreamSynchronize(s));
+    return TT_EMB_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ inspection
+
+extern "C" int tt_emb_grouping_counts(tt_emb_t h, int64_t* counts_host, tt_emb_stream_t stream)
+{
+    if (!h || !counts_host) return TT_EMB_ERR_ARG;
+    if (!h->bound || !h->have_forward) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int T = h->T, K = h->K;
+    uint32_t* tmp = (uint32_t*)malloc((size_t)(T + 1) * sizeof(uint32_t));
+    if (!tmp) return TT_EMB_ERR_ARG;
+    for (int k = 1; k <= K; ++k) {
+        cudaError_t e = cudaMemcpyAsync(tmp, h->v.tb[k], (size_t)(T + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) { free(tmp); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }
+        for (int t = 0; t < T; ++t) counts_host[t * K + (k - 1)] = (int64_t)tmp[t + 1] - (int64_t)tmp[t];
+    }
+    free(tmp);
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_export_level(tt_emb_t h, int32_t table, int32_t level, int64_t* vals, int32_t* row_counts,
+                                   int32_t* lookup_counts, tt_emb_stream_t stream)
+{
+    if (!h || table < 0 || table >= h->T || level < 1 || level > h->K) return TT_EMB_ERR_ARG;
+    if (!h->bound || !h->have_forward) return TT_EMB_ERR_STATE;
+    if (lookup_counts && !h->enable_backward) return TT_EMB_ERR_STATE;  // needs the cursor scratch array
+    cudaStream_t s = (cudaStream_t)stream;
+    TT_CUDA(tt_launch_export_level(h, table, level, vals, row_counts, lookup_counts, s));
+    TT_CUDA(cudaStreamSynchronize(s));
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_export_inverse(tt_emb_t h, int32_t table, int32_t* inv, tt_emb_stream_t stream)
+{
+    if (!h || !inv || table < 0 || table >= h->T) return TT_EMB_ERR_ARG;
+    if (!h->bound || !h->have_forward) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    TT_CUDA(tt_launch_export_inverse(h, table, inv, s));
+    TT_CUDA(cudaStreamSynchronize(s));
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_pack_core(tt_emb_t h, int32_t table, int32_t core, const float* rndr, float* canonical,
+                                tt_emb_stream_t stream)
+{
+    if (!h || !rndr || !canonical || table < 0 || table >= h->T || core < 0 || core >= h->K) return TT_EMB_ERR_ARG;
+    if (!device_ok(nullptr)) return TT_EMB_ERR_ARCH;
+    TT_CUDA(tt_launch_pack(h->tab[table], core, rndr, canonical, true, (cudaStream_t)stream));
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_unpack_core(tt_emb_t h, int32_t table, int32_t core, const float* canonical, float* rndr,
+                                  tt_emb_stream_t stream)
+{
+    if (!h || !rndr || !canonical || table < 0 || table >= h->T || core < 0 || core >= h->K) return TT_EMB_ERR_ARG;
+    if (!device_ok(nullptr)) return TT_EMB_ERR_ARCH;
+    TT_CUDA(tt_launch_pack(h->tab[table], core, canonical, rndr, false, (cudaStream_t)stream));
+    return TT_EMB_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ probes
+
+static __device__ float g_probe_sink[4];  // never-taken stores keep the probe loops alive
+
+__global__ void k_probe_fma(float* out, int iters, float a, float b)
+{
+    float x0 = threadIdx.x, x1 = x0 + 1.f, x2 = x0 + 2.f, x3 = x0 + 3.f, x4 = x0 + 4.f, x5 = x0 + 5.f, x6 = x0 + 6.f, x7 = x0 + 7.f;
+    for (int i = 0; i < iters; ++i) {
+        x0 = fmaf(x0, a, b); x1 = fmaf(x1, a, b); x2 = fmaf(x2, a, b); x3 = fmaf(x3, a, b);
+        x4 = fmaf(x4, a, b); x5 = fmaf(x5, a, b); x6 = fmaf(x6, a, b); x7 = fmaf(x7, a, b);
+    }
+    const float sum = x0 + x1 + x2 + x3 + x4 + x5 + x6 + x7;
+    if (sum == 123.456f) out[0] = sum;  // never true; keeps the chain alive
+}
+
+extern "C" int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t stream)
+{
+    if (!slots_per_second) return TT_EMB_ERR_ARG;
+    int sms = 0;
+    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    float* dsink = nullptr;
+    TT_CUDA(cudaGetSymbolAddress((void**)&dsink, g_probe_sink));
+    cudaEvent_t e0, e1;
+    TT_CUDA(cudaEventCreate(&e0));
+    TT_CUDA(cudaEventCreate(&e1));
+    const int iters = 20000;
+    double best = 0.0;
+    for (int rep = 0; rep < 4; ++rep) {
+        cudaEventRecord(e0, s);
+        k_probe_fma<<<sms * 8, 256, 0, s>>>(dsink, iters, 1.0001f, 0.5f);
+        cudaEventRecord(e1, s);
+        cudaError_t e = cudaEventSynchronize(e1);
+        if (e != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double rate = (double)sms * 8 * 256 * 8 * iters / (ms * 1e-3);
+        if (rep > 0 && rate > best) best = rate;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *slots_per_second = best;
+    return TT_EMB_OK;
+}
+
+__global__ void k_probe_fill(int32_t* idx, int64_t n, uint32_t rows)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        uint64_t x = (uint64_t)i * 0x9E3779B97F4A7C15ull;
+        x ^= x >> 29; x *= 0xBF58476D1CE4E5B9ull; x ^= x >> 32;
+        idx[i] = (int32_t)(x % rows);
+    }
+}
+
+__global__ void __launch_bounds__(256) k_probe_gather(const float4* __restrict__ buf, const int32_t* __restrict__ idx, int64_t n, float* sink)
+{
+    const int lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t i0 = warp * 32; i0 < n; i0 += nw * 32) {
+        const int mine = (i0 + lane < n) ? idx[i0 + lane] : -1;
+#pragma unroll 4
+        for (int j = 0; j < 32; j += 2) {
+            const int r = __shfl_sync(0xffffffffu, mine, j + half);
+            if (r >= 0) {
+                const float4 x = __ldg(buf + (size_t)r * 16 + l16);
+                acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+            }
+        }
+    }
+    if (acc.x + acc.y + acc.z + acc.w == 123.456f) sink[0] = acc.x;
+}
+
+extern "C" int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* scratch_idx, int64_t num_rows_read,
+                                   double* bytes_per_second, tt_emb_stream_t stream)
+{
+    if (!buffer || !scratch_idx || !bytes_per_second || bytes < 256 || num_rows_read < 1) return TT_EMB_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(buffer) & 15) return TT_EMB_ERR_ARG;
+    int sms = 0;
+    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    float* dsink = nullptr;
+    TT_CUDA(cudaGetSymbolAddress((void**)&dsink, g_probe_sink));
+    const size_t rows = bytes / 256;
+    if (rows >= (1ull << 31)) return TT_EMB_ERR_ARG;
+    k_probe_fill<<<sms * 4, 256, 0, s>>>(scratch_idx, num_rows_read, (uint32_t)rows);
+    cudaEvent_t e0, e1;
+    TT_CUDA(cudaEventCreate(&e0));
+    TT_CUDA(cudaEventCreate(&e1));
+    double best = 0.0;
+    for (int rep = 0; rep < 4; ++rep) {
+        cudaEventRecord(e0, s);
+        k_probe_gather<<<sms * 8, 256, 0, s>>>((const float4*)buffer, scratch_idx, num_rows_read, dsink);
+        cudaEventRecord(e1, s);
+        cudaError_t e = cudaEventSynchronize(e1);
+        if (e != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double rate = (double)num_rows_read * 256.0 / (ms * 1e-3);
+        if (rep > 0 && rate > best) best = rate;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *bytes_per_second = best;
+    return TT_EMB_OK;
+}

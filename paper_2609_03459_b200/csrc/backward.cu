@@ -1,0 +1,646 @@
+// Backward path (paper Sec. 3.2 backward, Eq. 2) and SGD.
+//
+//   1. sort:  the forward left one (slot, bag) pair per lookup; a counting sort by slot (counts -> exclusive
+//             scan -> scatter) groups the lookups of every distinct row.  Hot rows would serialise global
+//             atomics, so each CTA first aggregates its tile in a shared-memory hash table and issues one
+//             global atomic per distinct row per tile.
+//   2. dE:    segmented sum of grad_out rows over the sorted pairs.  Fixed-size chunks of sorted positions per
+//             warp (skew-proof); segments that cross chunk borders leave partial sums which a second kernel
+//             adds in position order.
+//   3. last level: per group, C is rebuilt in shared memory; every row contributes C^T.dE to the slice of
+//             the last core it selects and dE.D^T to the group's dC (summed over the rows sharing C before
+//             going up, Eq. 2).  Rows of one group select distinct slices, so a CTA-private copy of the
+//             last core's gradient in shared memory is updated without atomics; the copies are then added
+//             in a fixed order (segment reduction keyed by slice).
+//   4. middle cores: dP_{k-1} of a parent = sum over its (contiguous) children; the gradient of slice i_k
+//             = sum over the level-k nodes with that digit, enumerated by a second, digit-major bitmap sort.
+//             Each output has exactly one owner, which sums in sorted order: no atomics.
+#include "common.cuh"
+#include "scan.cuh"
+
+#define HT_SIZE 4096
+#define HT_TILE 2048
+#define HT_EMPTY 0xffffffffu
+#define RB 8  // rows per batch in the last-level kernel
+
+// ---------------------------------------------------------------------------------------------- small utilities
+
+__global__ void k_zero_u32_dev(uint32_t* p, const uint32_t* count, uint32_t extra)
+{
+    const uint32_t n = *count + extra;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0u;
+}
+
+// zero the gradients that are not fully written by an owner kernel: core 0 always, last core when the
+// table does not use the private copy
+__global__ void k_zero_grads(WsView w)
+{
+    const int t = blockIdx.y;
+    const TableDesc& td = w.tdesc[t];
+    const int K = w.K;
+    float* g0 = td.grad[0];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < td.core_floats[0]; i += (int64_t)gridDim.x * blockDim.x) g0[i] = 0.f;
+    if (!td.priv_ok) {
+        float* gl = td.grad[K - 1];
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < td.core_floats[K - 1]; i += (int64_t)gridDim.x * blockDim.x) gl[i] = 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- 1. sort by slot
+
+// MODE 0: cnt[slot] += occurrences.  MODE 1: pairs[seg_start[slot] + claimed position] = (slot, bag).
+template <int MODE>
+__global__ void __launch_bounds__(256) k_sort_pass(WsView w)
+{
+    const uint2* __restrict__ upairs = w.upairs;
+    const uint32_t capK = w.cap[w.K];
+    __shared__ uint32_t keys[HT_SIZE];
+    __shared__ uint32_t vals[HT_SIZE];
+    const int64_t L = w.L;
+    const int64_t ntiles = (L + HT_TILE - 1) / HT_TILE;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) { keys[i] = HT_EMPTY; vals[i] = 0u; }
+        __syncthreads();
+        uint2 pr[HT_TILE / 256];
+        uint32_t hh[HT_TILE / 256], rk[HT_TILE / 256];
+#pragma unroll
+        for (int j = 0; j < HT_TILE / 256; ++j) {
+            const int64_t l = tile * HT_TILE + j * 256 + threadIdx.x;
+            pr[j] = l < L ? __ldg(upairs + l) : make_uint2(HT_EMPTY, 0u);
+            if (pr[j].x >= capK || (int64_t)pr[j].y >= w.B) pr[j].x = HT_EMPTY;  // invalid lookup (or malformed offsets)
+        }
+#pragma unroll
+        for (int j = 0; j < HT_TILE / 256; ++j) {
+            if (pr[j].x == HT_EMPTY) continue;
+            uint32_t p = (pr[j].x * 2654435761u) >> 20;
+            for (int probe = 0; probe < HT_SIZE; ++probe) {
+                const uint32_t old = atomicCAS(&keys[p], HT_EMPTY, pr[j].x);
+                if (old == HT_EMPTY || old == pr[j].x) break;
+                p = (p + 1) & (HT_SIZE - 1);
+            }
+            hh[j] = p;
+            rk[j] = atomicAdd(&vals[p], 1u);
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) {
+            if (keys[i] != HT_EMPTY) {
+                if (MODE == 0) atomicAdd(&w.cnt[keys[i]], vals[i]);
+                else vals[i] = atomicAdd(&w.cursor[keys[i]], vals[i]);
+            }
+        }
+        if (MODE == 1) {
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < HT_TILE / 256; ++j) {
+                if (pr[j].x == HT_EMPTY) continue;
+                const uint32_t pos = w.cnt[pr[j].x] + vals[hh[j]] + rk[j];
+                w.pairs[pos] = pr[j];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+struct CntScan {
+    WsView w;
+    __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + w.K]; }
+    __device__ uint32_t value(uint32_t i) const { return w.cnt[i]; }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t) const { w.cnt[i] = excl; }
+    __device__ void total(uint32_t tot) const { w.cnt[size()] = tot; }
+};
+
+cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
+{
+    WsView& w = h->v;
+    const int zgrid = h->sm_count * 8;
+    k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cnt, w.counters + CTR_LEVEL0 + w.K, 1u);
+    k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cursor, w.counters + CTR_LEVEL0 + w.K, 0u);
+    const int64_t ntiles = (w.L + HT_TILE - 1) / HT_TILE;
+    int grid = (int)(ntiles < (int64_t)h->sm_count * 6 ? ntiles : (int64_t)h->sm_count * 6);
+    if (grid < 1) grid = 1;
+    k_sort_pass<0><<<grid, 256, 0, s>>>(w);
+    CntScan cs{w};
+    cudaError_t e = tt_scan(cs, w.cap[w.K], w.scan_tmp, s);
+    if (e != cudaSuccess) return e;
+    k_sort_pass<1><<<grid, 256, 0, s>>>(w);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------- 2. dE
+
+// lane l of the warp owns float4 chunks l, l+32, ... of a row (VEC) or floats l, l+32, ... (!VEC)
+template <bool VEC, int CPL>
+struct RowAcc {
+    float v[VEC ? 4 * CPL : CPL];
+    __device__ void clear()
+    {
+#pragma unroll
+        for (int i = 0; i < (VEC ? 4 * CPL : CPL); ++i) v[i] = 0.f;
+    }
+    __device__ void add_row(const float* __restrict__ row, int D, int lane)
+    {
+        if (VEC) {
+            const float4* r4 = reinterpret_cast<const float4*>(row);
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const int ch = lane + c * 32;
+                if (ch * 4 < D) {
+                    const float4 x = __ldg(r4 + ch);
+                    v[4 * c] += x.x; v[4 * c + 1] += x.y; v[4 * c + 2] += x.z; v[4 * c + 3] += x.w;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const int i = lane + c * 32;
+                if (i < D) v[c] += __ldg(row + i);
+            }
+        }
+    }
+    __device__ void store(float* __restrict__ row, int D, int lane) const
+    {
+        if (VEC) {
+            float4* r4 = reinterpret_cast<float4*>(row);
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const int ch = lane + c * 32;
+                if (ch * 4 < D) r4[ch] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const int i = lane + c * 32;
+                if (i < D) row[i] = v[c];
+            }
+        }
+    }
+};
+
+template <bool VEC, int CPL>
+__global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ grad_out)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
+    const uint32_t Ltot = w.cnt[U];
+    const int64_t a64 = chunk * TT_DE_CHUNK;
+    if (a64 >= Ltot) return;
+    const uint32_t a = (uint32_t)a64;
+    const uint32_t b = min(a + (uint32_t)TT_DE_CHUNK, Ltot);
+    const int D = w.D;
+    const size_t gstride = (size_t)w.T * D;
+    const uint32_t prev = a > 0 ? w.pairs[a - 1].x : HT_EMPTY;
+    const uint32_t next = b < Ltot ? w.pairs[b].x : HT_EMPTY;
+    RowAcc<VEC, CPL> acc;
+    acc.clear();
+    uint32_t cur = w.pairs[a].x;
+    int tcur = tt_find_table(w.tb[w.K], w.T, cur);
+    bool seg_first = true;
+    float* carry = w.carry + (size_t)chunk * 2 * D;
+    for (uint32_t p0 = a; p0 < b; p0 += 32) {
+        const uint2 mine = (p0 + lane < b) ? __ldg(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
+        const int n = (int)min(32u, b - p0);
+        for (int j = 0; j < n; ++j) {
+            const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j);
+            const uint32_t bag = __shfl_sync(0xffffffffu, mine.y, j);
+            if (sl != cur) {
+                const bool open_start = seg_first && prev == cur;
+                if (open_start) acc.store(carry, D, lane);  // head: started in an earlier chunk, ends here
+                else acc.store(w.E + (size_t)cur * D, D, lane);
+                acc.clear();
+                cur = sl;
+                tcur = tt_find_table(w.tb[w.K], w.T, cur);
+                seg_first = false;
+            }
+            acc.add_row(grad_out + (size_t)bag * gstride + (size_t)tcur * D, D, lane);
+        }
+    }
+    const bool open_start = seg_first && prev == cur;
+    const bool open_end = next == cur;
+    if (open_end) acc.store(carry + D, D, lane);        // tail: continues in the next chunk
+    else if (open_start) acc.store(carry, D, lane);     // head
+    else acc.store(w.E + (size_t)cur * D, D, lane);
+}
+
+// the chunk in which a border-crossing segment starts adds up the pieces in position order
+template <bool VEC, int CPL>
+__global__ void __launch_bounds__(256) k_dE_fix(WsView w)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
+    const uint32_t Ltot = w.cnt[U];
+    const int64_t a64 = chunk * TT_DE_CHUNK;
+    if (a64 >= Ltot) return;
+    const uint32_t a = (uint32_t)a64;
+    const uint32_t b = min(a + (uint32_t)TT_DE_CHUNK, Ltot);
+    if (b >= Ltot) return;
+    const uint32_t first = w.pairs[a].x, last = w.pairs[b - 1].x;
+    const uint32_t prev = a > 0 ? w.pairs[a - 1].x : HT_EMPTY;
+    const uint32_t next = w.pairs[b].x;
+    if (next != last) return;                         // nothing continues past this chunk
+    if (first == last && prev == first) return;       // the segment started earlier: not the owner
+    const int D = w.D;
+    RowAcc<VEC, CPL> acc;
+    acc.clear();
+    acc.add_row(w.carry + ((size_t)chunk * 2 + 1) * D, D, lane);
+    const int64_t nchunks = ((int64_t)Ltot + TT_DE_CHUNK - 1) / TT_DE_CHUNK;
+    for (int64_t c2 = chunk + 1; c2 < nchunks; ++c2) {
+        const uint32_t a2 = (uint32_t)(c2 * TT_DE_CHUNK);
+        const uint32_t b2 = min(a2 + (uint32_t)TT_DE_CHUNK, Ltot);
+        const uint32_t last2 = w.pairs[b2 - 1].x;
+        const uint32_t next2 = b2 < Ltot ? w.pairs[b2].x : HT_EMPTY;
+        if (last2 == last && next2 == last) {
+            acc.add_row(w.carry + ((size_t)c2 * 2 + 1) * D, D, lane);
+        } else {
+            acc.add_row(w.carry + (size_t)c2 * 2 * D, D, lane);
+            break;
+        }
+    }
+    acc.store(w.E + (size_t)last * D, D, lane);
+}
+
+template <bool VEC, int CPL>
+static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
+{
+    const int64_t chunks = (h->v.L + TT_DE_CHUNK - 1) / TT_DE_CHUNK;
+    const int grid = (int)((chunks + 7) / 8);
+    if (grid > 0) {
+        k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out);
+        k_dE_fix<VEC, CPL><<<grid, 256, 0, s>>>(h->v);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s)
+{
+    const int D = h->D;
+    const bool vec = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(grad_out) & 15) == 0);
+    if (vec) {
+        if (D <= 128) return launch_dE_t<true, 1>(h, grad_out, s);
+        if (D <= 256) return launch_dE_t<true, 2>(h, grad_out, s);
+        if (D <= 512) return launch_dE_t<true, 4>(h, grad_out, s);
+        return launch_dE_t<true, 8>(h, grad_out, s);
+    }
+    if (D <= 128) return launch_dE_t<false, 4>(h, grad_out, s);
+    if (D <= 256) return launch_dE_t<false, 8>(h, grad_out, s);
+    if (D <= 512) return launch_dE_t<false, 16>(h, grad_out, s);
+    return launch_dE_t<false, 32>(h, grad_out, s);
+}
+
+// ---------------------------------------------------------------------------------------------- 3. last level
+
+// same cost-balanced units as the forward sweep (forward.cu)
+__device__ __forceinline__ void tt_unit_range_b(const WsView& w, int unit, int& t_out, int& q_out, uint32_t& g0, uint32_t& g1)
+{
+    int t = 0;
+    for (int i = 0; i < w.T; ++i)
+        if (w.tdesc[i].unit_base <= unit) t = i;
+    const TableDesc& td = w.tdesc[t];
+    const int q = unit - td.unit_base, Q = td.units;
+    const int lvl = w.K - 1;
+    const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
+    const uint64_t ca = w.cost[a], cb = w.cost[b];
+    const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
+    auto lower = [&](uint64_t target) {
+        uint32_t lo = a, hi = b;
+        while (lo < hi) {
+            uint32_t mid = lo + ((hi - lo) >> 1);
+            if ((uint64_t)w.cost[mid] < target) lo = mid + 1; else hi = mid;
+        }
+        return lo;
+    };
+    g0 = q == 0 ? a : lower(lo_c);
+    g1 = q == Q - 1 ? b : lower(hi_c);
+    t_out = t;
+    q_out = q;
+}
+
+__device__ __forceinline__ void tt_mid_product_b(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
+                                                 int M, int ra, int cols)
+{
+    for (int c = threadIdx.x; c < cols; c += blockDim.x)
+        for (int m = 0; m < M; ++m) {
+            float acc = 0.f;
+            for (int a = 0; a < ra; ++a) acc = fmaf(Pl[m * ra + a], __ldg(Bsl + (size_t)a * cols + c), acc);
+            out[(size_t)m * cols + c] = acc;
+        }
+}
+
+__device__ __forceinline__ const float* tt_left_operand_b(const WsView& w, const TableDesc& td, int k, uint32_t v)
+{
+    if (k == 2) {
+        const uint32_t i1 = w.val[2][v] / (uint32_t)td.n[1];
+        return td.core[0] + (size_t)i1 * td.slice_floats[0];
+    }
+    return w.pbuf[k - 1] + (size_t)w.parent[k][v] * w.stride[k - 1];
+}
+
+__global__ void __launch_bounds__(256) k_sweep_bwd(WsView w, int pl_floats, int c_floats)
+{
+    extern __shared__ float sm[];
+    float* Pl = sm;
+    float* Cs = Pl + pl_floats;
+    float* dCs = Cs + c_floats;
+    float* dEs = dCs + c_floats;          // RB * D
+    float* priv = dEs + RB * w.D;         // n_K * slice_K (when priv_ok)
+    int t, q;
+    uint32_t g0, g1;
+    tt_unit_range_b(w, blockIdx.x, t, q, g0, g1);
+    const TableDesc& td = w.tdesc[t];
+    const int K = w.K, kl = K - 1, km = K - 2;
+    const int Pm = td.P[K - 1], rb = td.r[K - 1], dK = td.d[kl], D = w.D;
+    const int sliceK = td.slice_floats[kl];
+    const uint32_t nK = (uint32_t)td.n[kl];
+    const int priv_floats = (int)nK * sliceK;
+    const bool use_priv = td.priv_ok != 0;
+    if (use_priv)
+        for (int i = threadIdx.x; i < priv_floats; i += blockDim.x) priv[i] = 0.f;
+    for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) dCs[i] = 0.f;
+    __syncthreads();
+    for (uint32_t g = g0; g < g1; ++g) {
+        const uint32_t val = w.val[K - 1][g];
+        if (K >= 3) {
+            const int M = td.P[km], ra = td.r[km], cols = td.d[km] * rb;
+            const float* src = tt_left_operand_b(w, td, K - 1, g);
+            for (int i = threadIdx.x; i < M * ra; i += blockDim.x) Pl[i] = src[i];
+            __syncthreads();
+            const uint32_t im = val % (uint32_t)td.n[km];
+            tt_mid_product_b(Pl, td.core[km] + (size_t)im * td.slice_floats[km], Cs, M, ra, cols);
+        } else {
+            const float* src = td.core[0] + (size_t)val * td.slice_floats[0];
+            for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) Cs[i] = src[i];
+        }
+        __syncthreads();
+        const uint32_t u0 = w.cstart[K - 1][g], u1 = w.cstart[K - 1][g + 1];
+        for (uint32_t ub = u0; ub < u1; ub += RB) {
+            const int nr = (int)min((uint32_t)RB, u1 - ub);
+            for (int i = threadIdx.x; i < nr * D; i += blockDim.x) dEs[i] = w.E[(size_t)ub * D + i];
+            __syncthreads();
+            // dG_K[i_K][b][j] += sum_p C[p][b] * dE[p][j]     ("dD = C^T . dE")
+            for (int it = threadIdx.x; it < nr * sliceK; it += blockDim.x) {
+                const int rr = it / sliceK, e = it - rr * sliceK;
+                const int bb = e / dK, j = e - bb * dK;
+                const float* de = dEs + rr * D + j;
+                float acc = 0.f;
+                for (int p = 0; p < Pm; ++p) acc = fmaf(Cs[p * rb + bb], de[p * dK], acc);
+                const uint32_t iK = w.val[K][ub + rr] % nK;
+                if (use_priv) priv[iK * sliceK + e] += acc;      // rows of a group select distinct slices
+                else atomicAdd(td.grad[kl] + (size_t)iK * sliceK + e, acc);
+            }
+            // dC[p][b] += sum_j dE[p][j] * D[b][j]             ("dC = dE . D^T", summed over the group: Eq. 2)
+            for (int it = threadIdx.x; it < Pm * rb; it += blockDim.x) {
+                const int p = it / rb, bb = it - p * rb;
+                float acc = 0.f;
+                for (int rr = 0; rr < nr; ++rr) {
+                    const uint32_t iK = w.val[K][ub + rr] % nK;
+                    const float* Dsl = td.core[kl] + (size_t)iK * sliceK + bb * dK;
+                    const float* de = dEs + rr * D + p * dK;
+                    for (int j = 0; j < dK; ++j) acc = fmaf(de[j], __ldg(Dsl + j), acc);
+                }
+                dCs[it] += acc;
+            }
+            __syncthreads();
+        }
+        // hand dC to the level above (K = 2: it is the gradient of the first core's slice itself)
+        float* dst = K >= 3 ? w.dP[K - 1] + (size_t)g * w.stride[K - 1] : td.grad[0] + (size_t)val * td.slice_floats[0];
+        for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) { dst[i] = dCs[i]; dCs[i] = 0.f; }
+        __syncthreads();
+    }
+    if (use_priv) {
+        float* dst = w.gpart + td.gpart_off + (size_t)q * priv_floats;
+        for (int i = threadIdx.x; i < priv_floats; i += blockDim.x) dst[i] = priv[i];
+    }
+}
+
+// fixed-order sum of the per-unit copies of the last core's gradient
+__global__ void __launch_bounds__(256) k_reduce_gpart(WsView w)
+{
+    const int t = blockIdx.y;
+    const TableDesc& td = w.tdesc[t];
+    if (!td.priv_ok) return;
+    const int kl = w.K - 1;
+    const int64_t n = td.core_floats[kl];
+    const float* src = w.gpart + td.gpart_off;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        float s = 0.f;
+        for (int q = 0; q < td.units; ++q) s += src[(size_t)q * n + i];
+        td.grad[kl][i] = s;
+    }
+}
+
+cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
+{
+    WsView& w = h->v;
+    int max_pl = 1, max_c = 1;
+    for (int t = 0; t < h->T; ++t) {
+        const TableDesc& td = h->tab[t];
+        for (int k = 1; k < h->K; ++k) {
+            int f = td.P[k] * td.r[k];
+            if (k <= h->K - 2 && f > max_pl) max_pl = f;
+            if (k == h->K - 1 && f > max_c) max_c = f;
+        }
+    }
+    k_zero_grads<<<dim3(64, h->T), 256, 0, s>>>(w);
+    // P_k of the levels below K-1 are still in pbuf from the forward (K = 4 only)
+    const size_t smem = (size_t)(max_pl + 2 * max_c + RB * h->D + h->max_priv_floats) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_sweep_bwd<<<h->units_total, 256, smem, s>>>(w, max_pl, max_c);
+    k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------- 4. middle cores
+
+__device__ __forceinline__ uint32_t tt_tkey(const TableDesc& td, int k, uint32_t val)
+{
+    // digit-major key of a level-k node: i_k * (number of possible parents) + parent prefix value
+    const uint32_t nk = (uint32_t)td.n[k - 1];
+    return (val % nk) * td.prefix_space[k - 1] + val / nk;
+}
+
+__global__ void k_tmark(WsView w, int k)
+{
+    const uint32_t count = w.counters[CTR_LEVEL0 + k];
+    for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < count; v += gridDim.x * blockDim.x) {
+        const int t = tt_find_table(w.tb[k], w.T, v);
+        const TableDesc& td = w.tdesc[t];
+        const uint32_t key = tt_tkey(td, k, w.val[k][v]);
+        atomicOr(&w.tbm[k][td.tword_base[k] + (key >> 5)].x, 1u << (key & 31));
+    }
+}
+
+struct TPopScan {
+    WsView w;
+    int k;
+    __device__ uint32_t size() const { return w.ttotal_words[k]; }
+    __device__ uint32_t value(uint32_t i) const { return __popc(w.tbm[k][i].x); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t) const { w.tbm[k][i].y = excl; }
+    __device__ void total(uint32_t) const {}
+};
+
+__device__ __forceinline__ uint32_t tt_trank(const WsView& w, const TableDesc& td, int k, uint32_t key)
+{
+    const uint2 e = w.tbm[k][td.tword_base[k] + (key >> 5)];
+    return e.y + __popc(e.x & ((1u << (key & 31)) - 1u));
+}
+
+__global__ void k_tfill(WsView w, int k)
+{
+    const uint32_t count = w.counters[CTR_LEVEL0 + k];
+    for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < count; v += gridDim.x * blockDim.x) {
+        const int t = tt_find_table(w.tb[k], w.T, v);
+        const TableDesc& td = w.tdesc[t];
+        w.tnode[k][tt_trank(w, td, k, tt_tkey(td, k, w.val[k][v]))] = v;
+    }
+}
+
+// dP_{k-1}[parent] (or the first core's gradient slice when k = 2) = sum over children v of
+//   out[m][a] = sum_{j,b} dP_k[v][(m*d_k + j)*r_k + b] * G_k[i_k(v)][a][j][b]
+// one CTA per parent, children in sorted order; the slice is staged in shared memory (padded rows)
+__global__ void __launch_bounds__(256) k_mid_down(WsView w, int k)
+{
+    extern __shared__ float sm[];
+    const uint32_t count = w.counters[CTR_LEVEL0 + k - 1];
+    for (uint32_t pn = blockIdx.x; pn < count; pn += gridDim.x) {
+        const int t = tt_find_table(w.tb[k - 1], w.T, pn);
+        const TableDesc& td = w.tdesc[t];
+        const int kc = k - 1;
+        const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
+        const int ld = cols + 1;
+        float* Bs = sm;                  // ra * ld
+        float* dPs = sm + ra * ld;       // M * cols
+        const int nout = M * ra;
+        // each thread owns outputs o = tid, tid + 256, ... (at most 16 per thread: M*ra <= 4096)
+        float acc[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+        const uint32_t c0 = w.cstart[k - 1][pn], c1 = w.cstart[k - 1][pn + 1];
+        for (uint32_t v = c0; v < c1; ++v) {
+            const uint32_t ik = w.val[k][v] % (uint32_t)td.n[kc];
+            const float* Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
+            for (int i = threadIdx.x; i < ra * cols; i += blockDim.x) Bs[(i / cols) * ld + (i % cols)] = __ldg(Bsl + i);
+            const float* dp = w.dP[k] + (size_t)v * w.stride[k];
+            for (int i = threadIdx.x; i < M * cols; i += blockDim.x) dPs[i] = dp[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int o = threadIdx.x + i * 256;
+                if (o < nout) {
+                    const int m = o / ra, a = o - m * ra;
+                    const float* x = dPs + m * cols;
+                    const float* y = Bs + a * ld;
+                    float s = 0.f;
+                    for (int c = 0; c < cols; ++c) s = fmaf(x[c], y[c], s);
+                    acc[i] += s;
+                }
+            }
+            __syncthreads();
+        }
+        float* dst;
+        if (k == 2) dst = td.grad[0] + (size_t)w.val[1][pn] * td.slice_floats[0];
+        else dst = w.dP[k - 1] + (size_t)pn * w.stride[k - 1];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int o = threadIdx.x + i * 256;
+            if (o < nout) dst[o] = acc[i];
+        }
+    }
+}
+
+// gradient of slice i_k of core k (1-based, 2 <= k <= K-1) of table t:
+//   dG_k[i_k][a][c] = sum over level-k nodes v with digit i_k of sum_m P_{k-1}[parent(v)][m][a] * dP_k[v][m*cols + c]
+// one CTA per (table, slice); nodes come from the digit-major list, i.e. in ascending parent order
+__global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
+{
+    extern __shared__ float sm[];
+    const int t = blockIdx.y;
+    const TableDesc& td = w.tdesc[t];
+    const int kc = k - 1;
+    if ((int)blockIdx.x >= td.n[kc]) return;
+    const uint32_t ik = blockIdx.x;
+    const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
+    const int nout = ra * cols;
+    float* Pls = sm;             // M * ra
+    float* dPs = sm + M * ra;    // M * cols
+    const uint32_t space = td.prefix_space[k - 1];
+    const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
+    float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
+    for (int o0 = 0; o0 < nout; o0 += 256 * 16) {
+        float acc[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+        for (uint32_t jn = j0; jn < j1; ++jn) {
+            const uint32_t v = w.tnode[k][jn];
+            const float* pl = tt_left_operand_b(w, td, k, v);
+            for (int i = threadIdx.x; i < M * ra; i += blockDim.x) Pls[i] = pl[i];
+            const float* dp = w.dP[k] + (size_t)v * w.stride[k];
+            for (int i = threadIdx.x; i < M * cols; i += blockDim.x) dPs[i] = dp[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int o = o0 + threadIdx.x + i * 256;
+                if (o < nout) {
+                    const int a = o / cols, c = o - a * cols;
+                    float s = 0.f;
+                    for (int m = 0; m < M; ++m) s = fmaf(Pls[m * ra + a], dPs[m * cols + c], s);
+                    acc[i] += s;
+                }
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int o = o0 + threadIdx.x + i * 256;
+            if (o < nout) dst[o] = acc[i];
+        }
+    }
+}
+
+cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
+{
+    WsView& w = h->v;
+    cudaError_t e;
+    for (int k = h->K - 1; k >= 2; --k) {
+        int max_n = 1, max_down = 1, max_slice = 1;
+        for (int t = 0; t < h->T; ++t) {
+            const TableDesc& td = h->tab[t];
+            const int kc = k - 1;
+            const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
+            if (td.n[kc] > max_n) max_n = td.n[kc];
+            if (ra * (cols + 1) + M * cols > max_down) max_down = ra * (cols + 1) + M * cols;
+            if (M * ra + M * cols > max_slice) max_slice = M * ra + M * cols;
+        }
+        if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
+        const int g = h->sm_count * 8;
+        k_tmark<<<g, 256, 0, s>>>(w, k);
+        TPopScan tp{w, k};
+        if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
+        k_tfill<<<g, 256, 0, s>>>(w, k);
+        if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
+        k_mid_slice<<<dim3(max_n, h->T), 256, (size_t)max_slice * sizeof(float), s>>>(w, k);
+        if ((e = cudaFuncSetAttribute(k_mid_down, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_down * sizeof(float)))) != cudaSuccess) return e;
+        k_mid_down<<<h->sm_count * 8, 256, (size_t)max_down * sizeof(float), s>>>(w, k);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------- SGD
+
+__global__ void __launch_bounds__(256) k_sgd(WsView w, float lr)
+{
+    const int t = blockIdx.y / w.K, k = blockIdx.y % w.K;
+    const TableDesc& td = w.tdesc[t];
+    float* __restrict__ G = td.core[k];
+    const float* __restrict__ dG = td.grad[k];
+    const int64_t n = td.core_floats[k];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        G[i] = G[i] - lr * dG[i];
+}
+
+cudaError_t tt_launch_sgd(tt_emb* h, float lr, cudaStream_t s)
+{
+    k_sgd<<<dim3(64, h->T * h->K), 256, 0, s>>>(h->v, lr);
+    return cudaGetLastError();
+}

@@ -1,0 +1,135 @@
+// Internal declarations shared by the translation units of libtt_emb.so (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "tt_emb.h"
+
+#define TT_MAXK 4
+#define TT_SCAN_THREADS 256
+#define TT_SCAN_ITEMS 16
+#define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
+#define TT_DE_CHUNK 256                                  // sorted lookups per warp in the dE segment reduction
+#define TT_NUM_STAGES 9
+
+// Per-table descriptor, resident in the workspace.  k below is 0-based (core k+1 of the paper).
+struct TableDesc {
+    int64_t N;
+    int32_t n[TT_MAXK];
+    int32_t d[TT_MAXK];
+    int32_t r[TT_MAXK + 1];
+    int32_t P[TT_MAXK + 1];             // P[0] = 1, P[k] = d_1 * .. * d_k
+    int32_t slice_floats[TT_MAXK];      // r[k] * d[k] * r[k+1]
+    int64_t core_floats[TT_MAXK];       // n[k] * slice_floats[k]
+    float* core[TT_MAXK];
+    float* grad[TT_MAXK];
+    uint32_t word_base;                 // first 32-row word of this table in the presence bitmap
+    uint32_t num_words;
+    uint32_t tword_base[TT_MAXK];       // same for the digit-major ("transposed") node bitmaps, levels 2..K-1
+    uint32_t tnum_words[TT_MAXK];
+    uint32_t prefix_space[TT_MAXK + 1]; // n_1 * .. * n_k (number of possible length-k prefixes), k = 1..K-1
+    int64_t gpart_off;                  // float offset of this table's last-core gradient partials
+    int32_t units;                      // work units (CTAs) this table is cut into
+    int32_t unit_base;                  // first global unit id
+    int32_t priv_ok;                    // last-core gradient of this table fits the shared-memory private copy
+    int32_t pad;
+};
+
+// Device-side view of the workspace handed to kernels by value.
+struct WsView {
+    int32_t T, K, D;
+    int32_t stride[TT_MAXK + 1];        // floats per node of the level-k partial-product buffers (max over tables)
+    int64_t B, L;                       // current batch / lookups
+    int64_t capU;                       // capacity in distinct rows
+    uint32_t cap[TT_MAXK + 1];          // node capacity per level 1..K
+    uint32_t total_words;
+    uint32_t ttotal_words[TT_MAXK];
+    int32_t* status;
+    uint32_t* counters;                 // [k] = number of level-k nodes (k = 1..K); [8+k] transposed counts
+    TableDesc* tdesc;
+    int64_t* tl_start;                  // [T+1] first lookup of each table
+    uint2* bm;                          // {32 presence bits, number of set bits before this word (global)}
+    uint32_t* scan_tmp;
+    uint32_t* val[TT_MAXK + 1];         // level k: prefix value within the table (k = K: row id)
+    uint32_t* cstart[TT_MAXK + 1];      // level k < K: first child (level k+1 node); [count] = sentinel
+    uint32_t* parent[TT_MAXK + 1];      // level k >= 2: parent node at level k-1
+    uint32_t* tb[TT_MAXK + 1];          // [T+1] node range of each table at level k
+    uint32_t* cost;                     // [cap_{K-1}+1] exclusive scan of per-group cost (+ total)
+    float* pbuf[TT_MAXK + 1];           // partial products P_k of level-k nodes, 2 <= k <= K-2
+    float* E;                           // [capU][D] rows (forward) / dE (backward)
+    // backward
+    uint32_t* cnt;                      // [capU+1] lookups per distinct row -> exclusive scan
+    uint32_t* cursor;                   // [capU]
+    uint2* pairs;                       // [L] (slot, bag) sorted by slot
+    uint2* upairs;                      // [L] (slot, bag) in lookup order, written by the pooling kernel (null: forward only)
+    float* dP[TT_MAXK + 1];             // dP_k per level-k node, 2 <= k <= K-1
+    float* carry;                       // [chunks][2][D]
+    float* gpart;                       // last-core gradient partials
+    uint2* tbm[TT_MAXK + 1];            // digit-major node bitmaps, levels 2..K-1
+    uint32_t* tnode[TT_MAXK + 1];       // nodes of level k ordered by (table, i_k, parent prefix)
+    const int64_t* indices;
+    const int64_t* offsets;
+};
+
+enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16 };
+
+struct tt_emb {
+    int T, K, D;
+    int64_t max_batch, max_lookups, capU;
+    int enable_backward;
+    int sm_count;
+    int units_total;
+    int cost_shift;       // cost unit of the schedule = 2^cost_shift FMAs
+    TableDesc* tab;       // host copy [T]
+    size_t ws_bytes;
+    size_t off_status, off_counters, off_tdesc, off_tlstart, off_bm, off_scan, off_cost, off_E;
+    size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
+    size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
+    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart;
+    size_t scan_tmp_elems;
+    int64_t gpart_floats;
+    int max_priv_floats;  // largest n_K * slice_K among tables that use the private copy
+    WsView v;             // filled at bind
+    bool bound, have_forward;
+    bool timing;
+    cudaEvent_t ev[TT_NUM_STAGES][2];
+    bool ev_valid[TT_NUM_STAGES];
+    bool ev_created;
+};
+
+// ---- launchers implemented in the .cu files (all enqueue on `s`, return cudaGetLastError()) ----
+cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s);
+cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s);
+cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_sgd(tt_emb* h, float lr, cudaStream_t s);
+cudaError_t tt_launch_export_level(tt_emb* h, int table, int level, int64_t* vals, int32_t* rc, int32_t* lc, cudaStream_t s);
+cudaError_t tt_launch_export_inverse(tt_emb* h, int table, int32_t* inv, cudaStream_t s);
+cudaError_t tt_launch_pack(const TableDesc& td, int core, const float* src, float* dst, bool to_canonical, cudaStream_t s);
+
+// ---- small device helpers ----
+__device__ __forceinline__ int tt_find_table(const uint32_t* __restrict__ tb, int T, uint32_t v)
+{
+    // largest t with tb[t] <= v  (tb non-decreasing, tb[0] = 0)
+    int lo = 0, hi = T;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (tb[mid] <= v) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ int tt_find_table64(const int64_t* __restrict__ tb, int T, int64_t v)
+{
+    int lo = 0, hi = T;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (tb[mid] <= v) lo = mid; else hi = mid;
+    }
+    return lo;
+}

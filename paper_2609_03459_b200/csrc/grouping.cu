@@ -1,0 +1,274 @@
+// Prefix grouping (paper Sec. 3.3: sort, unique, mixed-radix conversion, run-length encoding), integer only.
+//
+// B200 design: the sort + unique of a table's row ids is a distribution (counting) sort over the row-id
+// domain with one presence bit per row.  The bitmaps of all tables (N_t / 8 bytes each) stay resident in
+// the 126 MB L2, so marking costs one L2 access per lookup, and an exclusive scan of the word popcounts
+// yields (a) the ascending list of distinct rows, (b) a rank structure {bits, base} that maps any row id
+// to its slot with one 8-byte load, so no per-lookup inverse map is ever written.  Prefix levels follow
+// by comparing neighbouring entries of the sorted lists (run-length encoding) and compacting with the
+// same scan.  No kernel waits on another CTA.
+#include "common.cuh"
+#include "scan.cuh"
+
+// ---------------------------------------------------------------------------------------------- prologue
+
+__global__ void k_check_offsets(WsView w)
+{
+    const int64_t nb = (int64_t)w.T * w.B;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i <= nb; i += stride) {
+        const int64_t o = w.offsets[i];
+        if (o < 0 || o > w.L) bad = true;
+        if (i == 0 && o != 0) bad = true;
+        if (i == nb && o != w.L) bad = true;
+        if (i < nb && w.offsets[i + 1] < o) bad = true;
+        if (i % w.B == 0 || i == nb) {
+            int64_t c = o < 0 ? 0 : (o > w.L ? w.L : o);
+            w.tl_start[i == nb ? w.T : i / w.B] = c;
+        }
+    }
+    if (bad) atomicOr(w.status, TT_EMB_STATUS_OFFSETS);
+}
+
+// ---------------------------------------------------------------------------------------------- mark
+
+__global__ void __launch_bounds__(256) k_mark(WsView w)
+{
+    const int64_t L = w.L;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x * 4;
+    int t = 0;
+    bool bad = false;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x * 4 + threadIdx.x; base < L; base += step) {
+        int64_t g[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t l = base + (int64_t)j * blockDim.x;
+            g[j] = l < L ? __ldg(w.indices + l) : -1;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t l = base + (int64_t)j * blockDim.x;
+            if (l >= L) continue;
+            if (!(w.tl_start[t] <= l && l < w.tl_start[t + 1])) t = tt_find_table64(w.tl_start, w.T, l);
+            const TableDesc& td = w.tdesc[t];
+            if (g[j] < 0 || g[j] >= td.N) { bad = true; continue; }
+            const uint32_t row = (uint32_t)g[j];
+            unsigned* word = &w.bm[td.word_base + (row >> 5)].x;
+            const unsigned m = 1u << (row & 31);
+            if (!(__ldcg(word) & m)) atomicOr(word, m);
+        }
+    }
+    if (bad) atomicOr(w.status, TT_EMB_STATUS_INDEX);
+}
+
+// ---------------------------------------------------------------------------------------------- level K: rows
+
+struct PopScan {
+    WsView w;
+    __device__ uint32_t size() const { return w.total_words; }
+    __device__ uint32_t value(uint32_t i) const { return __popc(w.bm[i].x); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v) const
+    {
+        w.bm[i].y = excl;
+        const int K = w.K;
+        // every table starts on a scan-tile boundary, so this search is uniform within a CTA
+        int t = 0;
+        {
+            int lo = 0, hi = w.T;
+            while (hi - lo > 1) {
+                int mid = (lo + hi) >> 1;
+                if (w.tdesc[mid].word_base <= i) lo = mid; else hi = mid;
+            }
+            t = lo;
+        }
+        const uint32_t wb = w.tdesc[t].word_base;
+        if (i == wb) w.tb[K][t] = excl < w.cap[K] ? excl : w.cap[K];
+        if (v) {
+            unsigned bits = w.bm[i].x;
+            uint32_t slot = excl;
+            const uint32_t row0 = (i - wb) << 5;
+            while (bits) {
+                const int b = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (slot < w.cap[K]) w.val[K][slot] = row0 + b;
+                ++slot;
+            }
+        }
+    }
+    __device__ void total(uint32_t tot) const
+    {
+        const int K = w.K;
+        if (tot > w.cap[K]) { atomicOr(w.status, TT_EMB_STATUS_OVERFLOW); tot = w.cap[K]; }
+        w.counters[CTR_LEVEL0 + K] = tot;
+        w.tb[K][w.T] = tot;
+    }
+};
+
+// ---------------------------------------------------------------------------------------------- level k from level k+1
+
+struct LevelUp {
+    WsView w;
+    int k;  // level being produced (1..K-1); reads level k+1
+    __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + k + 1]; }
+    __device__ uint32_t value(uint32_t v) const
+    {
+        const uint32_t* tbc = w.tb[k + 1];
+        const int t = tt_find_table(tbc, w.T, v);
+        const uint32_t nk = (uint32_t)w.tdesc[t].n[k];  // radix of digit k+1 (0-based core index k)
+        if (v == tbc[t]) return 1u;
+        return (w.val[k + 1][v] / nk != w.val[k + 1][v - 1] / nk) ? 1u : 0u;
+    }
+    __device__ void emit(uint32_t v, uint32_t excl, uint32_t flag) const
+    {
+        const uint32_t* tbc = w.tb[k + 1];
+        const int t = tt_find_table(tbc, w.T, v);
+        w.parent[k + 1][v] = excl + flag - 1u;
+        if (flag) {
+            w.val[k][excl] = w.val[k + 1][v] / (uint32_t)w.tdesc[t].n[k];
+            w.cstart[k][excl] = v;
+            if (v == tbc[t]) w.tb[k][t] = excl;
+        }
+    }
+    __device__ void total(uint32_t tot) const
+    {
+        w.counters[CTR_LEVEL0 + k] = tot;
+        w.cstart[k][tot] = size();
+        w.tb[k][w.T] = tot;
+    }
+};
+
+// tables without any node at level k+1 never had tb[k][t] written: inherit from the next table
+__global__ void k_fix_tb(WsView w, int k)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int t = w.T - 1; t >= 0; --t)
+            if (w.tb[k + 1][t] == w.tb[k + 1][t + 1]) w.tb[k][t] = w.tb[k][t + 1];
+    }
+}
+
+cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
+{
+    WsView& w = h->v;
+    cudaError_t e;
+    // status word + counters are adjacent; bitmap follows its own region
+    if ((e = cudaMemsetAsync(w.status, 0, (16 + 64) * sizeof(uint32_t), s)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(w.bm, 0, (size_t)w.total_words * sizeof(uint2), s)) != cudaSuccess) return e;
+    const int64_t nb = (int64_t)w.T * w.B + 1;
+    int g0 = (int)((nb + 255) / 256);
+    if (g0 > h->sm_count * 8) g0 = h->sm_count * 8;
+    k_check_offsets<<<g0, 256, 0, s>>>(w);
+    if (w.L > 0) {
+        int64_t want = (w.L + 1023) / 1024;
+        int g1 = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
+        k_mark<<<g1, 256, 0, s>>>(w);
+    }
+    PopScan ps{w};
+    if ((e = tt_scan(ps, w.total_words, w.scan_tmp, s)) != cudaSuccess) return e;
+    for (int k = w.K - 1; k >= 1; --k) {
+        LevelUp lu{w, k};
+        if ((e = tt_scan(lu, w.cap[k + 1], w.scan_tmp, s)) != cudaSuccess) return e;
+        k_fix_tb<<<1, 32, 0, s>>>(w, k);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------- export (inspection)
+
+// first leaf (level-K node) under node v of level k
+__device__ __forceinline__ uint32_t tt_first_leaf(const WsView& w, int k, uint32_t v)
+{
+    for (int j = k; j < w.K; ++j) v = w.cstart[j][v];
+    return v;
+}
+
+__global__ void k_export_mult(WsView w, int table)
+{
+    // lookups per distinct row of one table -> cursor[] (scratch), via the rank structure
+    const TableDesc& td = w.tdesc[table];
+    const int64_t lo = w.tl_start[table], hi = w.tl_start[table + 1];
+    for (int64_t l = lo + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < hi; l += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t g = w.indices[l];
+        if (g < 0 || g >= td.N) continue;
+        const uint2 e = w.bm[td.word_base + ((uint32_t)g >> 5)];
+        const uint32_t slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
+        if (slot < w.cap[w.K]) atomicAdd(&w.cursor[slot], 1u);
+    }
+}
+
+__global__ void k_export_level(WsView w, int table, int k, int64_t* vals, int32_t* rc, int32_t* lc, int have_mult)
+{
+    const uint32_t v0 = w.tb[k][table], v1 = w.tb[k][table + 1];
+    for (uint32_t v = v0 + blockIdx.x * blockDim.x + threadIdx.x; v < v1; v += gridDim.x * blockDim.x) {
+        if (vals) vals[v - v0] = (int64_t)w.val[k][v];
+        const uint32_t l0 = tt_first_leaf(w, k, v);
+        const uint32_t l1 = (v + 1 < w.counters[CTR_LEVEL0 + k]) ? tt_first_leaf(w, k, v + 1) : w.counters[CTR_LEVEL0 + w.K];
+        if (rc) rc[v - v0] = (int32_t)(l1 - l0);
+        if (lc && have_mult) {
+            uint32_t s = 0;
+            for (uint32_t u = l0; u < l1; ++u) s += w.cursor[u];
+            lc[v - v0] = (int32_t)s;
+        }
+    }
+}
+
+cudaError_t tt_launch_export_level(tt_emb* h, int table, int level, int64_t* vals, int32_t* rc, int32_t* lc, cudaStream_t s)
+{
+    WsView& w = h->v;
+    if (lc) {
+        cudaError_t e = cudaMemsetAsync(w.cursor, 0, (size_t)w.cap[w.K] * sizeof(uint32_t), s);
+        if (e != cudaSuccess) return e;
+        k_export_mult<<<h->sm_count * 4, 256, 0, s>>>(w, table);
+    }
+    k_export_level<<<h->sm_count * 4, 256, 0, s>>>(w, table, level, vals, rc, lc, lc ? 1 : 0);
+    return cudaGetLastError();
+}
+
+__global__ void k_export_inverse(WsView w, int table, int32_t* inv)
+{
+    const TableDesc& td = w.tdesc[table];
+    const int64_t lo = w.tl_start[table], hi = w.tl_start[table + 1];
+    const uint32_t base = w.tb[w.K][table];
+    for (int64_t l = lo + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < hi; l += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t g = w.indices[l];
+        int32_t r = -1;
+        if (g >= 0 && g < td.N) {
+            const uint2 e = w.bm[td.word_base + ((uint32_t)g >> 5)];
+            r = (int32_t)(e.y + __popc(e.x & ((1u << (g & 31)) - 1u)) - base);
+        }
+        inv[l - lo] = r;
+    }
+}
+
+cudaError_t tt_launch_export_inverse(tt_emb* h, int table, int32_t* inv, cudaStream_t s)
+{
+    k_export_inverse<<<h->sm_count * 4, 256, 0, s>>>(h->v, table, inv);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------- core layout conversion
+
+__global__ void k_pack(const float* __restrict__ src, float* __restrict__ dst, int rp, int n, int d, int rn, int to_canonical)
+{
+    // canonical [n][rp][d][rn]  <->  index order [rp][n][d][rn]
+    const int64_t total = (int64_t)rp * n * d * rn;
+    const int inner = d * rn;
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total; c += (int64_t)gridDim.x * blockDim.x) {
+        const int x = (int)(c % inner);
+        const int64_t q = c / inner;
+        const int a = (int)(q % rp);
+        const int i = (int)(q / rp);
+        const int64_t o = ((int64_t)a * n + i) * inner + x;
+        if (to_canonical) dst[c] = src[o]; else dst[o] = src[c];
+    }
+}
+
+cudaError_t tt_launch_pack(const TableDesc& td, int core, const float* src, float* dst, bool to_canonical, cudaStream_t s)
+{
+    const int64_t total = td.core_floats[core];
+    int grid = (int)((total + 255) / 256);
+    if (grid > 4096) grid = 4096;
+    if (grid < 1) grid = 1;
+    k_pack<<<grid, 256, 0, s>>>(src, dst, td.r[core], td.n[core], td.d[core], td.r[core + 1], to_canonical ? 1 : 0);
+    return cudaGetLastError();
+}

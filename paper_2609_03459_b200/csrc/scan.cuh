@@ -1,0 +1,109 @@
+// Device-wide exclusive scan of uint32 values produced by a functor, as three kernels
+// (tile sums -> scan of tile sums by one CTA -> per-tile scan + apply).  No inter-CTA waiting.
+//
+// Functor F:
+//   __device__ uint32_t size() const;                       number of elements (may read device memory)
+//   __device__ uint32_t value(uint32_t i) const;            input i
+//   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v) const;   called once per element in the apply pass
+//   __device__ void total(uint32_t tot) const;              called by one thread with the grand total
+#pragma once
+#include "common.cuh"
+
+__device__ __forceinline__ uint32_t tt_block_excl_scan(uint32_t x, uint32_t* sm /* [34] */, uint32_t& block_total)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    uint32_t incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) sm[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        uint32_t wv = lane < nw ? sm[lane] : 0u, wi = wv;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += y;
+        }
+        sm[lane] = wi - wv;
+        if (lane == 31) sm[33] = wi;
+    }
+    __syncthreads();
+    uint32_t res = sm[wid] + incl - x;
+    block_total = sm[33];
+    __syncthreads();
+    return res;
+}
+
+template <class F>
+__global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t* __restrict__ tile_sums)
+{
+    __shared__ uint32_t sm[34];
+    const uint32_t n = f.size();
+    const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
+    if (base >= n) return;
+    uint32_t s = 0;
+    const uint64_t i0 = base + (uint64_t)threadIdx.x * TT_SCAN_ITEMS;
+#pragma unroll 4
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j)
+        if (i0 + j < n) s += f.value((uint32_t)(i0 + j));
+    uint32_t tot;
+    tt_block_excl_scan(s, sm, tot);
+    if (threadIdx.x == 0) tile_sums[blockIdx.x] = tot;
+}
+
+template <class F>
+__global__ void __launch_bounds__(1024) tt_scan_spine(F f, uint32_t* __restrict__ tile_sums)
+{
+    __shared__ uint32_t sm[34];
+    const uint32_t n = f.size();
+    const uint32_t ntiles = (uint32_t)(((uint64_t)n + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
+    uint32_t carry = 0;
+    for (uint32_t b0 = 0; b0 < ntiles; b0 += blockDim.x) {
+        uint32_t i = b0 + threadIdx.x;
+        uint32_t x = i < ntiles ? tile_sums[i] : 0u;
+        uint32_t tot;
+        uint32_t ex = tt_block_excl_scan(x, sm, tot);
+        if (i < ntiles) tile_sums[i] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) f.total(carry);
+}
+
+template <class F>
+__global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
+{
+    __shared__ uint32_t sm[34];
+    const uint32_t n = f.size();
+    const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
+    if (base >= n) return;
+    uint32_t v[TT_SCAN_ITEMS];
+    uint32_t s = 0;
+    const uint64_t i0 = base + (uint64_t)threadIdx.x * TT_SCAN_ITEMS;
+#pragma unroll
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+        v[j] = (i0 + j < n) ? f.value((uint32_t)(i0 + j)) : 0u;
+        s += v[j];
+    }
+    uint32_t tot;
+    uint32_t ex = tile_sums[blockIdx.x] + tt_block_excl_scan(s, sm, tot);
+#pragma unroll
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+        if (i0 + j < n) f.emit((uint32_t)(i0 + j), ex, v[j]);
+        ex += v[j];
+    }
+}
+
+// capacity = host-known upper bound of f.size(); tmp must hold ceil(capacity / TT_SCAN_TILE) + 1 words
+template <class F>
+static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, cudaStream_t s)
+{
+    unsigned tiles = (unsigned)((capacity + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
+    if (tiles == 0) tiles = 1;
+    tt_scan_reduce<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    tt_scan_spine<F><<<1, 1024, 0, s>>>(f, tmp);
+    tt_scan_apply<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    return cudaGetLastError();
+}

@@ -1,0 +1,247 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 CPU oracle, on the same seeded inputs.
+
+Bar: integers (distinct rows, prefix groups, counts, inverse map) bit-exact after canonical ordering;
+fp32 tensors within max|err| <= 1e-5 * max|ref|, per output tensor."""
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from workloads import TableSpec
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def binding():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2609_03459_b200 import binding as b
+    return b
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def assert_close(got, ref, what):
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    scale = np.abs(ref).max() if ref.size else 0.0
+    err = np.abs(got - ref).max() if ref.size else 0.0
+    if scale == 0.0:
+        assert err == 0.0, f"{what}: reference is all zero but max|got| = {err}"
+    else:
+        assert err <= TOL * scale, f"{what}: max|err| = {err:.3e} > 1e-5 * {scale:.3e}"
+
+
+def run_forward(binding, wl, **kw):
+    emb = binding.from_workload(wl, **kw)
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    return emb, out.cpu().numpy()
+
+
+def check_grouping(emb, wl):
+    counts = emb.grouping_counts()
+    for t, s in enumerate(wl.tables):
+        idx, _ = wl.table_slice(t)
+        g = oracle.grouping(s.n, idx)
+        K = s.K
+        assert counts[t, K - 1] == g["uniq"].shape[0], (t, counts[t], g["uniq"].shape)
+        vals, rc, lc = emb.export_level(t, K, int(counts[t, K - 1]), with_lookup_counts=emb.enable_backward)
+        np.testing.assert_array_equal(vals, g["uniq"])
+        np.testing.assert_array_equal(rc, np.ones_like(rc))
+        if lc is not None:
+            np.testing.assert_array_equal(lc, g["mult"])
+        for k in range(1, K):
+            lev = g["levels"][k - 1]
+            assert counts[t, k - 1] == lev["vals"].shape[0]
+            vals, rc, lc = emb.export_level(t, k, int(counts[t, k - 1]), with_lookup_counts=emb.enable_backward)
+            np.testing.assert_array_equal(vals, lev["vals"])
+            np.testing.assert_array_equal(rc, lev["row_counts"])
+            if lc is not None:
+                np.testing.assert_array_equal(lc, lev["lookup_counts"])
+        inv = emb.export_inverse(t, idx.shape[0])
+        np.testing.assert_array_equal(inv, g["inv"])
+
+
+# ------------------------------------------------------------------------------------------ tiny forms of the five configs
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("mapping", ["identity", "scattered"])
+def test_tiny_configs_forward_and_grouping(binding, cfg, mapping):
+    wl = workloads.make(cfg, tiny=True, mapping=mapping)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"cfg{cfg}-tiny out")
+    check_grouping(emb, wl)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_tiny_configs_backward_and_sgd(binding, cfg):
+    wl = workloads.make(cfg, tiny=True)
+    rng = np.random.default_rng(cfg)
+    go = wl.grad_out if wl.grad_out is not None else rng.standard_normal((wl.B, wl.T * wl.D)).astype(np.float32)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    emb.backward(dev(go))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl, grad_out=go)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"cfg{cfg}-tiny dG[{t}][{k}]")
+    emb.sgd_step(0.01)
+    cores = emb.get_cores()
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref[t], 0.01)
+        for k in range(wl.tables[t].K):
+            assert_close(cores[t][k], want[k], f"cfg{cfg}-tiny core[{t}][{k}] after SGD")
+    assert emb.status() == 0
+
+
+# ------------------------------------------------------------------------------------------ medium cases: several tiles, ragged tails
+
+MEDIUM = [
+    # name, tables, B, pooling
+    ("k3-mixed", [TableSpec(200_003, (59, 59, 59), (4, 4, 4), (1, 16, 32, 1), 1.05, "normal", 0.05),
+                  TableSpec(1_500, (12, 12, 12), (4, 4, 4), (1, 32, 16, 1), 0.9, "normal", 0.05),
+                  TableSpec(150_000, (54, 54, 54), (4, 4, 4), (1, 7, 5, 1), 1.2, "normal", 0.05)], 300, (0, 40)),
+    ("k2", [TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 1.0, "uniform", 0.1)], 257, (1, 9)),
+    ("k4", [TableSpec(40_000, (15, 14, 14, 14), (2, 4, 4, 4), (1, 6, 9, 5, 1), 1.1, "normal", 0.05)], 200, 8),
+    ("odd-D", [TableSpec(30_000, (32, 32, 32), (3, 3, 5), (1, 4, 6, 1), 1.0, "normal", 0.1)], 123, (0, 12)),
+    ("wide-D", [TableSpec(5_000, (18, 18, 18), (8, 8, 8), (1, 4, 4, 1), 1.0, "normal", 0.1)], 64, (1, 6)),
+]
+
+
+@pytest.mark.parametrize("case", MEDIUM, ids=[c[0] for c in MEDIUM])
+def test_medium_forward_backward(binding, case):
+    name, tables, B, pooling = case
+    wl = workloads.custom(tables, B, pooling, seed=77, with_grad=True, name=name)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"{name} out")
+    check_grouping(emb, wl)
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"{name} dG[{t}][{k}]")
+
+
+def test_forward_only_handle_and_repeat_calls(binding):
+    # a forward-only handle (no backward workspace) gives the same output, and calling twice is idempotent
+    name, tables, B, pooling = MEDIUM[0]
+    wl = workloads.custom(tables, B, pooling, seed=5)
+    emb, out1 = run_forward(binding, wl, enable_backward=False)
+    out2 = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    np.testing.assert_array_equal(out1, out2)
+    assert_close(out1, oracle.forward_workload(wl), "forward-only out")
+    # a different batch through the same handle (smaller batch, fewer lookups)
+    wl2 = workloads.custom(tables, B // 2, pooling, seed=6)
+    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    out3 = emb.forward(dev(wl2.indices), dev(wl2.offsets), wl2.B).cpu().numpy()
+    wl2.cores = wl.cores
+    assert_close(out3, oracle.forward_workload(wl2), "second batch out")
+
+
+# ------------------------------------------------------------------------------------------ degenerate inputs
+
+def test_hot_row_and_long_segments(binding):
+    # one row takes ~70 % of 60k lookups: exercises chunk-crossing segments of the dE reduction,
+    # the hash-aggregated sort and a bag with thousands of lookups
+    spec = TableSpec(50_000, (37, 37, 37), (4, 4, 4), (1, 8, 16, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec], 40, (500, 2500), seed=3, with_grad=True)
+    rng = np.random.default_rng(0)
+    hot = rng.random(wl.L) < 0.7
+    wl.indices[hot] = 31_337
+    wl.indices[rng.random(wl.L) < 0.1] = 31_338
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert_close(out, oracle.forward_workload(wl), "hot out")
+    check_grouping(emb, wl)
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for k in range(3):
+        assert_close(grads[0][k], ref[0][k], f"hot dG[{k}]")
+
+
+def test_all_bags_empty(binding):
+    spec = TableSpec(1000, (10, 10, 10), (4, 4, 4), (1, 4, 4, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec, spec], 9, 0, seed=1, with_grad=True)
+    assert wl.L == 0
+    import torch
+    emb = binding.from_workload(wl, enable_backward=True)
+    idx = torch.zeros(1, dtype=torch.int64, device="cuda")[:0]
+    out = emb.forward(idx, dev(wl.offsets), wl.B).cpu().numpy()
+    assert emb.status() == 0
+    assert np.count_nonzero(out) == 0
+    emb.backward(dev(wl.grad_out))
+    for row in emb.get_grads():
+        for g in row:
+            assert np.count_nonzero(g) == 0
+
+
+def test_out_of_range_indices_are_flagged_and_ignored(binding):
+    spec = TableSpec(997, (10, 10, 10), (4, 4, 4), (1, 4, 4, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec], 20, (1, 6), seed=2, with_grad=True)
+    bad = wl.indices.copy()
+    bad[3] = 997       # first padding row: not a valid row id
+    bad[10] = -5
+    bad[11] = 1 << 40
+    wl_bad = workloads.Workload(wl.name, wl.tables, wl.B, bad, wl.offsets, wl.cores, wl.grad_out)
+    emb, out = run_forward(binding, wl_bad, enable_backward=True)
+    assert emb.status() & binding.STATUS_INDEX
+    assert_close(out, oracle.forward_workload(wl_bad), "oob out")   # the oracle skips them as well
+    emb.backward(dev(wl.grad_out))
+    ref = oracle.backward_workload(wl_bad)
+    grads = emb.get_grads()
+    for k in range(3):
+        assert_close(grads[0][k], ref[0][k], f"oob dG[{k}]")
+
+
+def test_bad_offsets_are_flagged(binding):
+    spec = TableSpec(997, (10, 10, 10), (4, 4, 4), (1, 4, 4, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec], 20, 3, seed=2)
+    off = wl.offsets.copy()
+    off[5], off[6] = off[6], off[5] - 1
+    emb = binding.from_workload(wl)
+    emb.forward(dev(wl.indices), dev(off), wl.B)
+    assert emb.status() & binding.STATUS_OFFSETS
+
+
+def test_unique_row_capacity_overflow_is_flagged(binding):
+    spec = TableSpec(5000, (18, 18, 18), (4, 4, 4), (1, 4, 4, 1), 0.5, "normal", 0.1)
+    wl = workloads.custom([spec], 50, 20, seed=4)
+    emb = binding.from_workload(wl, max_unique_rows=100)
+    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    assert emb.status() & binding.STATUS_OVERFLOW
+
+
+def test_pack_unpack_round_trip(binding):
+    wl = workloads.make(4, tiny=True)
+    emb = binding.from_workload(wl)
+    back = emb.get_cores()
+    for k in range(4):
+        np.testing.assert_array_equal(back[0][k], wl.cores[0][k])
+
+
+def test_invariants_index_order_and_bag_additivity(binding):
+    # results do not depend on the order of indices inside a bag; a bag holding two bags' lookups is their sum
+    spec = TableSpec(20_000, (28, 28, 28), (4, 4, 4), (1, 8, 8, 1), 1.1, "normal", 0.1)
+    wl = workloads.custom([spec], 64, 16, seed=9)
+    emb, out = run_forward(binding, wl)
+    rng = np.random.default_rng(1)
+    perm = wl.indices.reshape(64, 16).copy()
+    for b in range(64):
+        rng.shuffle(perm[b])
+    out_p = emb.forward(dev(perm.reshape(-1)), dev(wl.offsets), 64).cpu().numpy()
+    assert np.abs(out_p - out).max() <= 2e-6 * np.abs(out).max()
+    merged_off = wl.offsets[::2].copy()
+    out_m = emb.forward(dev(wl.indices), dev(merged_off), 32).cpu().numpy()
+    assert np.abs(out_m - (out[0::2] + out[1::2])).max() <= 2e-6 * np.abs(out).max()
