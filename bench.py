@@ -1,0 +1,446 @@
+#!/usr/bin/env python
+"""Benchmark of the TT-embedding path: pooled lookups/s on seeded synthetic workloads, with roofline.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2|cfg4|cfg1] [--impl reference]
+
+A step is one pass of the whole hot path over one batch: grouping, schedule, contraction, pooling and --
+for the training workload (cfg5, the default: the 60-table configuration with backward and SGD) --
+the backward pass and the SGD update.  Prints ONE JSON line on rank 0.
+
+  value      lookups/s of the whole job (all ranks), inputs resident in HBM before the timed region
+  e2e        the same through the public call with HOST (pinned) buffers: H2D of indices/offsets(/grad_out)
+             and D2H of `out` inside the timed region
+  roofline   the dominant kernel of the step against its own bound (measured peaks)
+  step_roofline  the whole step against max(FP32 slots / measured FP32 peak, HBM bytes / measured HBM peak)
+  cpu_baseline   the fp64 oracle, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
+
+`--impl reference` times the oracle alone on the host cores (same metric, bounded sample per step).
+With N > 1 (torchrun) every rank runs the same configuration on its own seeded batch (weak scaling,
+batch-sharded replicas); the training step all-reduces the core gradients (NCCL) before SGD.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "pooled TT-embedding lookups/sec at batch 32768 (fwd, fwd+bwd); % of roofline"
+UNIT = "lookups/s"
+WORKLOADS = {
+    "cfg1": (1, False, "config 1: 1 table 100x100x100, D=64, ranks [1,8,8,1], batch 1024, pooling 1, Zipf 1.05, forward"),
+    "cfg2": (2, False, "config 2: 1 table 200x250x200, D=128, ranks [1,32,32,1], batch 32768, pooling 20, Zipf 1.1, forward"),
+    "cfg3": (3, False, "config 3: 60 tables N~logU[1e4,4e7], D=64, ranks {16,32}, batch 32768, pooling U[1,100], Zipf U[0.8,1.2], forward"),
+    "cfg4": (4, False, "config 4: 1 table 64^4, D=128, ranks [1,64,64,64,1], batch 65536, pooling 8, Zipf 1.2, forward"),
+    "cfg5": (5, True, "config 5: config-3 tables and indices, forward + backward (grad_out N(0,1)) + SGD lr 0.01"),
+}
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (profiling recipe)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while a timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()  # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def sample_bags(wl, stride: int):
+    """Every stride-th bag of every table, as a list of per-table (indices, offsets, bag ids)."""
+    res = []
+    for t in range(wl.T):
+        idx, off = wl.table_slice(t)
+        bags = np.arange(0, wl.B, stride)
+        lens = (off[1:] - off[:-1])[bags]
+        sub_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        sub_idx = np.concatenate([idx[off[b]:off[b + 1]] for b in bags]) if len(bags) else np.zeros(0, np.int64)
+        res.append((sub_idx, sub_off, bags))
+    return res
+
+
+def oracle_pass(wl, sample, train: bool) -> int:
+    """One pass of the fp64 oracle (as it stands) over the sampled bags; returns lookups processed."""
+    import oracle
+    n = 0
+    D = wl.D
+    for t, (idx, off, bags) in enumerate(sample):
+        s = wl.tables[t]
+        oracle.forward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off)
+        if train:
+            g = oracle.backward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off, wl.grad_out[bags, t * D:(t + 1) * D])
+            oracle.sgd(wl.cores[t], g, wl.lr)
+        n += idx.shape[0]
+    return n
+
+
+def pick_stride(wl, train: bool) -> int:
+    # aim at roughly 10-30 s of CPU work for the sample (measured rates of the plain oracle: ~0.5 M lookups/s
+    # forward, ~0.1 M lookups/s with backward, at rank 32 on 8 cores; scaled by the contraction size)
+    spec = wl.tables[0]
+    K = spec.K
+    fma = 0
+    P = 1
+    for k in range(K):
+        fma += P * spec.r[k] * spec.d[k] * spec.r[k + 1]
+        P *= spec.d[k]
+    per_lookup = fma * (4.0 if train else 1.0)
+    budget = 15.0 * 5e9  # ~5 G fp64 FMA/s on a handful of cores
+    want = max(1.0, budget / per_lookup)
+    stride = int(max(1, round(wl.L / want)))
+    return min(stride, max(1, wl.B // 4))
+
+
+# ------------------------------------------------------------------------------------------------ algorithmic work
+
+def algorithmic_work(wl, counts, train: bool):
+    """FP32 slots (FMA or ADD lanes) and HBM bytes the method itself needs after de-duplication."""
+    T, K, D, L, B = wl.T, wl.tables[0].K, wl.D, wl.L, wl.B
+    s_contract = 0
+    touched_core_bytes = 0
+    seg_adds = 0
+    for t, s in enumerate(wl.tables):
+        P = 1
+        for k in range(1, K + 1):           # level k uses core k (1-based)
+            c_k = P * s.r[k - 1] * s.d[k - 1] * s.r[k]
+            if k >= 2:
+                s_contract += int(counts[t, k - 1]) * c_k
+            slice_f = s.r[k - 1] * s.d[k - 1] * s.r[k]
+            touched_core_bytes += min(int(counts[t, k - 1]), s.n[k - 1]) * slice_f * 4
+            seg_adds += int(counts[t, k - 1]) * slice_f
+            P *= s.d[k - 1]
+    U = int(counts[:, K - 1].sum())
+    core_bytes = sum(c.size * 4 for tc in wl.cores for c in tc)
+    fwd_slots = s_contract + L * D
+    fwd_bytes = 8 * L + 8 * (T * B + 1) + 8 * U + min(touched_core_bytes, core_bytes) + 4 * B * T * D
+    res = {"U_rows": U, "U_prefix": int(counts[:, K - 2].sum()), "fwd_slots": fwd_slots, "fwd_hbm_bytes": fwd_bytes,
+           "contract_slots": s_contract, "pool_slots": L * D,
+           "pool_kernel_bytes": 8 * L + 8 * (T * B + 1) + 4 * U * D + 4 * B * T * D}
+    if train:
+        # dE sums; dD and dC per row and the level above (2x the forward contractions), recompute of the
+        # on-chip intermediates (levels below K), segment-reduce adds of the slice gradients
+        recompute = 0
+        for t, s in enumerate(wl.tables):
+            P = 1
+            for k in range(1, K):
+                if k >= 2:
+                    recompute += int(counts[t, k - 1]) * P * s.r[k - 1] * s.d[k - 1] * s.r[k]
+                P *= s.d[k - 1]
+        bwd_slots = L * D + 2 * s_contract + recompute + seg_adds
+        bwd_bytes = 8 * L + 4 * B * T * D + core_bytes + 3 * core_bytes
+        res.update({"bwd_slots": bwd_slots, "bwd_hbm_bytes": bwd_bytes,
+                    "dE_kernel_bytes": 8 * L + 4 * B * T * D + 4 * U * D})
+    return res
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+
+def run_reference(args, wl, train, desc, rank, world):
+    if rank != 0:
+        return
+    stride = args.cpu_stride or pick_stride(wl, train)
+    sample = sample_bags(wl, stride)
+    cores = len(os.sched_getaffinity(0))
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle_pass(wl, sample, train)
+    t0 = time.perf_counter()
+    n = 0
+    for _ in range(args.steps):
+        n += oracle_pass(wl, sample, train)
+    dt = time.perf_counter() - t0
+    v = n / dt
+    sample_desc = f"every {stride}-th bag of every table ({n // args.steps} lookups per step), fp64 oracle, OpenMP over bags"
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": desc, "mapping": args.mapping, "sample": sample_desc},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_desc},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ main arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
+    ap.add_argument("--mapping", default="identity", choices=["identity", "scattered"])
+    ap.add_argument("--cpu-stride", type=int, default=0, help="bag stride of the oracle sample (0 = automatic)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg_id, train, desc = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        wl = workloads.make(cfg_id, mapping=args.mapping)
+        run_reference(args, wl, train, desc, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_03459_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    # every rank draws its own batch from the same recipe (weak scaling); tables/cores are identical
+    wl = workloads.make(cfg_id, mapping=args.mapping)
+    if rank > 0:
+        other = workloads.make(cfg_id, mapping=args.mapping, seed=workloads.BASE_SEED + 7919 * rank)
+        wl.indices, wl.offsets, wl.grad_out = other.indices, other.offsets, other.grad_out
+        del other
+    T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
+
+    emb = binding.from_workload(wl, enable_backward=train, device=device)
+    h_idx = torch.from_numpy(wl.indices).pin_memory()
+    h_off = torch.from_numpy(wl.offsets).pin_memory()
+    h_grad = torch.from_numpy(wl.grad_out).pin_memory() if train else None
+    h_out = torch.empty((B, T * D), dtype=torch.float32).pin_memory()
+    d_idx, d_off = h_idx.to(device), h_off.to(device)
+    d_grad = h_grad.to(device) if train else None
+    d_out = torch.empty((B, T * D), dtype=torch.float32, device=device)
+
+    def step(idx, off, grad):
+        emb.forward(idx, off, B, out=d_out)
+        if train:
+            emb.backward(grad)
+            if world > 1:
+                dist.all_reduce(emb.flat_grads)   # the one exchange of the data-parallel path
+            emb.sgd_step(wl.lr)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=device)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    # ---- roofline denominators measured in this run
+    fp32_peak = binding.probe_fp32()
+    l2_gather = binding.probe_gather(32 << 20, device=device)
+    hbm_gather = binding.probe_gather(2 << 30, device=device)
+    hbm_gbs, peak_src = measured_peaks()
+
+    for _ in range(args.warmup):
+        step(d_idx, d_off, d_grad)
+    torch.cuda.synchronize()
+    status = emb.status()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    # ---- device-resident timing of the whole step, per-stage events enabled
+    emb.enable_timing(True)
+    stage_tot = {}
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    stage_runs = []
+    for _ in range(args.steps):
+        step(d_idx, d_off, d_grad)
+        stage_runs.append(None)
+    e1.record()
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    # per-stage averages: events of the last step are still valid; re-run a few steps to average them
+    stage_acc = {}
+    for _ in range(min(args.steps, 5)):
+        step(d_idx, d_off, d_grad)
+        torch.cuda.synchronize()
+        for k, v in emb.stage_ms().items():
+            stage_acc.setdefault(k, []).append(v)
+    stage_ms = {k: float(np.mean(v)) for k, v in stage_acc.items()}
+    emb.enable_timing(False)
+    ms_t = torch.tensor([total_ms], device=device)
+    if world > 1:
+        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
+    total_ms = float(ms_t.item())
+    ms_per_step = total_ms / args.steps
+
+    # ---- forward only (same inputs)
+    fwd_ms = timed(lambda: emb.forward(d_idx, d_off, B, out=d_out), args.steps) / args.steps
+
+    # ---- end to end through host buffers
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step():
+            idx = h_idx.to(device, non_blocking=True)
+            off = h_off.to(device, non_blocking=True)
+            grad = h_grad.to(device, non_blocking=True) if train else None
+            step(idx, off, grad)
+            h_out.copy_(d_out, non_blocking=True)
+        for _ in range(2):
+            e2e_step()
+        e2e_ms = timed(e2e_step, args.steps) / args.steps
+        h2d = h_idx.numel() * 8 + h_off.numel() * 8 + (h_grad.numel() * 4 if train else 0)
+        e2e = {"value": world * L / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4)}
+    clocks = sampler.stop()
+
+    counts = emb_counts = None
+    emb.forward(d_idx, d_off, B, out=d_out)
+    torch.cuda.synchronize()
+    counts = emb.grouping_counts()
+    work = algorithmic_work(wl, counts, train)
+
+    # ---- roofline of the dominant kernel (stage) and of the whole step
+    def stage_roof(name, ms):
+        if name == "pooling":
+            ach = work["pool_kernel_bytes"] / (ms * 1e-3) / 1e9
+            return {"kernel": "k_pool_vec", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                    "frac": ach / hbm_gbs, "traffic": None, "peak_source": peak_src,
+                    "note": "algorithmic bytes: indices + offsets + each distinct row once + out; the per-lookup row "
+                            "gather (L*D*4 bytes, mostly L2 hits) is not counted",
+                    "l2_gather_GBs": wl.L * D * 4 / (ms * 1e-3) / 1e9, "l2_gather_peak_GBs": l2_gather / 1e9}
+        if name == "contraction":
+            ach = work["contract_slots"] / (ms * 1e-3) / 1e12
+            return {"kernel": "k_sweep_fwd", "bound": "alu", "achieved": ach, "peak": fp32_peak / 1e12,
+                    "unit": "T FP32 lane-ops/s", "frac": ach / (fp32_peak / 1e12), "traffic": None,
+                    "peak_source": "independent-FMA-chain probe in this run"}
+        if name == "bwd_dE" and train:
+            ach = work["dE_kernel_bytes"] / (ms * 1e-3) / 1e9
+            return {"kernel": "k_dE", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                    "frac": ach / hbm_gbs, "traffic": None, "peak_source": peak_src}
+        if name in ("bwd_contraction", "bwd_middle") and train:
+            slots = work["bwd_slots"] - wl.L * D
+            ach = slots / (ms * 1e-3) / 1e12
+            return {"kernel": "k_sweep_bwd" if name == "bwd_contraction" else "k_mid_slice+k_mid_down", "bound": "alu",
+                    "achieved": ach, "peak": fp32_peak / 1e12, "unit": "T FP32 lane-ops/s",
+                    "frac": ach / (fp32_peak / 1e12), "traffic": None,
+                    "peak_source": "independent-FMA-chain probe in this run",
+                    "note": "all backward contraction slots attributed to this stage (upper bound on its share)"}
+        ach = (8 * wl.L) / (ms * 1e-3) / 1e9
+        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s", "frac": ach / hbm_gbs,
+                "traffic": None, "peak_source": peak_src, "note": "algorithmic bytes: one pass over the indices"}
+
+    dominant = max(stage_ms, key=stage_ms.get) if stage_ms else "pooling"
+    roofline = stage_roof(dominant, stage_ms.get(dominant, ms_per_step))
+    tot_slots = work["fwd_slots"] + (work["bwd_slots"] if train else 0)
+    tot_bytes = work["fwd_hbm_bytes"] + (work["bwd_hbm_bytes"] if train else 0)
+    t_alu, t_hbm = tot_slots / fp32_peak, tot_bytes / (hbm_gbs * 1e9)
+    step_roof = {"t_alu_ms": t_alu * 1e3, "t_hbm_ms": t_hbm * 1e3, "bound": "alu" if t_alu >= t_hbm else "hbm",
+                 "t_roof_ms": max(t_alu, t_hbm) * 1e3, "frac": max(t_alu, t_hbm) * 1e3 / ms_per_step,
+                 "fp32_slots": tot_slots, "hbm_bytes": tot_bytes}
+    fwd_roof_t = max(work["fwd_slots"] / fp32_peak, work["fwd_hbm_bytes"] / (hbm_gbs * 1e9))
+
+    launches_fwd = 2 + 3 + 4 * (K - 1) + 3 + max(K - 3, 0) + 2
+    launches_bwd = 7 + 2 + 3 + 7 * (K - 2) + 1
+    line = {
+        "metric": METRIC, "value": world * L / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": desc, "mapping": args.mapping, "tables": T, "batch_per_gpu": B, "lookups_per_gpu": L,
+                   "step": "forward+backward+sgd" if train else "forward",
+                   "parallelism": f"dp{world} (batch-sharded replicas" + (", all-reduce of core gradients)" if train else ")"),
+                   "l2_policy": "inputs larger than L2 (indices alone are %.0f MB)" % (L * 8 / 1e6)},
+        "forward_only": {"value": world * L / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,
+                         "roofline_frac": fwd_roof_t * 1e3 / fwd_ms, "t_roof_ms": fwd_roof_t * 1e3},
+        "stage_ms": stage_ms, "roofline": roofline, "step_roofline": step_roof,
+        "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
+                  "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},
+        "work": work, "device_status": status, "clocks": clocks, "e2e": e2e,
+        "gpu_launches": launches_fwd + (launches_bwd if train else 0),
+        "workspace_GB": emb.workspace_bytes / 1e9,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        stride = args.cpu_stride or pick_stride(wl, train)
+        sample = sample_bags(wl, stride)
+        t0 = time.perf_counter()
+        n = oracle_pass(wl, sample, train)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                                "sample": f"every {stride}-th bag of every table ({n} lookups, {dt:.1f} s), fp64, "
+                                          "same step (forward" + ("+backward+sgd)" if train else ")")}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

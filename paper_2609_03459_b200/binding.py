@@ -159,21 +159,32 @@ class TTEmbeddingBag:
 
     # ---- set-up
     def set_cores(self, cores):
-        """cores[t][k]: fp32 array of shape (r_{k-1}, n_k, d_k, r_k).  Packs to slice-major and binds."""
+        """cores[t][k]: fp32 array of shape (r_{k-1}, n_k, d_k, r_k).  Packs to slice-major and binds.
+        All cores live in one flat device buffer (self.flat_cores), all gradients in another
+        (self.flat_grads), so a multi-GPU job can all-reduce the gradients with a single collective."""
         torch = self.torch
         with torch.cuda.device(self.device):
             s = _stream_ptr()
+            sizes = [int(np.prod(self.shapes[t][k])) for t in range(self.T) for k in range(self.K)]
+            offs, tot = [], 0
+            for n in sizes:
+                offs.append(tot)
+                tot += (n + 3) // 4 * 4  # keep every core 16-byte aligned
+            self.flat_cores = torch.empty(max(tot, 4), dtype=torch.float32, device=self.device)
             self.cores = []
+            i = 0
             for t in range(self.T):
                 row = []
                 for k in range(self.K):
-                    src = torch.as_tensor(np.ascontiguousarray(cores[t][k], dtype=np.float32)
-                                          if not torch.is_tensor(cores[t][k]) else cores[t][k])
+                    src = cores[t][k]
+                    if not torch.is_tensor(src):
+                        src = torch.from_numpy(np.ascontiguousarray(src, dtype=np.float32))
                     src = src.to(self.device, dtype=torch.float32).contiguous()
                     assert tuple(src.shape) == tuple(self.shapes[t][k]), (t, k, src.shape, self.shapes[t][k])
-                    dst = torch.empty(src.numel(), dtype=torch.float32, device=self.device)
+                    dst = self.flat_cores[offs[i]:offs[i] + sizes[i]]
                     _check(lib.tt_emb_pack_core(self.h, t, k, src.data_ptr(), dst.data_ptr(), s), "tt_emb_pack_core")
                     row.append(dst)
+                    i += 1
                 self.cores.append(row)
             torch.cuda.current_stream().synchronize()
             if self.workspace is None:
@@ -182,7 +193,14 @@ class TTEmbeddingBag:
             ptrs = (ctypes.c_void_p * (self.T * self.K))(*[c.data_ptr() for row in self.cores for c in row])
             _check(lib.tt_emb_bind(self.h, ptrs, base, self.workspace_bytes, s), "tt_emb_bind")
             if self.enable_backward:
-                self.grads = [[torch.empty_like(c) for c in row] for row in self.cores]
+                self.flat_grads = torch.zeros_like(self.flat_cores)
+                self.grads, i = [], 0
+                for t in range(self.T):
+                    row = []
+                    for k in range(self.K):
+                        row.append(self.flat_grads[offs[i]:offs[i] + sizes[i]])
+                        i += 1
+                    self.grads.append(row)
 
     def get_cores(self):
         """Cores back in index order [r_{k-1}, n_k, d_k, r_k] as numpy fp32."""

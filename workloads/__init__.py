@@ -19,6 +19,8 @@ Conventions
 from __future__ import annotations
 
 import math
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 from typing import List, Optional, Sequence, Tuple
 
@@ -88,9 +90,9 @@ def _scatter_multiplier(N: int) -> int:
 
 def zipf_rows(rng: np.random.Generator, N: int, alpha: float, size: int, mapping: str = "identity") -> np.ndarray:
     """`size` row ids in [0, N) whose popularity rank follows a bounded Zipf(alpha) law."""
-    k = np.arange(1, N + 1, dtype=np.float64)
-    w = k ** (-float(alpha))
-    cdf = np.cumsum(w)
+    cdf = np.arange(1, N + 1, dtype=np.float64)
+    np.power(cdf, -float(alpha), out=cdf)
+    np.cumsum(cdf, out=cdf)
     cdf /= cdf[-1]
     u = rng.random(size)
     rank0 = np.searchsorted(cdf, u, side="left").astype(np.int64)
@@ -131,17 +133,26 @@ def near_equal_factors3(N: int) -> Tuple[int, int, int]:
 def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None) -> Workload:
     """pooling: int (fixed) or (lo, hi) inclusive uniform per (table, bag)."""
     T = len(tables)
-    idx_parts, len_parts, cores = [], [], []
-    for t, spec in enumerate(tables):
+
+    def one_table(t):
+        # every table has its own generator, so the result does not depend on thread scheduling
+        spec = tables[t]
         rng = np.random.default_rng(seed0 + t)
-        cores.append(make_cores(rng, spec))
+        tc = make_cores(rng, spec)
         if isinstance(pooling, tuple):
             lens = rng.integers(pooling[0], pooling[1] + 1, size=B, dtype=np.int64)
         else:
             lens = np.full(B, int(pooling), dtype=np.int64)
-        Lt = int(lens.sum())
-        idx_parts.append(zipf_rows(rng, spec.N, spec.alpha, Lt, mapping))
-        len_parts.append(lens)
+        return tc, lens, zipf_rows(rng, spec.N, spec.alpha, int(lens.sum()), mapping)
+
+    if T > 1 and sum(s.N for s in tables) > 1_000_000:
+        with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+            parts = list(ex.map(one_table, range(T)))
+    else:
+        parts = [one_table(t) for t in range(T)]
+    cores = [p[0] for p in parts]
+    len_parts = [p[1] for p in parts]
+    idx_parts = [p[2] for p in parts]
     lens = np.concatenate(len_parts)
     offsets = np.zeros(T * B + 1, dtype=np.int64)
     np.cumsum(lens, out=offsets[1:])
