@@ -230,6 +230,8 @@ def main():
     ap.add_argument("--cpu-stride", type=int, default=0, help="bag stride of the oracle sample (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--num-tables", type=int, default=0, help="reduced case for profiler captures: fewer tables (cfg3/cfg5)")
+    ap.add_argument("--batch", type=int, default=0, help="reduced case for profiler captures: smaller batch")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -258,9 +260,12 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     # every rank draws its own batch from the same recipe (weak scaling); tables/cores are identical
-    wl = workloads.make(cfg_id, mapping=args.mapping)
+    shrink = dict(num_tables=args.num_tables or None, batch=args.batch or None)
+    wl = workloads.make(cfg_id, mapping=args.mapping, **shrink)
+    if shrink["num_tables"] or shrink["batch"]:
+        desc += f" [REDUCED: tables={wl.T}, batch={wl.B}]"
     if rank > 0:
-        other = workloads.make(cfg_id, mapping=args.mapping, seed=workloads.BASE_SEED + 7919 * rank)
+        other = workloads.make(cfg_id, mapping=args.mapping, seed=workloads.BASE_SEED + 7919 * rank, **shrink)
         wl.indices, wl.offsets, wl.grad_out = other.indices, other.offsets, other.grad_out
         del other
     T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
@@ -319,10 +324,8 @@ def main():
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    stage_runs = []
     for _ in range(args.steps):
         step(d_idx, d_off, d_grad)
-        stage_runs.append(None)
     e1.record()
     barrier()
     total_ms = e0.elapsed_time(e1)
@@ -361,7 +364,6 @@ def main():
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4)}
     clocks = sampler.stop()
 
-    counts = emb_counts = None
     emb.forward(d_idx, d_off, B, out=d_out)
     torch.cuda.synchronize()
     counts = emb.grouping_counts()

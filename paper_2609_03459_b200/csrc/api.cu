@@ -139,26 +139,44 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->capU = (cfg->max_unique_rows > 0 && cfg->max_unique_rows < bound) ? cfg->max_unique_rows : bound;
 
     // work units: every table is cut into `units` equal-cost slices, one CTA each
-    int Q = (4 * h->sm_count + T - 1) / T;
-    if (Q < 4) Q = 4;
-    if (Q > 1024) Q = 1024;
+    int Q = (16 * h->sm_count + T - 1) / T;
+    if (Q < 8) Q = 8;
+    if (Q > 2048) Q = 2048;
     int unit_base = 0;
-    const int priv_budget = (227 * 1024 - 1024) / 4 - (max_pl + 2 * max_c + 8 * D);
     int64_t gpart = 0;
     h->max_priv_floats = 0;
     for (int t = 0; t < T; ++t) {
         TableDesc& td = h->tab[t];
         td.units = Q;
+        td.fast = -1;
+        if (K >= 3 && td.d[K - 1] == 4) {
+            // (P_{K-1}, r_{K-1}, P_{K-2}) combinations with a register-tiled variant (see forward.cu)
+            const int PMv = td.P[K - 1], RBv = td.r[K - 1], Mv = td.P[K - 2];
+            if (PMv == 16 && Mv == 4 && RBv == 32) td.fast = 0;
+            else if (PMv == 16 && Mv == 4 && RBv == 16) td.fast = 1;
+            else if (PMv == 16 && Mv == 4 && RBv == 8) td.fast = 2;
+            else if (PMv == 32 && Mv == 4 && RBv == 32) td.fast = 3;
+            else if (PMv == 32 && Mv == 8 && RBv == 64) td.fast = 4;
+        }
         td.unit_base = unit_base;
         unit_base += Q;
-        td.priv_ok = (td.core_floats[K - 1] <= priv_budget) ? 1 : 0;
+        td.priv_ok = 0;
         td.gpart_off = gpart;
-        if (td.priv_ok) {
-            gpart += (int64_t)Q * td.core_floats[K - 1];
-            if (td.core_floats[K - 1] > h->max_priv_floats) h->max_priv_floats = (int)td.core_floats[K - 1];
-        }
+        gpart += (td.core_floats[K - 1] + 3) / 4 * 4;
     }
     h->units_total = unit_base;
+    h->units_per_table = Q;
+    h->vlist_host = (int32_t*)calloc((size_t)T, sizeof(int32_t));
+    if (!h->vlist_host) return fail(TT_EMB_ERR_ARG);
+    {
+        int pos = 0;
+        for (int vi = 0; vi <= TT_NUM_VARIANTS; ++vi) {
+            h->vbase[vi] = pos;
+            for (int t = 0; t < T; ++t)
+                if (h->tab[t].fast == vi - 1) h->vlist_host[pos++] = t;
+            h->vcount[vi] = pos - h->vbase[vi];
+        }
+    }
     h->gpart_floats = gpart;
 
     WsView& v = h->v;
@@ -189,6 +207,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->off_counters = h->off_status + 16 * sizeof(uint32_t);
     h->off_tdesc = take((size_t)T * sizeof(TableDesc));
     h->off_tlstart = take((size_t)(T + 1) * sizeof(int64_t));
+    h->off_vlist = take((size_t)T * sizeof(int32_t));
     h->off_bm = take((size_t)words * sizeof(uint2));
     uint64_t scan_max = words;
     for (int k = 1; k <= K; ++k) if (v.cap[k] > scan_max) scan_max = v.cap[k];
@@ -214,7 +233,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
         }
         h->off_carry = take(((size_t)(h->max_lookups / TT_DE_CHUNK) + 2) * 2 * D * sizeof(float));
-        h->off_gpart = take((size_t)(gpart > 0 ? gpart : 1) * sizeof(float));
+        h->off_gpart = take((size_t)TT_STRIPES * (size_t)(gpart > 0 ? gpart : 4) * sizeof(float));
     }
     h->ws_bytes = off;
     *out_handle = h;
@@ -227,6 +246,7 @@ extern "C" int tt_emb_destroy(tt_emb_t h)
     if (h->ev_created)
         for (int i = 0; i < TT_NUM_STAGES; ++i) { cudaEventDestroy(h->ev[i][0]); cudaEventDestroy(h->ev[i][1]); }
     free(h->tab);
+    free(h->vlist_host);
     delete h;
     return TT_EMB_OK;
 }
@@ -276,6 +296,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     v.counters = (uint32_t*)(base + h->off_counters);
     v.tdesc = (TableDesc*)(base + h->off_tdesc);
     v.tl_start = (int64_t*)(base + h->off_tlstart);
+    v.vlist = (int32_t*)(base + h->off_vlist);
     v.bm = (uint2*)(base + h->off_bm);
     v.scan_tmp = (uint32_t*)(base + h->off_scan);
     for (int k = 1; k <= K; ++k) {
@@ -300,9 +321,11 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
         }
         v.carry = (float*)(base + h->off_carry);
         v.gpart = (float*)(base + h->off_gpart);
+        v.gpart_stride = h->gpart_floats > 0 ? h->gpart_floats : 4;
     }
     // pageable source: the runtime stages it before returning, so h->tab may change afterwards
     TT_CUDA(cudaMemcpyAsync(v.tdesc, h->tab, (size_t)T * sizeof(TableDesc), cudaMemcpyHostToDevice, s));
+    TT_CUDA(cudaMemcpyAsync(v.vlist, h->vlist_host, (size_t)T * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     TT_CUDA(cudaMemsetAsync(v.status, 0, (16 + 64) * sizeof(uint32_t), s));
     h->bound = true;
     h->have_forward = false;

@@ -31,8 +31,8 @@ __global__ void k_zero_u32_dev(uint32_t* p, const uint32_t* count, uint32_t extr
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0u;
 }
 
-// zero the gradients that are not fully written by an owner kernel: core 0 always, last core when the
-// table does not use the private copy
+// zero the gradient that is not fully written by an owner kernel: core 0 (only the slices of present
+// first digits are written later)
 __global__ void k_zero_grads(WsView w)
 {
     const int t = blockIdx.y;
@@ -40,10 +40,7 @@ __global__ void k_zero_grads(WsView w)
     const int K = w.K;
     float* g0 = td.grad[0];
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < td.core_floats[0]; i += (int64_t)gridDim.x * blockDim.x) g0[i] = 0.f;
-    if (!td.priv_ok) {
-        float* gl = td.grad[K - 1];
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < td.core_floats[K - 1]; i += (int64_t)gridDim.x * blockDim.x) gl[i] = 0.f;
-    }
+    (void)K;
 }
 
 // ---------------------------------------------------------------------------------------------- 1. sort by slot
@@ -291,13 +288,10 @@ cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s)
 // ---------------------------------------------------------------------------------------------- 3. last level
 
 // same cost-balanced units as the forward sweep (forward.cu)
-__device__ __forceinline__ void tt_unit_range_b(const WsView& w, int unit, int& t_out, int& q_out, uint32_t& g0, uint32_t& g1)
+__device__ __forceinline__ void tt_unit_range_b(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
 {
-    int t = 0;
-    for (int i = 0; i < w.T; ++i)
-        if (w.tdesc[i].unit_base <= unit) t = i;
     const TableDesc& td = w.tdesc[t];
-    const int q = unit - td.unit_base, Q = td.units;
+    const int Q = td.units;
     const int lvl = w.K - 1;
     const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
     const uint64_t ca = w.cost[a], cb = w.cost[b];
@@ -312,8 +306,6 @@ __device__ __forceinline__ void tt_unit_range_b(const WsView& w, int unit, int& 
     };
     g0 = q == 0 ? a : lower(lo_c);
     g1 = q == Q - 1 ? b : lower(hi_c);
-    t_out = t;
-    q_out = q;
 }
 
 __device__ __forceinline__ void tt_mid_product_b(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
@@ -336,26 +328,14 @@ __device__ __forceinline__ const float* tt_left_operand_b(const WsView& w, const
     return w.pbuf[k - 1] + (size_t)w.parent[k][v] * w.stride[k - 1];
 }
 
-__global__ void __launch_bounds__(256) k_sweep_bwd(WsView w, int pl_floats, int c_floats)
+// generic fallback (any shape): the whole CTA works on one group at a time
+__device__ __forceinline__ void tt_sweep_bwd_generic(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1,
+                                                     float* gk, float* Pl, float* Cs, float* dCs, float* dEs)
 {
-    extern __shared__ float sm[];
-    float* Pl = sm;
-    float* Cs = Pl + pl_floats;
-    float* dCs = Cs + c_floats;
-    float* dEs = dCs + c_floats;          // RB * D
-    float* priv = dEs + RB * w.D;         // n_K * slice_K (when priv_ok)
-    int t, q;
-    uint32_t g0, g1;
-    tt_unit_range_b(w, blockIdx.x, t, q, g0, g1);
-    const TableDesc& td = w.tdesc[t];
     const int K = w.K, kl = K - 1, km = K - 2;
     const int Pm = td.P[K - 1], rb = td.r[K - 1], dK = td.d[kl], D = w.D;
     const int sliceK = td.slice_floats[kl];
     const uint32_t nK = (uint32_t)td.n[kl];
-    const int priv_floats = (int)nK * sliceK;
-    const bool use_priv = td.priv_ok != 0;
-    if (use_priv)
-        for (int i = threadIdx.x; i < priv_floats; i += blockDim.x) priv[i] = 0.f;
     for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) dCs[i] = 0.f;
     __syncthreads();
     for (uint32_t g = g0; g < g1; ++g) {
@@ -385,8 +365,7 @@ __global__ void __launch_bounds__(256) k_sweep_bwd(WsView w, int pl_floats, int 
                 float acc = 0.f;
                 for (int p = 0; p < Pm; ++p) acc = fmaf(Cs[p * rb + bb], de[p * dK], acc);
                 const uint32_t iK = w.val[K][ub + rr] % nK;
-                if (use_priv) priv[iK * sliceK + e] += acc;      // rows of a group select distinct slices
-                else atomicAdd(td.grad[kl] + (size_t)iK * sliceK + e, acc);
+                atomicAdd(gk + (size_t)iK * sliceK + e, acc);
             }
             // dC[p][b] += sum_j dE[p][j] * D[b][j]             ("dC = dE . D^T", summed over the group: Eq. 2)
             for (int it = threadIdx.x; it < Pm * rb; it += blockDim.x) {
@@ -407,46 +386,277 @@ __global__ void __launch_bounds__(256) k_sweep_bwd(WsView w, int pl_floats, int 
         for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) { dst[i] = dCs[i]; dCs[i] = 0.f; }
         __syncthreads();
     }
-    if (use_priv) {
-        float* dst = w.gpart + td.gpart_off + (size_t)q * priv_floats;
-        for (int i = threadIdx.x; i < priv_floats; i += blockDim.x) dst[i] = priv[i];
+}
+
+// ---- register-tiled backward of the last two levels (same shape variants as the forward sweep) ----------------
+//
+// One warp per group.  C is rebuilt in shared memory, then two passes over the group's rows:
+//   pass A  dC[p][b] += sum_j dE_u[p][j] * D_u[b][j]: a lane owns TP rows p for all b (TP*RB accumulators) and
+//           one of 32*TP/PM concurrent rows; D streams as float4 (16 FMAs per load at TP = 4).  The row-slots
+//           are then combined by a reduce-scatter of warp shuffles and each lane writes its share of dC (Eq. 2:
+//           the sum over the rows sharing C is formed before anything moves up a level).
+//   pass B  dG_K[i_K][b][j] += sum_p C[p][b] * dE_u[p][j]: a lane owns RB*TP/PM values of b for all p
+//           (PM*RB*TP/PM registers of C) and streams the float4 rows of dE (8*TP FMAs per load at PM = 16).
+//           The lane's 4*RB*TP/PM results are contiguous in the slice and go out as vector reductions.
+
+__device__ __forceinline__ void tt_red_v4(float* p, float x, float y, float z, float wv)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(wv) : "memory");
+}
+
+template <int M, int CPL>
+__device__ __forceinline__ void tt_warp_mid_b(const float* As, const float* __restrict__ Bsl, float* Cs, int ra, int cols, int lane)
+{
+    const int c4n = cols >> 2;
+    const int LA = (c4n / CPL) < 32 ? (c4n / CPL) : 32;
+    const int NS = 32 / LA;
+    const int s = lane / LA, ll = lane - s * LA;
+    float acc[CPL][M][4];
+#pragma unroll
+    for (int i = 0; i < CPL; ++i)
+#pragma unroll
+        for (int m = 0; m < M; ++m) { acc[i][m][0] = 0.f; acc[i][m][1] = 0.f; acc[i][m][2] = 0.f; acc[i][m][3] = 0.f; }
+    const float4* __restrict__ B4 = reinterpret_cast<const float4*>(Bsl);
+#pragma unroll 8
+    for (int a = s; a < ra; a += NS) {
+        float4 b[CPL];
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) b[i] = __ldg(B4 + (size_t)a * c4n + ll + i * LA);
+        float av[M];
+#pragma unroll
+        for (int m4 = 0; m4 < M / 4; ++m4) {
+            const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
+            av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+        }
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                acc[i][m][0] = fmaf(av[m], b[i].x, acc[i][m][0]);
+                acc[i][m][1] = fmaf(av[m], b[i].y, acc[i][m][1]);
+                acc[i][m][2] = fmaf(av[m], b[i].z, acc[i][m][2]);
+                acc[i][m][3] = fmaf(av[m], b[i].w, acc[i][m][3]);
+            }
+    }
+    for (int o = LA; o < 32; o <<= 1)
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[i][m][x] += __shfl_xor_sync(0xffffffffu, acc[i][m][x], o);
+    if (s == 0) {
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+                *reinterpret_cast<float4*>(Cs + m * cols + 4 * (ll + i * LA)) = make_float4(acc[i][m][0], acc[i][m][1], acc[i][m][2], acc[i][m][3]);
     }
 }
 
-// fixed-order sum of the per-unit copies of the last core's gradient
+template <int PM, int RB_, int TP>
+__device__ __forceinline__ void tt_warp_rows_dC(const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1, uint32_t row_base,
+                                                float* dPdst, int lane)
+{
+    constexpr int LR = PM / TP, RW = 32 / LR, NV = TP * RB_;
+    const int q = lane % LR, slot = lane / LR;
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
+    float dc[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) dc[i] = 0.f;
+    for (uint32_t ub = u0; ub < u1; ub += RW) {
+        const uint32_t u = ub + slot;
+        const bool act = u < u1;
+        const uint32_t iK = act ? rows[u] - row_base : 0u;
+        const float4* __restrict__ D4 = reinterpret_cast<const float4*>(GK + (size_t)iK * (RB_ * 4));
+        float4 e[TP];
+#pragma unroll
+        for (int i = 0; i < TP; ++i) e[i] = act ? __ldg(E4 + (size_t)u * PM + TP * q + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int b = 0; b < RB_; ++b) {
+            const float4 d = __ldg(D4 + b);
+#pragma unroll
+            for (int i = 0; i < TP; ++i) {
+                float a = dc[i * RB_ + b];
+                a = fmaf(e[i].x, d.x, a); a = fmaf(e[i].y, d.y, a); a = fmaf(e[i].z, d.z, a); a = fmaf(e[i].w, d.w, a);
+                dc[i * RB_ + b] = a;
+            }
+        }
+    }
+    // reduce-scatter over the RW row-slots: after the step with lane bit o, a lane keeps the half selected by that bit
+    int base = 0;
+    int n = NV;
+#pragma unroll
+    for (int o = 16; o >= LR; o >>= 1) {
+        n >>= 1;
+        const bool hi = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < NV / 2; ++i) {
+            if (i < n) {
+                const float send = hi ? dc[i] : dc[i + n];
+                const float recv = __shfl_xor_sync(0xffffffffu, send, o);
+                dc[i] = (hi ? dc[i + n] : dc[i]) + recv;
+            }
+        }
+        base += hi ? n : 0;
+    }
+    // the lane now holds dc[0..n) = dC values [base, base+n) of its TP rows (value v <-> row v / RB_, column v % RB_)
+    constexpr int NF = NV / RW;
+    float* dst = dPdst + (TP * q + base / RB_) * RB_ + base % RB_;
+#pragma unroll
+    for (int i = 0; i < NF / 4; ++i)
+        *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(dc[4 * i], dc[4 * i + 1], dc[4 * i + 2], dc[4 * i + 3]);
+}
+
+template <int PM, int RB_, int TP>
+__device__ __forceinline__ void tt_warp_rows_dG(const float* Cs, const WsView& w, uint32_t u0, uint32_t u1, uint32_t row_base,
+                                                float* gk, int lane)
+{
+    constexpr int LR = PM / TP, RW = 32 / LR, BQ = RB_ / LR;
+    const int q = lane % LR, slot = lane / LR;
+    const uint32_t* __restrict__ rows = w.val[w.K];
+    const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
+    float c2[PM][BQ];
+#pragma unroll
+    for (int p = 0; p < PM; ++p)
+#pragma unroll
+        for (int bi = 0; bi < BQ; ++bi) c2[p][bi] = Cs[p * RB_ + BQ * q + bi];
+    for (uint32_t ub = u0; ub < u1; ub += RW) {
+        const uint32_t u = ub + slot;
+        const bool act = u < u1;
+        const uint32_t ur = act ? u : u0;
+        float4 acc[BQ];
+#pragma unroll
+        for (int bi = 0; bi < BQ; ++bi) acc[bi] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int p = 0; p < PM; ++p) {
+            const float4 e = __ldg(E4 + (size_t)ur * PM + p);
+#pragma unroll
+            for (int bi = 0; bi < BQ; ++bi) {
+                acc[bi].x = fmaf(c2[p][bi], e.x, acc[bi].x);
+                acc[bi].y = fmaf(c2[p][bi], e.y, acc[bi].y);
+                acc[bi].z = fmaf(c2[p][bi], e.z, acc[bi].z);
+                acc[bi].w = fmaf(c2[p][bi], e.w, acc[bi].w);
+            }
+        }
+        if (act) {
+            const uint32_t iK = rows[u] - row_base;
+            float* dst = gk + (size_t)iK * (RB_ * 4) + (BQ * q) * 4;
+#pragma unroll
+            for (int bi = 0; bi < BQ; ++bi) tt_red_v4(dst + 4 * bi, acc[bi].x, acc[bi].y, acc[bi].z, acc[bi].w);
+        }
+    }
+}
+
+template <int PM, int RB_, int TP, int M, int CPL>
+__device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* gk,
+                                                  float* As, float* Cs, int lane, int wid, int nw)
+{
+    const int K = w.K, km = K - 2;
+    const int ra = td.r[km], cols = td.d[km] * RB_;
+    const uint32_t nK = (uint32_t)td.n[K - 1];
+    for (uint32_t g = g0 + wid; g < g1; g += nw) {
+        const uint32_t val = w.val[K - 1][g];
+        const float* src = tt_left_operand_b(w, td, K - 1, g);
+        for (int i = lane; i < M * ra; i += 32) {
+            const int m = i / ra, a = i - m * ra;
+            As[a * M + m] = __ldg(src + i);
+        }
+        __syncwarp();
+        const uint32_t im = val % (uint32_t)td.n[km];
+        tt_warp_mid_b<M, CPL>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
+        __syncwarp();
+        const uint32_t u0 = w.cstart[K - 1][g], u1 = w.cstart[K - 1][g + 1];
+        tt_warp_rows_dC<PM, RB_, TP>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
+        tt_warp_rows_dG<PM, RB_, TP>(Cs, w, u0, u1, val * nK, gk, lane);
+        __syncwarp();
+    }
+}
+
+// One CTA (4 warps) per work unit (table, q); last-core gradients go to one of TT_STRIPES L2-resident partial
+// copies with vector reductions, added up in fixed stripe order by k_reduce_gpart.
+template <int V>
+__global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int c_floats, int vbase)
+{
+    extern __shared__ __align__(16) float sm[];
+    const int t = w.vlist[vbase + blockIdx.y], q = blockIdx.x;
+    uint32_t g0, g1;
+    tt_unit_range_b(w, t, q, g0, g1);
+    const TableDesc& td = w.tdesc[t];
+    const int stripe = (blockIdx.x + blockIdx.y) % TT_STRIPES;
+    float* gk = w.gpart + (size_t)stripe * w.gpart_stride + td.gpart_off;
+    if (V < 0) {
+        float* Pl = sm;
+        float* Cs = Pl + pl_floats;
+        float* dCs = Cs + c_floats;
+        float* dEs = dCs + c_floats;
+        tt_sweep_bwd_generic(w, td, g0, g1, gk, Pl, Cs, dCs, dEs);
+        return;
+    }
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    float* As = sm + (size_t)wid * (pl_floats + c_floats);
+    float* Cs = As + pl_floats;
+    if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+}
+
+// fixed-order sum of the partial copies of the last core's gradient
 __global__ void __launch_bounds__(256) k_reduce_gpart(WsView w)
 {
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
-    if (!td.priv_ok) return;
     const int kl = w.K - 1;
     const int64_t n = td.core_floats[kl];
     const float* src = w.gpart + td.gpart_off;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         float s = 0.f;
-        for (int q = 0; q < td.units; ++q) s += src[(size_t)q * n + i];
+#pragma unroll
+        for (int q = 0; q < TT_STRIPES; ++q) s += src[(size_t)q * w.gpart_stride + i];
         td.grad[kl][i] = s;
     }
+}
+
+template <int V>
+static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream_t s)
+{
+    const int n = h->vcount[V + 1];
+    if (n == 0) return cudaSuccess;
+    const size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
+                              : (size_t)4 * (max_pl + max_c) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_sweep_bwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    return cudaGetLastError();
 }
 
 cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
-    int max_pl = 1, max_c = 1;
+    int max_pl = 4, max_c = 4;
     for (int t = 0; t < h->T; ++t) {
         const TableDesc& td = h->tab[t];
         for (int k = 1; k < h->K; ++k) {
-            int f = td.P[k] * td.r[k];
+            int f = (td.P[k] * td.r[k] + 3) / 4 * 4;
             if (k <= h->K - 2 && f > max_pl) max_pl = f;
             if (k == h->K - 1 && f > max_c) max_c = f;
         }
     }
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(w.gpart, 0, (size_t)TT_STRIPES * w.gpart_stride * sizeof(float), s)) != cudaSuccess) return e;
     k_zero_grads<<<dim3(64, h->T), 256, 0, s>>>(w);
     // P_k of the levels below K-1 are still in pbuf from the forward (K = 4 only)
-    const size_t smem = (size_t)(max_pl + 2 * max_c + RB * h->D + h->max_priv_floats) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k_sweep_bwd<<<h->units_total, 256, smem, s>>>(w, max_pl, max_c);
+    if ((e = launch_sweep_bwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<0>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<2>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<3>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<4>(h, max_pl, max_c, s)) != cudaSuccess) return e;
     k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
     return cudaGetLastError();
 }

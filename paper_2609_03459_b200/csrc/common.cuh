@@ -12,6 +12,8 @@
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
 #define TT_DE_CHUNK 256                                  // sorted lookups per warp in the dE segment reduction
 #define TT_NUM_STAGES 9
+#define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
+#define TT_NUM_VARIANTS 5                                // register-tiled shape variants (forward.cu)
 
 // Per-table descriptor, resident in the workspace.  k below is 0-based (core k+1 of the paper).
 struct TableDesc {
@@ -29,11 +31,11 @@ struct TableDesc {
     uint32_t tword_base[TT_MAXK];       // same for the digit-major ("transposed") node bitmaps, levels 2..K-1
     uint32_t tnum_words[TT_MAXK];
     uint32_t prefix_space[TT_MAXK + 1]; // n_1 * .. * n_k (number of possible length-k prefixes), k = 1..K-1
-    int64_t gpart_off;                  // float offset of this table's last-core gradient partials
+    int64_t gpart_off;                  // float offset of this table's last core inside one stripe
     int32_t units;                      // work units (CTAs) this table is cut into
     int32_t unit_base;                  // first global unit id
     int32_t priv_ok;                    // last-core gradient of this table fits the shared-memory private copy
-    int32_t pad;
+    int32_t fast;                       // register-tiled kernel variant for this table's shapes, -1 = generic path
 };
 
 // Device-side view of the workspace handed to kernels by value.
@@ -48,6 +50,7 @@ struct WsView {
     int32_t* status;
     uint32_t* counters;                 // [k] = number of level-k nodes (k = 1..K); [8+k] transposed counts
     TableDesc* tdesc;
+    int32_t* vlist;                     // table ids grouped by kernel variant (generic first)
     int64_t* tl_start;                  // [T+1] first lookup of each table
     uint2* bm;                          // {32 presence bits, number of set bits before this word (global)}
     uint32_t* scan_tmp;
@@ -65,7 +68,8 @@ struct WsView {
     uint2* upairs;                      // [L] (slot, bag) in lookup order, written by the pooling kernel (null: forward only)
     float* dP[TT_MAXK + 1];             // dP_k per level-k node, 2 <= k <= K-1
     float* carry;                       // [chunks][2][D]
-    float* gpart;                       // last-core gradient partials
+    float* gpart;                       // [TT_STRIPES][gpart_stride] partial copies of all tables' last-core gradients
+    int64_t gpart_stride;               // floats per stripe
     uint2* tbm[TT_MAXK + 1];            // digit-major node bitmaps, levels 2..K-1
     uint32_t* tnode[TT_MAXK + 1];       // nodes of level k ordered by (table, i_k, parent prefix)
     const int64_t* indices;
@@ -80,6 +84,11 @@ struct tt_emb {
     int enable_backward;
     int sm_count;
     int units_total;
+    int units_per_table;
+    int vcount[TT_NUM_VARIANTS + 1];   // tables per variant, index 0 = generic (-1)
+    int vbase[TT_NUM_VARIANTS + 1];    // first entry of each variant in vlist
+    int32_t* vlist_host;
+    size_t off_vlist;
     int cost_shift;       // cost unit of the schedule = 2^cost_shift FMAs
     TableDesc* tab;       // host copy [T]
     size_t ws_bytes;

@@ -46,13 +46,10 @@ cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s)
 }
 
 // group range [g0, g1) of work unit `unit` (global id) -- equal-cost slice of its table
-__device__ __forceinline__ void tt_unit_range(const WsView& w, int unit, int& t_out, uint32_t& g0, uint32_t& g1)
+__device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
 {
-    int t = 0;
-    for (int i = 0; i < w.T; ++i)
-        if (w.tdesc[i].unit_base <= unit) t = i;
     const TableDesc& td = w.tdesc[t];
-    const int q = unit - td.unit_base, Q = td.units;
+    const int Q = td.units;
     const int lvl = w.K - 1;
     const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
     const uint64_t ca = w.cost[a], cb = w.cost[b];
@@ -68,7 +65,6 @@ __device__ __forceinline__ void tt_unit_range(const WsView& w, int unit, int& t_
     };
     g0 = q == 0 ? a : lower(lo_c);
     g1 = q == Q - 1 ? b : lower(hi_c);
-    t_out = t;
 }
 
 // ---------------------------------------------------------------------------------------------- products
@@ -126,16 +122,146 @@ __global__ void __launch_bounds__(128) k_mid_level(WsView w, int k)
     }
 }
 
-// fused levels K-1 and K: C in shared memory, rows to w.E
-__global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats)
+// ---- register-tiled warp-level products (fast path) ---------------------------------------------------------
+//
+// One warp owns one group at a time.  FP32 FMA throughput is only reachable when every float that enters
+// a lane's registers feeds >= 4 FMAs (the shared-memory / L1 path delivers 32 floats per clock per SM, the
+// FMA pipes retire 128 lane-FMAs per clock), so:
+//   * mid product  C = Pl . B : a lane owns 4 (or 8) consecutive columns of B for all M rows of Pl; B streams
+//     through once as float4, Pl comes as float4 broadcasts from shared memory.
+//   * last product E = C . D  : a lane keeps TP rows of C (TP x RB floats) in registers for the whole group
+//     and streams the float4 rows of each child's D slice: 4*TP FMAs per loaded float4; PM/TP lanes cover a
+//     row, so a warp produces 32*TP/PM rows at a time and each lane stores 4*TP consecutive floats of E.
+
+// Cs[m*cols + c] = sum_a Pl[m][a] * Bsl[a*cols + c];  As holds Pl transposed: As[a*M + m].
+// cols/4 must be a power of two and cols <= 128*CPL.
+template <int M, int CPL>
+__device__ __forceinline__ void tt_warp_mid(const float* As, const float* __restrict__ Bsl, float* Cs, int ra, int cols, int lane)
 {
-    extern __shared__ float sm[];
-    float* Pl = sm;
-    float* Cs = sm + pl_floats;
-    int t;
-    uint32_t g0, g1;
-    tt_unit_range(w, blockIdx.x, t, g0, g1);
-    const TableDesc& td = w.tdesc[t];
+    const int c4n = cols >> 2;
+    const int LA = (c4n / CPL) < 32 ? (c4n / CPL) : 32;  // lanes that cover one row of B
+    const int NS = 32 / LA;                              // the a-range is split over NS lane groups
+    const int s = lane / LA, ll = lane - s * LA;
+    float acc[CPL][M][4];
+#pragma unroll
+    for (int i = 0; i < CPL; ++i)
+#pragma unroll
+        for (int m = 0; m < M; ++m) { acc[i][m][0] = 0.f; acc[i][m][1] = 0.f; acc[i][m][2] = 0.f; acc[i][m][3] = 0.f; }
+    const float4* __restrict__ B4 = reinterpret_cast<const float4*>(Bsl);
+#pragma unroll 4
+    for (int a = s; a < ra; a += NS) {
+        float4 b[CPL];
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) b[i] = __ldg(B4 + (size_t)a * c4n + ll + i * LA);
+        float av[M];
+#pragma unroll
+        for (int m4 = 0; m4 < M / 4; ++m4) {
+            const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
+            av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+        }
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                acc[i][m][0] = fmaf(av[m], b[i].x, acc[i][m][0]);
+                acc[i][m][1] = fmaf(av[m], b[i].y, acc[i][m][1]);
+                acc[i][m][2] = fmaf(av[m], b[i].z, acc[i][m][2]);
+                acc[i][m][3] = fmaf(av[m], b[i].w, acc[i][m][3]);
+            }
+    }
+    for (int o = LA; o < 32; o <<= 1)
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[i][m][x] += __shfl_xor_sync(0xffffffffu, acc[i][m][x], o);
+    if (s == 0) {
+#pragma unroll
+        for (int i = 0; i < CPL; ++i)
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+                *reinterpret_cast<float4*>(Cs + m * cols + 4 * (ll + i * LA)) = make_float4(acc[i][m][0], acc[i][m][1], acc[i][m][2], acc[i][m][3]);
+    }
+}
+
+// E rows u0..u1 of the group whose C (PM x RB, row-major) is in Cs.  d_K = 4.
+template <int PM, int RB, int TP>
+__device__ __forceinline__ void tt_warp_rows(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
+                                             uint32_t row_base, int lane)
+{
+    constexpr int LR = PM / TP;   // lanes per row
+    constexpr int RW = 32 / LR;   // rows per batch
+    const int q = lane % LR, slot = lane / LR;
+    float c[TP][RB];
+#pragma unroll
+    for (int i = 0; i < TP; ++i)
+#pragma unroll
+        for (int b4 = 0; b4 < RB / 4; ++b4) {
+            const float4 t = *reinterpret_cast<const float4*>(Cs + (TP * q + i) * RB + 4 * b4);
+            c[i][4 * b4] = t.x; c[i][4 * b4 + 1] = t.y; c[i][4 * b4 + 2] = t.z; c[i][4 * b4 + 3] = t.w;
+        }
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    for (uint32_t ub = u0; ub < u1; ub += RW) {
+        const uint32_t u = ub + slot;
+        const bool act = u < u1;
+        const uint32_t iK = act ? rows[u] - row_base : 0u;
+        const float4* __restrict__ D4 = reinterpret_cast<const float4*>(GK + (size_t)iK * (RB * 4));
+        float acc[TP][4];
+#pragma unroll
+        for (int i = 0; i < TP; ++i) { acc[i][0] = 0.f; acc[i][1] = 0.f; acc[i][2] = 0.f; acc[i][3] = 0.f; }
+#pragma unroll
+        for (int b = 0; b < RB; ++b) {
+            const float4 d = __ldg(D4 + b);
+#pragma unroll
+            for (int i = 0; i < TP; ++i) {
+                acc[i][0] = fmaf(c[i][b], d.x, acc[i][0]);
+                acc[i][1] = fmaf(c[i][b], d.y, acc[i][1]);
+                acc[i][2] = fmaf(c[i][b], d.z, acc[i][2]);
+                acc[i][3] = fmaf(c[i][b], d.w, acc[i][3]);
+            }
+        }
+        if (act) {
+            float4* e = reinterpret_cast<float4*>(w.E + (size_t)u * (PM * 4) + TP * q * 4);
+#pragma unroll
+            for (int i = 0; i < TP; ++i) e[i] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        }
+    }
+}
+
+// one warp: groups fetched dynamically from the CTA's range through a shared counter
+template <int PM, int RB, int TP, int M, int CPL>
+__device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& td, uint32_t g1, float* As, float* Cs,
+                                              uint32_t* next, int lane)
+{
+    const int K = w.K, km = K - 2;
+    const int ra = td.r[km], cols = td.d[km] * RB;
+    const uint32_t nK = (uint32_t)td.n[K - 1];
+    for (;;) {
+        uint32_t g = 0;
+        if (lane == 0) g = atomicAdd(next, 1u);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        if (g >= g1) break;
+        const uint32_t val = w.val[K - 1][g];
+        const float* src = tt_left_operand(w, td, K - 1, g);
+        for (int i = lane; i < M * ra; i += 32) {
+            const int m = i / ra, a = i - m * ra;
+            As[a * M + m] = __ldg(src + i);
+        }
+        __syncwarp();
+        const uint32_t im = val % (uint32_t)td.n[km];
+        tt_warp_mid<M, CPL>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
+        __syncwarp();
+        tt_warp_rows<PM, RB, TP>(Cs, w, td, w.cstart[K - 1][g], w.cstart[K - 1][g + 1], val * nK, lane);
+        __syncwarp();
+    }
+}
+
+// generic fallback: the whole CTA works on one group at a time (any shape)
+__device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* Pl, float* Cs)
+{
     const int K = w.K, kl = K - 1, km = K - 2;
     const int Pm = td.P[K - 1], rb = td.r[K - 1], dK = td.d[kl], D = w.D;
     const uint32_t nK = (uint32_t)td.n[kl];
@@ -170,14 +296,54 @@ __global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats)
     }
 }
 
+// fused levels K-1 and K: C stays on chip, rows go to w.E.  One CTA (4 warps) per work unit (table, q);
+// one instantiation per shape variant V so that each gets its own register budget.  blockIdx.y walks the
+// tables of variant V (w.vlist), blockIdx.x the table's equal-cost slices.
+template <int V>
+__global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
+{
+    extern __shared__ __align__(16) float sm[];
+    __shared__ uint32_t next;
+    const int t = w.vlist[vbase + blockIdx.y];
+    uint32_t g0, g1;
+    tt_unit_range(w, t, blockIdx.x, g0, g1);
+    const TableDesc& td = w.tdesc[t];
+    if (V < 0) {
+        tt_sweep_generic(w, td, g0, g1, sm, sm + pl_floats);
+        return;
+    }
+    if (threadIdx.x == 0) next = g0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    float* As = sm + (size_t)wid * (pl_floats + c_floats);
+    float* Cs = As + pl_floats;
+    if (V == 0) tt_sweep_fast<16, 32, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
+    if (V == 1) tt_sweep_fast<16, 16, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
+    if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
+    if (V == 3) tt_sweep_fast<32, 32, 4, 4, 2>(w, td, g1, As, Cs, &next, lane);
+    if (V == 4) tt_sweep_fast<32, 64, 2, 8, 2>(w, td, g1, As, Cs, &next, lane);
+}
+
+template <int V>
+static cudaError_t launch_sweep_fwd(tt_emb* h, int max_pl, int max_c, cudaStream_t s)
+{
+    const int n = h->vcount[V + 1];
+    if (n == 0) return cudaSuccess;
+    const size_t smem = (size_t)4 * (max_pl + max_c) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(k_sweep_fwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_sweep_fwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    return cudaGetLastError();
+}
+
 cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
-    int max_pl = 1, max_c = 1;
+    int max_pl = 4, max_c = 4;
     for (int t = 0; t < h->T; ++t) {
         const TableDesc& td = h->tab[t];
         for (int k = 1; k < h->K; ++k) {
-            int f = td.P[k] * td.r[k];
+            int f = (td.P[k] * td.r[k] + 3) / 4 * 4;
             if (k <= h->K - 2 && f > max_pl) max_pl = f;
             if (k == h->K - 1 && f > max_c) max_c = f;
         }
@@ -186,8 +352,13 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
         int grid = h->sm_count * 16;
         k_mid_level<<<grid, 128, (size_t)max_pl * sizeof(float), s>>>(w, k);
     }
-    const size_t smem = (size_t)(max_pl + max_c) * sizeof(float);
-    k_sweep_fwd<<<h->units_total, 128, smem, s>>>(w, max_pl);
+    cudaError_t e;
+    if ((e = launch_sweep_fwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<0>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<2>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<3>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<4>(h, max_pl, max_c, s)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
