@@ -158,6 +158,14 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (PMv == 32 && Mv == 4 && RBv == 32) td.fast = 3;
             else if (PMv == 32 && Mv == 8 && RBv == 64) td.fast = 4;
         }
+        for (int k = 0; k < TT_MAXK; ++k) td.midfast[k] = -1;
+        for (int k = 2; k <= K - 1; ++k) {
+            const int Mv = td.P[k - 1], rav = td.r[k - 1], colsv = td.d[k - 1] * td.r[k];
+            if (Mv == 4 && rav == 32 && colsv == 128) td.midfast[k] = 0;
+            else if (Mv == 4 && rav == 16 && colsv == 128) td.midfast[k] = 1;
+            else if (Mv == 4 && rav == 32 && colsv == 64) td.midfast[k] = 2;
+            else if (Mv == 4 && rav == 16 && colsv == 64) td.midfast[k] = 3;
+        }
         td.unit_base = unit_base;
         unit_base += Q;
         td.priv_ok = 0;
@@ -229,6 +237,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         h->off_pairs = take((size_t)2 * (size_t)(h->max_lookups + 1) * sizeof(uint2));
         for (int k = 2; k <= K - 1; ++k) {
             h->off_dP[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
+            h->off_Y[k] = take((size_t)v.cap[k] * stride[k - 1] * sizeof(float));
             h->off_tbm[k] = take((size_t)twords[k] * sizeof(uint2));
             h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
         }
@@ -316,6 +325,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
         v.upairs = v.pairs + (h->max_lookups + 1);
         for (int k = 2; k <= K - 1; ++k) {
             v.dP[k] = (float*)(base + h->off_dP[k]);
+            v.Y[k] = (float*)(base + h->off_Y[k]);
             v.tbm[k] = (uint2*)(base + h->off_tbm[k]);
             v.tnode[k] = (uint32_t*)(base + h->off_tnode[k]);
         }

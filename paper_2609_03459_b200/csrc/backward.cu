@@ -716,6 +716,7 @@ __global__ void __launch_bounds__(256) k_mid_down(WsView w, int k)
     for (uint32_t pn = blockIdx.x; pn < count; pn += gridDim.x) {
         const int t = tt_find_table(w.tb[k - 1], w.T, pn);
         const TableDesc& td = w.tdesc[t];
+        if (td.midfast[k] >= 0) continue;  // handled by k_mid_fused + k_mid_sum
         const int kc = k - 1;
         const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
         const int ld = cols + 1;
@@ -768,7 +769,7 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
     const int kc = k - 1;
-    if ((int)blockIdx.x >= td.n[kc]) return;
+    if ((int)blockIdx.x >= td.n[kc] || td.midfast[k] >= 0) return;
     const uint32_t ik = blockIdx.x;
     const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
     const int nout = ra * cols;
@@ -808,12 +809,144 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
     }
 }
 
+// ---- register-tiled middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ------
+//
+// One CTA of 128 threads per (table, slice i_k).  The slice G_k[i_k] (RA x COLS) never changes inside the CTA,
+// so each thread keeps its APT x 4 tile of it in registers.  The nodes with digit i_k arrive in ascending parent
+// order from the digit-major list; per node the CTA stages dP_k (4 x COLS) and the parent's P_{k-1} (4 x RA)
+// in shared memory (double-buffered, one barrier per node) and every thread does, for its tile,
+//     dG_k[a][c] += sum_m P_{k-1}[m][a] * dP_k[m][c]               (accumulated in registers over all nodes)
+//     Y[m][a]     = sum_c dP_k[m][c] * G_k[a][c]                    (partial over its 4 columns)
+// The Y partials are combined over the TC lanes that share an a-range by a reduce-scatter of warp shuffles and
+// written once per node; k_mid_sum then adds the Y rows of each parent's (contiguous) children.
+template <int NVAL, int W>
+__device__ __forceinline__ int tt_reduce_scatter(float (&v)[NVAL], int lane)
+{
+    int idx = 0;
+    int n = NVAL;
+#pragma unroll
+    for (int o = W / 2; o >= 1; o >>= 1) {
+        if (n > 1) {
+            n >>= 1;
+            const bool hi = (lane & o) != 0;
+#pragma unroll
+            for (int i = 0; i < NVAL / 2; ++i) {
+                if (i < n) {
+                    const float send = hi ? v[i] : v[i + n];
+                    const float recv = __shfl_xor_sync(0xffffffffu, send, o);
+                    v[i] = (hi ? v[i + n] : v[i]) + recv;
+                }
+            }
+            idx += hi ? n : 0;
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+        }
+    }
+    return idx;
+}
+
+template <int RA, int COLS>
+__global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
+{
+    constexpr int M = 4, TC = COLS / 4, AG = 128 / TC, APT = RA / AG, NVAL = M * APT;
+    constexpr int REP = TC / NVAL > 0 ? TC / NVAL : 1;  // lanes that end up with the same reduced value
+    __shared__ __align__(16) float sA[2][M * RA];
+    __shared__ __align__(16) float sD[2][M * COLS];
+    const int t = blockIdx.y;
+    const TableDesc& td = w.tdesc[t];
+    const int kc = k - 1;
+    if (td.midfast[k] != variant || (int)blockIdx.x >= td.n[kc]) return;
+    const uint32_t ik = blockIdx.x;
+    const int tid = threadIdx.x, cl = tid % TC, ag = tid / TC, a0 = ag * APT;
+    const float* __restrict__ Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
+    float4 breg[APT], acc[APT];
+#pragma unroll
+    for (int i = 0; i < APT; ++i) {
+        breg[i] = __ldg(reinterpret_cast<const float4*>(Bsl + (size_t)(a0 + i) * COLS) + cl);
+        acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const uint32_t space = td.prefix_space[k - 1];
+    const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
+    const int strideY = w.stride[k - 1];
+    float4 rd = make_float4(0.f, 0.f, 0.f, 0.f), rav = rd;
+    uint32_t vnext = 0;
+    auto fetch = [&](uint32_t jn) {
+        vnext = w.tnode[k][jn];
+        if (tid < M * COLS / 4) rd = __ldg(reinterpret_cast<const float4*>(w.dP[k] + (size_t)vnext * w.stride[k]) + tid);
+        if (tid < M * RA / 4) rav = __ldg(reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, vnext)) + tid);
+    };
+    auto stage = [&](int buf) {
+        if (tid < M * COLS / 4) reinterpret_cast<float4*>(sD[buf])[tid] = rd;
+        if (tid < M * RA / 4) reinterpret_cast<float4*>(sA[buf])[tid] = rav;
+    };
+    uint32_t vcur = 0;
+    if (j0 < j1) { fetch(j0); stage(0); vcur = vnext; }
+    __syncthreads();
+    for (uint32_t jn = j0; jn < j1; ++jn) {
+        const int cur = (int)((jn - j0) & 1u);
+        const bool more = jn + 1 < j1;
+        if (more) fetch(jn + 1);
+        float y[NVAL];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float4 d = reinterpret_cast<const float4*>(sD[cur])[m * TC + cl];
+#pragma unroll
+            for (int i = 0; i < APT; ++i) {
+                const float av = sA[cur][m * RA + a0 + i];
+                acc[i].x = fmaf(av, d.x, acc[i].x); acc[i].y = fmaf(av, d.y, acc[i].y);
+                acc[i].z = fmaf(av, d.z, acc[i].z); acc[i].w = fmaf(av, d.w, acc[i].w);
+                float yy = d.x * breg[i].x;
+                yy = fmaf(d.y, breg[i].y, yy); yy = fmaf(d.z, breg[i].z, yy); yy = fmaf(d.w, breg[i].w, yy);
+                y[m * APT + i] = yy;
+            }
+        }
+        const int idx = tt_reduce_scatter<NVAL, TC>(y, cl);
+        if ((cl % REP) == 0) {
+            const int m = idx / APT, i = idx - m * APT;
+            w.Y[k][(size_t)vcur * strideY + m * RA + a0 + i] = y[0];
+        }
+        if (more) stage(cur ^ 1);
+        vcur = vnext;
+        __syncthreads();
+    }
+    float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
+#pragma unroll
+    for (int i = 0; i < APT; ++i) reinterpret_cast<float4*>(dst + (size_t)(a0 + i) * COLS)[cl] = acc[i];
+}
+
+// dP_{k-1}[parent] (k = 2: the first core's gradient slice) = sum of the Y rows of the parent's children,
+// which are contiguous in sorted order; one warp per parent
+__global__ void __launch_bounds__(256) k_mid_sum(WsView w, int k)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t count = w.counters[CTR_LEVEL0 + k - 1];
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int strideY = w.stride[k - 1];
+    for (uint32_t pn = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; pn < count; pn += nwarps) {
+        const int t = tt_find_table(w.tb[k - 1], w.T, pn);
+        const TableDesc& td = w.tdesc[t];
+        if (td.midfast[k] < 0) continue;
+        const int nout4 = td.P[k - 1] * td.r[k - 1] / 4;
+        const uint32_t c0 = w.cstart[k - 1][pn], c1 = w.cstart[k - 1][pn + 1];
+        float* dst = k == 2 ? td.grad[0] + (size_t)w.val[1][pn] * td.slice_floats[0] : w.dP[k - 1] + (size_t)pn * w.stride[k - 1];
+        for (int f = lane; f < nout4; f += 32) {
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t v = c0; v < c1; ++v) {
+                const float4 x = __ldg(reinterpret_cast<const float4*>(w.Y[k] + (size_t)v * strideY) + f);
+                s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
+            }
+            reinterpret_cast<float4*>(dst)[f] = s;
+        }
+    }
+}
+
 cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
     cudaError_t e;
     for (int k = h->K - 1; k >= 2; --k) {
         int max_n = 1, max_down = 1, max_slice = 1;
+        bool any_generic = false, any_fast[4] = {false, false, false, false};
         for (int t = 0; t < h->T; ++t) {
             const TableDesc& td = h->tab[t];
             const int kc = k - 1;
@@ -821,6 +954,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
             if (td.n[kc] > max_n) max_n = td.n[kc];
             if (ra * (cols + 1) + M * cols > max_down) max_down = ra * (cols + 1) + M * cols;
             if (M * ra + M * cols > max_slice) max_slice = M * ra + M * cols;
+            if (td.midfast[k] < 0) any_generic = true; else any_fast[td.midfast[k]] = true;
         }
         if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
         const int g = h->sm_count * 8;
@@ -828,10 +962,18 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         TPopScan tp{w, k};
         if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
         k_tfill<<<g, 256, 0, s>>>(w, k);
-        if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
-        k_mid_slice<<<dim3(max_n, h->T), 256, (size_t)max_slice * sizeof(float), s>>>(w, k);
-        if ((e = cudaFuncSetAttribute(k_mid_down, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_down * sizeof(float)))) != cudaSuccess) return e;
-        k_mid_down<<<h->sm_count * 8, 256, (size_t)max_down * sizeof(float), s>>>(w, k);
+        const dim3 sg(max_n, h->T);
+        if (any_fast[0]) k_mid_fused<32, 128><<<sg, 128, 0, s>>>(w, k, 0);
+        if (any_fast[1]) k_mid_fused<16, 128><<<sg, 128, 0, s>>>(w, k, 1);
+        if (any_fast[2]) k_mid_fused<32, 64><<<sg, 128, 0, s>>>(w, k, 2);
+        if (any_fast[3]) k_mid_fused<16, 64><<<sg, 128, 0, s>>>(w, k, 3);
+        if (any_fast[0] || any_fast[1] || any_fast[2] || any_fast[3]) k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k);
+        if (any_generic) {
+            if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
+            k_mid_slice<<<sg, 256, (size_t)max_slice * sizeof(float), s>>>(w, k);
+            if ((e = cudaFuncSetAttribute(k_mid_down, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_down * sizeof(float)))) != cudaSuccess) return e;
+            k_mid_down<<<h->sm_count * 8, 256, (size_t)max_down * sizeof(float), s>>>(w, k);
+        }
     }
     return cudaGetLastError();
 }

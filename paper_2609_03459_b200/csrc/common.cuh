@@ -36,6 +36,7 @@ struct TableDesc {
     int32_t unit_base;                  // first global unit id
     int32_t priv_ok;                    // last-core gradient of this table fits the shared-memory private copy
     int32_t fast;                       // register-tiled kernel variant for this table's shapes, -1 = generic path
+    int32_t midfast[TT_MAXK];           // same for the middle-core backward of level k (index k), -1 = generic
 };
 
 // Device-side view of the workspace handed to kernels by value.
@@ -67,6 +68,7 @@ struct WsView {
     uint2* pairs;                       // [L] (slot, bag) sorted by slot
     uint2* upairs;                      // [L] (slot, bag) in lookup order, written by the pooling kernel (null: forward only)
     float* dP[TT_MAXK + 1];             // dP_k per level-k node, 2 <= k <= K-1
+    float* Y[TT_MAXK + 1];              // per level-k node: its contribution to dP_{k-1} of its parent
     float* carry;                       // [chunks][2][D]
     float* gpart;                       // [TT_STRIPES][gpart_stride] partial copies of all tables' last-core gradients
     int64_t gpart_stride;               // floats per stripe
@@ -95,6 +97,7 @@ struct tt_emb {
     size_t off_status, off_counters, off_tdesc, off_tlstart, off_bm, off_scan, off_cost, off_E;
     size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
+    size_t off_Y[TT_MAXK + 1];
     size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart;
     size_t scan_tmp_elems;
     int64_t gpart_floats;

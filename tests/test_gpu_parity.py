@@ -111,6 +111,15 @@ MEDIUM = [
     ("k3-mixed", [TableSpec(200_003, (59, 59, 59), (4, 4, 4), (1, 16, 32, 1), 1.05, "normal", 0.05),
                   TableSpec(1_500, (12, 12, 12), (4, 4, 4), (1, 32, 16, 1), 0.9, "normal", 0.05),
                   TableSpec(150_000, (54, 54, 54), (4, 4, 4), (1, 7, 5, 1), 1.2, "normal", 0.05)], 300, (0, 40)),
+    # every register-tiled shape variant: (r1, r2) in {16,32}^2 and rank 8 with d = 4x4x4, the d = 4x8x4 rank-32
+    # shape, and the 4-core rank-64 shape
+    ("tiled-r16-r32", [TableSpec(30_000, (32, 32, 32), (4, 4, 4), (1, 32, 32, 1), 1.1, "normal", 0.05),
+                       TableSpec(20_000, (28, 28, 28), (4, 4, 4), (1, 16, 16, 1), 0.9, "normal", 0.05),
+                       TableSpec(25_000, (30, 30, 30), (4, 4, 4), (1, 16, 32, 1), 1.0, "normal", 0.05),
+                       TableSpec(12_000, (23, 23, 23), (4, 4, 4), (1, 32, 16, 1), 1.2, "normal", 0.05),
+                       TableSpec(8_000, (20, 20, 20), (4, 4, 4), (1, 8, 8, 1), 1.05, "uniform", 0.1)], 150, (0, 30)),
+    ("tiled-d484", [TableSpec(10_000, (20, 25, 20), (4, 8, 4), (1, 32, 32, 1), 1.1, "normal", 0.05)], 100, 20),
+    ("tiled-k4-r64", [TableSpec(20_736, (12, 12, 12, 12), (2, 4, 4, 4), (1, 64, 64, 64, 1), 1.2, "normal", 0.02)], 120, 8),
     ("k2", [TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 1.0, "uniform", 0.1)], 257, (1, 9)),
     ("k4", [TableSpec(40_000, (15, 14, 14, 14), (2, 4, 4, 4), (1, 6, 9, 5, 1), 1.1, "normal", 0.05)], 200, 8),
     ("odd-D", [TableSpec(30_000, (32, 32, 32), (3, 3, 5), (1, 4, 6, 1), 1.0, "normal", 0.1)], 123, (0, 12)),
