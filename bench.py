@@ -261,13 +261,12 @@ def main():
 
     # every rank draws its own batch from the same recipe (weak scaling); tables/cores are identical
     shrink = dict(num_tables=args.num_tables or None, batch=args.batch or None)
-    wl = workloads.make(cfg_id, mapping=args.mapping, **shrink)
+    wl = workloads.make(cfg_id, mapping=args.mapping, **shrink) if rank == 0 else None
     if shrink["num_tables"] or shrink["batch"]:
-        desc += f" [REDUCED: tables={wl.T}, batch={wl.B}]"
+        desc += f" [REDUCED: tables={shrink['num_tables'] or 'all'}, batch={shrink['batch'] or 'full'}]"
+    from paper_2609_03459_b200 import dist as ttd
     if rank > 0:
-        other = workloads.make(cfg_id, mapping=args.mapping, seed=workloads.BASE_SEED + 7919 * rank, **shrink)
-        wl.indices, wl.offsets, wl.grad_out = other.indices, other.offsets, other.grad_out
-        del other
+        wl = workloads.make(cfg_id, mapping=args.mapping, batch_seed=ttd.rank_seed(workloads.BASE_SEED, rank), **shrink)
     T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
 
     emb = binding.from_workload(wl, enable_backward=train, device=device)
@@ -283,8 +282,7 @@ def main():
         emb.forward(idx, off, B, out=d_out)
         if train:
             emb.backward(grad)
-            if world > 1:
-                dist.all_reduce(emb.flat_grads)   # the one exchange of the data-parallel path
+            ttd.allreduce_core_grads(emb.flat_grads)   # the one exchange of the data-parallel path
             emb.sgd_step(wl.lr)
 
     def barrier():

@@ -257,13 +257,90 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
     acc.store(w.E + (size_t)last * D, D, lane);
 }
 
+// Fast variant for D/4 <= 32 float4 chunks per row: LPR lanes cover a row, 32/LPR rows per load instruction,
+// NF load instructions issued back to back (the kernel is latency-bound), then the rows are folded in
+// position order; each sub-warp keeps its own partial sum and the sub-warps are combined at a segment end.
+template <int LPR>
+__global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restrict__ grad_out)
+{
+    constexpr int RPI = 32 / LPR, NF = 8;
+    const int lane = threadIdx.x & 31, sub = lane / LPR, lr = lane % LPR;
+    const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
+    const uint32_t Ltot = w.cnt[U];
+    const int64_t a64 = chunk * TT_DE_CHUNK;
+    if (a64 >= Ltot) return;
+    const uint32_t a = (uint32_t)a64;
+    const uint32_t b = min(a + (uint32_t)TT_DE_CHUNK, Ltot);
+    const int D = w.D, D4 = D >> 2;
+    const bool lane_on = lr < D4;
+    const uint32_t prev = a > 0 ? w.pairs[a - 1].x : HT_EMPTY;
+    const uint32_t next = b < Ltot ? w.pairs[b].x : HT_EMPTY;
+    const float4* __restrict__ G4 = reinterpret_cast<const float4*>(grad_out);
+    float4* __restrict__ E4 = reinterpret_cast<float4*>(w.E);
+    float4* carry4 = reinterpret_cast<float4*>(w.carry + (size_t)chunk * 2 * D);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t cur = w.pairs[a].x;
+    bool seg_first = true;
+    // combine the sub-warps and store (sub-warp 0 writes), then clear
+    auto flush = [&](float4* dst) {
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+        }
+        if (sub == 0 && lane_on) dst[lr] = acc;
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    for (uint32_t p0 = a; p0 < b; p0 += 32) {
+        const uint2 mine = (p0 + lane < b) ? __ldg(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
+        // row index of this lane's pair inside grad_out viewed as [B*T][D]
+        const uint32_t grow = mine.x != HT_EMPTY ? mine.y * (uint32_t)w.T + (uint32_t)tt_find_table(w.tb[w.K], w.T, mine.x) : 0u;
+        const int n = (int)min(32u, b - p0);
+        for (int j0 = 0; j0 < n; j0 += NF * RPI) {
+            float4 v[NF];
+#pragma unroll
+            for (int jj = 0; jj < NF; ++jj) {
+                const int j = j0 + jj * RPI + sub;
+                const uint32_t gr = __shfl_sync(0xffffffffu, grow, j & 31);
+                v[jj] = (j < n && lane_on) ? __ldg(G4 + (size_t)gr * D4 + lr) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int jj = 0; jj < NF; ++jj) {
+#pragma unroll
+                for (int h = 0; h < RPI; ++h) {
+                    const int j = j0 + jj * RPI + h;
+                    const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j & 31);
+                    if (j < n) {
+                        if (sl != cur) {
+                            if (seg_first && prev == cur) flush(carry4);            // head: began in an earlier chunk
+                            else flush(E4 + (size_t)cur * D4);
+                            cur = sl;
+                            seg_first = false;
+                        }
+                        if (sub == h) { acc.x += v[jj].x; acc.y += v[jj].y; acc.z += v[jj].z; acc.w += v[jj].w; }
+                    }
+                }
+            }
+        }
+    }
+    const bool open_start = seg_first && prev == cur;
+    if (next == cur) flush(carry4 + D4);          // tail: continues in the next chunk
+    else if (open_start) flush(carry4);           // head
+    else flush(E4 + (size_t)cur * D4);
+}
+
 template <bool VEC, int CPL>
 static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
 {
     const int64_t chunks = (h->v.L + TT_DE_CHUNK - 1) / TT_DE_CHUNK;
     const int grid = (int)((chunks + 7) / 8);
     if (grid > 0) {
-        k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out);
+        const int D4 = h->D / 4;
+        if (VEC && D4 <= 8) k_dE_fast<8><<<grid, 256, 0, s>>>(h->v, grad_out);
+        else if (VEC && D4 <= 16) k_dE_fast<16><<<grid, 256, 0, s>>>(h->v, grad_out);
+        else if (VEC && D4 <= 32) k_dE_fast<32><<<grid, 256, 0, s>>>(h->v, grad_out);
+        else k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out);
         k_dE_fix<VEC, CPL><<<grid, 256, 0, s>>>(h->v);
     }
     return cudaGetLastError();

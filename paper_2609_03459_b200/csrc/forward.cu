@@ -365,21 +365,40 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
 // ---------------------------------------------------------------------------------------------- pooling
 
 // One warp per bag.  A row of D floats is read as D/4 float4 chunks by a sub-warp of LPR lanes
-// (LPR = power of two >= min(32, D/4)); 32/LPR rows are in flight per load instruction, and the
-// sub-warps' partial sums are combined with __shfl_xor at the end.
+// (LPR = power of two >= min(32, D/4)); 32/LPR rows are fetched per load instruction, up to NF such
+// instructions are issued back to back before any result is consumed (the kernel is bound by memory
+// latency, so bytes in flight per warp are what counts), the rank look-ups of the next 32 lookups are
+// started before the current ones are gathered, and the sub-warps' partial sums are combined with
+// __shfl_xor at the end.
+__device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableDesc& td, int64_t l, uint32_t capK)
+{
+    const int64_t g = __ldg(w.indices + l);
+    uint32_t slot = 0xffffffffu;
+    if (g >= 0 && g < td.N) {
+        const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
+        if (e.x >> (g & 31) & 1u) {
+            slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
+            if (slot >= capK) slot = 0xffffffffu;
+        }
+    }
+    return slot;
+}
+
 template <int LPR, int CPL>  // lanes per row, float4 chunks per lane
 __global__ void __launch_bounds__(256) k_pool_vec(WsView w, float* __restrict__ out)
 {
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPR, lr = lane % LPR;
-    constexpr int RPI = 32 / LPR;  // rows per iteration
+    constexpr int RPI = 32 / LPR;                       // rows per load instruction
+    constexpr int NIT = 32 / RPI;                       // load instructions per 32 lookups
+    constexpr int NF = (NIT * CPL > 16) ? (16 / CPL > 0 ? 16 / CPL : 1) : NIT;  // instructions in flight
     const int D4 = w.D >> 2;
     const int64_t nb = (int64_t)w.T * w.B;
-    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
     const uint32_t capK = w.cap[w.K];
-    bool bad = false;
-    for (int64_t bag = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); bag < nb; bag += nwarps) {
+    // one warp per bag, plain grid: the hardware block scheduler balances bags of very different sizes
+    const int64_t bag = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (bag < nb) {
         const int t = (int)(bag / w.B);
         const int64_t b = bag - (int64_t)t * w.B;
         const TableDesc& td = w.tdesc[t];
@@ -389,34 +408,34 @@ __global__ void __launch_bounds__(256) k_pool_vec(WsView w, float* __restrict__ 
         float4 acc[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        uint32_t slot_next = (lo + lane < hi) ? tt_lookup_slot(w, td, lo + lane, capK) : 0xffffffffu;
         for (int64_t l0 = lo; l0 < hi; l0 += 32) {
-            uint32_t slot = 0xffffffffu;
-            if (l0 + lane < hi) {
-                const int64_t g = __ldg(w.indices + l0 + lane);
-                if (g >= 0 && g < td.N) {
-                    const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
-                    if (e.x >> (g & 31) & 1u) {
-                        slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
-                        if (slot >= capK) slot = 0xffffffffu;
-                    }
-                }
-                if (w.upairs) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);  // kept for the backward sort
-            }
+            const uint32_t slot = slot_next;
+            if (w.upairs && l0 + lane < hi) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);  // kept for the backward sort
+            slot_next = (l0 + 32 + lane < hi) ? tt_lookup_slot(w, td, l0 + 32 + lane, capK) : 0xffffffffu;
             const int n = (int)min((int64_t)32, hi - l0);
-#pragma unroll 4
-            for (int j = 0; j < n; j += RPI) {
-                const uint32_t sl = __shfl_sync(0xffffffffu, slot, (j + sub) & 31);
-                if (j + sub < n && sl != 0xffffffffu) {
-                    const float4* row = E4 + (size_t)sl * D4;
+#pragma unroll
+            for (int j0 = 0; j0 < NIT; j0 += NF) {
+                if (j0 * RPI >= n) break;
+                float4 v[NF][CPL];
+#pragma unroll
+                for (int jj = 0; jj < NF; ++jj) {
+                    const int j = (j0 + jj) * RPI + sub;
+                    const uint32_t sl = __shfl_sync(0xffffffffu, slot, j & 31);
+                    const bool ok = j < n && sl != 0xffffffffu;
+                    const float4* row = E4 + (size_t)(ok ? sl : 0u) * D4;
 #pragma unroll
                     for (int c = 0; c < CPL; ++c) {
                         const int ch = lr + c * LPR;
-                        if (ch < D4) {
-                            const float4 v = __ldg(row + ch);
-                            acc[c].x += v.x; acc[c].y += v.y; acc[c].z += v.z; acc[c].w += v.w;
-                        }
+                        v[jj][c] = (ok && ch < D4) ? __ldg(row + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
+#pragma unroll
+                for (int jj = 0; jj < NF; ++jj)
+#pragma unroll
+                    for (int c = 0; c < CPL; ++c) {
+                        acc[c].x += v[jj][c].x; acc[c].y += v[jj][c].y; acc[c].z += v[jj][c].z; acc[c].w += v[jj][c].w;
+                    }
             }
         }
 #pragma unroll
@@ -438,7 +457,6 @@ __global__ void __launch_bounds__(256) k_pool_vec(WsView w, float* __restrict__ 
             }
         }
     }
-    (void)bad;
 }
 
 // any D (scalar path): lane handles elements lane, lane+32, ...
@@ -499,13 +517,14 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
 {
     WsView& w = h->v;
     const int64_t nb = (int64_t)w.T * w.B;
-    int64_t want = (nb + 7) / 8;  // 8 warps per CTA
-    int grid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
+    const int64_t want = (nb + 7) / 8;  // 8 warps per CTA, one warp per bag
+    int grid = (int)want;
     if (grid < 1) grid = 1;
     const int D = w.D;
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0);
     if (!vec_ok) {
-        k_pool_scalar<<<grid, 256, 0, s>>>(w, out);
+        int pgrid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
+        k_pool_scalar<<<pgrid < 1 ? 1 : pgrid, 256, 0, s>>>(w, out);
         return cudaGetLastError();
     }
     const int D4 = D / 4;

@@ -130,8 +130,10 @@ def near_equal_factors3(N: int) -> Tuple[int, int, int]:
     return (n1, n, n)
 
 
-def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None) -> Workload:
-    """pooling: int (fixed) or (lo, hi) inclusive uniform per (table, bag)."""
+def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None, batch_seed0=None) -> Workload:
+    """pooling: int (fixed) or (lo, hi) inclusive uniform per (table, bag).
+    batch_seed0: draw the batch (bag lengths, indices, grad_out) from another stream while the cores stay
+    those of seed0 (used for the per-rank batches of a multi-GPU run)."""
     T = len(tables)
 
     def one_table(t):
@@ -139,6 +141,8 @@ def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None) ->
         spec = tables[t]
         rng = np.random.default_rng(seed0 + t)
         tc = make_cores(rng, spec)
+        if batch_seed0 is not None:
+            rng = np.random.default_rng(batch_seed0 + t)
         if isinstance(pooling, tuple):
             lens = rng.integers(pooling[0], pooling[1] + 1, size=B, dtype=np.int64)
         else:
@@ -159,7 +163,7 @@ def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None) ->
     indices = np.concatenate(idx_parts).astype(np.int64) if idx_parts else np.zeros(0, np.int64)
     grad = None
     if with_grad:
-        rng = np.random.default_rng(seed0 + 999)
+        rng = np.random.default_rng((seed0 if batch_seed0 is None else batch_seed0) + 999)
         D = tables[0].D
         grad = rng.standard_normal(size=(B, T * D)).astype(np.float32)
     return Workload(name=name, tables=tables, B=B, indices=indices, offsets=offsets, cores=cores,
@@ -182,27 +186,29 @@ def _cfg3_tables(rng: np.random.Generator, T: int, n_cap: Optional[int] = None) 
 
 
 def make(config: int, *, tiny: bool = False, mapping: str = "identity", seed: Optional[int] = None,
-         batch: Optional[int] = None, num_tables: Optional[int] = None) -> Workload:
+         batch: Optional[int] = None, num_tables: Optional[int] = None, batch_seed: Optional[int] = None) -> Workload:
     """Build one of the five benchmark configurations (1..5).
 
     tiny=True keeps the structure (K, dim factors, skew, pooling law) but shrinks row factors to <= 6
     and the batch to <= 16 so that a dense materialisation of the table is affordable.
     `batch` / `num_tables` override B / T (used for reduced-size parity cases and bounded CPU timing).
+    `batch_seed` draws another batch (bag lengths, indices, grad_out) for the same tables and cores.
     """
     seed0 = (BASE_SEED if seed is None else seed) + 1000 * config
+    bs0 = None if batch_seed is None else batch_seed + 1000 * config
     if config == 1:
         n = (5, 6, 4) if tiny else (100, 100, 100)
         N = int(np.prod(n)) - (3 if tiny else 0)
         spec = TableSpec(N=N, n=n, d=(4, 4, 4), r=(1, 8, 8, 1), alpha=1.05, core_dist="uniform", core_scale=0.1)
         B = batch or (16 if tiny else 1024)
-        return _assemble("cfg1" + ("-tiny" if tiny else ""), [spec], B, 1, seed0, mapping, False)
+        return _assemble("cfg1" + ("-tiny" if tiny else ""), [spec], B, 1, seed0, mapping, False, batch_seed0=bs0)
     if config == 2:
         n = (4, 5, 6) if tiny else (200, 250, 200)
         N = int(np.prod(n))
         r = (1, 5, 3, 1) if tiny else (1, 32, 32, 1)
         spec = TableSpec(N=N, n=n, d=(4, 8, 4), r=r, alpha=1.1, core_dist="normal", core_scale=0.05)
         B = batch or (12 if tiny else 32768)
-        return _assemble("cfg2" + ("-tiny" if tiny else ""), [spec], B, 20, seed0, mapping, False)
+        return _assemble("cfg2" + ("-tiny" if tiny else ""), [spec], B, 20, seed0, mapping, False, batch_seed0=bs0)
     if config in (3, 5):
         # tables are drawn from the config-3 stream for both 3 and 5 so that 5 trains on 3's tables
         seed3 = (BASE_SEED if seed is None else seed) + 1000 * 3
@@ -215,14 +221,14 @@ def make(config: int, *, tiny: bool = False, mapping: str = "identity", seed: Op
         B = batch or (16 if tiny else 32768)
         pooling = (1, 9) if tiny else (1, 100)
         return _assemble(f"cfg{config}" + ("-tiny" if tiny else ""), tables, B, pooling, seed3, mapping,
-                         with_grad=(config == 5))
+                         with_grad=(config == 5), batch_seed0=None if batch_seed is None else batch_seed + 3000)
     if config == 4:
         n = (3, 4, 3, 4) if tiny else (64, 64, 64, 64)
         N = int(np.prod(n))
         r = (1, 3, 4, 2, 1) if tiny else (1, 64, 64, 64, 1)
         spec = TableSpec(N=N, n=n, d=(2, 4, 4, 4), r=r, alpha=1.2, core_dist="normal", core_scale=0.02)
         B = batch or (16 if tiny else 65536)
-        return _assemble("cfg4" + ("-tiny" if tiny else ""), [spec], B, 8, seed0, mapping, False)
+        return _assemble("cfg4" + ("-tiny" if tiny else ""), [spec], B, 8, seed0, mapping, False, batch_seed0=bs0)
     raise ValueError("config must be 1..5")
 
 
