@@ -17,6 +17,7 @@
 //             Each output has exactly one owner, which sums in sorted order: no atomics.
 #include "common.cuh"
 #include "scan.cuh"
+#include "mma.cuh"
 
 #define HT_SIZE 4096
 #define HT_TILE 2048
@@ -258,12 +259,13 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
 }
 
 // Fast variant for D/4 <= 32 float4 chunks per row: LPR lanes cover a row, 32/LPR rows per load instruction,
-// NF load instructions issued back to back (the kernel is latency-bound), then the rows are folded in
-// position order; each sub-warp keeps its own partial sum and the sub-warps are combined at a segment end.
+// NF load instructions issued back to back, then the rows are folded in position order.  Each sub-warp keeps
+// its own partial sum; the sub-warps are combined only when a segment ends.  Segment starts inside a batch of
+// 32 positions are found once with a ballot, so a window without a start costs 4 adds per load and nothing else.
 template <int LPR>
 __global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restrict__ grad_out)
 {
-    constexpr int RPI = 32 / LPR, NF = 8;
+    constexpr int RPI = 32 / LPR, NF = 4;
     const int lane = threadIdx.x & 31, sub = lane / LPR, lr = lane % LPR;
     const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
@@ -282,8 +284,9 @@ __global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restri
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     uint32_t cur = w.pairs[a].x;
     bool seg_first = true;
-    // combine the sub-warps and store (sub-warp 0 writes), then clear
-    auto flush = [&](float4* dst) {
+    // close the running segment: combine the sub-warps, store (sub-warp 0 writes), clear
+    auto close_segment = [&]() {
+        float4* dst = (seg_first && prev == cur) ? carry4 : E4 + (size_t)cur * D4;   // head piece or whole segment
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
             acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
@@ -291,12 +294,18 @@ __global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restri
         }
         if (sub == 0 && lane_on) dst[lr] = acc;
         acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        seg_first = false;
     };
+    uint32_t last_slot = cur;  // slot of the position before the current batch
     for (uint32_t p0 = a; p0 < b; p0 += 32) {
         const uint2 mine = (p0 + lane < b) ? __ldg(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
-        // row index of this lane's pair inside grad_out viewed as [B*T][D]
-        const uint32_t grow = mine.x != HT_EMPTY ? mine.y * (uint32_t)w.T + (uint32_t)tt_find_table(w.tb[w.K], w.T, mine.x) : 0u;
         const int n = (int)min(32u, b - p0);
+        // row index of this lane's pair inside grad_out viewed as [B*T][D]
+        const uint32_t grow = lane < n ? mine.y * (uint32_t)w.T + (uint32_t)tt_find_table(w.tb[w.K], w.T, mine.x) : 0u;
+        uint32_t before = __shfl_up_sync(0xffffffffu, mine.x, 1);
+        if (lane == 0) before = last_slot;
+        const unsigned starts = __ballot_sync(0xffffffffu, lane < n && mine.x != before);  // bit j: position j opens a segment
+        last_slot = __shfl_sync(0xffffffffu, mine.x, n - 1);
         for (int j0 = 0; j0 < n; j0 += NF * RPI) {
             float4 v[NF];
 #pragma unroll
@@ -307,16 +316,15 @@ __global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restri
             }
 #pragma unroll
             for (int jj = 0; jj < NF; ++jj) {
+                const int j = j0 + jj * RPI;
+                if (((starts >> j) & ((1u << RPI) - 1u)) == 0u) {
+                    acc.x += v[jj].x; acc.y += v[jj].y; acc.z += v[jj].z; acc.w += v[jj].w;
+                } else {
 #pragma unroll
-                for (int h = 0; h < RPI; ++h) {
-                    const int j = j0 + jj * RPI + h;
-                    const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j & 31);
-                    if (j < n) {
-                        if (sl != cur) {
-                            if (seg_first && prev == cur) flush(carry4);            // head: began in an earlier chunk
-                            else flush(E4 + (size_t)cur * D4);
-                            cur = sl;
-                            seg_first = false;
+                    for (int h = 0; h < RPI; ++h) {
+                        if ((starts >> (j + h)) & 1u) {
+                            close_segment();
+                            cur = __shfl_sync(0xffffffffu, mine.x, (j + h) & 31);
                         }
                         if (sub == h) { acc.x += v[jj].x; acc.y += v[jj].y; acc.z += v[jj].z; acc.w += v[jj].w; }
                     }
@@ -324,10 +332,17 @@ __global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restri
             }
         }
     }
-    const bool open_start = seg_first && prev == cur;
-    if (next == cur) flush(carry4 + D4);          // tail: continues in the next chunk
-    else if (open_start) flush(carry4);           // head
-    else flush(E4 + (size_t)cur * D4);
+    // last segment of the chunk
+    {
+        const bool open_start = seg_first && prev == cur;
+        float4* dst = next == cur ? carry4 + D4 : (open_start ? carry4 : E4 + (size_t)cur * D4);  // tail / head / whole
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+        }
+        if (sub == 0 && lane_on) dst[lr] = acc;
+    }
 }
 
 template <bool VEC, int CPL>
@@ -628,7 +643,125 @@ __device__ __forceinline__ void tt_warp_rows_dG(const float* Cs, const WsView& w
     }
 }
 
-template <int PM, int RB_, int TP, int M, int CPL>
+// ---- tensor-core (3xTF32, m16n8k8) forms of the two row passes, d_K = 4 ---------------------------------------
+//
+// pass A  dC[p][b] = sum over the group's rows u and j of dE_u[p][j] * D_u[b][j]:  M = 16 rows p, N = 8 values of b,
+//         K = 8 = two rows x 4 columns j.  The sum over the rows that share C (Eq. 2) is the accumulation over
+//         k-steps, so dC ends up complete in the accumulator fragments (PM*RB/32 registers) and is written once:
+//         no cross-lane reduction at all.
+// pass B  dG_K[i_K(u)][b][j] += sum_p C[p][b] * dE_u[p][j]:  M = 16 values of b, K = 8 rows p, N = 8 = two rows x 4
+//         columns j; C^T fragments are fixed per group.  Results leave as 8-byte vector reductions.
+__device__ __forceinline__ void tt_red_v2(float* p, float x, float y)
+{
+    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(x), "f"(y) : "memory");
+}
+
+template <int PM, int RB_>
+__device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1, uint32_t row_base,
+                                                    float* dPdst, int lane)
+{
+    constexpr int MT = PM / 16, NT = RB_ / 8;
+    const int g = lane >> 2, t = lane & 3;
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    float acc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f; }
+    for (uint32_t ub = u0; ub < u1; ub += 2) {
+        const bool two = ub + 1 < u1;
+        const uint32_t ua = ub, uc = two ? ub + 1 : ub;
+        const float* __restrict__ Ea = w.E + (size_t)ua * (PM * 4) + t;
+        const float* __restrict__ Ec = w.E + (size_t)uc * (PM * 4) + t;
+        const float* __restrict__ Da = GK + (size_t)(rows[ua] - row_base) * (RB_ * 4) + t;
+        const float* __restrict__ Dc = GK + (size_t)(rows[uc] - row_base) * (RB_ * 4) + t;
+        Tf32Pair a[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            a[mt][0] = tt_split_tf32(__ldg(Ea + (16 * mt + g) * 4));
+            a[mt][1] = tt_split_tf32(__ldg(Ea + (16 * mt + g + 8) * 4));
+            a[mt][2] = tt_split_tf32(two ? __ldg(Ec + (16 * mt + g) * 4) : 0.f);
+            a[mt][3] = tt_split_tf32(two ? __ldg(Ec + (16 * mt + g + 8) * 4) : 0.f);
+        }
+        float bv[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            bv[nt][0] = __ldg(Da + (8 * nt + g) * 4);
+            bv[nt][1] = __ldg(Dc + (8 * nt + g) * 4);
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            Tf32Pair b[2];
+            b[0] = tt_split_tf32(bv[nt][0]);
+            b[1] = tt_split_tf32(bv[nt][1]);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt][nt], a[mt], b);
+        }
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        }
+}
+
+template <int PM, int RB_>
+__device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsView& w, uint32_t u0, uint32_t u1, uint32_t row_base,
+                                                    float* gk, int lane)
+{
+    constexpr int MT = RB_ / 16, KT = PM / 8;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t* __restrict__ rows = w.val[w.K];
+    Tf32Pair a[MT][KT][4];   // A[m = b][k = p] = C[p][b]
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            a[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g]);
+            a[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g + 8]);
+            a[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g]);
+            a[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g + 8]);
+        }
+    const int rb_ = g >> 2, jb = g & 3;       // B fragment: row rb_ of the pair, column jb of dE
+    const int rc = t >> 1, jc = 2 * (t & 1);  // C fragment: row rc of the pair, columns jc, jc+1
+    for (uint32_t ub = u0; ub < u1; ub += 2) {
+        const uint32_t ul = min(ub + (uint32_t)rb_, u1 - 1);
+        const bool valid = ub + (uint32_t)rb_ < u1;
+        const float* __restrict__ El = w.E + (size_t)ul * (PM * 4) + jb;
+        float acc[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) { acc[mt][0] = 0.f; acc[mt][1] = 0.f; acc[mt][2] = 0.f; acc[mt][3] = 0.f; }
+        float bv[KT][2];
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            bv[kt][0] = valid ? __ldg(El + (8 * kt + t) * 4) : 0.f;
+            bv[kt][1] = valid ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
+        }
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            Tf32Pair b[2];
+            b[0] = tt_split_tf32(bv[kt][0]);
+            b[1] = tt_split_tf32(bv[kt][1]);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt], a[mt][kt], b);
+        }
+        const uint32_t us = ub + (uint32_t)rc;
+        if (us < u1) {
+            float* dst = gk + (size_t)(rows[us] - row_base) * (RB_ * 4) + jc;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                tt_red_v2(dst + (16 * mt + g) * 4, acc[mt][0], acc[mt][1]);
+                tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
+            }
+        }
+    }
+}
+
+template <int PM, int RB_, int TP, int M, int CPL, bool MMA>
 __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* gk,
                                                   float* As, float* Cs, int lane, int wid, int nw)
 {
@@ -647,8 +780,13 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
         tt_warp_mid_b<M, CPL>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
         __syncwarp();
         const uint32_t u0 = w.cstart[K - 1][g], u1 = w.cstart[K - 1][g + 1];
-        tt_warp_rows_dC<PM, RB_, TP>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
-        tt_warp_rows_dG<PM, RB_, TP>(Cs, w, u0, u1, val * nK, gk, lane);
+        if constexpr (MMA) {
+            tt_warp_rows_dC_mma<PM, RB_>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
+            tt_warp_rows_dG_mma<PM, RB_>(Cs, w, u0, u1, val * nK, gk, lane);
+        } else {
+            tt_warp_rows_dC<PM, RB_, TP>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
+            tt_warp_rows_dG<PM, RB_, TP>(Cs, w, u0, u1, val * nK, gk, lane);
+        }
         __syncwarp();
     }
 }
@@ -676,11 +814,11 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
-    if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
 }
 
 // fixed-order sum of the partial copies of the last core's gradient

@@ -11,6 +11,7 @@
 //     reduces them in registers; lanes of different sub-warps are combined with warp shuffles.  No atomics.
 #include "common.cuh"
 #include "scan.cuh"
+#include "mma.cuh"
 
 // ---------------------------------------------------------------------------------------------- schedule
 
@@ -231,8 +232,67 @@ __device__ __forceinline__ void tt_warp_rows(const float* Cs, const WsView& w, c
     }
 }
 
+// Tensor-core form of the last product (d_K = 4): E_u[p][j] = sum_b C[p][b] * D_u[b][j] as m16n8k8 tiles with
+// M = 16 rows p of C, K = 8 values of b, N = 8 = two child rows x 4 columns j.  The fragments of C (split into TF32
+// head and tail) stay in PM*RB/8 registers for the whole group; each child's slice is read exactly once per warp
+// (two coalesced 64-byte pieces per load instruction), so the shared-memory / L1 path carries 4x fewer bytes per
+// FMA than the FP32-pipe form and a warp needs ~1/3 of its registers.
+template <int PM, int RB>
+__device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
+                                                 uint32_t row_base, int lane)
+{
+    constexpr int MT = PM / 16, KT = RB / 8;
+    const int g = lane >> 2, t = lane & 3;
+    Tf32Pair a[MT][KT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            a[mt][kt][0] = tt_split_tf32(Cs[(16 * mt + g) * RB + 8 * kt + t]);
+            a[mt][kt][1] = tt_split_tf32(Cs[(16 * mt + g + 8) * RB + 8 * kt + t]);
+            a[mt][kt][2] = tt_split_tf32(Cs[(16 * mt + g) * RB + 8 * kt + t + 4]);
+            a[mt][kt][3] = tt_split_tf32(Cs[(16 * mt + g + 8) * RB + 8 * kt + t + 4]);
+        }
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    const int rb_ = g >> 2, jb = g & 3;   // this lane's B-fragment column: child row rb_ of the pair, output column jb
+    const int rc = t >> 1, jc = 2 * (t & 1);  // this lane's C-fragment columns: child row rc, output columns jc, jc+1
+    for (uint32_t ub = u0; ub < u1; ub += 2) {
+        const uint32_t ul = min(ub + (uint32_t)rb_, u1 - 1);   // an odd tail repeats the last row (not stored twice)
+        const uint32_t iK = rows[ul] - row_base;
+        const float* __restrict__ Dl = GK + (size_t)iK * (RB * 4) + jb;
+        float bv[KT][2];
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            bv[kt][0] = __ldg(Dl + (8 * kt + t) * 4);
+            bv[kt][1] = __ldg(Dl + (8 * kt + t + 4) * 4);
+        }
+        float acc[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) { acc[mt][0] = 0.f; acc[mt][1] = 0.f; acc[mt][2] = 0.f; acc[mt][3] = 0.f; }
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+            Tf32Pair b[2];
+            b[0] = tt_split_tf32(bv[kt][0]);
+            b[1] = tt_split_tf32(bv[kt][1]);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt], a[mt][kt], b);
+        }
+        const uint32_t us = ub + (uint32_t)rc;
+        if (us < u1) {
+            float* e = w.E + (size_t)us * (PM * 4) + jc;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                *reinterpret_cast<float2*>(e + (16 * mt + g) * 4) = make_float2(acc[mt][0], acc[mt][1]);
+                *reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4) = make_float2(acc[mt][2], acc[mt][3]);
+            }
+        }
+    }
+}
+
 // one warp: groups fetched dynamically from the CTA's range through a shared counter
-template <int PM, int RB, int TP, int M, int CPL>
+template <int PM, int RB, int TP, int M, int CPL, bool MMA>
 __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& td, uint32_t g1, float* As, float* Cs,
                                               uint32_t* next, int lane)
 {
@@ -254,7 +314,8 @@ __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& 
         const uint32_t im = val % (uint32_t)td.n[km];
         tt_warp_mid<M, CPL>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
         __syncwarp();
-        tt_warp_rows<PM, RB, TP>(Cs, w, td, w.cstart[K - 1][g], w.cstart[K - 1][g + 1], val * nK, lane);
+        if constexpr (MMA) tt_warp_rows_mma<PM, RB>(Cs, w, td, w.cstart[K - 1][g], w.cstart[K - 1][g + 1], val * nK, lane);
+        else tt_warp_rows<PM, RB, TP>(Cs, w, td, w.cstart[K - 1][g], w.cstart[K - 1][g + 1], val * nK, lane);
         __syncwarp();
     }
 }
@@ -317,11 +378,11 @@ __global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats, int 
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
-    if (V == 0) tt_sweep_fast<16, 32, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
-    if (V == 1) tt_sweep_fast<16, 16, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
-    if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1>(w, td, g1, As, Cs, &next, lane);
-    if (V == 3) tt_sweep_fast<32, 32, 4, 4, 2>(w, td, g1, As, Cs, &next, lane);
-    if (V == 4) tt_sweep_fast<32, 64, 2, 8, 2>(w, td, g1, As, Cs, &next, lane);
+    if (V == 0) tt_sweep_fast<16, 32, 4, 4, 1, true>(w, td, g1, As, Cs, &next, lane);
+    if (V == 1) tt_sweep_fast<16, 16, 4, 4, 1, true>(w, td, g1, As, Cs, &next, lane);
+    if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 3) tt_sweep_fast<32, 32, 4, 4, 2, true>(w, td, g1, As, Cs, &next, lane);
+    if (V == 4) tt_sweep_fast<32, 64, 2, 8, 2, false>(w, td, g1, As, Cs, &next, lane);
 }
 
 template <int V>
@@ -385,35 +446,59 @@ __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableD
 }
 
 template <int LPR, int CPL>  // lanes per row, float4 chunks per lane
-__global__ void __launch_bounds__(256) k_pool_vec(WsView w, float* __restrict__ out)
+__global__ void __launch_bounds__(256, (CPL == 1 ? 5 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
 {
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPR, lr = lane % LPR;
     constexpr int RPI = 32 / LPR;                       // rows per load instruction
     constexpr int NIT = 32 / RPI;                       // load instructions per 32 lookups
-    constexpr int NF = (NIT * CPL > 16) ? (16 / CPL > 0 ? 16 / CPL : 1) : NIT;  // instructions in flight
+    constexpr int NF = NIT < 4 ? NIT : 4;               // load instructions in flight
     const int D4 = w.D >> 2;
     const int64_t nb = (int64_t)w.T * w.B;
     const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
     const uint32_t capK = w.cap[w.K];
-    // one warp per bag, plain grid: the hardware block scheduler balances bags of very different sizes
-    const int64_t bag = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (bag < nb) {
-        const int t = (int)(bag / w.B);
+    // Skew-aware split: the grid is exactly resident (persistent warps); warp wi takes the bags whose first
+    // lookup falls into the wi-th equal share of the L lookups (offsets is the cost prefix sum).
+    const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int64_t b0, b1;
+    {
+        const int64_t target = lane == 0 ? (w.L * wi) / W : (w.L * (wi + 1)) / W;
+        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target
+        if (lane < 2)
+            while (lo < hi) {
+                const int64_t mid = (lo + hi) >> 1;
+                if (__ldg(w.offsets + mid) < target) lo = mid + 1; else hi = mid;
+            }
+        b0 = __shfl_sync(0xffffffffu, lo, 0);
+        b1 = __shfl_sync(0xffffffffu, lo, 1);
+        if (wi == 0) b0 = 0;
+        if (wi == W - 1) b1 = nb;
+    }
+    if (b0 >= b1) return;
+    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
+    if (o_hi < o_lo) o_hi = o_lo;
+    int t = (int)(b0 / w.B);
+    uint32_t slot_next = (o_lo + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], o_lo + lane, capK) : 0xffffffffu;
+    for (int64_t bag = b0; bag < b1; ++bag) {
         const int64_t b = bag - (int64_t)t * w.B;
-        const TableDesc& td = w.tdesc[t];
-        int64_t lo = w.offsets[bag], hi = w.offsets[bag + 1];
-        lo = lo < 0 ? 0 : (lo > w.L ? w.L : lo);
-        hi = hi < lo ? lo : (hi > w.L ? w.L : hi);
+        // next bag (for the prefetch of its first 32 rank look-ups)
+        const bool has_next = bag + 1 < b1;
+        int64_t n_hi = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_hi;
+        if (n_hi < o_hi) n_hi = o_hi;
+        const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
         float4 acc[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        uint32_t slot_next = (lo + lane < hi) ? tt_lookup_slot(w, td, lo + lane, capK) : 0xffffffffu;
-        for (int64_t l0 = lo; l0 < hi; l0 += 32) {
+        if (o_lo >= o_hi && has_next)
+            slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+        for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
-            if (w.upairs && l0 + lane < hi) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);  // kept for the backward sort
-            slot_next = (l0 + 32 + lane < hi) ? tt_lookup_slot(w, td, l0 + 32 + lane, capK) : 0xffffffffu;
-            const int n = (int)min((int64_t)32, hi - l0);
+            if (w.upairs && l0 + lane < o_hi) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);  // kept for the backward sort
+            if (l0 + 32 < o_hi) slot_next = (l0 + 32 + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], l0 + 32 + lane, capK) : 0xffffffffu;
+            else if (has_next) slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+            const int n = (int)min((int64_t)32, o_hi - l0);
 #pragma unroll
             for (int j0 = 0; j0 < NIT; j0 += NF) {
                 if (j0 * RPI >= n) break;
@@ -456,7 +541,26 @@ __global__ void __launch_bounds__(256) k_pool_vec(WsView w, float* __restrict__ 
                 if (ch < D4) o4[ch] = acc[c];
             }
         }
+        o_lo = o_hi;
+        o_hi = n_hi;
+        t = tn;
     }
+}
+
+template <int LPR, int CPL>
+static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
+{
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_vec<LPR, CPL>, 256, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const int64_t nb = (int64_t)h->v.T * h->v.B;
+    int64_t grid = (int64_t)per_sm * h->sm_count;
+    const int64_t need = (nb + 7) / 8;
+    if (grid > need) grid = need;
+    if (grid < 1) grid = 1;
+    k_pool_vec<LPR, CPL><<<(int)grid, 256, 0, s>>>(h->v, out);
+    return cudaGetLastError();
 }
 
 // any D (scalar path): lane handles elements lane, lane+32, ...
@@ -528,12 +632,12 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
         return cudaGetLastError();
     }
     const int D4 = D / 4;
-    if (D4 <= 4) k_pool_vec<4, 1><<<grid, 256, 0, s>>>(w, out);
-    else if (D4 <= 8) k_pool_vec<8, 1><<<grid, 256, 0, s>>>(w, out);
-    else if (D4 <= 16) k_pool_vec<16, 1><<<grid, 256, 0, s>>>(w, out);
-    else if (D4 <= 32) k_pool_vec<32, 1><<<grid, 256, 0, s>>>(w, out);
-    else if (D4 <= 64) k_pool_vec<32, 2><<<grid, 256, 0, s>>>(w, out);
-    else if (D4 <= 128) k_pool_vec<32, 4><<<grid, 256, 0, s>>>(w, out);
-    else k_pool_vec<32, 8><<<grid, 256, 0, s>>>(w, out);
-    return cudaGetLastError();
+    (void)grid;
+    if (D4 <= 4) return launch_pool_vec<4, 1>(h, out, s);
+    if (D4 <= 8) return launch_pool_vec<8, 1>(h, out, s);
+    if (D4 <= 16) return launch_pool_vec<16, 1>(h, out, s);
+    if (D4 <= 32) return launch_pool_vec<32, 1>(h, out, s);
+    if (D4 <= 64) return launch_pool_vec<32, 2>(h, out, s);
+    if (D4 <= 128) return launch_pool_vec<32, 4>(h, out, s);
+    return launch_pool_vec<32, 8>(h, out, s);
 }
