@@ -139,9 +139,10 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->capU = (cfg->max_unique_rows > 0 && cfg->max_unique_rows < bound) ? cfg->max_unique_rows : bound;
 
     // work units: every table is cut into `units` equal-cost slices, one CTA each
-    int Q = (16 * h->sm_count + T - 1) / T;
+    // about 8 waves of 8 resident CTAs per SM: fine enough that the last wave and table-size differences do not matter
+    int Q = (64 * h->sm_count + T - 1) / T;
     if (Q < 8) Q = 8;
-    if (Q > 2048) Q = 2048;
+    if (Q > 16384) Q = 16384;
     int unit_base = 0;
     int64_t gpart = 0;
     h->max_priv_floats = 0;

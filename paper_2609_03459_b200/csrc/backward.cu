@@ -396,8 +396,11 @@ __device__ __forceinline__ void tt_unit_range_b(const WsView& w, int t, int q, u
         }
         return lo;
     };
-    g0 = q == 0 ? a : lower(lo_c);
-    g1 = q == Q - 1 ? b : lower(hi_c);
+    const bool odd = (threadIdx.x & 1) != 0;
+    const uint32_t mine = lower(odd ? hi_c : lo_c);
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
+    g0 = q == 0 ? a : (odd ? other : mine);
+    g1 = q == Q - 1 ? b : (odd ? mine : other);
 }
 
 __device__ __forceinline__ void tt_mid_product_b(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
@@ -509,7 +512,7 @@ __device__ __forceinline__ void tt_warp_mid_b(const float* As, const float* __re
 #pragma unroll
         for (int m = 0; m < M; ++m) { acc[i][m][0] = 0.f; acc[i][m][1] = 0.f; acc[i][m][2] = 0.f; acc[i][m][3] = 0.f; }
     const float4* __restrict__ B4 = reinterpret_cast<const float4*>(Bsl);
-#pragma unroll 8
+#pragma unroll 16
     for (int a = s; a < ra; a += NS) {
         float4 b[CPL];
 #pragma unroll

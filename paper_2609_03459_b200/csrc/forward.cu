@@ -64,8 +64,12 @@ __device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uin
         }
         return lo;
     };
-    g0 = q == 0 ? a : lower(lo_c);
-    g1 = q == Q - 1 ? b : lower(hi_c);
+    // every thread needs both bounds; even and odd lanes each search one and exchange it
+    const bool odd = (threadIdx.x & 1) != 0;
+    const uint32_t mine = lower(odd ? hi_c : lo_c);
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
+    g0 = q == 0 ? a : (odd ? other : mine);
+    g1 = q == Q - 1 ? b : (odd ? mine : other);
 }
 
 // ---------------------------------------------------------------------------------------------- products
@@ -149,7 +153,7 @@ __device__ __forceinline__ void tt_warp_mid(const float* As, const float* __rest
 #pragma unroll
         for (int m = 0; m < M; ++m) { acc[i][m][0] = 0.f; acc[i][m][1] = 0.f; acc[i][m][2] = 0.f; acc[i][m][3] = 0.f; }
     const float4* __restrict__ B4 = reinterpret_cast<const float4*>(Bsl);
-#pragma unroll 4
+#pragma unroll 16
     for (int a = s; a < ra; a += NS) {
         float4 b[CPL];
 #pragma unroll
@@ -258,34 +262,42 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
     const uint32_t* __restrict__ rows = w.val[K];
     const int rb_ = g >> 2, jb = g & 3;   // this lane's B-fragment column: child row rb_ of the pair, output column jb
     const int rc = t >> 1, jc = 2 * (t & 1);  // this lane's C-fragment columns: child row rc, output columns jc, jc+1
-    for (uint32_t ub = u0; ub < u1; ub += 2) {
-        const uint32_t ul = min(ub + (uint32_t)rb_, u1 - 1);   // an odd tail repeats the last row (not stored twice)
-        const uint32_t iK = rows[ul] - row_base;
-        const float* __restrict__ Dl = GK + (size_t)iK * (RB * 4) + jb;
-        float bv[KT][2];
+    constexpr int NP = 2;   // row pairs in flight
+    for (uint32_t ub = u0; ub < u1; ub += 2 * NP) {
+        float bv[NP][KT][2];
 #pragma unroll
-        for (int kt = 0; kt < KT; ++kt) {
-            bv[kt][0] = __ldg(Dl + (8 * kt + t) * 4);
-            bv[kt][1] = __ldg(Dl + (8 * kt + t + 4) * 4);
+        for (int np = 0; np < NP; ++np) {
+            // an odd tail (or a missing second pair) repeats the last row; it is computed but not stored
+            const uint32_t ul = min(ub + 2 * np + (uint32_t)rb_, u1 - 1);
+            const uint32_t iK = rows[ul] - row_base;
+            const float* __restrict__ Dl = GK + (size_t)iK * (RB * 4) + jb;
+#pragma unroll
+            for (int kt = 0; kt < KT; ++kt) {
+                bv[np][kt][0] = __ldg(Dl + (8 * kt + t) * 4);
+                bv[np][kt][1] = __ldg(Dl + (8 * kt + t + 4) * 4);
+            }
         }
-        float acc[MT][4];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) { acc[mt][0] = 0.f; acc[mt][1] = 0.f; acc[mt][2] = 0.f; acc[mt][3] = 0.f; }
+        for (int np = 0; np < NP; ++np) {
+            float acc[MT][4];
 #pragma unroll
-        for (int kt = 0; kt < KT; ++kt) {
-            Tf32Pair b[2];
-            b[0] = tt_split_tf32(bv[kt][0]);
-            b[1] = tt_split_tf32(bv[kt][1]);
+            for (int mt = 0; mt < MT; ++mt) { acc[mt][0] = 0.f; acc[mt][1] = 0.f; acc[mt][2] = 0.f; acc[mt][3] = 0.f; }
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt], a[mt][kt], b);
-        }
-        const uint32_t us = ub + (uint32_t)rc;
-        if (us < u1) {
-            float* e = w.E + (size_t)us * (PM * 4) + jc;
+            for (int kt = 0; kt < KT; ++kt) {
+                Tf32Pair b[2];
+                b[0] = tt_split_tf32(bv[np][kt][0]);
+                b[1] = tt_split_tf32(bv[np][kt][1]);
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                *reinterpret_cast<float2*>(e + (16 * mt + g) * 4) = make_float2(acc[mt][0], acc[mt][1]);
-                *reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4) = make_float2(acc[mt][2], acc[mt][3]);
+                for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt], a[mt][kt], b);
+            }
+            const uint32_t us = ub + 2 * np + (uint32_t)rc;
+            if (us < u1) {
+                float* e = w.E + (size_t)us * (PM * 4) + jc;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    *reinterpret_cast<float2*>(e + (16 * mt + g) * 4) = make_float2(acc[mt][0], acc[mt][1]);
+                    *reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4) = make_float2(acc[mt][2], acc[mt][3]);
+                }
             }
         }
     }
