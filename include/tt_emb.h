@@ -118,6 +118,22 @@ int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, i
  */
 int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads, tt_emb_stream_t stream);
 
+/*
+ * Forward for callers that cannot allocate device memory (no counterpart in the paper; added for embedding in
+ * hosts with a fixed memory pool, plug-ins that only receive raw pointers, and allocation-frozen regions).
+ * Same result as tt_emb_bind(core_ptrs, <workspace>) followed by tt_emb_forward(...), but the workspace is a
+ * fixed 32 MiB array inside the library (tt_emb_static_workspace_limit()); nothing is allocated.
+ *   - returns TT_EMB_ERR_WORKSPACE, launching nothing, if tt_emb_workspace_bytes(h) exceeds that limit;
+ *   - the first call on a device looks up the array's address: make it outside any stream capture;
+ *   - all calls on a device share the array (it keeps the previous call's contents; what must start at zero is
+ *     cleared by the call); calls whose GPU work overlaps (other streams, other handles) race: serialise them;
+ *   - afterwards the handle is bound to the array.
+ * core_ptrs as in tt_emb_bind; the remaining arguments as in tt_emb_forward.  Asynchronous.
+ */
+int tt_emb_forward_static(tt_emb_t h, float* const* core_ptrs, const int64_t* indices, const int64_t* offsets,
+                          int64_t batch, int64_t num_lookups, float* out, tt_emb_stream_t stream);
+size_t tt_emb_static_workspace_limit(void);
+
 /* Plain SGD on every bound core: G <- G - lr * dG, elementwise fp32.  Asynchronous. */
 int tt_emb_sgd_step(tt_emb_t h, float* const* core_grads, float lr, tt_emb_stream_t stream);
 

@@ -64,6 +64,8 @@ _SIGS = {
     "tt_emb_dim": (ctypes.c_int, [_vp, ctypes.POINTER(_i32)]),
     "tt_emb_bind": (ctypes.c_int, [_vp, _vp, _vp, ctypes.c_size_t, _vp]),
     "tt_emb_forward": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
+    "tt_emb_forward_static": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp]),
+    "tt_emb_static_workspace_limit": (ctypes.c_size_t, []),
     "tt_emb_backward": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "tt_emb_sgd_step": (ctypes.c_int, [_vp, _vp, _f32, _vp]),
     "tt_emb_status": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), _vp]),
@@ -235,6 +237,20 @@ class TTEmbeddingBag:
         self._keep = (indices, offsets)
         _check(lib.tt_emb_forward(self.h, indices.data_ptr(), offsets.data_ptr(), int(batch), int(indices.numel()),
                                   out.data_ptr(), _stream_ptr()), "tt_emb_forward")
+        return out
+
+    def forward_static(self, indices, offsets, batch: int, out=None):
+        """Forward through the library's built-in 32 MiB workspace: for callers that must not allocate device
+        memory.  Only for configurations whose workspace fits (TTEmbError with ERR_WORKSPACE otherwise).  Calls
+        must not overlap on the GPU; the handle stays bound to the built-in workspace afterwards."""
+        torch = self.torch
+        assert indices.dtype == torch.int64 and offsets.dtype == torch.int64 and indices.is_cuda and offsets.is_cuda
+        if out is None:
+            out = torch.empty((batch, self.T * self.D), dtype=torch.float32, device=self.device)
+        self._keep = (indices, offsets)
+        ptrs = (ctypes.c_void_p * (self.T * self.K))(*[c.data_ptr() for row in self.cores for c in row])
+        _check(lib.tt_emb_forward_static(self.h, ptrs, indices.data_ptr(), offsets.data_ptr(), int(batch),
+                                         int(indices.numel()), out.data_ptr(), _stream_ptr()), "tt_emb_forward_static")
         return out
 
     def backward(self, grad_out):
