@@ -113,8 +113,10 @@ int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, i
  * grad_out   device fp32[batch][T*D]
  * core_grads HOST array of T*K DEVICE pointers, each shaped like the matching core (slice-major);
  *            fully OVERWRITTEN (untouched slices become zero), not accumulated.
- * Gradients of one slice are combined by segment reductions over sorted keys, not by per-element
- * global atomics.  Needs enable_backward = 1.  Asynchronous.
+ * Lookups are sorted by row and reduced by segments (dE); first- and middle-core slices each have a single
+ * owner that sums its sorted contributions; last-core slices are accumulated with vector reductions into a
+ * few L2-resident partial copies that are then added in a fixed order.  Needs enable_backward = 1.
+ * Asynchronous.
  */
 int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads, tt_emb_stream_t stream);
 

@@ -9,9 +9,10 @@
 //             adds in position order.
 //   3. last level: per group, C is rebuilt in shared memory; every row contributes C^T.dE to the slice of
 //             the last core it selects and dE.D^T to the group's dC (summed over the rows sharing C before
-//             going up, Eq. 2).  Rows of one group select distinct slices, so a CTA-private copy of the
-//             last core's gradient in shared memory is updated without atomics; the copies are then added
-//             in a fixed order (segment reduction keyed by slice).
+//             going up, Eq. 2; the sum is the k-loop of the tensor-core product, so dC is written once).
+//             The last core's slices are accumulated with vector reductions into TT_STRIPES L2-resident
+//             partial copies, which are then added in a fixed order (shared-memory fp32 atomics measured
+//             at 2.6 per clock per SM on this part, too slow for a CTA-private copy).
 //   4. middle cores: dP_{k-1} of a parent = sum over its (contiguous) children; the gradient of slice i_k
 //             = sum over the level-k nodes with that digit, enumerated by a second, digit-major bitmap sort.
 //             Each output has exactly one owner, which sums in sorted order: no atomics.
