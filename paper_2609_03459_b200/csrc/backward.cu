@@ -244,15 +244,25 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
     acc.clear();
     acc.add_row(w.carry + ((size_t)chunk * 2 + 1) * D, D, lane);
     const int64_t nchunks = ((int64_t)Ltot + TT_DE_CHUNK - 1) / TT_DE_CHUNK;
-    for (int64_t c2 = chunk + 1; c2 < nchunks; ++c2) {
-        const uint32_t a2 = (uint32_t)(c2 * TT_DE_CHUNK);
-        const uint32_t b2 = min(a2 + (uint32_t)TT_DE_CHUNK, Ltot);
-        const uint32_t last2 = w.pairs[b2 - 1].x;
-        const uint32_t next2 = b2 < Ltot ? w.pairs[b2].x : HT_EMPTY;
-        if (last2 == last && next2 == last) {
-            acc.add_row(w.carry + ((size_t)c2 * 2 + 1) * D, D, lane);
-        } else {
-            acc.add_row(w.carry + (size_t)c2 * 2 * D, D, lane);
+    // A popular row spans thousands of chunks.  Look at 32 following chunks at once: every lane classifies one
+    // ("whole chunk is this row and it goes on" = a tail piece to add; otherwise its head piece ends the row),
+    // a ballot finds where the row ends, and the pieces are added in position order.
+    for (int64_t c0 = chunk + 1; c0 < nchunks; c0 += 32) {
+        const int64_t c2 = c0 + lane;
+        bool through = false;
+        if (c2 < nchunks) {
+            const uint32_t a2 = (uint32_t)(c2 * TT_DE_CHUNK);
+            const uint32_t b2 = min(a2 + (uint32_t)TT_DE_CHUNK, Ltot);
+            const uint32_t last2 = w.pairs[b2 - 1].x;
+            const uint32_t next2 = b2 < Ltot ? w.pairs[b2].x : HT_EMPTY;
+            through = last2 == last && next2 == last;
+        }
+        const unsigned stops = __ballot_sync(0xffffffffu, !through);   // chunks beyond the end count as stops
+        const int nthrough = stops ? __ffs(stops) - 1 : 32;
+#pragma unroll 8
+        for (int i = 0; i < nthrough; ++i) acc.add_row(w.carry + ((size_t)(c0 + i) * 2 + 1) * D, D, lane);
+        if (nthrough < 32) {
+            if (c0 + nthrough < nchunks) acc.add_row(w.carry + (size_t)(c0 + nthrough) * 2 * D, D, lane);
             break;
         }
     }
