@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
 // its own partial sum; the sub-warps are combined only when a segment ends.  Segment starts inside a batch of
 // 32 positions are found once with a ballot, so a window without a start costs 4 adds per load and nothing else.
 template <int LPR>
-__global__ void __launch_bounds__(256) k_dE_fast(WsView w, const float* __restrict__ grad_out)
+__global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __restrict__ grad_out)
 {
     constexpr int RPI = 32 / LPR, NF = 4;
     const int lane = threadIdx.x & 31, sub = lane / LPR, lr = lane % LPR;

@@ -458,7 +458,7 @@ __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableD
 }
 
 template <int LPR, int CPL>  // lanes per row, float4 chunks per lane
-__global__ void __launch_bounds__(256, (CPL == 1 ? 5 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
+__global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
 {
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPR, lr = lane % LPR;
