@@ -1,6 +1,7 @@
 // Warp-level 16x8x8 tensor-core products in "3xTF32": every fp32 operand is split into a TF32 head and a TF32
 // tail, and a.b is accumulated as a_lo.b_hi + a_hi.b_lo + a_hi.b_hi in fp32.  The dropped tail.tail term is
-// ~2^-22 relative, which keeps the contractions inside the 1e-5 tolerance (a single TF32 pass misses it ~40x).
+// ~2^-22 relative and the truncated tails ~2^-21, which keeps the contractions inside the 1e-5 tolerance (a single
+// TF32 pass misses it ~40x).
 //
 // Fragment layout of mma.sync.aligned.m16n8k8.row.col (g = lane / 4, t = lane % 4):
 //   A (16x8, row-major):  a0 = A[g][t]      a1 = A[g+8][t]    a2 = A[g][t+4]    a3 = A[g+8][t+4]
@@ -13,12 +14,16 @@ struct Tf32Pair {
     uint32_t hi, lo;
 };
 
+// head = x rounded to TF32 (10 explicit mantissa bits) with integer arithmetic on the bit pattern: add half a TF32
+// ulp, clear the 13 low bits.  tail = x - head is exact in fp32 and is handed over as it is: the tensor core reads
+// only the TF32 part of an operand register, i.e. it truncates the tail to its own top bits (error <= 2^-21 |x|).
+// cvt.rna.tf32.f32 would do the same rounding but runs on the quarter-rate conversion pipe, which made the split
+// the bottleneck of the row stage.
 __device__ __forceinline__ Tf32Pair tt_split_tf32(float x)
 {
     Tf32Pair p;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(p.hi) : "f"(x));
-    const float rest = x - __uint_as_float(p.hi);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(p.lo) : "f"(rest));
+    p.hi = (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
+    p.lo = __float_as_uint(x - __uint_as_float(p.hi));
     return p;
 }
 
