@@ -142,7 +142,7 @@ def pick_stride(wl, train: bool) -> int:
         fma += P * spec.r[k] * spec.d[k] * spec.r[k + 1]
         P *= spec.d[k]
     per_lookup = fma * (4.0 if train else 1.0)
-    budget = 15.0 * 5e9  # ~5 G fp64 FMA/s on a handful of cores
+    budget = 15.0 * 14e9  # the plain oracle sustains ~14 G fp64 FMA/s on the 16 host cores of the GPU machine
     want = max(1.0, budget / per_lookup)
     stride = int(max(1, round(wl.L / want)))
     return min(stride, max(1, wl.B // 4))
@@ -367,38 +367,73 @@ def main():
     counts = emb.grouping_counts()
     work = algorithmic_work(wl, counts, train)
 
-    # ---- roofline of the dominant kernel (stage) and of the whole step
-    def stage_roof(name, ms):
-        if name == "pooling":
-            ach = work["pool_kernel_bytes"] / (ms * 1e-3) / 1e9
-            return {"kernel": "k_pool_vec", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                    "frac": ach / hbm_gbs, "traffic": None, "peak_source": peak_src,
-                    "note": "algorithmic bytes: indices + offsets + each distinct row once + out; the per-lookup row "
-                            "gather (L*D*4 bytes, mostly L2 hits) is not counted",
-                    "l2_gather_GBs": wl.L * D * 4 / (ms * 1e-3) / 1e9, "l2_gather_peak_GBs": l2_gather / 1e9}
-        if name == "contraction":
-            ach = work["contract_slots"] / (ms * 1e-3) / 1e12
-            return {"kernel": "k_sweep_fwd", "bound": "alu", "achieved": ach, "peak": fp32_peak / 1e12,
-                    "unit": "T FP32 lane-ops/s", "frac": ach / (fp32_peak / 1e12), "traffic": None,
-                    "peak_source": "independent-FMA-chain probe in this run"}
-        if name == "bwd_dE" and train:
-            ach = work["dE_kernel_bytes"] / (ms * 1e-3) / 1e9
-            return {"kernel": "k_dE", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                    "frac": ach / hbm_gbs, "traffic": None, "peak_source": peak_src}
-        if name in ("bwd_contraction", "bwd_middle") and train:
-            slots = work["bwd_slots"] - wl.L * D
-            ach = slots / (ms * 1e-3) / 1e12
-            return {"kernel": "k_sweep_bwd" if name == "bwd_contraction" else "k_mid_slice+k_mid_down", "bound": "alu",
-                    "achieved": ach, "peak": fp32_peak / 1e12, "unit": "T FP32 lane-ops/s",
-                    "frac": ach / (fp32_peak / 1e12), "traffic": None,
-                    "peak_source": "independent-FMA-chain probe in this run",
-                    "note": "all backward contraction slots attributed to this stage (upper bound on its share)"}
-        ach = (8 * wl.L) / (ms * 1e-3) / 1e9
-        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s", "frac": ach / hbm_gbs,
-                "traffic": None, "peak_source": peak_src, "note": "algorithmic bytes: one pass over the indices"}
+    # ---- roofline of the dominant kernel and of the whole step
+    # DRAM traffic per lookup / per distinct row of the top kernels, from the ncu capture of the reduced case
+    # (8 tables; profiles/ncu_full_cfg5_reduced.md), scaled to this launch by the units it processes.
+    NCU_TRAFFIC = {"k_pool_vec": ("lookup", 124.5), "k_dE_fast": ("lookup", 71.9),
+                   "k_sweep_fwd": ("row", 226.6), "k_sweep_bwd": ("row", 364.0)}
 
-    dominant = max(stage_ms, key=stage_ms.get) if stage_ms else "pooling"
-    roofline = stage_roof(dominant, stage_ms.get(dominant, ms_per_step))
+    def traffic_of(kernel, share=1.0):
+        unit, per = NCU_TRAFFIC[kernel]
+        return per * (wl.L if unit == "lookup" else work["U_rows"] * share)
+
+    variant_rows = {}   # distinct rows handled by each sweep variant
+    for t, s in enumerate(wl.tables):
+        v = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4}.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
+            if (s.d[-1] == 4 and K >= 3) else -1
+        variant_rows[v] = variant_rows.get(v, 0) + int(counts[t, K - 1])
+
+    def variant_slots(v, backward):
+        tot = 0
+        for t, s in enumerate(wl.tables):
+            vv = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4}.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
+                if (s.d[-1] == 4 and K >= 3) else -1
+            if vv != v:
+                continue
+            P = int(np.prod(s.d[:K - 2])) if K >= 3 else 1
+            c_mid = P * s.r[K - 2] * s.d[K - 2] * s.r[K - 1] if K >= 3 else 0
+            c_last = int(np.prod(s.d[:K - 1])) * s.r[K - 1] * s.d[K - 1]
+            g, u = int(counts[t, K - 2]), int(counts[t, K - 1])
+            tot += (g * c_mid + 2 * u * c_last) if backward else (g * c_mid + u * c_last)
+        return tot
+
+    kernels = {}
+    if "pooling" in stage_ms:
+        ms = stage_ms["pooling"]
+        ach = work["pool_kernel_bytes"] / (ms * 1e-3) / 1e9
+        kernels["k_pool_vec"] = (ms, {"kernel": "k_pool_vec", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                                      "frac": ach / hbm_gbs, "traffic": traffic_of("k_pool_vec"), "peak_source": peak_src,
+                                      "note": "algorithmic bytes: indices + offsets + every distinct row once + out "
+                                              "(+ one (slot,bag) pair per lookup when the backward is enabled); the "
+                                              "per-lookup row gather (L*D*4 bytes) is on-chip / re-read traffic and is "
+                                              "not counted; traffic scaled from the reduced-case ncu capture",
+                                      "row_gather_GBs": wl.L * D * 4 / (ms * 1e-3) / 1e9,
+                                      "row_gather_peak_l2_GBs": l2_gather / 1e9, "row_gather_peak_hbm_GBs": hbm_gather / 1e9})
+    if train and "bwd_dE" in stage_ms:
+        ms = stage_ms["bwd_dE"]
+        ach = work["dE_kernel_bytes"] / (ms * 1e-3) / 1e9
+        kernels["k_dE_fast"] = (ms, {"kernel": "k_dE_fast (+k_dE_fix)", "bound": "hbm", "achieved": ach, "peak": hbm_gbs,
+                                     "unit": "GB/s", "frac": ach / hbm_gbs, "traffic": traffic_of("k_dE_fast"),
+                                     "peak_source": peak_src})
+    for name, ms in stage_ms.items():
+        if name.startswith("k_sweep_"):
+            v = int(name[name.index("<") + 1:name.index(">")])
+            bwd = name.startswith("k_sweep_bwd")
+            slots = variant_slots(v, bwd)
+            ach = slots / (ms * 1e-3) / 1e12
+            share = variant_rows.get(v, 0) / max(work["U_rows"], 1)
+            kernels[name] = (ms, {"kernel": name, "bound": "alu", "achieved": ach, "peak": fp32_peak / 1e12,
+                                  "unit": "T FP32 lane-ops/s", "frac": ach / (fp32_peak / 1e12),
+                                  "traffic": traffic_of("k_sweep_bwd" if bwd else "k_sweep_fwd", share),
+                                  "peak_source": "independent-FMA-chain probe in this run",
+                                  "note": "FMA-equivalent slots of the contractions this kernel performs; the row stages "
+                                          "run as 3xTF32 tensor-core products, the peak is the FP32 pipe"})
+    if kernels:
+        dominant = max(kernels, key=lambda k: kernels[k][0])
+        roofline = dict(kernels[dominant][1], ms_per_launch=kernels[dominant][0])
+    else:
+        roofline = None
+    kernel_rooflines = {k: {"ms": v[0], "frac": v[1]["frac"], "bound": v[1]["bound"]} for k, v in kernels.items()}
     tot_slots = work["fwd_slots"] + (work["bwd_slots"] if train else 0)
     tot_bytes = work["fwd_hbm_bytes"] + (work["bwd_hbm_bytes"] if train else 0)
     t_alu, t_hbm = tot_slots / fp32_peak, tot_bytes / (hbm_gbs * 1e9)
@@ -419,7 +454,7 @@ def main():
                    "l2_policy": "inputs larger than L2 (indices alone are %.0f MB)" % (L * 8 / 1e6)},
         "forward_only": {"value": world * L / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,
                          "roofline_frac": fwd_roof_t * 1e3 / fwd_ms, "t_roof_ms": fwd_roof_t * 1e3},
-        "stage_ms": stage_ms, "roofline": roofline, "step_roofline": step_roof,
+        "stage_ms": stage_ms, "roofline": roofline, "kernel_rooflines": kernel_rooflines, "step_roofline": step_roof,
         "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
                   "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},
         "work": work, "device_status": status, "clocks": clocks, "e2e": e2e,

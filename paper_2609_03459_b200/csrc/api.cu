@@ -345,6 +345,20 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
 
 // ------------------------------------------------------------------------------------------------ timing helpers
 
+cudaError_t tt_stage_begin(tt_emb* h, int stage, cudaStream_t s)
+{
+    if (!h->timing || !h->ev_created) return cudaSuccess;
+    return cudaEventRecord(h->ev[stage][0], s);
+}
+
+cudaError_t tt_stage_end(tt_emb* h, int stage, cudaStream_t s)
+{
+    if (!h->timing || !h->ev_created) return cudaSuccess;
+    cudaError_t e = cudaEventRecord(h->ev[stage][1], s);
+    if (e == cudaSuccess) h->ev_valid[stage] = true;
+    return e;
+}
+
 static int stage_begin(tt_emb* h, int stage, cudaStream_t s)
 {
     if (!h->timing) return TT_EMB_OK;
@@ -403,6 +417,7 @@ extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t*
     v.indices = indices; v.offsets = offsets;
     h->have_forward = false;
     for (int i = 0; i < 4; ++i) h->ev_valid[i] = false;
+    for (int i = 9; i < 15; ++i) h->ev_valid[i] = false;
     TT_STAGE(h, 0, s, tt_launch_grouping(h, s));
     TT_STAGE(h, 1, s, tt_launch_schedule(h, s));
     TT_STAGE(h, 2, s, tt_launch_contraction(h, s));
@@ -432,6 +447,7 @@ extern "C" int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* 
     int r = upload_grads(h, core_grads, s);
     if (r) return r;
     for (int i = 4; i < 8; ++i) h->ev_valid[i] = false;
+    for (int i = 15; i < 21; ++i) h->ev_valid[i] = false;
     TT_STAGE(h, 4, s, tt_launch_bwd_sort(h, s));
     TT_STAGE(h, 5, s, tt_launch_bwd_dE(h, grad_out, s));
     TT_STAGE(h, 6, s, tt_launch_bwd_contraction(h, s));

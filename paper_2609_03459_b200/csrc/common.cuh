@@ -11,7 +11,7 @@
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
 #define TT_DE_CHUNK 256                                  // sorted lookups per warp in the dE segment reduction
-#define TT_NUM_STAGES 9
+#define TT_NUM_STAGES 21                                // 0..8 pipeline stages, 9..14 forward sweep variants, 15..20 backward sweep variants
 #define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
 #define TT_NUM_VARIANTS 5                                // register-tiled shape variants (forward.cu)
 
@@ -109,6 +109,10 @@ struct tt_emb {
     bool ev_valid[TT_NUM_STAGES];
     bool ev_created;
 };
+
+// stage timing (api.cu): no-ops unless timing is enabled
+cudaError_t tt_stage_begin(tt_emb* h, int stage, cudaStream_t s);
+cudaError_t tt_stage_end(tt_emb* h, int stage, cudaStream_t s);
 
 // ---- launchers implemented in the .cu files (all enqueue on `s`, return cudaGetLastError()) ----
 cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s);

@@ -405,7 +405,9 @@ static cudaError_t launch_sweep_fwd(tt_emb* h, int max_pl, int max_c, cudaStream
     const size_t smem = (size_t)4 * (max_pl + max_c) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_sweep_fwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    if ((e = tt_stage_begin(h, 9 + V + 1, s)) != cudaSuccess) return e;
     k_sweep_fwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    if ((e = tt_stage_end(h, 9 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
