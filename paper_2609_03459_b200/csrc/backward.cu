@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 #pragma unroll
         for (int j = 0; j < HT_TILE / 256; ++j) {
             const int64_t l = tile * HT_TILE + j * 256 + threadIdx.x;
-            pr[j] = l < L ? __ldg(upairs + l) : make_uint2(HT_EMPTY, 0u);
+            pr[j] = l < L ? __ldcs(upairs + l) : make_uint2(HT_EMPTY, 0u);
             if (pr[j].x >= capK || (int64_t)pr[j].y >= w.B) pr[j].x = HT_EMPTY;  // invalid lookup (or malformed offsets)
         }
 #pragma unroll
@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
     };
     uint32_t last_slot = cur;  // slot of the position before the current batch
     for (uint32_t p0 = a; p0 < b; p0 += 32) {
-        const uint2 mine = (p0 + lane < b) ? __ldg(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
+        const uint2 mine = (p0 + lane < b) ? __ldcs(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
         const int n = (int)min(32u, b - p0);
         // row index of this lane's pair inside grad_out viewed as [B*T][D]
         const uint32_t grow = lane < n ? mine.y * (uint32_t)w.T + (uint32_t)tt_find_table(w.tb[w.K], w.T, mine.x) : 0u;

@@ -295,8 +295,8 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
                 float* e = w.E + (size_t)us * (PM * 4) + jc;
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
-                    *reinterpret_cast<float2*>(e + (16 * mt + g) * 4) = make_float2(acc[mt][0], acc[mt][1]);
-                    *reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4) = make_float2(acc[mt][2], acc[mt][3]);
+                    __stcs(reinterpret_cast<float2*>(e + (16 * mt + g) * 4), make_float2(acc[mt][0], acc[mt][1]));
+                    __stcs(reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4), make_float2(acc[mt][2], acc[mt][3]));
                 }
             }
         }
@@ -447,7 +447,7 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
 // __shfl_xor at the end.
 __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableDesc& td, int64_t l, uint32_t capK)
 {
-    const int64_t g = __ldg(w.indices + l);
+    const int64_t g = __ldcs(w.indices + l);   // streamed once: evict-first, keeps L2 for rows and rank words
     uint32_t slot = 0xffffffffu;
     if (g >= 0 && g < td.N) {
         const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
@@ -509,7 +509,7 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
             slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
         for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
-            if (w.upairs && l0 + lane < o_hi) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);  // kept for the backward sort
+            if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));  // kept for the backward sort
             if (l0 + 32 < o_hi) slot_next = (l0 + 32 + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], l0 + 32 + lane, capK) : 0xffffffffu;
             else if (has_next) slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
             const int n = (int)min((int64_t)32, o_hi - l0);
@@ -552,13 +552,119 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 const int ch = lr + c * LPR;
-                if (ch < D4) o4[ch] = acc[c];
+                if (ch < D4) __stcs(o4 + ch, acc[c]);
             }
         }
         o_lo = o_hi;
         o_hi = n_hi;
         t = tn;
     }
+}
+
+// Rows of up to 256 bytes (D <= 64): the gather is bound by bytes in flight, and registers cap what LDG can keep in
+// flight.  Here every warp owns an 8 KB shared-memory buffer and fills it with cp.async (16 bytes per lane, two
+// rows per instruction, no staging registers): the 32 rows of a batch are all in flight at once.  Same bag
+// partition (equal shares of the lookups per warp), same prefetch of the next batch's rank look-ups.
+__device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
+__global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restrict__ out)
+{
+    extern __shared__ __align__(16) float4 pool_buf[];   // [8 warps][32 rows][16 float4]
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int sub = lane >> 4, lr = lane & 15;
+    float4* buf = pool_buf + (size_t)wid * 32 * 16;
+    const int D4 = w.D >> 2;
+    const bool lane_on = lr < D4;
+    const int64_t nb = (int64_t)w.T * w.B;
+    const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
+    const uint32_t capK = w.cap[w.K];
+    const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int64_t b0, b1;
+    {
+        const int64_t target = lane == 0 ? (w.L * wi) / W : (w.L * (wi + 1)) / W;
+        int64_t lo = 0, hi = nb;
+        if (lane < 2)
+            while (lo < hi) {
+                const int64_t mid = (lo + hi) >> 1;
+                if (__ldg(w.offsets + mid) < target) lo = mid + 1; else hi = mid;
+            }
+        b0 = __shfl_sync(0xffffffffu, lo, 0);
+        b1 = __shfl_sync(0xffffffffu, lo, 1);
+        if (wi == 0) b0 = 0;
+        if (wi == W - 1) b1 = nb;
+    }
+    if (b0 >= b1) return;
+    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
+    if (o_hi < o_lo) o_hi = o_lo;
+    int t = (int)(b0 / w.B);
+    uint32_t slot_next = (o_lo + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], o_lo + lane, capK) : 0xffffffffu;
+    for (int64_t bag = b0; bag < b1; ++bag) {
+        const int64_t b = bag - (int64_t)t * w.B;
+        const bool has_next = bag + 1 < b1;
+        int64_t n_hi = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_hi;
+        if (n_hi < o_hi) n_hi = o_hi;
+        const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (o_lo >= o_hi && has_next)
+            slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+        for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
+            const uint32_t slot = slot_next;
+            if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));
+            const int n = (int)min((int64_t)32, o_hi - l0);
+            const unsigned valid = __ballot_sync(0xffffffffu, lane < n && slot != 0xffffffffu);
+            // all rows of the batch in flight
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+                const int j = 2 * jj + sub;
+                const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
+                if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * 16 + lr, E4 + (size_t)sl * D4 + lr);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            // the rank look-ups of the next batch (or of the next bag) overlap the gather
+            if (l0 + 32 < o_hi) slot_next = (l0 + 32 + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], l0 + 32 + lane, capK) : 0xffffffffu;
+            else if (has_next) slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+                const int j = 2 * jj + sub;
+                if (((valid >> j) & 1u) && lane_on) {
+                    const float4 v = buf[j * 16 + lr];
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+            }
+            __syncwarp();
+        }
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+        if (sub == 0 && lane_on) __stcs(reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr, acc);
+        o_lo = o_hi;
+        o_hi = n_hi;
+        t = tn;
+    }
+}
+
+static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
+{
+    const size_t smem = (size_t)8 * 32 * 16 * sizeof(float4);
+    cudaError_t e = cudaFuncSetAttribute(k_pool_async, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async, 256, smem)) != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const int64_t nb = (int64_t)h->v.T * h->v.B;
+    int64_t grid = (int64_t)per_sm * h->sm_count;
+    const int64_t need = (nb + 7) / 8;
+    if (grid > need) grid = need;
+    if (grid < 1) grid = 1;
+    k_pool_async<<<(int)grid, 256, smem, s>>>(h->v, out);
+    return cudaGetLastError();
 }
 
 template <int LPR, int CPL>
@@ -647,6 +753,7 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
     }
     const int D4 = D / 4;
     (void)grid;
+    if (D4 > 8 && D4 <= 16) return launch_pool_async(h, out, s);
     if (D4 <= 4) return launch_pool_vec<4, 1>(h, out, s);
     if (D4 <= 8) return launch_pool_vec<8, 1>(h, out, s);
     if (D4 <= 16) return launch_pool_vec<16, 1>(h, out, s);
