@@ -81,10 +81,12 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
             rk[j] = atomicAdd(&vals[p], 1u);
         }
         __syncthreads();
+        // one global atomic per distinct row of the tile.  MODE 1 claims a run of positions directly on the scanned
+        // count array: cnt[slot] starts as the segment start and ends as the segment end (= next segment's start)
         for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) {
             if (keys[i] != HT_EMPTY) {
                 if (MODE == 0) atomicAdd(&w.cnt[keys[i]], vals[i]);
-                else vals[i] = atomicAdd(&w.cursor[keys[i]], vals[i]);
+                else vals[i] = atomicAdd(&w.cnt[keys[i]], vals[i]);
             }
         }
         if (MODE == 1) {
@@ -92,8 +94,7 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 #pragma unroll
             for (int j = 0; j < HT_TILE / 256; ++j) {
                 if (pr[j].x == HT_EMPTY) continue;
-                const uint32_t pos = w.cnt[pr[j].x] + vals[hh[j]] + rk[j];
-                w.pairs[pos] = pr[j];
+                w.pairs[vals[hh[j]] + rk[j]] = pr[j];
             }
         }
         __syncthreads();
@@ -113,15 +114,20 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
     WsView& w = h->v;
     const int zgrid = h->sm_count * 8;
     k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cnt, w.counters + CTR_LEVEL0 + w.K, 1u);
-    k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cursor, w.counters + CTR_LEVEL0 + w.K, 0u);
     const int64_t ntiles = (w.L + HT_TILE - 1) / HT_TILE;
-    int grid = (int)(ntiles < (int64_t)h->sm_count * 6 ? ntiles : (int64_t)h->sm_count * 6);
-    if (grid < 1) grid = 1;
-    k_sort_pass<0><<<grid, 256, 0, s>>>(w);
+    cudaError_t e;
+    int per_sm0 = 0, per_sm1 = 0;   // persistent grids sized to what is actually resident (no partial second wave)
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm0, k_sort_pass<0>, 256, 0)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm1, k_sort_pass<1>, 256, 0)) != cudaSuccess) return e;
+    auto grid_of = [&](int per_sm) {
+        int64_t g = (int64_t)(per_sm < 1 ? 1 : per_sm) * h->sm_count;
+        if (g > ntiles) g = ntiles;
+        return (int)(g < 1 ? 1 : g);
+    };
+    k_sort_pass<0><<<grid_of(per_sm0), 256, 0, s>>>(w);
     CntScan cs{w};
-    cudaError_t e = tt_scan(cs, w.cap[w.K], w.scan_tmp, s);
-    if (e != cudaSuccess) return e;
-    k_sort_pass<1><<<grid, 256, 0, s>>>(w);
+    if ((e = tt_scan(cs, w.cap[w.K], w.scan_tmp, s)) != cudaSuccess) return e;
+    k_sort_pass<1><<<grid_of(per_sm1), 256, 0, s>>>(w);
     return cudaGetLastError();
 }
 
