@@ -232,6 +232,10 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->off_cost = take(((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
     for (int k = 2; k <= K - 2; ++k) h->off_pbuf[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
     h->off_E = take((size_t)h->capU * D * sizeof(float));
+    for (int k = 2; k <= K - 1; ++k) {   // digit-major node lists: level K-1 orders the sweeps, the others serve the backward
+        h->off_tbm[k] = take((size_t)twords[k] * sizeof(uint2));
+        h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+    }
     if (h->enable_backward) {
         h->off_cnt = take(((size_t)h->capU + 1) * sizeof(uint32_t));
         h->off_cursor = take((size_t)h->capU * sizeof(uint32_t));
@@ -239,8 +243,6 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         for (int k = 2; k <= K - 1; ++k) {
             h->off_dP[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
             h->off_Y[k] = take((size_t)v.cap[k] * stride[k - 1] * sizeof(float));
-            h->off_tbm[k] = take((size_t)twords[k] * sizeof(uint2));
-            h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
         }
         h->off_carry = take(((size_t)(h->max_lookups / TT_DE_CHUNK) + 2) * 2 * D * sizeof(float));
         h->off_gpart = take((size_t)TT_STRIPES * (size_t)(gpart > 0 ? gpart : 4) * sizeof(float));
@@ -319,6 +321,10 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     for (int k = 2; k <= K - 2; ++k) v.pbuf[k] = (float*)(base + h->off_pbuf[k]);
     v.E = (float*)(base + h->off_E);
     v.upairs = nullptr;
+    for (int k = 2; k <= K - 1; ++k) {
+        v.tbm[k] = (uint2*)(base + h->off_tbm[k]);
+        v.tnode[k] = (uint32_t*)(base + h->off_tnode[k]);
+    }
     if (h->enable_backward) {
         v.cnt = (uint32_t*)(base + h->off_cnt);
         v.cursor = (uint32_t*)(base + h->off_cursor);
@@ -327,8 +333,6 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
         for (int k = 2; k <= K - 1; ++k) {
             v.dP[k] = (float*)(base + h->off_dP[k]);
             v.Y[k] = (float*)(base + h->off_Y[k]);
-            v.tbm[k] = (uint2*)(base + h->off_tbm[k]);
-            v.tnode[k] = (uint32_t*)(base + h->off_tnode[k]);
         }
         v.carry = (float*)(base + h->off_carry);
         v.gpart = (float*)(base + h->off_gpart);

@@ -450,7 +450,8 @@ __device__ __forceinline__ void tt_sweep_bwd_generic(const WsView& w, const Tabl
     const uint32_t nK = (uint32_t)td.n[kl];
     for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) dCs[i] = 0.f;
     __syncthreads();
-    for (uint32_t g = g0; g < g1; ++g) {
+    for (uint32_t jpos = g0; jpos < g1; ++jpos) {
+        const uint32_t g = K >= 3 ? w.tnode[K - 1][jpos] : jpos;
         const uint32_t val = w.val[K - 1][g];
         if (K >= 3) {
             const int M = td.P[km], ra = td.r[km], cols = td.d[km] * rb;
@@ -788,7 +789,8 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
     const int K = w.K, km = K - 2;
     const int ra = td.r[km], cols = td.d[km] * RB_;
     const uint32_t nK = (uint32_t)td.n[K - 1];
-    for (uint32_t g = g0 + wid; g < g1; g += nw) {
+    for (uint32_t j = g0 + wid; j < g1; j += nw) {
+        const uint32_t g = w.tnode[K - 1][j];   // units are cut from the digit-major order (see forward.cu)
         const uint32_t val = w.val[K - 1][g];
         const float* src = tt_left_operand_b(w, td, K - 1, g);
         for (int i = lane; i < M * ra; i += 32) {
@@ -1177,6 +1179,21 @@ __global__ void __launch_bounds__(256) k_mid_sum(WsView w, int k)
     }
 }
 
+// Digit-major ("transposed") list of the level-k nodes: a second presence-bitmap sort, keyed by
+// (i_k, parent prefix) instead of (parent prefix, i_k); tnode[k][rank] = node.
+cudaError_t tt_launch_tlist(tt_emb* h, int k, cudaStream_t s)
+{
+    WsView& w = h->v;
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
+    const int g = h->sm_count * 8;
+    k_tmark<<<g, 256, 0, s>>>(w, k);
+    TPopScan tp{w, k};
+    if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
+    k_tfill<<<g, 256, 0, s>>>(w, k);
+    return cudaGetLastError();
+}
+
 cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
@@ -1193,12 +1210,8 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
             if (M * ra + M * cols > max_slice) max_slice = M * ra + M * cols;
             if (td.midfast[k] < 0) any_generic = true; else any_fast[td.midfast[k]] = true;
         }
-        if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
-        const int g = h->sm_count * 8;
-        k_tmark<<<g, 256, 0, s>>>(w, k);
-        TPopScan tp{w, k};
-        if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
-        k_tfill<<<g, 256, 0, s>>>(w, k);
+        // level K-1's digit-major list already exists: the forward built it to order its sweep
+        if (k != h->K - 1 && (e = tt_launch_tlist(h, k, s)) != cudaSuccess) return e;
         const dim3 sg(max_n, h->T);
         if (any_fast[0]) k_mid_fused<32, 128><<<sg, 128, 0, s>>>(w, k, 0);
         if (any_fast[1]) k_mid_fused<16, 128><<<sg, 128, 0, s>>>(w, k, 1);

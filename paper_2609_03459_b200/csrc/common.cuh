@@ -117,6 +117,7 @@ cudaError_t tt_stage_end(tt_emb* h, int stage, cudaStream_t s);
 // ---- launchers implemented in the .cu files (all enqueue on `s`, return cudaGetLastError()) ----
 cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s);
 cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s);
+cudaError_t tt_launch_tlist(tt_emb* h, int k, cudaStream_t s);   // digit-major list of the level-k nodes
 cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s);
 cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s);
 cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s);

@@ -19,10 +19,13 @@ struct CostScan {
     WsView w;
     int shift;
     __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + w.K - 1]; }
-    __device__ uint32_t value(uint32_t g) const
+    __device__ uint32_t value(uint32_t j) const
     {
+        // position j of the sweep order: digit-major for K >= 3 (groups that share the big slice of core K-1 are
+        // neighbours, so that slice is fetched from L2 once per run instead of once per group), natural for K = 2
         const int K = w.K;
-        const int t = tt_find_table(w.tb[K - 1], w.T, g);
+        const int t = tt_find_table(w.tb[K - 1], w.T, j);
+        const uint32_t g = K >= 3 ? w.tnode[K - 1][j] : j;
         const TableDesc& td = w.tdesc[t];
         const uint32_t nchild = w.cstart[K - 1][g + 1] - w.cstart[K - 1][g];
         // c_k = P_{k-1} r_{k-1} d_k r_k
@@ -41,6 +44,10 @@ struct CostScan {
 
 cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s)
 {
+    if (h->K >= 3) {
+        cudaError_t e = tt_launch_tlist(h, h->K - 1, s);
+        if (e != cudaSuccess) return e;
+    }
     // cost unit: 2^shift FMAs, chosen at create time so that the worst-case total fits 32 bits
     CostScan cs{h->v, h->cost_shift};
     return tt_scan(cs, h->v.cap[h->v.K - 1], h->v.scan_tmp, s);
@@ -316,6 +323,7 @@ __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& 
         if (lane == 0) g = atomicAdd(next, 1u);
         g = __shfl_sync(0xffffffffu, g, 0);
         if (g >= g1) break;
+        g = w.tnode[K - 1][g];   // position in the digit-major order -> group
         const uint32_t val = w.val[K - 1][g];
         const float* src = tt_left_operand(w, td, K - 1, g);
         for (int i = lane; i < M * ra; i += 32) {
@@ -338,7 +346,8 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
     const int K = w.K, kl = K - 1, km = K - 2;
     const int Pm = td.P[K - 1], rb = td.r[K - 1], dK = td.d[kl], D = w.D;
     const uint32_t nK = (uint32_t)td.n[kl];
-    for (uint32_t g = g0; g < g1; ++g) {
+    for (uint32_t jpos = g0; jpos < g1; ++jpos) {
+        const uint32_t g = K >= 3 ? w.tnode[K - 1][jpos] : jpos;
         const uint32_t val = w.val[K - 1][g];
         if (K >= 3) {
             const int M = td.P[km], ra = td.r[km], cols = td.d[km] * rb;
