@@ -782,6 +782,112 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
     }
 }
 
+// Both row passes in one loop over the group's row pairs: the row ids and the dE rows come from memory once (the
+// second fragment layout of dE is served by L1), dC accumulates across the loop, dG_K tiles leave per pair.
+template <int PM, int RB_>
+__device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
+                                                     uint32_t row_base, float* dPdst, float* gk, int lane)
+{
+    constexpr int MT = PM / 16, NT = RB_ / 8;     // dC tiles: rows p, columns b
+    constexpr int MT2 = RB_ / 16, KT2 = PM / 8;   // dG tiles: rows b, k = p
+    const int g = lane >> 2, t = lane & 3;
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    Tf32Pair ct[MT2][KT2][4];   // A[m = b][k = p] = C[p][b]
+#pragma unroll
+    for (int mt = 0; mt < MT2; ++mt)
+#pragma unroll
+        for (int kt = 0; kt < KT2; ++kt) {
+            ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g]);
+            ct[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g + 8]);
+            ct[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g]);
+            ct[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g + 8]);
+        }
+    float dc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { dc[mt][nt][0] = 0.f; dc[mt][nt][1] = 0.f; dc[mt][nt][2] = 0.f; dc[mt][nt][3] = 0.f; }
+    const int rb_ = g >> 2, jb = g & 3;       // dG B fragment: row rb_ of the pair, column jb of dE
+    const int rc = t >> 1, jc = 2 * (t & 1);  // dG C fragment: row rc of the pair, columns jc, jc+1
+    for (uint32_t ub = u0; ub < u1; ub += 2) {
+        const bool two = ub + 1 < u1;
+        const uint32_t ua = ub, uc = two ? ub + 1 : ub;
+        const uint32_t iKa = rows[ua] - row_base, iKc = rows[uc] - row_base;
+        const float* __restrict__ Ea = w.E + (size_t)ua * (PM * 4);
+        const float* __restrict__ Ec = w.E + (size_t)uc * (PM * 4);
+        // ---- loads: dE as A fragments (dC), slices as B fragments (dC), dE as B fragments (dG)
+        float av[MT][4], bv[NT][2], ev[KT2][2];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            av[mt][0] = __ldg(Ea + (16 * mt + g) * 4 + t);
+            av[mt][1] = __ldg(Ea + (16 * mt + g + 8) * 4 + t);
+            av[mt][2] = two ? __ldg(Ec + (16 * mt + g) * 4 + t) : 0.f;
+            av[mt][3] = two ? __ldg(Ec + (16 * mt + g + 8) * 4 + t) : 0.f;
+        }
+        const float* __restrict__ Da = GK + (size_t)iKa * (RB_ * 4) + t;
+        const float* __restrict__ Dc = GK + (size_t)iKc * (RB_ * 4) + t;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            bv[nt][0] = __ldg(Da + (8 * nt + g) * 4);
+            bv[nt][1] = __ldg(Dc + (8 * nt + g) * 4);
+        }
+        const bool valid = rb_ == 0 || two;
+        const float* __restrict__ El = (rb_ == 0 ? Ea : Ec) + jb;
+#pragma unroll
+        for (int kt = 0; kt < KT2; ++kt) {
+            ev[kt][0] = valid ? __ldg(El + (8 * kt + t) * 4) : 0.f;
+            ev[kt][1] = valid ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
+        }
+        // ---- dC += dE . D^T
+        {
+            Tf32Pair a[MT][4];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) a[mt][x] = tt_split_tf32(av[mt][x]);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                Tf32Pair b[2];
+                b[0] = tt_split_tf32(bv[nt][0]);
+                b[1] = tt_split_tf32(bv[nt][1]);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(dc[mt][nt], a[mt], b);
+            }
+        }
+        // ---- dG_K[i_K] += C^T . dE
+        {
+            float acc[MT2][4];
+#pragma unroll
+            for (int mt = 0; mt < MT2; ++mt) { acc[mt][0] = 0.f; acc[mt][1] = 0.f; acc[mt][2] = 0.f; acc[mt][3] = 0.f; }
+#pragma unroll
+            for (int kt = 0; kt < KT2; ++kt) {
+                Tf32Pair b[2];
+                b[0] = tt_split_tf32(ev[kt][0]);
+                b[1] = tt_split_tf32(ev[kt][1]);
+#pragma unroll
+                for (int mt = 0; mt < MT2; ++mt) tt_mma_3xtf32(acc[mt], ct[mt][kt], b);
+            }
+            if (rc == 0 || two) {
+                float* dst = gk + (size_t)(rc == 0 ? iKa : iKc) * (RB_ * 4) + jc;
+#pragma unroll
+                for (int mt = 0; mt < MT2; ++mt) {
+                    tt_red_v2(dst + (16 * mt + g) * 4, acc[mt][0], acc[mt][1]);
+                    tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dc[mt][nt][0], dc[mt][nt][1]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dc[mt][nt][2], dc[mt][nt][3]);
+        }
+}
+
 template <int PM, int RB_, int TP, int M, int CPL, bool MMA>
 __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* gk,
                                                   float* As, float* Cs, int lane, int wid, int nw)
@@ -803,8 +909,14 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
         __syncwarp();
         const uint32_t u0 = w.cstart[K - 1][g], u1 = w.cstart[K - 1][g + 1];
         if constexpr (MMA) {
-            tt_warp_rows_dC_mma<PM, RB_>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
-            tt_warp_rows_dG_mma<PM, RB_>(Cs, w, u0, u1, val * nK, gk, lane);
+            // small C (rank 16): one fused loop over the row pairs is faster; larger C: two passes keep the register
+            // footprint low enough for twice the resident warps (measured on the 60-table configuration)
+            if constexpr (PM * RB_ <= 256) {
+                tt_warp_rows_bwd_mma<PM, RB_>(Cs, w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], gk, lane);
+            } else {
+                tt_warp_rows_dC_mma<PM, RB_>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
+                tt_warp_rows_dG_mma<PM, RB_>(Cs, w, u0, u1, val * nK, gk, lane);
+            }
         } else {
             tt_warp_rows_dC<PM, RB_, TP>(w, td, u0, u1, val * nK, w.dP[K - 1] + (size_t)g * w.stride[K - 1], lane);
             tt_warp_rows_dG<PM, RB_, TP>(Cs, w, u0, u1, val * nK, gk, lane);
