@@ -348,12 +348,35 @@ def main():
     # ---- end to end through host buffers
     e2e = None
     if not args.no_e2e:
+        # the call a user makes with host buffers: indices/offsets go up first, grad_out goes up on a second
+        # stream while the forward runs, `out` comes down while the backward runs
+        copy_stream = torch.cuda.Stream(device)
+        e_idx, e_off = torch.empty_like(d_idx), torch.empty_like(d_off)
+        e_grad = torch.empty_like(d_grad) if train else None
+
         def e2e_step():
-            idx = h_idx.to(device, non_blocking=True)
-            off = h_off.to(device, non_blocking=True)
-            grad = h_grad.to(device, non_blocking=True) if train else None
-            step(idx, off, grad)
-            h_out.copy_(d_out, non_blocking=True)
+            main = torch.cuda.current_stream()
+            e_idx.copy_(h_idx, non_blocking=True)
+            e_off.copy_(h_off, non_blocking=True)
+            ev_in = main.record_event()
+            ev_grad = None
+            if train:
+                copy_stream.wait_event(ev_in)
+                with torch.cuda.stream(copy_stream):
+                    e_grad.copy_(h_grad, non_blocking=True)
+                    ev_grad = copy_stream.record_event()
+            emb.forward(e_idx, e_off, B, out=d_out)
+            ev_fwd = main.record_event()
+            copy_stream.wait_event(ev_fwd)
+            with torch.cuda.stream(copy_stream):
+                h_out.copy_(d_out, non_blocking=True)
+                ev_out = copy_stream.record_event()
+            if train:
+                main.wait_event(ev_grad)
+                emb.backward(e_grad)
+                ttd.allreduce_core_grads(emb.flat_grads)
+                emb.sgd_step(wl.lr)
+            main.wait_event(ev_out)
         for _ in range(2):
             e2e_step()
         e2e_ms = timed(e2e_step, args.steps) / args.steps
