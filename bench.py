@@ -230,6 +230,8 @@ def main():
     ap.add_argument("--cpu-stride", type=int, default=0, help="bag stride of the oracle sample (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--ablation", default="none", choices=["none", "unique-only", "static", "unique-only+static"],
+                    help="study switches (forward workloads only): no prefix reuse / equal-count schedule")
     ap.add_argument("--num-tables", type=int, default=0, help="reduced case for profiler captures: fewer tables (cfg3/cfg5)")
     ap.add_argument("--batch", type=int, default=0, help="reduced case for profiler captures: smaller batch")
     args = ap.parse_args()
@@ -269,7 +271,10 @@ def main():
         wl = workloads.make(cfg_id, mapping=args.mapping, batch_seed=ttd.rank_seed(workloads.BASE_SEED, rank), **shrink)
     T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
 
-    emb = binding.from_workload(wl, enable_backward=train, device=device)
+    abl = {"none": 0, "unique-only": 1, "static": 2, "unique-only+static": 3}[args.ablation]
+    if abl and train:
+        raise SystemExit("--ablation needs a forward workload (cfg1..cfg4)")
+    emb = binding.from_workload(wl, enable_backward=train, ablation=abl, device=device)
     h_idx = torch.from_numpy(wl.indices).pin_memory()
     h_off = torch.from_numpy(wl.offsets).pin_memory()
     h_grad = torch.from_numpy(wl.grad_out).pin_memory() if train else None
@@ -472,7 +477,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": desc, "mapping": args.mapping, "tables": T, "batch_per_gpu": B, "lookups_per_gpu": L,
-                   "step": "forward+backward+sgd" if train else "forward",
+                   "step": "forward+backward+sgd" if train else "forward", "ablation": args.ablation,
                    "parallelism": f"dp{world} (batch-sharded replicas" + (", all-reduce of core gradients)" if train else ")"),
                    "l2_policy": "inputs larger than L2 (indices alone are %.0f MB)" % (L * 8 / 1e6)},
         "forward_only": {"value": world * L / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,

@@ -71,7 +71,11 @@ typedef struct {
     int64_t max_lookups;        /* upper bound on `num_lookups` (all tables together) */
     int64_t max_unique_rows;    /* upper bound on distinct (table,row) pairs per call; 0 = min(max_lookups, sum N_t) */
     int32_t enable_backward;    /* 0: forward only (smaller workspace); 1: tt_emb_backward may be called */
-    int32_t reserved;
+    int32_t ablation;           /* 0 = the full method.  Study switches (forward only, tt_emb_backward returns
+                                   TT_EMB_ERR_STATE): bit 0 = no prefix reuse, every distinct row forms its own group and
+                                   rebuilds its prefix product ("unique only", cf. the paper's reuse ablation);
+                                   bit 1 = static schedule, every table cut into units of equal group COUNT instead of
+                                   equal cost (cf. the paper's scheduling ablation) */
 } tt_emb_config_t;
 
 /* Host only.  Copies everything it needs out of *cfg.  [data model: Sec. 2.1] */

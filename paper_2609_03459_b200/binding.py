@@ -41,7 +41,7 @@ class tt_emb_config_t(ctypes.Structure):
         ("max_lookups", ctypes.c_int64),
         ("max_unique_rows", ctypes.c_int64),
         ("enable_backward", ctypes.c_int32),
-        ("reserved", ctypes.c_int32),
+        ("ablation", ctypes.c_int32),
     ]
 
 
@@ -106,7 +106,7 @@ def _check(code: int, where: str):
 
 def make_config(num_rows: Sequence[int], row_factors: Sequence[Sequence[int]], dim_factors: Sequence[Sequence[int]],
                 ranks: Sequence[Sequence[int]], max_batch: int, max_lookups: int, max_unique_rows: int = 0,
-                enable_backward: bool = False):
+                enable_backward: bool = False, ablation: int = 0):
     """Returns (tt_emb_config_t, keepalive list of numpy arrays)."""
     T = len(num_rows)
     K = len(row_factors[0])
@@ -115,7 +115,7 @@ def make_config(num_rows: Sequence[int], row_factors: Sequence[Sequence[int]], d
     df = np.ascontiguousarray(np.asarray(dim_factors, dtype=np.int32).reshape(T * K))
     rk = np.ascontiguousarray(np.asarray(ranks, dtype=np.int32).reshape(T * (K + 1)))
     cfg = tt_emb_config_t(T, K, nr.ctypes.data, rf.ctypes.data, df.ctypes.data, rk.ctypes.data,
-                          int(max_batch), int(max_lookups), int(max_unique_rows), 1 if enable_backward else 0, 0)
+                          int(max_batch), int(max_lookups), int(max_unique_rows), 1 if enable_backward else 0, int(ablation))
     return cfg, [nr, rf, df, rk]
 
 
@@ -130,7 +130,7 @@ class TTEmbeddingBag:
     (numpy or torch, fp32) and converted on the device to the library's slice-major layout."""
 
     def __init__(self, num_rows, row_factors, dim_factors, ranks, max_batch, max_lookups, *,
-                 max_unique_rows: int = 0, enable_backward: bool = False, device="cuda:0"):
+                 max_unique_rows: int = 0, enable_backward: bool = False, ablation: int = 0, device="cuda:0"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -139,7 +139,7 @@ class TTEmbeddingBag:
                        for t in range(self.T)]
         self.enable_backward = enable_backward
         cfg, keep = make_config(num_rows, row_factors, dim_factors, ranks, max_batch, max_lookups,
-                                max_unique_rows, enable_backward)
+                                max_unique_rows, enable_backward, ablation)
         h = ctypes.c_void_p()
         _check(lib.tt_emb_create(ctypes.byref(cfg), ctypes.byref(h)), "tt_emb_create")
         self.h = h
@@ -314,11 +314,12 @@ class TTEmbeddingBag:
         return res
 
 
-def from_workload(wl, *, enable_backward: bool = False, max_unique_rows: int = 0, device="cuda:0") -> TTEmbeddingBag:
+def from_workload(wl, *, enable_backward: bool = False, max_unique_rows: int = 0, ablation: int = 0,
+                  device="cuda:0") -> TTEmbeddingBag:
     """Build a TTEmbeddingBag for a workloads.Workload-like object (tables with N, n, d, r; B; L; cores)."""
     emb = TTEmbeddingBag([s.N for s in wl.tables], [s.n for s in wl.tables], [s.d for s in wl.tables],
                          [s.r for s in wl.tables], wl.B, max(wl.L, 1), max_unique_rows=max_unique_rows,
-                         enable_backward=enable_backward, device=device)
+                         enable_backward=enable_backward, ablation=ablation, device=device)
     emb.set_cores(wl.cores)
     return emb
 

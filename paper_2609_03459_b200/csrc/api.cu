@@ -68,6 +68,8 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->T = T; h->K = K;
     h->max_batch = cfg->max_batch; h->max_lookups = cfg->max_lookups;
     h->enable_backward = cfg->enable_backward ? 1 : 0;
+    h->ablation = cfg->ablation & 3;
+    if (h->ablation && h->enable_backward) return fail(TT_EMB_ERR_ARG);   // the study switches are forward only
     h->sm_count = 148;
     { int sms = 0; if (device_ok(&sms) && sms > 0) h->sm_count = sms; }
 
@@ -190,9 +192,11 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
 
     WsView& v = h->v;
     v.T = T; v.K = K; v.D = D;
+    v.ablation = h->ablation;
     v.capU = h->capU;
     for (int k = 1; k <= K; ++k) {
         uint64_t c = level_space[k] < (uint64_t)h->capU ? level_space[k] : (uint64_t)h->capU;
+        if ((h->ablation & 1) && k == K - 1) c = (uint64_t)h->capU;   // one group per distinct row
         v.cap[k] = (uint32_t)c;
         v.stride[k] = stride[k];
     }

@@ -42,6 +42,7 @@ struct TableDesc {
 // Device-side view of the workspace handed to kernels by value.
 struct WsView {
     int32_t T, K, D;
+    int32_t ablation;                   // study switches: bit 0 no prefix reuse, bit 1 static (equal-count) schedule
     int32_t stride[TT_MAXK + 1];        // floats per node of the level-k partial-product buffers (max over tables)
     int64_t B, L;                       // current batch / lookups
     int64_t capU;                       // capacity in distinct rows
@@ -84,6 +85,7 @@ struct tt_emb {
     int T, K, D;
     int64_t max_batch, max_lookups, capU;
     int enable_backward;
+    int ablation;
     int sm_count;
     int units_total;
     int units_per_table;

@@ -25,7 +25,7 @@ struct CostScan {
         // neighbours, so that slice is fetched from L2 once per run instead of once per group), natural for K = 2
         const int K = w.K;
         const int t = tt_find_table(w.tb[K - 1], w.T, j);
-        const uint32_t g = K >= 3 ? w.tnode[K - 1][j] : j;
+        const uint32_t g = (K >= 3 && !(w.ablation & 1)) ? w.tnode[K - 1][j] : j;
         const TableDesc& td = w.tdesc[t];
         const uint32_t nchild = w.cstart[K - 1][g + 1] - w.cstart[K - 1][g];
         // c_k = P_{k-1} r_{k-1} d_k r_k
@@ -44,7 +44,7 @@ struct CostScan {
 
 cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s)
 {
-    if (h->K >= 3) {
+    if (h->K >= 3 && !(h->ablation & 1)) {
         cudaError_t e = tt_launch_tlist(h, h->K - 1, s);
         if (e != cudaSuccess) return e;
     }
@@ -61,6 +61,11 @@ __device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uin
     const int lvl = w.K - 1;
     const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
     const uint64_t ca = w.cost[a], cb = w.cost[b];
+    if (w.ablation & 2) {   // study switch: static schedule, equal group counts
+        g0 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)q / Q);
+        g1 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)(q + 1) / Q);
+        return;
+    }
     const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
     // first group whose exclusive cost >= target
     auto lower = [&](uint64_t target) {
@@ -323,7 +328,7 @@ __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& 
         if (lane == 0) g = atomicAdd(next, 1u);
         g = __shfl_sync(0xffffffffu, g, 0);
         if (g >= g1) break;
-        g = w.tnode[K - 1][g];   // position in the digit-major order -> group
+        if (!(w.ablation & 1)) g = w.tnode[K - 1][g];   // position in the digit-major order -> group
         const uint32_t val = w.val[K - 1][g];
         const float* src = tt_left_operand(w, td, K - 1, g);
         for (int i = lane; i < M * ra; i += 32) {
@@ -347,7 +352,7 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
     const int Pm = td.P[K - 1], rb = td.r[K - 1], dK = td.d[kl], D = w.D;
     const uint32_t nK = (uint32_t)td.n[kl];
     for (uint32_t jpos = g0; jpos < g1; ++jpos) {
-        const uint32_t g = K >= 3 ? w.tnode[K - 1][jpos] : jpos;
+        const uint32_t g = (K >= 3 && !(w.ablation & 1)) ? w.tnode[K - 1][jpos] : jpos;
         const uint32_t val = w.val[K - 1][g];
         if (K >= 3) {
             const int M = td.P[km], ra = td.r[km], cols = td.d[km] * rb;

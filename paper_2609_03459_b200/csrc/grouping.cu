@@ -117,6 +117,7 @@ struct LevelUp {
         const int t = tt_find_table(tbc, w.T, v);
         const uint32_t nk = (uint32_t)w.tdesc[t].n[k];  // radix of digit k+1 (0-based core index k)
         if (v == tbc[t]) return 1u;
+        if ((w.ablation & 1) && k == w.K - 1) return 1u;   // study switch: no prefix reuse, every row opens a group
         return (w.val[k + 1][v] / nk != w.val[k + 1][v - 1] / nk) ? 1u : 0u;
     }
     __device__ void emit(uint32_t v, uint32_t excl, uint32_t flag) const

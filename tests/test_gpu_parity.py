@@ -159,6 +159,22 @@ def test_forward_only_handle_and_repeat_calls(binding):
     assert_close(out3, oracle.forward_workload(wl2), "second batch out")
 
 
+@pytest.mark.parametrize("flags", [1, 2, 3])
+def test_ablation_switches_keep_the_result(binding, flags):
+    # the study switches (no prefix reuse / static schedule) change cost, never values
+    name, tables, B, pooling = MEDIUM[1]
+    wl = workloads.custom(tables, B, pooling, seed=21)
+    emb = binding.from_workload(wl, ablation=flags)
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"ablation {flags} out")
+    counts = emb.grouping_counts()
+    if flags & 1:   # every distinct row is its own group
+        assert np.array_equal(counts[:, 1], counts[:, 2])
+    with pytest.raises(binding.TTEmbError):
+        binding.from_workload(wl, ablation=flags, enable_backward=True)
+
+
 # ------------------------------------------------------------------------------------------ degenerate inputs
 
 def test_hot_row_and_long_segments(binding):
