@@ -327,8 +327,10 @@ def main():
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    binding.launch_count(reset=True)
     for _ in range(args.steps):
         step(d_idx, d_off, d_grad)
+    launches_per_step = binding.launch_count() / max(args.steps, 1)   # counted at the library's launch sites
     e1.record()
     barrier()
     total_ms = e0.elapsed_time(e1)
@@ -470,8 +472,6 @@ def main():
                  "fp32_slots": tot_slots, "hbm_bytes": tot_bytes}
     fwd_roof_t = max(work["fwd_slots"] / fp32_peak, work["fwd_hbm_bytes"] / (hbm_gbs * 1e9))
 
-    launches_fwd = 2 + 3 + 4 * (K - 1) + 3 + max(K - 3, 0) + 2
-    launches_bwd = 7 + 2 + 3 + 7 * (K - 2) + 1
     line = {
         "metric": METRIC, "value": world * L / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -486,7 +486,7 @@ def main():
         "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
                   "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},
         "work": work, "device_status": status, "clocks": clocks, "e2e": e2e,
-        "gpu_launches": launches_fwd + (launches_bwd if train else 0),
+        "gpu_launches": int(round(launches_per_step)),
         "workspace_GB": emb.workspace_bytes / 1e9,
     }
 

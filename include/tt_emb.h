@@ -200,6 +200,9 @@ int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t stream);
 int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* scratch_idx, int64_t num_rows_read,
                         double* bytes_per_second, tt_emb_stream_t stream);
 
+/* Kernels launched by this thread's library calls since the last reset (counted at the launch sites). */
+int tt_emb_launch_count(int64_t* count, int32_t reset);
+
 const char* tt_emb_strerror(int code);
 /* cudaError_t of the last failing CUDA call made by this thread's most recent library call (0 = none). */
 int tt_emb_last_cuda_error(void);

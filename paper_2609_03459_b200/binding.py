@@ -78,6 +78,7 @@ _SIGS = {
     "tt_emb_stage_ms": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_f32)]),
     "tt_emb_probe_fp32": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_probe_gather": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp, _i64, ctypes.POINTER(ctypes.c_double), _vp]),
+    "tt_emb_launch_count": (ctypes.c_int, [ctypes.POINTER(_i64), _i32]),
     "tt_emb_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "tt_emb_last_cuda_error": (ctypes.c_int, []),
 }
@@ -322,6 +323,12 @@ def from_workload(wl, *, enable_backward: bool = False, max_unique_rows: int = 0
                          enable_backward=enable_backward, ablation=ablation, device=device)
     emb.set_cores(wl.cores)
     return emb
+
+
+def launch_count(reset: bool = False) -> int:
+    v = ctypes.c_int64()
+    _check(lib.tt_emb_launch_count(ctypes.byref(v), 1 if reset else 0), "tt_emb_launch_count")
+    return int(v.value)
 
 
 def probe_fp32() -> float:

@@ -6,6 +6,17 @@
 #include "common.cuh"
 
 static thread_local int g_last_cuda_error = 0;
+static thread_local long long g_launches = 0;
+
+void tt_note_launch(int n) { g_launches += n; }
+
+extern "C" int tt_emb_launch_count(int64_t* count, int32_t reset)
+{
+    if (!count) return TT_EMB_ERR_ARG;
+    *count = (int64_t)g_launches;
+    if (reset) g_launches = 0;
+    return TT_EMB_OK;
+}
 
 #define TT_CUDA(x)                                   \
     do {                                             \
@@ -147,7 +158,6 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     if (Q > 16384) Q = 16384;
     int unit_base = 0;
     int64_t gpart = 0;
-    h->max_priv_floats = 0;
     for (int t = 0; t < T; ++t) {
         TableDesc& td = h->tab[t];
         td.units = Q;
@@ -171,7 +181,6 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         }
         td.unit_base = unit_base;
         unit_base += Q;
-        td.priv_ok = 0;
         td.gpart_off = gpart;
         gpart += (td.core_floats[K - 1] + 3) / 4 * 4;
     }
@@ -577,6 +586,7 @@ extern "C" int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t strea
     for (int rep = 0; rep < 4; ++rep) {
         cudaEventRecord(e0, s);
         k_probe_fma<<<sms * 8, 256, 0, s>>>(dsink, iters, 1.0001f, 0.5f);
+        tt_note_launch();
         cudaEventRecord(e1, s);
         cudaError_t e = cudaEventSynchronize(e1);
         if (e != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }
@@ -633,6 +643,7 @@ extern "C" int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* sc
     const size_t rows = bytes / 256;
     if (rows >= (1ull << 31)) return TT_EMB_ERR_ARG;
     k_probe_fill<<<sms * 4, 256, 0, s>>>(scratch_idx, num_rows_read, (uint32_t)rows);
+    tt_note_launch();
     cudaEvent_t e0, e1;
     TT_CUDA(cudaEventCreate(&e0));
     TT_CUDA(cudaEventCreate(&e1));
@@ -640,6 +651,7 @@ extern "C" int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* sc
     for (int rep = 0; rep < 4; ++rep) {
         cudaEventRecord(e0, s);
         k_probe_gather<<<sms * 8, 256, 0, s>>>((const float4*)buffer, scratch_idx, num_rows_read, dsink);
+        tt_note_launch();
         cudaEventRecord(e1, s);
         cudaError_t e = cudaEventSynchronize(e1);
         if (e != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }

@@ -114,6 +114,7 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
     WsView& w = h->v;
     const int zgrid = h->sm_count * 8;
     k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cnt, w.counters + CTR_LEVEL0 + w.K, 1u);
+    tt_note_launch();
     const int64_t ntiles = (w.L + HT_TILE - 1) / HT_TILE;
     cudaError_t e;
     int per_sm0 = 0, per_sm1 = 0;   // persistent grids sized to what is actually resident (no partial second wave)
@@ -125,9 +126,11 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
         return (int)(g < 1 ? 1 : g);
     };
     k_sort_pass<0><<<grid_of(per_sm0), 256, 0, s>>>(w);
+    tt_note_launch();
     CntScan cs{w};
     if ((e = tt_scan(cs, w.cap[w.K], w.scan_tmp, s)) != cudaSuccess) return e;
     k_sort_pass<1><<<grid_of(per_sm1), 256, 0, s>>>(w);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -369,11 +372,12 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
     const int grid = (int)((chunks + 7) / 8);
     if (grid > 0) {
         const int D4 = h->D / 4;
-        if (VEC && D4 <= 8) k_dE_fast<8><<<grid, 256, 0, s>>>(h->v, grad_out);
-        else if (VEC && D4 <= 16) k_dE_fast<16><<<grid, 256, 0, s>>>(h->v, grad_out);
-        else if (VEC && D4 <= 32) k_dE_fast<32><<<grid, 256, 0, s>>>(h->v, grad_out);
-        else k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out);
+        if (VEC && D4 <= 8) { k_dE_fast<8><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        else if (VEC && D4 <= 16) { k_dE_fast<16><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        else if (VEC && D4 <= 32) { k_dE_fast<32><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        else { k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         k_dE_fix<VEC, CPL><<<grid, 256, 0, s>>>(h->v);
+        tt_note_launch();
     }
     return cudaGetLastError();
 }
@@ -982,6 +986,7 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     if (e != cudaSuccess) return e;
     if ((e = tt_stage_begin(h, 15 + V + 1, s)) != cudaSuccess) return e;
     k_sweep_bwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    tt_note_launch();
     if ((e = tt_stage_end(h, 15 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -1001,6 +1006,7 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     cudaError_t e;
     if ((e = cudaMemsetAsync(w.gpart, 0, (size_t)TT_STRIPES * w.gpart_stride * sizeof(float), s)) != cudaSuccess) return e;
     k_zero_grads<<<dim3(64, h->T), 256, 0, s>>>(w);
+    tt_note_launch();
     // P_k of the levels below K-1 are still in pbuf from the forward (K = 4 only)
     if ((e = launch_sweep_bwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<0>(h, max_pl, max_c, s)) != cudaSuccess) return e;
@@ -1009,6 +1015,7 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_bwd<3>(h, max_pl, max_c, s)) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<4>(h, max_pl, max_c, s)) != cudaSuccess) return e;
     k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -1300,9 +1307,11 @@ cudaError_t tt_launch_tlist(tt_emb* h, int k, cudaStream_t s)
     if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
     const int g = h->sm_count * 8;
     k_tmark<<<g, 256, 0, s>>>(w, k);
+    tt_note_launch();
     TPopScan tp{w, k};
     if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
     k_tfill<<<g, 256, 0, s>>>(w, k);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -1325,16 +1334,18 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // level K-1's digit-major list already exists: the forward built it to order its sweep
         if (k != h->K - 1 && (e = tt_launch_tlist(h, k, s)) != cudaSuccess) return e;
         const dim3 sg(max_n, h->T);
-        if (any_fast[0]) k_mid_fused<32, 128><<<sg, 128, 0, s>>>(w, k, 0);
-        if (any_fast[1]) k_mid_fused<16, 128><<<sg, 128, 0, s>>>(w, k, 1);
-        if (any_fast[2]) k_mid_fused<32, 64><<<sg, 128, 0, s>>>(w, k, 2);
-        if (any_fast[3]) k_mid_fused<16, 64><<<sg, 128, 0, s>>>(w, k, 3);
-        if (any_fast[0] || any_fast[1] || any_fast[2] || any_fast[3]) k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k);
+        if (any_fast[0]) { k_mid_fused<32, 128><<<sg, 128, 0, s>>>(w, k, 0); tt_note_launch(); }
+        if (any_fast[1]) { k_mid_fused<16, 128><<<sg, 128, 0, s>>>(w, k, 1); tt_note_launch(); }
+        if (any_fast[2]) { k_mid_fused<32, 64><<<sg, 128, 0, s>>>(w, k, 2); tt_note_launch(); }
+        if (any_fast[3]) { k_mid_fused<16, 64><<<sg, 128, 0, s>>>(w, k, 3); tt_note_launch(); }
+        if (any_fast[0] || any_fast[1] || any_fast[2] || any_fast[3]) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {
             if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
             k_mid_slice<<<sg, 256, (size_t)max_slice * sizeof(float), s>>>(w, k);
+            tt_note_launch();
             if ((e = cudaFuncSetAttribute(k_mid_down, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_down * sizeof(float)))) != cudaSuccess) return e;
             k_mid_down<<<h->sm_count * 8, 256, (size_t)max_down * sizeof(float), s>>>(w, k);
+            tt_note_launch();
         }
     }
     return cudaGetLastError();
@@ -1356,5 +1367,6 @@ __global__ void __launch_bounds__(256) k_sgd(WsView w, float lr)
 cudaError_t tt_launch_sgd(tt_emb* h, float lr, cudaStream_t s)
 {
     k_sgd<<<dim3(64, h->T * h->K), 256, 0, s>>>(h->v, lr);
+    tt_note_launch();
     return cudaGetLastError();
 }

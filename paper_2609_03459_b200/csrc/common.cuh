@@ -34,7 +34,7 @@ struct TableDesc {
     int64_t gpart_off;                  // float offset of this table's last core inside one stripe
     int32_t units;                      // work units (CTAs) this table is cut into
     int32_t unit_base;                  // first global unit id
-    int32_t priv_ok;                    // last-core gradient of this table fits the shared-memory private copy
+    int32_t pad0;
     int32_t fast;                       // register-tiled kernel variant for this table's shapes, -1 = generic path
     int32_t midfast[TT_MAXK];           // same for the middle-core backward of level k (index k), -1 = generic
 };
@@ -103,7 +103,6 @@ struct tt_emb {
     size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart;
     size_t scan_tmp_elems;
     int64_t gpart_floats;
-    int max_priv_floats;  // largest n_K * slice_K among tables that use the private copy
     WsView v;             // filled at bind
     bool bound, have_forward;
     bool timing;
@@ -111,6 +110,9 @@ struct tt_emb {
     bool ev_valid[TT_NUM_STAGES];
     bool ev_created;
 };
+
+// every kernel launch of the library is noted here (api.cu); read with tt_emb_launch_count
+void tt_note_launch(int n = 1);
 
 // stage timing (api.cu): no-ops unless timing is enabled
 cudaError_t tt_stage_begin(tt_emb* h, int stage, cudaStream_t s);

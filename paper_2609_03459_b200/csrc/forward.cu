@@ -421,6 +421,7 @@ static cudaError_t launch_sweep_fwd(tt_emb* h, int max_pl, int max_c, cudaStream
     if (e != cudaSuccess) return e;
     if ((e = tt_stage_begin(h, 9 + V + 1, s)) != cudaSuccess) return e;
     k_sweep_fwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    tt_note_launch();
     if ((e = tt_stage_end(h, 9 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -440,6 +441,7 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
     for (int k = 2; k <= h->K - 2; ++k) {
         int grid = h->sm_count * 16;
         k_mid_level<<<grid, 128, (size_t)max_pl * sizeof(float), s>>>(w, k);
+        tt_note_launch();
     }
     cudaError_t e;
     if ((e = launch_sweep_fwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
@@ -678,6 +680,7 @@ static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
     k_pool_async<<<(int)grid, 256, smem, s>>>(h->v, out);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -694,6 +697,7 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
     k_pool_vec<LPR, CPL><<<(int)grid, 256, 0, s>>>(h->v, out);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -763,6 +767,7 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
     if (!vec_ok) {
         int pgrid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
         k_pool_scalar<<<pgrid < 1 ? 1 : pgrid, 256, 0, s>>>(w, out);
+        tt_note_launch();
         return cudaGetLastError();
     }
     const int D4 = D / 4;

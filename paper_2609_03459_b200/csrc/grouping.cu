@@ -159,10 +159,12 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
     int g0 = (int)((nb + 255) / 256);
     if (g0 > h->sm_count * 8) g0 = h->sm_count * 8;
     k_check_offsets<<<g0, 256, 0, s>>>(w);
+    tt_note_launch();
     if (w.L > 0) {
         int64_t want = (w.L + 1023) / 1024;
         int g1 = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
         k_mark<<<g1, 256, 0, s>>>(w);
+        tt_note_launch();
     }
     PopScan ps{w};
     if ((e = tt_scan(ps, w.total_words, w.scan_tmp, s)) != cudaSuccess) return e;
@@ -170,6 +172,7 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
         LevelUp lu{w, k};
         if ((e = tt_scan(lu, w.cap[k + 1], w.scan_tmp, s)) != cudaSuccess) return e;
         k_fix_tb<<<1, 32, 0, s>>>(w, k);
+        tt_note_launch();
     }
     return cudaGetLastError();
 }
@@ -220,8 +223,10 @@ cudaError_t tt_launch_export_level(tt_emb* h, int table, int level, int64_t* val
         cudaError_t e = cudaMemsetAsync(w.cursor, 0, (size_t)w.cap[w.K] * sizeof(uint32_t), s);
         if (e != cudaSuccess) return e;
         k_export_mult<<<h->sm_count * 4, 256, 0, s>>>(w, table);
+        tt_note_launch();
     }
     k_export_level<<<h->sm_count * 4, 256, 0, s>>>(w, table, level, vals, rc, lc, lc ? 1 : 0);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -244,6 +249,7 @@ __global__ void k_export_inverse(WsView w, int table, int32_t* inv)
 cudaError_t tt_launch_export_inverse(tt_emb* h, int table, int32_t* inv, cudaStream_t s)
 {
     k_export_inverse<<<h->sm_count * 4, 256, 0, s>>>(h->v, table, inv);
+    tt_note_launch();
     return cudaGetLastError();
 }
 
@@ -271,5 +277,6 @@ cudaError_t tt_launch_pack(const TableDesc& td, int core, const float* src, floa
     if (grid > 4096) grid = 4096;
     if (grid < 1) grid = 1;
     k_pack<<<grid, 256, 0, s>>>(src, dst, td.r[core], td.n[core], td.d[core], td.r[core + 1], to_canonical ? 1 : 0);
+    tt_note_launch();
     return cudaGetLastError();
 }

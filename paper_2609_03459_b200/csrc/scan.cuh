@@ -103,7 +103,10 @@ static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, 
     unsigned tiles = (unsigned)((capacity + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
     if (tiles == 0) tiles = 1;
     tt_scan_reduce<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    tt_note_launch();
     tt_scan_spine<F><<<1, 1024, 0, s>>>(f, tmp);
+    tt_note_launch();
     tt_scan_apply<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    tt_note_launch();
     return cudaGetLastError();
 }
