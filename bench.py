@@ -457,7 +457,9 @@ def main():
                                   "traffic": traffic_of("k_sweep_bwd" if bwd else "k_sweep_fwd", share),
                                   "peak_source": "independent-FMA-chain probe in this run",
                                   "note": "FMA-equivalent slots of the contractions this kernel performs; the row stages "
-                                          "run as 3xTF32 tensor-core products, the peak is the FP32 pipe"})
+                                          "run as 3xTF32 tensor-core products, the peak is the FP32 pipe; the kernels of "
+                                          "different shape variants run concurrently on forked streams, so each one's "
+                                          "duration includes sharing the GPU (the fraction is a lower bound)"})
     if kernels:
         dominant = max(kernels, key=lambda k: kernels[k][0])
         roofline = dict(kernels[dominant][1], ms_per_launch=kernels[dominant][0])

@@ -270,6 +270,10 @@ extern "C" int tt_emb_destroy(tt_emb_t h)
     if (!h) return TT_EMB_ERR_ARG;
     if (h->ev_created)
         for (int i = 0; i < TT_NUM_STAGES; ++i) { cudaEventDestroy(h->ev[i][0]); cudaEventDestroy(h->ev[i][1]); }
+    if (h->side_created) {
+        for (int i = 0; i < 4; ++i) cudaStreamDestroy(h->side[i]);
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(h->side_ev[i]);
+    }
     free(h->tab);
     free(h->vlist_host);
     delete h;
@@ -361,6 +365,32 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
 }
 
 // ------------------------------------------------------------------------------------------------ timing helpers
+
+cudaError_t tt_fork(tt_emb* h, cudaStream_t s, int n)
+{
+    cudaError_t e;
+    if (!h->side_created) {
+        for (int i = 0; i < 4; ++i)
+            if ((e = cudaStreamCreateWithFlags(&h->side[i], cudaStreamNonBlocking)) != cudaSuccess) return e;
+        for (int i = 0; i < 5; ++i)
+            if ((e = cudaEventCreateWithFlags(&h->side_ev[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+        h->side_created = true;
+    }
+    if ((e = cudaEventRecord(h->side_ev[4], s)) != cudaSuccess) return e;
+    for (int i = 0; i < n; ++i)
+        if ((e = cudaStreamWaitEvent(h->side[i], h->side_ev[4], 0)) != cudaSuccess) return e;
+    return cudaSuccess;
+}
+
+cudaError_t tt_join(tt_emb* h, cudaStream_t s, int n)
+{
+    cudaError_t e;
+    for (int i = 0; i < n; ++i) {
+        if ((e = cudaEventRecord(h->side_ev[i], h->side[i])) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(s, h->side_ev[i], 0)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
 
 cudaError_t tt_stage_begin(tt_emb* h, int stage, cudaStream_t s)
 {

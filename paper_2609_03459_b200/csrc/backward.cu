@@ -1008,12 +1008,20 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     k_zero_grads<<<dim3(64, h->T), 256, 0, s>>>(w);
     tt_note_launch();
     // P_k of the levels below K-1 are still in pbuf from the forward (K = 4 only)
-    if ((e = launch_sweep_bwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_bwd<0>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_bwd<1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_bwd<2>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_bwd<3>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_bwd<4>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    // tables of different shape variants are independent: their kernels run side by side on forked streams
+    int nvar = 0;
+    for (int vi = 0; vi <= TT_NUM_VARIANTS; ++vi) nvar += h->vcount[vi] > 0 ? 1 : 0;
+    const bool fork = nvar > 1;
+    if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
+    int slot = 0;
+    auto next_stream = [&](int vi) { return (fork && h->vcount[vi] > 0) ? h->side[(slot++) & 3] : s; };
+    if ((e = launch_sweep_bwd<-1>(h, max_pl, max_c, next_stream(0))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<0>(h, max_pl, max_c, next_stream(1))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<1>(h, max_pl, max_c, next_stream(2))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<2>(h, max_pl, max_c, next_stream(3))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<3>(h, max_pl, max_c, next_stream(4))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<4>(h, max_pl, max_c, next_stream(5))) != cudaSuccess) return e;
+    if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
     tt_note_launch();
     return cudaGetLastError();
@@ -1172,11 +1180,17 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 // One CTA of 128 threads per (table, slice i_k).  The slice G_k[i_k] (RA x COLS) never changes inside the CTA,
 // so each thread keeps its APT x 4 tile of it in registers.  The nodes with digit i_k arrive in ascending parent
 // order from the digit-major list; per node the CTA stages dP_k (4 x COLS) and the parent's P_{k-1} (4 x RA)
-// in shared memory (double-buffered, one barrier per node) and every thread does, for its tile,
+// in shared memory (a 4-stage cp.async pipeline, one barrier per node) and every thread does, for its tile,
 //     dG_k[a][c] += sum_m P_{k-1}[m][a] * dP_k[m][c]               (accumulated in registers over all nodes)
 //     Y[m][a]     = sum_c dP_k[m][c] * G_k[a][c]                    (partial over its 4 columns)
 // The Y partials are combined over the TC lanes that share an a-range by a reduce-scatter of warp shuffles and
 // written once per node; k_mid_sum then adds the Y rows of each parent's (contiguous) children.
+__device__ __forceinline__ void tt_cp_async16_b(void* smem_dst, const void* gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
 template <int NVAL, int W>
 __device__ __forceinline__ int tt_reduce_scatter(float (&v)[NVAL], int lane)
 {
@@ -1208,8 +1222,9 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
 {
     constexpr int M = 4, TC = COLS / 4, AG = 128 / TC, APT = RA / AG, NVAL = M * APT;
     constexpr int REP = TC / NVAL > 0 ? TC / NVAL : 1;  // lanes that end up with the same reduced value
-    __shared__ __align__(16) float sA[2][M * RA];
-    __shared__ __align__(16) float sD[2][M * COLS];
+    constexpr int ST = 4;   // stages of the node pipeline (cp.async, no staging registers)
+    __shared__ __align__(16) float sA[ST][M * RA];
+    __shared__ __align__(16) float sD[ST][M * COLS];
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
     const int kc = k - 1;
@@ -1226,24 +1241,28 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
     const uint32_t space = td.prefix_space[k - 1];
     const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
     const int strideY = w.stride[k - 1];
-    float4 rd = make_float4(0.f, 0.f, 0.f, 0.f), rav = rd;
-    uint32_t vnext = 0;
-    auto fetch = [&](uint32_t jn) {
-        vnext = w.tnode[k][jn];
-        if (tid < M * COLS / 4) rd = __ldg(reinterpret_cast<const float4*>(w.dP[k] + (size_t)vnext * w.stride[k]) + tid);
-        if (tid < M * RA / 4) rav = __ldg(reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, vnext)) + tid);
+    // node jn of the list -> stage jn % ST (always commits a group so that the group count stays in step)
+    auto issue = [&](uint32_t jn) {
+        if (jn < j1) {
+            const uint32_t v = w.tnode[k][jn];
+            const int buf = (int)((jn - j0) % ST);
+            if (tid < M * COLS / 4)
+                tt_cp_async16_b(reinterpret_cast<float4*>(sD[buf]) + tid,
+                                reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k]) + tid);
+            if (tid < M * RA / 4)
+                tt_cp_async16_b(reinterpret_cast<float4*>(sA[buf]) + tid,
+                                reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, v)) + tid);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    auto stage = [&](int buf) {
-        if (tid < M * COLS / 4) reinterpret_cast<float4*>(sD[buf])[tid] = rd;
-        if (tid < M * RA / 4) reinterpret_cast<float4*>(sA[buf])[tid] = rav;
-    };
-    uint32_t vcur = 0;
-    if (j0 < j1) { fetch(j0); stage(0); vcur = vnext; }
-    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < ST - 1; ++i) issue(j0 + i);
     for (uint32_t jn = j0; jn < j1; ++jn) {
-        const int cur = (int)((jn - j0) & 1u);
-        const bool more = jn + 1 < j1;
-        if (more) fetch(jn + 1);
+        const int cur = (int)((jn - j0) % ST);
+        asm volatile("cp.async.wait_group %0;" ::"n"(ST - 2) : "memory");
+        __syncthreads();            // node jn has landed for everyone; everyone is done with node jn-1
+        issue(jn + ST - 1);         // refills the stage node jn-1 used
+        const uint32_t vcur = w.tnode[k][jn];
         float y[NVAL];
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -1263,10 +1282,8 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
             const int m = idx / APT, i = idx - m * APT;
             w.Y[k][(size_t)vcur * strideY + m * RA + a0 + i] = y[0];
         }
-        if (more) stage(cur ^ 1);
-        vcur = vnext;
-        __syncthreads();
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
 #pragma unroll
     for (int i = 0; i < APT; ++i) reinterpret_cast<float4*>(dst + (size_t)(a0 + i) * COLS)[cl] = acc[i];
@@ -1334,10 +1351,15 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // level K-1's digit-major list already exists: the forward built it to order its sweep
         if (k != h->K - 1 && (e = tt_launch_tlist(h, k, s)) != cudaSuccess) return e;
         const dim3 sg(max_n, h->T);
-        if (any_fast[0]) { k_mid_fused<32, 128><<<sg, 128, 0, s>>>(w, k, 0); tt_note_launch(); }
-        if (any_fast[1]) { k_mid_fused<16, 128><<<sg, 128, 0, s>>>(w, k, 1); tt_note_launch(); }
-        if (any_fast[2]) { k_mid_fused<32, 64><<<sg, 128, 0, s>>>(w, k, 2); tt_note_launch(); }
-        if (any_fast[3]) { k_mid_fused<16, 64><<<sg, 128, 0, s>>>(w, k, 3); tt_note_launch(); }
+        // the shape variants are independent (different tables): run them side by side so that the tail of one
+        // (a few long node lists) overlaps the others
+        const bool fork = (int)any_fast[0] + (int)any_fast[1] + (int)any_fast[2] + (int)any_fast[3] > 1;
+        if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
+        if (any_fast[0]) { k_mid_fused<32, 128><<<sg, 128, 0, fork ? h->side[0] : s>>>(w, k, 0); tt_note_launch(); }
+        if (any_fast[1]) { k_mid_fused<16, 128><<<sg, 128, 0, fork ? h->side[1] : s>>>(w, k, 1); tt_note_launch(); }
+        if (any_fast[2]) { k_mid_fused<32, 64><<<sg, 128, 0, fork ? h->side[2] : s>>>(w, k, 2); tt_note_launch(); }
+        if (any_fast[3]) { k_mid_fused<16, 64><<<sg, 128, 0, fork ? h->side[3] : s>>>(w, k, 3); tt_note_launch(); }
+        if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (any_fast[0] || any_fast[1] || any_fast[2] || any_fast[3]) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {
             if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;

@@ -109,10 +109,18 @@ struct tt_emb {
     cudaEvent_t ev[TT_NUM_STAGES][2];
     bool ev_valid[TT_NUM_STAGES];
     bool ev_created;
+    // side streams for kernels of different shape variants that may overlap (created on first use)
+    cudaStream_t side[4];
+    cudaEvent_t side_ev[5];
+    bool side_created;
 };
 
 // every kernel launch of the library is noted here (api.cu); read with tt_emb_launch_count
 void tt_note_launch(int n = 1);
+
+// fork/join helpers (api.cu): side streams wait for everything enqueued on `s` so far / `s` waits for the side streams
+cudaError_t tt_fork(tt_emb* h, cudaStream_t s, int n);
+cudaError_t tt_join(tt_emb* h, cudaStream_t s, int n);
 
 // stage timing (api.cu): no-ops unless timing is enabled
 cudaError_t tt_stage_begin(tt_emb* h, int stage, cudaStream_t s);

@@ -444,12 +444,20 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
         tt_note_launch();
     }
     cudaError_t e;
-    if ((e = launch_sweep_fwd<-1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_fwd<0>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_fwd<1>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_fwd<2>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_fwd<3>(h, max_pl, max_c, s)) != cudaSuccess) return e;
-    if ((e = launch_sweep_fwd<4>(h, max_pl, max_c, s)) != cudaSuccess) return e;
+    // tables of different shape variants are independent: their kernels run side by side on forked streams
+    int nvar = 0;
+    for (int vi = 0; vi <= TT_NUM_VARIANTS; ++vi) nvar += h->vcount[vi] > 0 ? 1 : 0;
+    const bool fork = nvar > 1;
+    if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
+    int slot = 0;
+    auto next_stream = [&](int vi) { return (fork && h->vcount[vi] > 0) ? h->side[(slot++) & 3] : s; };
+    if ((e = launch_sweep_fwd<-1>(h, max_pl, max_c, next_stream(0))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<0>(h, max_pl, max_c, next_stream(1))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<1>(h, max_pl, max_c, next_stream(2))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<2>(h, max_pl, max_c, next_stream(3))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<3>(h, max_pl, max_c, next_stream(4))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<4>(h, max_pl, max_c, next_stream(5))) != cudaSuccess) return e;
+    if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
