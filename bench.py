@@ -400,8 +400,9 @@ def main():
     # ---- roofline of the dominant kernel and of the whole step
     # DRAM traffic per lookup / per distinct row of the top kernels, from the ncu capture of the reduced case
     # (8 tables; profiles/ncu_full_cfg5_reduced.md), scaled to this launch by the units it processes.
-    NCU_TRAFFIC = {"k_pool_vec": ("lookup", 124.5), "k_dE_fast": ("lookup", 71.9),
-                   "k_sweep_fwd": ("row", 226.6), "k_sweep_bwd": ("row", 364.0)}
+    NCU_TRAFFIC = {"k_pool": ("lookup", 118.6), "k_dE_fast": ("lookup", 71.5),
+                   "k_sweep_fwd": ("row", 226.0), "k_sweep_bwd": ("row", 345.0)}
+    pool_kernel = "k_pool_async" if 32 < D <= 64 and D % 4 == 0 else "k_pool_vec"
 
     def traffic_of(kernel, share=1.0):
         unit, per = NCU_TRAFFIC[kernel]
@@ -431,8 +432,8 @@ def main():
     if "pooling" in stage_ms:
         ms = stage_ms["pooling"]
         ach = work["pool_kernel_bytes"] / (ms * 1e-3) / 1e9
-        kernels["k_pool_vec"] = (ms, {"kernel": "k_pool_vec", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                                      "frac": ach / hbm_gbs, "traffic": traffic_of("k_pool_vec"), "peak_source": peak_src,
+        kernels[pool_kernel] = (ms, {"kernel": pool_kernel, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                                      "frac": ach / hbm_gbs, "traffic": traffic_of("k_pool"), "peak_source": peak_src,
                                       "note": "algorithmic bytes: indices + offsets + every distinct row once + out "
                                               "(+ one (slot,bag) pair per lookup when the backward is enabled); the "
                                               "per-lookup row gather (L*D*4 bytes) is on-chip / re-read traffic and is "

@@ -154,6 +154,11 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     // work units: every table is cut into `units` equal-cost slices, one CTA each
     // about 8 waves of 8 resident CTAs per SM: fine enough that the last wave and table-size differences do not matter
     int Q = (64 * h->sm_count + T - 1) / T;
+    {   // ... but not so fine that a unit holds only a handful of groups (each unit pays two binary searches)
+        uint64_t groups = level_space[K - 1] < (uint64_t)h->capU ? level_space[K - 1] : (uint64_t)h->capU;
+        const int64_t by_groups = (int64_t)(groups / (uint64_t)T / 64);
+        if (Q > by_groups) Q = (int)by_groups;
+    }
     if (Q < 8) Q = 8;
     if (Q > 16384) Q = 16384;
     int unit_base = 0;
