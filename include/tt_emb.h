@@ -187,6 +187,9 @@ int tt_emb_unpack_core(tt_emb_t h, int32_t table, int32_t core, const float* can
  * 6 backward contraction, 7 backward middle cores + reductions, 8 sgd; 9..14 the forward sweep kernel of shape
  * variant -1 (generic), 0..4; 15..20 the backward sweep kernel of the same variants (TT_EMB_ERR_STATE for a
  * variant no table uses).
+ * on = 0: no events; 1: events, normal execution; 2: events, and kernels of different shape variants, which
+ * normally run side by side on forked streams, run one after the other, so that a per-kernel duration is that
+ * kernel's alone (the step is slower in this mode; it is for per-kernel figures, not for throughput).
  */
 int tt_emb_enable_timing(tt_emb_t h, int32_t on);
 int tt_emb_stage_ms(tt_emb_t h, int32_t stage, float* ms);

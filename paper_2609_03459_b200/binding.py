@@ -303,8 +303,9 @@ class TTEmbeddingBag:
         _check(lib.tt_emb_export_inverse(self.h, table, inv.data_ptr(), _stream_ptr()), "tt_emb_export_inverse")
         return inv.cpu().numpy()[:num_lookups]
 
-    def enable_timing(self, on: bool = True):
-        _check(lib.tt_emb_enable_timing(self.h, 1 if on else 0), "tt_emb_enable_timing")
+    def enable_timing(self, on=True):
+        """False/0: off; True/1: stage events; 2: stage events with the shape-variant kernels serialised."""
+        _check(lib.tt_emb_enable_timing(self.h, int(on)), "tt_emb_enable_timing")
 
     def stage_ms(self) -> dict:
         res = {}

@@ -434,6 +434,7 @@ extern "C" int tt_emb_enable_timing(tt_emb_t h, int32_t on)
 {
     if (!h) return TT_EMB_ERR_ARG;
     h->timing = on != 0;
+    h->serial = on == 2;
     return TT_EMB_OK;
 }
 

@@ -1011,7 +1011,7 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     // tables of different shape variants are independent: their kernels run side by side on forked streams
     int nvar = 0;
     for (int vi = 0; vi <= TT_NUM_VARIANTS; ++vi) nvar += h->vcount[vi] > 0 ? 1 : 0;
-    const bool fork = nvar > 1;
+    const bool fork = nvar > 1 && !h->serial;
     if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
     int slot = 0;
     auto next_stream = [&](int vi) { return (fork && h->vcount[vi] > 0) ? h->side[(slot++) & 3] : s; };
@@ -1353,7 +1353,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         const dim3 sg(max_n, h->T);
         // the shape variants are independent (different tables): run them side by side so that the tail of one
         // (a few long node lists) overlaps the others
-        const bool fork = (int)any_fast[0] + (int)any_fast[1] + (int)any_fast[2] + (int)any_fast[3] > 1;
+        const bool fork = (int)any_fast[0] + (int)any_fast[1] + (int)any_fast[2] + (int)any_fast[3] > 1 && !h->serial;
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         if (any_fast[0]) { k_mid_fused<32, 128><<<sg, 128, 0, fork ? h->side[0] : s>>>(w, k, 0); tt_note_launch(); }
         if (any_fast[1]) { k_mid_fused<16, 128><<<sg, 128, 0, fork ? h->side[1] : s>>>(w, k, 1); tt_note_launch(); }

@@ -106,6 +106,7 @@ struct tt_emb {
     WsView v;             // filled at bind
     bool bound, have_forward;
     bool timing;
+    bool serial;          // timing mode 2: shape-variant kernels run one after the other (per-kernel durations)
     cudaEvent_t ev[TT_NUM_STAGES][2];
     bool ev_valid[TT_NUM_STAGES];
     bool ev_created;

@@ -447,7 +447,7 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
     // tables of different shape variants are independent: their kernels run side by side on forked streams
     int nvar = 0;
     for (int vi = 0; vi <= TT_NUM_VARIANTS; ++vi) nvar += h->vcount[vi] > 0 ? 1 : 0;
-    const bool fork = nvar > 1;
+    const bool fork = nvar > 1 && !h->serial;
     if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
     int slot = 0;
     auto next_stream = [&](int vi) { return (fork && h->vcount[vi] > 0) ? h->side[(slot++) & 3] : s; };
@@ -483,6 +483,16 @@ __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableD
     return slot;
 }
 
+// Pooling partition: the lookups are cut into C = W * chunks equal shares and warp wi takes shares wi, wi + W, ...
+// (whole bags, found by bisection on offsets).  All resident warps therefore work inside one moving window of
+// about W shares at a time - a few tables - so the rows that several bags share are still in L2 when the next
+// bag asks for them; one contiguous share per warp would spread the warps over all tables at once.
+__device__ __forceinline__ int64_t tt_pool_chunks(int64_t L, int64_t W)
+{
+    const int64_t c = L / (W * 512);                    // at least 512 lookups per share
+    return c < 1 ? 1 : (c > 8 ? 8 : c);
+}
+
 template <int LPR, int CPL>  // lanes per row, float4 chunks per lane
 __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
 {
@@ -495,14 +505,18 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
     const int64_t nb = (int64_t)w.T * w.B;
     const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
     const uint32_t capK = w.cap[w.K];
-    // Skew-aware split: the grid is exactly resident (persistent warps); warp wi takes the bags whose first
-    // lookup falls into the wi-th equal share of the L lookups (offsets is the cost prefix sum).
+    // Skew-aware split: the grid is exactly resident (persistent warps); a share holds the bags whose first
+    // lookup falls into it (offsets is the cost prefix sum).
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t C = W * tt_pool_chunks(w.L, W);
+    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    int64_t b_prev = 0;
+    for (int64_t ci = wi; ci < C; ci += W) {
     int64_t b0, b1;
     {
-        const int64_t target = lane == 0 ? (w.L * wi) / W : (w.L * (wi + 1)) / W;
-        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target
+        const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
+        int64_t lo = b_prev, hi = nb;                   // first bag with offsets[bag] >= target
         if (lane < 2)
             while (lo < hi) {
                 const int64_t mid = (lo + hi) >> 1;
@@ -510,11 +524,11 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
             }
         b0 = __shfl_sync(0xffffffffu, lo, 0);
         b1 = __shfl_sync(0xffffffffu, lo, 1);
-        if (wi == 0) b0 = 0;
-        if (wi == W - 1) b1 = nb;
+        if (ci == 0) b0 = 0;
+        if (ci == C - 1) b1 = nb;
+        b_prev = b1;
     }
-    if (b0 >= b1) return;
-    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    if (b0 >= b1) continue;
     int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
     if (o_hi < o_lo) o_hi = o_lo;
     int t = (int)(b0 / w.B);
@@ -583,6 +597,7 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
         o_hi = n_hi;
         t = tn;
     }
+    }
 }
 
 // Rows of up to 256 bytes (D <= 64): the gather is bound by bytes in flight, and registers cap what LDG can keep in
@@ -608,10 +623,14 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
     const uint32_t capK = w.cap[w.K];
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t C = W * tt_pool_chunks(w.L, W);
+    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    int64_t b_prev = 0;
+    for (int64_t ci = wi; ci < C; ci += W) {
     int64_t b0, b1;
     {
-        const int64_t target = lane == 0 ? (w.L * wi) / W : (w.L * (wi + 1)) / W;
-        int64_t lo = 0, hi = nb;
+        const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
+        int64_t lo = b_prev, hi = nb;                   // first bag with offsets[bag] >= target
         if (lane < 2)
             while (lo < hi) {
                 const int64_t mid = (lo + hi) >> 1;
@@ -619,11 +638,11 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
             }
         b0 = __shfl_sync(0xffffffffu, lo, 0);
         b1 = __shfl_sync(0xffffffffu, lo, 1);
-        if (wi == 0) b0 = 0;
-        if (wi == W - 1) b1 = nb;
+        if (ci == 0) b0 = 0;
+        if (ci == C - 1) b1 = nb;
+        b_prev = b1;
     }
-    if (b0 >= b1) return;
-    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    if (b0 >= b1) continue;
     int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
     if (o_hi < o_lo) o_hi = o_lo;
     int t = (int)(b0 / w.B);
@@ -671,6 +690,7 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
         o_lo = o_hi;
         o_hi = n_hi;
         t = tn;
+    }
     }
 }
 

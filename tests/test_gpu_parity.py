@@ -143,6 +143,22 @@ def test_medium_forward_backward(binding, case):
             assert_close(grads[t][k], ref[t][k], f"{name} dG[{t}][{k}]")
 
 
+@pytest.mark.parametrize("D,rank", [(16, 8), (16, 32), (32, 16), (32, 32), (64, 8), (64, 32)])
+def test_sweep_point_shapes(binding, D, rank):
+    # the shapes of the dimension / rank sweep (dim factors 2x2x4, 2x4x4, 4x4x4) at a batch the oracle finishes fast
+    wl = workloads.sweep_point(D, rank, 96, num_tables=3, with_grad=True)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"sweep D{D} r{rank} out")
+    check_grouping(emb, wl)
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        for k in range(3):
+            assert_close(grads[t][k], ref[t][k], f"sweep D{D} r{rank} dG[{t}][{k}]")
+
+
 def test_forward_only_handle_and_repeat_calls(binding):
     # a forward-only handle (no backward workspace) gives the same output, and calling twice is idempotent
     name, tables, B, pooling = MEDIUM[0]

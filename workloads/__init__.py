@@ -236,3 +236,26 @@ def custom(tables: Sequence[TableSpec], B: int, pooling, *, seed: int = 1234, ma
            with_grad: bool = False, name: str = "custom") -> Workload:
     """Arbitrary shapes for unit tests (pooling: int or (lo, hi); lo may be 0 to get empty bags)."""
     return _assemble(name, list(tables), B, pooling, seed, mapping, with_grad)
+
+
+SWEEP_DIM_FACTORS = {16: (2, 2, 4), 32: (2, 4, 4), 64: (4, 4, 4), 128: (4, 8, 4)}
+
+
+def sweep_point(D: int, rank: int, batch: int, *, num_tables: int = 8, with_grad: bool = False,
+                mapping: str = "identity", seed: Optional[int] = None) -> Workload:
+    """One point of the embedding-dimension / TT-rank / batch-size sweep (3 cores).
+
+    Tables: the first `num_tables` row counts and Zipf exponents of the config-3 stream (row counts
+    log-uniform in [1e4, 4e7], three near-equal row factors), every table with dim factors
+    SWEEP_DIM_FACTORS[D] and ranks (1, rank, rank, 1); cores N(0, 0.05); pooling factor uniform in
+    [1, 100] per (table, bag).  The same tables serve every (D, rank, batch), so points differ only in
+    the swept quantity.
+    """
+    if D not in SWEEP_DIM_FACTORS:
+        raise ValueError(f"D must be one of {sorted(SWEEP_DIM_FACTORS)}")
+    seed3 = (BASE_SEED if seed is None else seed) + 1000 * 3
+    base = _cfg3_tables(np.random.default_rng(seed3 + 500), num_tables)
+    tables = [TableSpec(N=s.N, n=s.n, d=SWEEP_DIM_FACTORS[D], r=(1, rank, rank, 1), alpha=s.alpha,
+                        core_dist="normal", core_scale=0.05) for s in base]
+    return _assemble(f"sweep-D{D}-r{rank}-B{batch}", tables, batch, (1, 100), seed3 + 7 * D + rank, mapping,
+                     with_grad=with_grad)
