@@ -1,0 +1,98 @@
+// Intermediate products (paper Sec. 3.2, "Intermediate Computation") of up to four prefix groups at once on the
+// tensor cores.
+//
+// Groups are walked in digit-major order, so neighbours share the slice B = G_{K-1}[i_{K-1}] (r_a x cols).  With
+// P_{K-2} of four rows per group, four groups stack into one 16 x r_a operand, and
+//     [C_0; C_1; C_2; C_3] = [P_0; P_1; P_2; P_3] . B
+// is a 16 x cols product of m16n8k8 tiles in 3xTF32 (see mma.cuh).  The slice then enters the SM once per four
+// groups instead of once per group (the FP32-pipe form of this product was bound by the L1 operand path), and the
+// product leaves the FP32 pipe.  Groups of the quad that use another slice (a run boundary) are handled in a
+// further pass; rows of groups that are not part of a pass are zero and their result is not stored.
+#pragma once
+#include "mma.cuh"
+
+// One pass.  Lane (g = lane / 4, t = lane % 4) feeds rows g and g + 8 of the stacked operand: row g belongs to group
+// g / 4 (source srcA, taken when selA), row g + 8 to group 2 + g / 4 (srcB, selB); m = g % 4 is the row of P inside
+// the group.  src points at P (4 x ra, row-major).  ra <= 32, any value (the k range is padded with zeros).
+// Results go to Cs4 + q * 4 * COLS + m * COLS + column for group q (C_q as [4][COLS] = [PM][RB] row-major).
+//
+// Column mapping: a block of 32 columns is one float4 load per lane and k row (8 lanes x 16 bytes = 128 bytes per
+// row); tile j of the block takes component j, i.e. tile column n' stands for slice column 32 * block + 4 n' + j, so
+// that a lane ends up with 8 consecutive columns of each of its two rows (two float4 stores per row).
+template <int COLS>
+__device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
+                                                const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane)
+{
+    constexpr int KTMAX = 4;
+    const int g = lane >> 2, t = lane & 3, m = g & 3;
+    const int kta = (ra + 7) >> 3;
+    Tf32Pair a[KTMAX][4];
+#pragma unroll
+    for (int kt = 0; kt < KTMAX; ++kt) {
+        const int k0 = 8 * kt + t, k1 = k0 + 4;
+        const float a0 = (selA && k0 < ra) ? __ldg(srcA + m * ra + k0) : 0.f;
+        const float a1 = (selB && k0 < ra) ? __ldg(srcB + m * ra + k0) : 0.f;
+        const float a2 = (selA && k1 < ra) ? __ldg(srcA + m * ra + k1) : 0.f;
+        const float a3 = (selB && k1 < ra) ? __ldg(srcB + m * ra + k1) : 0.f;
+        a[kt][0] = tt_split_tf32(a0); a[kt][1] = tt_split_tf32(a1); a[kt][2] = tt_split_tf32(a2); a[kt][3] = tt_split_tf32(a3);
+    }
+    const float4* __restrict__ B4 = reinterpret_cast<const float4*>(B);
+    constexpr int C4N = COLS / 4;
+    float* dstA = Cs4 + (size_t)(g >> 2) * (4 * COLS) + m * COLS + 8 * t;
+    float* dstB = Cs4 + (size_t)(2 + (g >> 2)) * (4 * COLS) + m * COLS + 8 * t;
+#pragma unroll 1
+    for (int nb = 0; nb < COLS / 32; ++nb) {
+        float4 f[KTMAX][2];
+#pragma unroll
+        for (int kt = 0; kt < KTMAX; ++kt) {
+            const int k0 = 8 * kt + t, k1 = k0 + 4;
+            f[kt][0] = k0 < ra ? __ldg(B4 + (size_t)k0 * C4N + 8 * nb + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+            f[kt][1] = k1 < ra ? __ldg(B4 + (size_t)k1 * C4N + 8 * nb + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float acc[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
+#pragma unroll
+        for (int kt = 0; kt < KTMAX; ++kt) {
+            if (kt < kta) {
+                const float v0[4] = {f[kt][0].x, f[kt][0].y, f[kt][0].z, f[kt][0].w};
+                const float v1[4] = {f[kt][1].x, f[kt][1].y, f[kt][1].z, f[kt][1].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    Tf32Pair b[2];
+                    b[0] = tt_split_tf32(v0[j]);
+                    b[1] = tt_split_tf32(v1[j]);
+                    tt_mma_3xtf32(acc[j], a[kt], b);
+                }
+            }
+        }
+        if (selA) {
+            *reinterpret_cast<float4*>(dstA + 32 * nb) = make_float4(acc[0][0], acc[1][0], acc[2][0], acc[3][0]);
+            *reinterpret_cast<float4*>(dstA + 32 * nb + 4) = make_float4(acc[0][1], acc[1][1], acc[2][1], acc[3][1]);
+        }
+        if (selB) {
+            *reinterpret_cast<float4*>(dstB + 32 * nb) = make_float4(acc[0][2], acc[1][2], acc[2][2], acc[3][2]);
+            *reinterpret_cast<float4*>(dstB + 32 * nb + 4) = make_float4(acc[0][3], acc[1][3], acc[2][3], acc[3][3]);
+        }
+    }
+}
+
+// All passes of one quad.  Lane q < cnt holds group q's slice index (imq) and operand pointer (srcq).
+template <int COLS>
+__device__ __forceinline__ void tt_quad_mid(const float* __restrict__ core_mid, size_t slice_floats, int ra, int cnt, uint32_t imq,
+                                            const float* srcq, float* Cs4, int lane)
+{
+    const int g = lane >> 2;
+    const unsigned long long sp = (unsigned long long)reinterpret_cast<uintptr_t>(srcq);
+    const float* srcA = reinterpret_cast<const float*>((uintptr_t)__shfl_sync(0xffffffffu, sp, g >> 2));
+    const float* srcB = reinterpret_cast<const float*>((uintptr_t)__shfl_sync(0xffffffffu, sp, 2 + (g >> 2)));
+    unsigned remaining = (1u << cnt) - 1u;
+    while (remaining) {
+        const int first = __ffs(remaining) - 1;
+        const uint32_t im = __shfl_sync(0xffffffffu, imq, first);
+        const unsigned sel = __ballot_sync(0xffffffffu, lane < 4 && ((remaining >> lane) & 1u) && imq == im) & 0xfu;
+        const bool selA = (sel >> (g >> 2)) & 1u, selB = (sel >> (2 + (g >> 2))) & 1u;
+        tt_quad_mid_mma<COLS>(core_mid + (size_t)im * slice_floats, ra, srcA, srcB, selA, selB, Cs4, lane);
+        remaining &= ~sel;
+    }
+}

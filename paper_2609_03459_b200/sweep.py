@@ -59,15 +59,14 @@ def time_point(D: int, rank: int, batch: int, train: bool, steps: int, warmup: i
         return float(np.mean(ms)), float(np.median(ms))
 
     fwd_mean, fwd_med = timed(fwd)
+    counts = emb.grouping_counts()         # of the forward that just ran
     res = {"D": D, "rank": rank, "batch": batch, "tables": wl.T, "lookups": int(wl.L),
            "forward_ms": fwd_mean, "forward_ms_median": fwd_med,
-           "forward_lookups_per_s": wl.L / (fwd_mean * 1e-3)}
+           "forward_lookups_per_s": wl.L / (fwd_mean * 1e-3),
+           "distinct_rows": int(counts[:, -1].sum()), "prefix_groups": int(counts[:, -2].sum())}
     if train:
         st_mean, st_med = timed(step)
         res.update({"step_ms": st_mean, "step_ms_median": st_med, "step_lookups_per_s": wl.L / (st_mean * 1e-3)})
-    counts = emb.grouping_counts()
-    res["distinct_rows"] = int(counts[:, -1].sum())
-    res["prefix_groups"] = int(counts[:, -2].sum())
     status = emb.status()
     if status != 0:
         raise RuntimeError(f"device status {status} at D={D} rank={rank} batch={batch}")

@@ -117,7 +117,10 @@ MEDIUM = [
                        TableSpec(20_000, (28, 28, 28), (4, 4, 4), (1, 16, 16, 1), 0.9, "normal", 0.05),
                        TableSpec(25_000, (30, 30, 30), (4, 4, 4), (1, 16, 32, 1), 1.0, "normal", 0.05),
                        TableSpec(12_000, (23, 23, 23), (4, 4, 4), (1, 32, 16, 1), 1.2, "normal", 0.05),
-                       TableSpec(8_000, (20, 20, 20), (4, 4, 4), (1, 8, 8, 1), 1.05, "uniform", 0.1)], 150, (0, 30)),
+                       TableSpec(8_000, (20, 20, 20), (4, 4, 4), (1, 8, 8, 1), 1.05, "uniform", 0.1),
+                       # first ranks that are not multiples of 8: the stacked tensor-core product pads its k range
+                       TableSpec(9_000, (21, 21, 21), (4, 4, 4), (1, 12, 32, 1), 1.0, "normal", 0.05),
+                       TableSpec(7_000, (19, 20, 19), (4, 4, 4), (1, 21, 16, 1), 1.1, "normal", 0.05)], 150, (0, 30)),
     ("tiled-d484", [TableSpec(10_000, (20, 25, 20), (4, 8, 4), (1, 32, 32, 1), 1.1, "normal", 0.05)], 100, 20),
     ("tiled-k4-r64", [TableSpec(20_736, (12, 12, 12, 12), (2, 4, 4, 4), (1, 64, 64, 64, 1), 1.2, "normal", 0.02)], 120, 8),
     ("k2", [TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 1.0, "uniform", 0.1)], 257, (1, 9)),
