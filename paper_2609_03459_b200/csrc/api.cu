@@ -169,14 +169,15 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         td.fast = -1;
         if (K >= 3 && td.d[K - 1] == 4) {
             // (P_{K-1}, r_{K-1}, P_{K-2}) combinations with a register-tiled variant (see forward.cu)
-            // the tensor-core variants (0, 1, 3) stack four groups' P_{K-2} (four rows each, r_{K-2} <= 32 columns)
+            // the tensor-core variants stack the P_{K-2} of four groups (0, 1, 3: four rows each, r_{K-2} <= 32) or of
+            // two groups (4: eight rows each, r_{K-2} <= 64)
             const int PMv = td.P[K - 1], RBv = td.r[K - 1], Mv = td.P[K - 2];
             const bool quad_ok = td.r[K - 2] <= 32;
             if (PMv == 16 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 0;
             else if (PMv == 16 && Mv == 4 && RBv == 16 && quad_ok) td.fast = 1;
             else if (PMv == 16 && Mv == 4 && RBv == 8) td.fast = 2;
             else if (PMv == 32 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 3;
-            else if (PMv == 32 && Mv == 8 && RBv == 64) td.fast = 4;
+            else if (PMv == 32 && Mv == 8 && RBv == 64 && td.r[K - 2] <= 64) td.fast = 4;
         }
         for (int k = 0; k < TT_MAXK; ++k) td.midfast[k] = -1;
         for (int k = 2; k <= K - 1; ++k) {

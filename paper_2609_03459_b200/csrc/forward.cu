@@ -346,21 +346,24 @@ __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& 
     }
 }
 
-// Tensor-core variants: a warp takes four consecutive groups of the digit-major order at a time; their intermediate
-// products are formed together (quad_mid.cuh), then each group's rows are produced from its C in shared memory.
-template <int PM, int RB>
+// Tensor-core variants: a warp takes NG = 16 / MROWS consecutive groups of the digit-major order at a time; their
+// intermediate products are formed together (quad_mid.cuh), then each group's rows are produced from its C in shared
+// memory: on the tensor cores too (TP = 0), or on the FP32 pipe with TP rows of C per lane where C is too large for
+// register-resident fragments.
+template <int PM, int RB, int MROWS, int KTMAX, int TP>
 __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& td, uint32_t g1, float* Cs4, uint32_t* next, int lane)
 {
-    constexpr int COLS = PM / 4 * RB;   // d_{K-1} * r_{K-1}; P_{K-2} has four rows
+    constexpr int COLS = PM / MROWS * RB;   // d_{K-1} * r_{K-1}
+    constexpr int NG = 16 / MROWS;
     const int K = w.K, km = K - 2;
     const int ra = td.r[km];
     const uint32_t nK = (uint32_t)td.n[K - 1];
     for (;;) {
         uint32_t base = 0;
-        if (lane == 0) base = atomicAdd(next, 4u);
+        if (lane == 0) base = atomicAdd(next, (uint32_t)NG);
         base = __shfl_sync(0xffffffffu, base, 0);
         if (base >= g1) break;
-        const int cnt = (int)min(4u, g1 - base);
+        const int cnt = (int)min((uint32_t)NG, g1 - base);
         uint32_t valq = 0, imq = 0, u0q = 0, u1q = 0;
         const float* srcq = nullptr;
         if (lane < cnt) {
@@ -372,12 +375,13 @@ __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& 
             u0q = w.cstart[K - 1][gq];
             u1q = w.cstart[K - 1][gq + 1];
         }
-        tt_quad_mid<COLS>(td.core[km], td.slice_floats[km], ra, cnt, imq, srcq, Cs4, lane);
+        tt_quad_mid<COLS, MROWS, KTMAX>(td.core[km], td.slice_floats[km], ra, cnt, imq, srcq, Cs4, lane);
         __syncwarp();
         for (int q = 0; q < cnt; ++q) {
             const uint32_t val = __shfl_sync(0xffffffffu, valq, q);
             const uint32_t u0 = __shfl_sync(0xffffffffu, u0q, q), u1 = __shfl_sync(0xffffffffu, u1q, q);
-            tt_warp_rows_mma<PM, RB>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
+            if constexpr (TP == 0) tt_warp_rows_mma<PM, RB>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
+            else tt_warp_rows<PM, RB, TP>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
         }
         __syncwarp();
     }
@@ -440,13 +444,13 @@ __global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats, int 
     if (threadIdx.x == 0) next = g0;
     __syncthreads();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    if (V == 0) tt_sweep_quad<16, 32>(w, td, g1, sm + (size_t)wid * (4 * 16 * 32), &next, lane);
-    if (V == 1) tt_sweep_quad<16, 16>(w, td, g1, sm + (size_t)wid * (4 * 16 * 16), &next, lane);
-    if (V == 3) tt_sweep_quad<32, 32>(w, td, g1, sm + (size_t)wid * (4 * 32 * 32), &next, lane);
+    if (V == 0) tt_sweep_quad<16, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 32), &next, lane);
+    if (V == 1) tt_sweep_quad<16, 16, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 16), &next, lane);
+    if (V == 3) tt_sweep_quad<32, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 32 * 32), &next, lane);
+    if (V == 4) tt_sweep_quad<32, 64, 8, 8, 2>(w, td, g1, sm + (size_t)wid * (2 * 32 * 64), &next, lane);
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
     if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1, false>(w, td, g1, As, Cs, &next, lane);
-    if (V == 4) tt_sweep_fast<32, 64, 2, 8, 2, false>(w, td, g1, As, Cs, &next, lane);
 }
 
 // dynamic shared memory of k_sweep_fwd<V> / k_sweep_bwd<V>: four C tiles per warp for the tensor-core variants
@@ -455,6 +459,7 @@ static size_t tt_sweep_smem(int V, int max_pl, int max_c)
     if (V == 0) return (size_t)4 * 4 * 16 * 32 * sizeof(float);
     if (V == 1) return (size_t)4 * 4 * 16 * 16 * sizeof(float);
     if (V == 3) return (size_t)4 * 4 * 32 * 32 * sizeof(float);
+    if (V == 4) return (size_t)4 * 2 * 32 * 64 * sizeof(float);
     return (size_t)4 * (max_pl + max_c) * sizeof(float);
 }
 
