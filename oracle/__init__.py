@@ -79,8 +79,16 @@ def row(n, d, r, cores, g: int) -> np.ndarray:
     return E
 
 
-def forward(n, d, r, N, cores, indices, offsets) -> np.ndarray:
-    """Pooled rows of one table: fp64 [B, D]."""
+def _weights_arg(weights, L):
+    if weights is None:
+        return None, ctypes.c_void_p(None)
+    w = np.ascontiguousarray(np.asarray(weights, dtype=np.float64))
+    assert w.shape == (L,)
+    return w, _p(w)
+
+
+def forward(n, d, r, N, cores, indices, offsets, weights=None, mode: str = "sum") -> np.ndarray:
+    """Pooled rows of one table: fp64 [B, D].  weights: per-lookup factors [L]; mode "sum" (the paper) or "mean"."""
     _check(n, d, r, cores)
     nn, dd, rr = _i64(n), _i64(d), _i64(r)
     idx, off = _i64(indices), _i64(offsets)
@@ -88,12 +96,14 @@ def forward(n, d, r, N, cores, indices, offsets) -> np.ndarray:
     D = int(np.prod(d))
     keep, cp = _core_ptrs(cores)
     out = np.zeros((B, D), dtype=np.float64)
+    wkeep, wp = _weights_arg(weights, idx.shape[0])
     lib().tt_oracle_forward(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
-                            _p(idx), _p(off), ctypes.c_int64(B), _p(out), ctypes.c_int64(D))
+                            _p(idx), _p(off), ctypes.c_int64(B), _p(out), ctypes.c_int64(D), wp,
+                            ctypes.c_int(1 if mode == "mean" else 0))
     return out
 
 
-def backward(n, d, r, N, cores, indices, offsets, grad_out) -> List[np.ndarray]:
+def backward(n, d, r, N, cores, indices, offsets, grad_out, weights=None, mode: str = "sum") -> List[np.ndarray]:
     """Core gradients of one table for loss = sum(grad_out * out): list of fp64 arrays shaped like the cores."""
     _check(n, d, r, cores)
     nn, dd, rr = _i64(n), _i64(d), _i64(r)
@@ -105,8 +115,10 @@ def backward(n, d, r, N, cores, indices, offsets, grad_out) -> List[np.ndarray]:
     keep, cp = _core_ptrs(cores)
     grads = [np.zeros(c.shape, dtype=np.float64) for c in keep]
     gp = (ctypes.c_void_p * len(grads))(*[g.ctypes.data for g in grads])
+    wkeep, wp = _weights_arg(weights, idx.shape[0])
     lib().tt_oracle_backward(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
-                             _p(idx), _p(off), ctypes.c_int64(B), _p(go), ctypes.c_int64(D), gp)
+                             _p(idx), _p(off), ctypes.c_int64(B), _p(go), ctypes.c_int64(D), gp, wp,
+                             ctypes.c_int(1 if mode == "mean" else 0))
     return grads
 
 
@@ -132,25 +144,35 @@ def sgd(cores: Sequence[np.ndarray], grads: Sequence[np.ndarray], lr: float) -> 
 
 # ----------------------------------------------------------------------------- multi-table wrappers
 
-def forward_workload(wl, tables=None, bags=None) -> np.ndarray:
-    """out fp64 [B, T*D] for a workloads.Workload (optionally only some tables; others stay zero)."""
+def _table_weights(wl, t, weights):
+    if weights is None:
+        return None
+    lo, hi = int(wl.offsets[t * wl.B]), int(wl.offsets[(t + 1) * wl.B])
+    return np.asarray(weights)[lo:hi]
+
+
+def forward_workload(wl, tables=None, bags=None, weights=None, mode: str = "sum") -> np.ndarray:
+    """out fp64 [B, T*D] for a workloads.Workload (optionally only some tables; others stay zero).
+    weights: per-lookup factors aligned with wl.indices."""
     D = wl.D
     out = np.zeros((wl.B, wl.T * D), dtype=np.float64)
     for t in (range(wl.T) if tables is None else tables):
         s = wl.tables[t]
         idx, off = wl.table_slice(t)
-        out[:, t * D:(t + 1) * D] = forward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off)
+        out[:, t * D:(t + 1) * D] = forward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off,
+                                            _table_weights(wl, t, weights), mode)
     return out
 
 
-def backward_workload(wl, grad_out=None, tables=None) -> List[List[np.ndarray]]:
+def backward_workload(wl, grad_out=None, tables=None, weights=None, mode: str = "sum") -> List[List[np.ndarray]]:
     go = wl.grad_out if grad_out is None else grad_out
     D = wl.D
     res = []
     for t in (range(wl.T) if tables is None else tables):
         s = wl.tables[t]
         idx, off = wl.table_slice(t)
-        res.append(backward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off, go[:, t * D:(t + 1) * D]))
+        res.append(backward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off, go[:, t * D:(t + 1) * D],
+                            _table_weights(wl, t, weights), mode))
     return res
 
 

@@ -110,13 +110,15 @@ void tt_oracle_row(int K, const int64_t* n, const int64_t* d, const int64_t* r,
 }
 
 /*
- * Pooled forward of ONE table: out[b*out_stride + j] = sum over lookups l in bag b of row(indices[l])[j]
- * (sum pooling, duplicates counted, empty bag -> zeros).  offsets has B+1 entries.
+ * Pooled forward of ONE table: out[b*out_stride + j] = sum over lookups l in bag b of a_l * row(indices[l])[j]
+ * (duplicates counted, empty bag -> zeros).  offsets has B+1 entries.  The paper pools by plain sum (a_l = 1:
+ * weights == NULL, mean == 0).  Two extensions follow the usual embedding-bag operator: per-lookup weights
+ * (a_l = weights[l]) and mean pooling (a_l = 1 / number of lookups of the bag, invalid ones included).
  * Returns the number of indices outside [0, N) (they contribute nothing).
  */
 int64_t tt_oracle_forward(int K, const int64_t* n, const int64_t* d, const int64_t* r, int64_t N,
                           const double* const* cores, const int64_t* indices, const int64_t* offsets,
-                          int64_t B, double* out, int64_t out_stride)
+                          int64_t B, double* out, int64_t out_stride, const double* weights, int mean)
 {
     int64_t D = 1;
     for (int k = 0; k < K; ++k) D *= d[k];
@@ -131,12 +133,15 @@ int64_t tt_oracle_forward(int K, const int64_t* n, const int64_t* d, const int64
         for (int64_t b = 0; b < B; ++b) {
             double* o = out + b * out_stride;
             for (int64_t j = 0; j < D; ++j) o[j] = 0.0;
+            const int64_t len = offsets[b + 1] - offsets[b];
             for (int64_t l = offsets[b]; l < offsets[b + 1]; ++l) {
                 int64_t g = indices[l];
                 if (g < 0 || g >= N) { ++bad; continue; }
+                double a = weights ? weights[l] : 1.0;
+                if (mean) a /= (double)len;
                 tt_oracle_digits(g, K, n, dig);
                 row_forward(K, n, d, r, cores, dig, P_all, P_off, E);
-                for (int64_t j = 0; j < D; ++j) o[j] += E[j];
+                for (int64_t j = 0; j < D; ++j) o[j] += a * E[j];
             }
         }
         free(P_all);
@@ -152,13 +157,15 @@ int64_t tt_oracle_forward(int K, const int64_t* n, const int64_t* d, const int64
  *                  dP_{k-1}[p][a]       = sum_{j,b'} dP_k[(p,j)][b'] * G_k[a][i_k][j][b']  ("dC = dE.D^T")
  *   dG_1[0][i_1][j][b'] += dP_1[j][b']
  * No regrouping by shared prefix (Eq. 2) is used here; that the regrouped form agrees is a test.
+ * With per-lookup weights or mean pooling (see tt_oracle_forward) dP_K = a_l * grad_out[b].
  * core_grads[k] has the shape of cores[k] and is ACCUMULATED INTO (caller zeroes it).
  * Bags are spread over OpenMP threads; each thread accumulates into a private fp64 copy which is
  * added to core_grads at the end (with one thread this is exactly the lookup order).
  */
 int64_t tt_oracle_backward(int K, const int64_t* n, const int64_t* d, const int64_t* r, int64_t N,
                            const double* const* cores, const int64_t* indices, const int64_t* offsets,
-                           int64_t B, const double* grad_out, int64_t grad_stride, double* const* core_grads)
+                           int64_t B, const double* grad_out, int64_t grad_stride, double* const* core_grads,
+                           const double* weights, int mean)
 {
     int64_t D = 1;
     for (int k = 0; k < K; ++k) D *= d[k];
@@ -178,12 +185,15 @@ int64_t tt_oracle_backward(int K, const int64_t* n, const int64_t* d, const int6
 #pragma omp for schedule(dynamic, 16)
         for (int64_t b = 0; b < B; ++b) {
             const double* go = grad_out + b * grad_stride;
+            const int64_t len = offsets[b + 1] - offsets[b];
             for (int64_t l = offsets[b]; l < offsets[b + 1]; ++l) {
                 int64_t g = indices[l];
                 if (g < 0 || g >= N) { ++bad; continue; }
+                double a = weights ? weights[l] : 1.0;
+                if (mean) a /= (double)len;
                 tt_oracle_digits(g, K, n, dig);
                 row_forward(K, n, d, r, cores, dig, P_all, P_off, NULL);
-                for (int64_t e = 0; e < D; ++e) dP[e] = go[e];
+                for (int64_t e = 0; e < D; ++e) dP[e] = a * go[e];
                 int64_t rows = D; /* rows of the partial product after core k */
                 for (int k = K - 1; k >= 1; --k) {
                     int64_t prow = rows / d[k]; /* rows of the partial product before core k */

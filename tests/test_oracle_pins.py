@@ -224,6 +224,42 @@ def test_backward_matches_torch_autograd(rng):
         np.testing.assert_allclose(grads[k], tc[k].grad.numpy(), rtol=1e-11, atol=1e-12)
 
 
+@pytest.mark.parametrize("mode,weighted", [("sum", True), ("mean", False)])
+def test_weighted_and_mean_pooling_match_library_embedding_bag(rng, mode, weighted):
+    # extensions beyond the paper's plain sum: forward against torch's embedding_bag on the brute-force table,
+    # backward against autograd through that same library call (gradient w.r.t. the dense table, contracted with
+    # the other cores by the brute-force definition of d table / d core entry)
+    n, d, r = (3, 4, 3), (2, 3, 2), (1, 3, 2, 1)
+    N = 33
+    cores = rand_cores(rng, n, d, r, 0.5)
+    W = oracle.dense(n, d, r, cores)
+    lens = np.array([4, 0, 1, 6, 2]); off = np.concatenate([[0], np.cumsum(lens)])
+    idx = rng.integers(0, N, size=off[-1]); idx[5] = idx[6]
+    wts = rng.normal(size=off[-1]) if weighted else None
+    go = rng.normal(size=(len(lens), 12))
+    out = oracle.forward(n, d, r, N, cores, idx, off, wts, mode)
+    Wt = torch.from_numpy(W).clone().requires_grad_(True)
+    eb = torch.nn.functional.embedding_bag(torch.from_numpy(idx), Wt, torch.from_numpy(off[:-1]), mode=mode,
+                                           per_sample_weights=None if wts is None else torch.from_numpy(wts))
+    np.testing.assert_allclose(out, eb.detach().numpy(), rtol=1e-12, atol=1e-13)
+    (eb * torch.from_numpy(go)).sum().backward()
+    dW = Wt.grad.numpy()
+    grads = oracle.backward(n, d, r, N, cores, idx, off, go, wts, mode)
+    pick = np.random.default_rng(5)
+    for k in range(3):
+        for e in pick.choice(cores[k].size, size=12, replace=False):
+            c2 = [c.copy() for c in cores]
+            c2[k] = np.zeros_like(cores[k]); c2[k].reshape(-1)[e] = 1.0
+            want = float((oracle.dense(n, d, r, c2) * dW).sum())   # the table is linear in each core
+            assert abs(want - grads[k].reshape(-1)[e]) < 1e-10 * max(1.0, abs(want))
+    # special cases that reduce to the plain sum: unit weights; mean over bags of one lookup
+    ones = oracle.forward(n, d, r, N, cores, idx, off, np.ones(off[-1]), "sum")
+    np.testing.assert_allclose(ones, oracle.forward(n, d, r, N, cores, idx, off), rtol=0, atol=0)
+    off1 = np.arange(off[-1] + 1)
+    np.testing.assert_allclose(oracle.forward(n, d, r, N, cores, idx, off1, None, "mean"),
+                               oracle.forward(n, d, r, N, cores, idx, off1), rtol=0, atol=0)
+
+
 def test_backward_prefix_regrouping_identity_eq2(rng):
     # Eq. 2: for lookups that share the first two digits, (sum_n dC_n).B^T equals sum_n (dC_n.B^T):
     # the gradient of one bag holding all rows of a prefix group equals the sum over single-row bags
