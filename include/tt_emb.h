@@ -76,6 +76,8 @@ typedef struct {
                                    rebuilds its prefix product ("unique only", cf. the paper's reuse ablation);
                                    bit 1 = static schedule, every table cut into units of equal group COUNT instead of
                                    equal cost (cf. the paper's scheduling ablation) */
+    int32_t enable_weighted;    /* 1: tt_emb_set_pooling may select mean pooling or per-lookup weights (with the
+                                   backward enabled the workspace grows by 4 bytes per lookup) */
 } tt_emb_config_t;
 
 /* Host only.  Copies everything it needs out of *cfg.  [data model: Sec. 2.1] */
@@ -110,6 +112,19 @@ int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace, size_t wor
  */
 int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
                    int64_t num_lookups, float* out, tt_emb_stream_t stream);
+
+/*
+ * Pooling mode of the forward / backward calls that follow (default: TT_EMB_POOL_SUM without weights, the paper's
+ * pooling [Sec. 3.2]).  The two other forms are extensions that follow the usual embedding-bag operator; the paper
+ * has no counterpart.
+ *   TT_EMB_POOL_MEAN    out = bag's sum / number of lookups of the bag (an empty bag gives zeros)
+ *   per_sample_weights  device fp32[num_lookups] (or NULL): lookup l contributes weights[l] * row; sum mode only.
+ *                       Must stay valid and unchanged until the backward of the forward that used it has completed.
+ * The backward differentiates the mode its forward used.  Needs cfg.enable_weighted (TT_EMB_ERR_STATE otherwise,
+ * unless mode is SUM and the pointer NULL); weights together with MEAN is TT_EMB_ERR_ARG.  Host only.
+ */
+enum tt_emb_pooling { TT_EMB_POOL_SUM = 0, TT_EMB_POOL_MEAN = 1 };
+int tt_emb_set_pooling(tt_emb_t h, int32_t mode, const float* per_sample_weights);
 
 /*
  * Backward of the most recent forward on this handle, for loss = sum(grad_out * out).

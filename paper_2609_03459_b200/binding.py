@@ -42,6 +42,7 @@ class tt_emb_config_t(ctypes.Structure):
         ("max_unique_rows", ctypes.c_int64),
         ("enable_backward", ctypes.c_int32),
         ("ablation", ctypes.c_int32),
+        ("enable_weighted", ctypes.c_int32),
     ]
 
 
@@ -74,6 +75,7 @@ _SIGS = {
     "tt_emb_export_inverse": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "tt_emb_pack_core": (ctypes.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "tt_emb_unpack_core": (ctypes.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
+    "tt_emb_set_pooling": (ctypes.c_int, [_vp, _i32, _vp]),
     "tt_emb_enable_timing": (ctypes.c_int, [_vp, _i32]),
     "tt_emb_stage_ms": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_f32)]),
     "tt_emb_probe_fp32": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
@@ -107,7 +109,7 @@ def _check(code: int, where: str):
 
 def make_config(num_rows: Sequence[int], row_factors: Sequence[Sequence[int]], dim_factors: Sequence[Sequence[int]],
                 ranks: Sequence[Sequence[int]], max_batch: int, max_lookups: int, max_unique_rows: int = 0,
-                enable_backward: bool = False, ablation: int = 0):
+                enable_backward: bool = False, ablation: int = 0, enable_weighted: bool = False):
     """Returns (tt_emb_config_t, keepalive list of numpy arrays)."""
     T = len(num_rows)
     K = len(row_factors[0])
@@ -116,7 +118,8 @@ def make_config(num_rows: Sequence[int], row_factors: Sequence[Sequence[int]], d
     df = np.ascontiguousarray(np.asarray(dim_factors, dtype=np.int32).reshape(T * K))
     rk = np.ascontiguousarray(np.asarray(ranks, dtype=np.int32).reshape(T * (K + 1)))
     cfg = tt_emb_config_t(T, K, nr.ctypes.data, rf.ctypes.data, df.ctypes.data, rk.ctypes.data,
-                          int(max_batch), int(max_lookups), int(max_unique_rows), 1 if enable_backward else 0, int(ablation))
+                          int(max_batch), int(max_lookups), int(max_unique_rows), 1 if enable_backward else 0, int(ablation),
+                          1 if enable_weighted else 0)
     return cfg, [nr, rf, df, rk]
 
 
@@ -131,7 +134,8 @@ class TTEmbeddingBag:
     (numpy or torch, fp32) and converted on the device to the library's slice-major layout."""
 
     def __init__(self, num_rows, row_factors, dim_factors, ranks, max_batch, max_lookups, *,
-                 max_unique_rows: int = 0, enable_backward: bool = False, ablation: int = 0, device="cuda:0"):
+                 max_unique_rows: int = 0, enable_backward: bool = False, ablation: int = 0,
+                 enable_weighted: bool = False, device="cuda:0"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -140,7 +144,7 @@ class TTEmbeddingBag:
                        for t in range(self.T)]
         self.enable_backward = enable_backward
         cfg, keep = make_config(num_rows, row_factors, dim_factors, ranks, max_batch, max_lookups,
-                                max_unique_rows, enable_backward, ablation)
+                                max_unique_rows, enable_backward, ablation, enable_weighted)
         h = ctypes.c_void_p()
         _check(lib.tt_emb_create(ctypes.byref(cfg), ctypes.byref(h)), "tt_emb_create")
         self.h = h
@@ -240,6 +244,17 @@ class TTEmbeddingBag:
                                   out.data_ptr(), _stream_ptr()), "tt_emb_forward")
         return out
 
+    def set_pooling(self, mode: str = "sum", per_sample_weights=None):
+        """Pooling of the following forward/backward calls: "sum" (default), "mean", or "sum" with per-lookup
+        weights (fp32 device tensor [L]).  Needs enable_weighted=True unless plain sum is selected."""
+        torch = self.torch
+        if per_sample_weights is not None:
+            assert per_sample_weights.dtype == torch.float32 and per_sample_weights.is_cuda and per_sample_weights.is_contiguous()
+        self._keep_w = per_sample_weights
+        _check(lib.tt_emb_set_pooling(self.h, {"sum": 0, "mean": 1}[mode],
+                                      None if per_sample_weights is None else per_sample_weights.data_ptr()),
+               "tt_emb_set_pooling")
+
     def forward_static(self, indices, offsets, batch: int, out=None):
         """Forward through the library's built-in 32 MiB workspace: for callers that must not allocate device
         memory.  Only for configurations whose workspace fits (TTEmbError with ERR_WORKSPACE otherwise).  Calls
@@ -317,11 +332,11 @@ class TTEmbeddingBag:
 
 
 def from_workload(wl, *, enable_backward: bool = False, max_unique_rows: int = 0, ablation: int = 0,
-                  device="cuda:0") -> TTEmbeddingBag:
+                  enable_weighted: bool = False, device="cuda:0") -> TTEmbeddingBag:
     """Build a TTEmbeddingBag for a workloads.Workload-like object (tables with N, n, d, r; B; L; cores)."""
     emb = TTEmbeddingBag([s.N for s in wl.tables], [s.n for s in wl.tables], [s.d for s in wl.tables],
                          [s.r for s in wl.tables], wl.B, max(wl.L, 1), max_unique_rows=max_unique_rows,
-                         enable_backward=enable_backward, ablation=ablation, device=device)
+                         enable_backward=enable_backward, ablation=ablation, enable_weighted=enable_weighted, device=device)
     emb.set_cores(wl.cores)
     return emb
 

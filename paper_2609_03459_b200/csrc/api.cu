@@ -80,6 +80,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->max_batch = cfg->max_batch; h->max_lookups = cfg->max_lookups;
     h->enable_backward = cfg->enable_backward ? 1 : 0;
     h->ablation = cfg->ablation & 3;
+    h->enable_weighted = cfg->enable_weighted != 0;
     if (h->ablation && h->enable_backward) return fail(TT_EMB_ERR_ARG);   // the study switches are forward only
     h->sm_count = 148;
     { int sms = 0; if (device_ok(&sms) && sms > 0) h->sm_count = sms; }
@@ -261,6 +262,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         h->off_cnt = take(((size_t)h->capU + 1) * sizeof(uint32_t));
         h->off_cursor = take((size_t)h->capU * sizeof(uint32_t));
         h->off_pairs = take((size_t)2 * (size_t)(h->max_lookups + 1) * sizeof(uint2));
+        h->off_wsorted = h->enable_weighted ? take((size_t)(h->max_lookups + 1) * sizeof(float)) : 0;
         for (int k = 2; k <= K - 1; ++k) {
             h->off_dP[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
             h->off_Y[k] = take((size_t)v.cap[k] * stride[k - 1] * sizeof(float));
@@ -346,6 +348,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     for (int k = 2; k <= K - 2; ++k) v.pbuf[k] = (float*)(base + h->off_pbuf[k]);
     v.E = (float*)(base + h->off_E);
     v.upairs = nullptr;
+    v.wsorted = nullptr;
     for (int k = 2; k <= K - 1; ++k) {
         v.tbm[k] = (uint2*)(base + h->off_tbm[k]);
         v.tnode[k] = (uint32_t*)(base + h->off_tnode[k]);
@@ -355,6 +358,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
         v.cursor = (uint32_t*)(base + h->off_cursor);
         v.pairs = (uint2*)(base + h->off_pairs);
         v.upairs = v.pairs + (h->max_lookups + 1);
+        v.wsorted = h->enable_weighted ? (float*)(base + h->off_wsorted) : nullptr;
         for (int k = 2; k <= K - 1; ++k) {
             v.dP[k] = (float*)(base + h->off_dP[k]);
             v.Y[k] = (float*)(base + h->off_Y[k]);
@@ -479,6 +483,17 @@ extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t*
     TT_STAGE(h, 2, s, tt_launch_contraction(h, s));
     TT_STAGE(h, 3, s, tt_launch_pooling(h, out, s));
     h->have_forward = true;
+    return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_set_pooling(tt_emb_t h, int32_t mode, const float* per_sample_weights)
+{
+    if (!h || (mode != TT_EMB_POOL_SUM && mode != TT_EMB_POOL_MEAN)) return TT_EMB_ERR_ARG;
+    if (mode == TT_EMB_POOL_MEAN && per_sample_weights) return TT_EMB_ERR_ARG;
+    if ((mode != TT_EMB_POOL_SUM || per_sample_weights) && !h->enable_weighted) return TT_EMB_ERR_STATE;
+    h->v.pool_mean = mode == TT_EMB_POOL_MEAN ? 1 : 0;
+    h->v.psw = per_sample_weights;
+    h->have_forward = false;   // a backward must follow a forward of the same mode
     return TT_EMB_OK;
 }
 

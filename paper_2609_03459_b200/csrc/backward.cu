@@ -94,7 +94,18 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 #pragma unroll
             for (int j = 0; j < HT_TILE / 256; ++j) {
                 if (pr[j].x == HT_EMPTY) continue;
-                w.pairs[vals[hh[j]] + rk[j]] = pr[j];
+                const uint32_t pos = vals[hh[j]] + rk[j];
+                w.pairs[pos] = pr[j];
+                if (w.wsorted && (w.psw || w.pool_mean)) {   // weighted / mean pooling: the pair's factor travels with it
+                    const int64_t l = tile * HT_TILE + j * 256 + threadIdx.x;
+                    float a = w.psw ? __ldg(w.psw + l) : 1.f;
+                    if (w.pool_mean) {
+                        const int64_t gb = (int64_t)tt_find_table(w.tb[w.K], w.T, pr[j].x) * w.B + pr[j].y;
+                        const int64_t len = __ldg(w.offsets + gb + 1) - __ldg(w.offsets + gb);
+                        a /= (float)(len > 0 ? len : 1);
+                    }
+                    w.wsorted[pos] = a;
+                }
             }
         }
         __syncthreads();
@@ -145,7 +156,8 @@ struct RowAcc {
 #pragma unroll
         for (int i = 0; i < (VEC ? 4 * CPL : CPL); ++i) v[i] = 0.f;
     }
-    __device__ void add_row(const float* __restrict__ row, int D, int lane)
+    // v += a * row (a = 1 gives exactly v + row)
+    __device__ void add_row(const float* __restrict__ row, int D, int lane, float a = 1.f)
     {
         if (VEC) {
             const float4* r4 = reinterpret_cast<const float4*>(row);
@@ -154,14 +166,15 @@ struct RowAcc {
                 const int ch = lane + c * 32;
                 if (ch * 4 < D) {
                     const float4 x = __ldg(r4 + ch);
-                    v[4 * c] += x.x; v[4 * c + 1] += x.y; v[4 * c + 2] += x.z; v[4 * c + 3] += x.w;
+                    v[4 * c] = fmaf(a, x.x, v[4 * c]); v[4 * c + 1] = fmaf(a, x.y, v[4 * c + 1]);
+                    v[4 * c + 2] = fmaf(a, x.z, v[4 * c + 2]); v[4 * c + 3] = fmaf(a, x.w, v[4 * c + 3]);
                 }
             }
         } else {
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 const int i = lane + c * 32;
-                if (i < D) v[c] += __ldg(row + i);
+                if (i < D) v[c] = fmaf(a, __ldg(row + i), v[c]);
             }
         }
     }
@@ -207,10 +220,13 @@ __global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ 
     float* carry = w.carry + (size_t)chunk * 2 * D;
     for (uint32_t p0 = a; p0 < b; p0 += 32) {
         const uint2 mine = (p0 + lane < b) ? __ldg(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
+        const bool weighted = w.wsorted && (w.psw || w.pool_mean);
+        const float wmine = (weighted && p0 + lane < b) ? __ldg(&w.wsorted[p0 + lane]) : 1.f;
         const int n = (int)min(32u, b - p0);
         for (int j = 0; j < n; ++j) {
             const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j);
             const uint32_t bag = __shfl_sync(0xffffffffu, mine.y, j);
+            const float wj = __shfl_sync(0xffffffffu, wmine, j);
             if (sl != cur) {
                 const bool open_start = seg_first && prev == cur;
                 if (open_start) acc.store(carry, D, lane);  // head: started in an earlier chunk, ends here
@@ -220,7 +236,7 @@ __global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ 
                 tcur = tt_find_table(w.tb[w.K], w.T, cur);
                 seg_first = false;
             }
-            acc.add_row(grad_out + (size_t)bag * gstride + (size_t)tcur * D, D, lane);
+            acc.add_row(grad_out + (size_t)bag * gstride + (size_t)tcur * D, D, lane, wj);
         }
     }
     const bool open_start = seg_first && prev == cur;
@@ -282,7 +298,7 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
 // NF load instructions issued back to back, then the rows are folded in position order.  Each sub-warp keeps
 // its own partial sum; the sub-warps are combined only when a segment ends.  Segment starts inside a batch of
 // 32 positions are found once with a ballot, so a window without a start costs 4 adds per load and nothing else.
-template <int LPR>
+template <int LPR, bool WT>
 __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __restrict__ grad_out)
 {
     constexpr int RPI = 32 / LPR, NF = 4;
@@ -319,6 +335,7 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
     uint32_t last_slot = cur;  // slot of the position before the current batch
     for (uint32_t p0 = a; p0 < b; p0 += 32) {
         const uint2 mine = (p0 + lane < b) ? __ldcs(&w.pairs[p0 + lane]) : make_uint2(HT_EMPTY, 0u);
+        const float wmine = (WT && p0 + lane < b) ? __ldcs(&w.wsorted[p0 + lane]) : 1.f;   // factor of this lane's pair
         const int n = (int)min(32u, b - p0);
         // row index of this lane's pair inside grad_out viewed as [B*T][D]
         const uint32_t grow = lane < n ? mine.y * (uint32_t)w.T + (uint32_t)tt_find_table(w.tb[w.K], w.T, mine.x) : 0u;
@@ -333,6 +350,10 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
                 const int j = j0 + jj * RPI + sub;
                 const uint32_t gr = __shfl_sync(0xffffffffu, grow, j & 31);
                 v[jj] = (j < n && lane_on) ? __ldg(G4 + (size_t)gr * D4 + lr) : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (WT) {
+                    const float wj = __shfl_sync(0xffffffffu, wmine, j & 31);
+                    v[jj].x *= wj; v[jj].y *= wj; v[jj].z *= wj; v[jj].w *= wj;
+                }
             }
 #pragma unroll
             for (int jj = 0; jj < NF; ++jj) {
@@ -372,9 +393,10 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
     const int grid = (int)((chunks + 7) / 8);
     if (grid > 0) {
         const int D4 = h->D / 4;
-        if (VEC && D4 <= 8) { k_dE_fast<8><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
-        else if (VEC && D4 <= 16) { k_dE_fast<16><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
-        else if (VEC && D4 <= 32) { k_dE_fast<32><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        const bool wt = h->v.wsorted && (h->v.psw || h->v.pool_mean);
+        if (VEC && D4 <= 8) { if (wt) k_dE_fast<8, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<8, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        else if (VEC && D4 <= 16) { if (wt) k_dE_fast<16, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<16, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
+        else if (VEC && D4 <= 32) { if (wt) k_dE_fast<32, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<32, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else { k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         k_dE_fix<VEC, CPL><<<grid, 256, 0, s>>>(h->v);
         tt_note_launch();

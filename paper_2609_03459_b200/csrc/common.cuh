@@ -77,6 +77,10 @@ struct WsView {
     uint32_t* tnode[TT_MAXK + 1];       // nodes of level k ordered by (table, i_k, parent prefix)
     const int64_t* indices;
     const int64_t* offsets;
+    // pooling beyond the plain sum (tt_emb_set_pooling)
+    const float* psw;                   // per-lookup weights [L] or null
+    float* wsorted;                     // [L] factor of every sorted pair (weight, or 1 / bag length), backward only
+    int32_t pool_mean;                  // 1: mean pooling
 };
 
 enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16 };
@@ -85,6 +89,7 @@ struct tt_emb {
     int T, K, D;
     int64_t max_batch, max_lookups, capU;
     int enable_backward;
+    int enable_weighted;
     int ablation;
     int sm_count;
     int units_total;
@@ -100,7 +105,7 @@ struct tt_emb {
     size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
     size_t off_Y[TT_MAXK + 1];
-    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart;
+    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted;
     size_t scan_tmp_elems;
     int64_t gpart_floats;
     WsView v;             // filled at bind

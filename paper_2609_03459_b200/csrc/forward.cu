@@ -545,7 +545,7 @@ __device__ __forceinline__ int64_t tt_pool_chunks(int64_t L, int64_t W)
     return c < 1 ? 1 : (c > 8 ? 8 : c);
 }
 
-template <int LPR, int CPL>  // lanes per row, float4 chunks per lane
+template <int LPR, int CPL, bool WT>  // lanes per row, float4 chunks per lane, weighted / mean pooling
 __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
 {
     const int lane = threadIdx.x & 31;
@@ -584,7 +584,13 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
     int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
     if (o_hi < o_lo) o_hi = o_lo;
     int t = (int)(b0 / w.B);
-    uint32_t slot_next = (o_lo + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], o_lo + lane, capK) : 0xffffffffu;
+    uint32_t slot_next;
+    float wt_next = 1.f;
+    auto fetch = [&](int64_t base, int64_t lim, int tt) {   // rank look-up (and weight) of lookup base + lane
+        slot_next = (base + lane < lim) ? tt_lookup_slot(w, w.tdesc[tt], base + lane, capK) : 0xffffffffu;
+        if (WT) wt_next = (w.psw && base + lane < lim) ? __ldg(w.psw + base + lane) : 1.f;
+    };
+    fetch(o_lo, o_hi, t);
     for (int64_t bag = b0; bag < b1; ++bag) {
         const int64_t b = bag - (int64_t)t * w.B;
         // next bag (for the prefetch of its first 32 rank look-ups)
@@ -595,13 +601,13 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
         float4 acc[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (o_lo >= o_hi && has_next)
-            slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+        if (o_lo >= o_hi && has_next) fetch(o_hi, n_hi, tn);
         for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
+            const float wt = wt_next;
             if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));  // kept for the backward sort
-            if (l0 + 32 < o_hi) slot_next = (l0 + 32 + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], l0 + 32 + lane, capK) : 0xffffffffu;
-            else if (has_next) slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+            if (l0 + 32 < o_hi) fetch(l0 + 32, o_hi, t);
+            else if (has_next) fetch(o_hi, n_hi, tn);
             const int n = (int)min((int64_t)32, o_hi - l0);
 #pragma unroll
             for (int j0 = 0; j0 < NIT; j0 += NF) {
@@ -620,11 +626,18 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
                     }
                 }
 #pragma unroll
-                for (int jj = 0; jj < NF; ++jj)
+                for (int jj = 0; jj < NF; ++jj) {
+                    const float wj = WT ? __shfl_sync(0xffffffffu, wt, ((j0 + jj) * RPI + sub) & 31) : 1.f;
 #pragma unroll
                     for (int c = 0; c < CPL; ++c) {
-                        acc[c].x += v[jj][c].x; acc[c].y += v[jj][c].y; acc[c].z += v[jj][c].z; acc[c].w += v[jj][c].w;
+                        if (WT) {
+                            acc[c].x = fmaf(wj, v[jj][c].x, acc[c].x); acc[c].y = fmaf(wj, v[jj][c].y, acc[c].y);
+                            acc[c].z = fmaf(wj, v[jj][c].z, acc[c].z); acc[c].w = fmaf(wj, v[jj][c].w, acc[c].w);
+                        } else {
+                            acc[c].x += v[jj][c].x; acc[c].y += v[jj][c].y; acc[c].z += v[jj][c].z; acc[c].w += v[jj][c].w;
+                        }
                     }
+                }
             }
         }
 #pragma unroll
@@ -639,9 +652,11 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
         }
         if (sub == 0) {
             float4* o4 = reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D);
+            const float inv = (WT && w.pool_mean && o_hi > o_lo) ? 1.f / (float)(o_hi - o_lo) : 1.f;
 #pragma unroll
             for (int c = 0; c < CPL; ++c) {
                 const int ch = lr + c * LPR;
+                if (WT) { acc[c].x *= inv; acc[c].y *= inv; acc[c].z *= inv; acc[c].w *= inv; }
                 if (ch < D4) __stcs(o4 + ch, acc[c]);
             }
         }
@@ -662,6 +677,7 @@ __device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
 
+template <bool WT>
 __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restrict__ out)
 {
     extern __shared__ __align__(16) float4 pool_buf[];   // [8 warps][32 rows][16 float4]
@@ -698,7 +714,13 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
     int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
     if (o_hi < o_lo) o_hi = o_lo;
     int t = (int)(b0 / w.B);
-    uint32_t slot_next = (o_lo + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], o_lo + lane, capK) : 0xffffffffu;
+    uint32_t slot_next;
+    float wt_next = 1.f;
+    auto fetch = [&](int64_t base, int64_t lim, int tt) {   // rank look-up (and weight) of lookup base + lane
+        slot_next = (base + lane < lim) ? tt_lookup_slot(w, w.tdesc[tt], base + lane, capK) : 0xffffffffu;
+        if (WT) wt_next = (w.psw && base + lane < lim) ? __ldg(w.psw + base + lane) : 1.f;
+    };
+    fetch(o_lo, o_hi, t);
     for (int64_t bag = b0; bag < b1; ++bag) {
         const int64_t b = bag - (int64_t)t * w.B;
         const bool has_next = bag + 1 < b1;
@@ -706,10 +728,10 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
         if (n_hi < o_hi) n_hi = o_hi;
         const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (o_lo >= o_hi && has_next)
-            slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+        if (o_lo >= o_hi && has_next) fetch(o_hi, n_hi, tn);
         for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
+            const float wt = wt_next;
             if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));
             const int n = (int)min((int64_t)32, o_hi - l0);
             const unsigned valid = __ballot_sync(0xffffffffu, lane < n && slot != 0xffffffffu);
@@ -722,22 +744,28 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             // the rank look-ups of the next batch (or of the next bag) overlap the gather
-            if (l0 + 32 < o_hi) slot_next = (l0 + 32 + lane < o_hi) ? tt_lookup_slot(w, w.tdesc[t], l0 + 32 + lane, capK) : 0xffffffffu;
-            else if (has_next) slot_next = (o_hi + lane < n_hi) ? tt_lookup_slot(w, w.tdesc[tn], o_hi + lane, capK) : 0xffffffffu;
+            if (l0 + 32 < o_hi) fetch(l0 + 32, o_hi, t);
+            else if (has_next) fetch(o_hi, n_hi, tn);
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) {
                 const int j = 2 * jj + sub;
+                const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
                 if (((valid >> j) & 1u) && lane_on) {
                     const float4 v = buf[j * 16 + lr];
-                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    if (WT) { acc.x = fmaf(wj, v.x, acc.x); acc.y = fmaf(wj, v.y, acc.y); acc.z = fmaf(wj, v.z, acc.z); acc.w = fmaf(wj, v.w, acc.w); }
+                    else { acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
                 }
             }
             __syncwarp();
         }
         acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
         acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+        if (WT && w.pool_mean && o_hi > o_lo) {
+            const float inv = 1.f / (float)(o_hi - o_lo);
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        }
         if (sub == 0 && lane_on) __stcs(reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr, acc);
         o_lo = o_hi;
         o_hi = n_hi;
@@ -746,29 +774,30 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
     }
 }
 
+template <bool WT>
 static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
 {
     const size_t smem = (size_t)8 * 32 * 16 * sizeof(float4);
-    cudaError_t e = cudaFuncSetAttribute(k_pool_async, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_pool_async<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async, 256, smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async<WT>, 256, smem)) != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const int64_t nb = (int64_t)h->v.T * h->v.B;
     int64_t grid = (int64_t)per_sm * h->sm_count;
     const int64_t need = (nb + 7) / 8;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_async<<<(int)grid, 256, smem, s>>>(h->v, out);
+    k_pool_async<WT><<<(int)grid, 256, smem, s>>>(h->v, out);
     tt_note_launch();
     return cudaGetLastError();
 }
 
-template <int LPR, int CPL>
+template <int LPR, int CPL, bool WT>
 static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
 {
     int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_vec<LPR, CPL>, 256, 0);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_vec<LPR, CPL, WT>, 256, 0);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const int64_t nb = (int64_t)h->v.T * h->v.B;
@@ -776,7 +805,7 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
     const int64_t need = (nb + 7) / 8;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_vec<LPR, CPL><<<(int)grid, 256, 0, s>>>(h->v, out);
+    k_pool_vec<LPR, CPL, WT><<<(int)grid, 256, 0, s>>>(h->v, out);
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -820,19 +849,34 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
                 const uint32_t slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
                 if (slot >= capK) continue;
                 const float* row = w.E + (size_t)slot * D;
+                const float a = w.psw ? __ldg(w.psw + l) : 1.f;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const int idx = e0 + lane + c * 32;
-                    if (idx < D) acc[c] += __ldg(row + idx);
+                    if (idx < D) acc[c] = fmaf(a, __ldg(row + idx), acc[c]);
                 }
             }
+            const float inv = (w.pool_mean && hi > lo) ? 1.f / (float)(hi - lo) : 1.f;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int idx = e0 + lane + c * 32;
-                if (idx < D) o[idx] = acc[c];
+                if (idx < D) o[idx] = acc[c] * inv;
             }
         }
     }
+}
+
+template <bool WT>
+static cudaError_t launch_pool_sized(tt_emb* h, int D4, float* out, cudaStream_t s)
+{
+    if (D4 > 8 && D4 <= 16) return launch_pool_async<WT>(h, out, s);
+    if (D4 <= 4) return launch_pool_vec<4, 1, WT>(h, out, s);
+    if (D4 <= 8) return launch_pool_vec<8, 1, WT>(h, out, s);
+    if (D4 <= 16) return launch_pool_vec<16, 1, WT>(h, out, s);
+    if (D4 <= 32) return launch_pool_vec<32, 1, WT>(h, out, s);
+    if (D4 <= 64) return launch_pool_vec<32, 2, WT>(h, out, s);
+    if (D4 <= 128) return launch_pool_vec<32, 4, WT>(h, out, s);
+    return launch_pool_vec<32, 8, WT>(h, out, s);
 }
 
 cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
@@ -852,12 +896,5 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
     }
     const int D4 = D / 4;
     (void)grid;
-    if (D4 > 8 && D4 <= 16) return launch_pool_async(h, out, s);
-    if (D4 <= 4) return launch_pool_vec<4, 1>(h, out, s);
-    if (D4 <= 8) return launch_pool_vec<8, 1>(h, out, s);
-    if (D4 <= 16) return launch_pool_vec<16, 1>(h, out, s);
-    if (D4 <= 32) return launch_pool_vec<32, 1>(h, out, s);
-    if (D4 <= 64) return launch_pool_vec<32, 2>(h, out, s);
-    if (D4 <= 128) return launch_pool_vec<32, 4>(h, out, s);
-    return launch_pool_vec<32, 8>(h, out, s);
+    return (w.psw || w.pool_mean) ? launch_pool_sized<true>(h, D4, out, s) : launch_pool_sized<false>(h, D4, out, s);
 }

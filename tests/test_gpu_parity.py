@@ -162,6 +162,48 @@ def test_sweep_point_shapes(binding, D, rank):
             assert_close(grads[t][k], ref[t][k], f"sweep D{D} r{rank} dG[{t}][{k}]")
 
 
+POOLING_CASES = [MEDIUM[0], MEDIUM[1], MEDIUM[2], MEDIUM[4], MEDIUM[6], MEDIUM[7]]   # D = 64 (cp.async pooling), D = 128, K = 2, odd D, wide D
+
+
+@pytest.mark.parametrize("mode", ["weighted", "mean"])
+@pytest.mark.parametrize("case", POOLING_CASES, ids=[c[0] for c in POOLING_CASES])
+def test_weighted_and_mean_pooling(binding, case, mode):
+    # per-lookup weights and mean pooling (extensions beyond the plain sum), forward and backward
+    name, tables, B, pooling = case
+    wl = workloads.custom(tables, B, pooling, seed=91, with_grad=True, name=name)
+    wts = np.random.default_rng(17).normal(size=wl.L).astype(np.float32) if mode == "weighted" else None
+    omode = "mean" if mode == "mean" else "sum"
+    emb = binding.from_workload(wl, enable_backward=True, enable_weighted=True)
+    emb.set_pooling(omode, None if wts is None else dev(wts))
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl, weights=wts, mode=omode), f"{name} {mode} out")
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl, weights=wts, mode=omode)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"{name} {mode} dG[{t}][{k}]")
+    # back to the plain sum on the same handle
+    emb.set_pooling("sum")
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    assert_close(out, oracle.forward_workload(wl), f"{name} sum after {mode}")
+
+
+def test_pooling_modes_need_the_config_flag(binding):
+    name, tables, B, pooling = MEDIUM[0]
+    wl = workloads.custom(tables, B, pooling, seed=5)
+    emb = binding.from_workload(wl)
+    emb.set_pooling("sum")                       # the default is always allowed
+    with pytest.raises(binding.TTEmbError):
+        emb.set_pooling("mean")
+    emb2 = binding.from_workload(wl, enable_weighted=True)
+    with pytest.raises(binding.TTEmbError):     # weights go with the sum mode only
+        import ctypes
+        from paper_2609_03459_b200.binding import lib, _check
+        _check(lib.tt_emb_set_pooling(emb2.h, 1, dev(np.ones(4, np.float32)).data_ptr()), "tt_emb_set_pooling")
+
+
 def test_forward_only_handle_and_repeat_calls(binding):
     # a forward-only handle (no backward workspace) gives the same output, and calling twice is idempotent
     name, tables, B, pooling = MEDIUM[0]
