@@ -1247,7 +1247,7 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
     constexpr int ST = 4;   // stages of the node pipeline (cp.async, no staging registers)
     __shared__ __align__(16) float sA[ST][M * RA];
     __shared__ __align__(16) float sD[ST][M * COLS];
-    const int t = blockIdx.y;
+    const int t = w.vlist[w.T + blockIdx.y];   // largest tables first: their long node lists start early
     const TableDesc& td = w.tdesc[t];
     const int kc = k - 1;
     if (td.midfast[k] != variant || (int)blockIdx.x >= td.n[kc]) return;

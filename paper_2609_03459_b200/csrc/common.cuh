@@ -52,7 +52,8 @@ struct WsView {
     int32_t* status;
     uint32_t* counters;                 // [k] = number of level-k nodes (k = 1..K); [8+k] transposed counts
     TableDesc* tdesc;
-    int32_t* vlist;                     // table ids grouped by kernel variant (generic first)
+    int32_t* vlist;                     // [0,T): table ids grouped by kernel variant (generic first); [T,2T): all tables;
+                                        // largest tables first inside each list
     int64_t* tl_start;                  // [T+1] first lookup of each table
     uint2* bm;                          // {32 presence bits, number of set bits before this word (global)}
     uint32_t* scan_tmp;
