@@ -147,6 +147,12 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
 
 // ---------------------------------------------------------------------------------------------- 2. dE
 
+__device__ __forceinline__ void tt_cp_async16_b(void* smem_dst, const void* gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
 // lane l of the warp owns float4 chunks l, l+32, ... of a row (VEC) or floats l, l+32, ... (!VEC)
 template <bool VEC, int CPL>
 struct RowAcc {
@@ -386,6 +392,98 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
     }
 }
 
+// D = 64 (256-byte rows): the 32 grad_out rows of a batch of sorted positions are fetched into an 8 KB per-warp
+// buffer with cp.async (all in flight at once, no staging registers), then every lane walks the batch in position
+// order owning two of the 64 columns: one shared-memory load and two adds per row, a coalesced 256-byte store when a
+// segment ends, and no shuffles to combine partial sums.  About half the instructions per lookup of k_dE_fast, which
+// was bound by instruction issue.  Chunks, carries and the fix-up pass are those of k_dE / k_dE_fast.
+template <bool WT>
+__global__ void __launch_bounds__(256, 3) k_dE_stage(WsView w, const float* __restrict__ grad_out)
+{
+    extern __shared__ __align__(16) float4 de_buf[];   // [8 warps][32 rows][16 float4]
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane >> 4, lr = lane & 15;
+    float4* buf = de_buf + (size_t)wid * 32 * 16;
+    const float2* buf2 = reinterpret_cast<const float2*>(buf);
+    const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
+    const uint32_t Ltot = w.cnt[U];
+    const int64_t a64 = chunk * TT_DE_CHUNK;
+    if (a64 >= Ltot) return;
+    const uint32_t a = (uint32_t)a64;
+    const uint32_t b = min(a + (uint32_t)TT_DE_CHUNK, Ltot);
+    const uint32_t prev = a > 0 ? w.pairs[a - 1].x : HT_EMPTY;
+    const uint32_t next = b < Ltot ? w.pairs[b].x : HT_EMPTY;
+    const float4* __restrict__ G4 = reinterpret_cast<const float4*>(grad_out);
+    float2* __restrict__ E2 = reinterpret_cast<float2*>(w.E);
+    float2* carry2 = reinterpret_cast<float2*>(w.carry + (size_t)chunk * 2 * 64);
+    const uint32_t* __restrict__ tbK = w.tb[w.K];
+    float2 acc = make_float2(0.f, 0.f);
+    uint32_t cur = w.pairs[a].x;
+    bool seg_first = true;
+    uint32_t last_slot = cur;
+    // slot range of the table the chunk is in: positions are sorted, so a batch rarely leaves it
+    int tcur = tt_find_table(tbK, w.T, cur);
+    uint32_t t_lo = tbK[tcur], t_hi = tbK[tcur + 1];
+    auto close_segment = [&]() {
+        float2* dst = (seg_first && prev == cur) ? carry2 : E2 + (size_t)cur * 32;   // head piece or whole segment
+        dst[lane] = acc;
+        acc = make_float2(0.f, 0.f);
+        seg_first = false;
+    };
+    uint2 mine = (a + lane < b) ? __ldcs(&w.pairs[a + lane]) : make_uint2(HT_EMPTY, 0u);
+    float wmine = (WT && a + lane < b) ? __ldcs(&w.wsorted[a + lane]) : 1.f;
+    for (uint32_t p0 = a; p0 < b; p0 += 32) {
+        const int n = (int)min(32u, b - p0);
+        int tl = tcur;
+        if (!__all_sync(0xffffffffu, lane >= n || (mine.x >= t_lo && mine.x < t_hi))) {
+            tl = lane < n ? tt_find_table(tbK, w.T, mine.x) : tcur;
+            tcur = __shfl_sync(0xffffffffu, tl, n - 1);
+            t_lo = tbK[tcur];
+            t_hi = tbK[tcur + 1];
+        }
+        const uint32_t grow = mine.y * (uint32_t)w.T + (uint32_t)tl;   // row of grad_out viewed as [B*T][64]
+        uint32_t before = __shfl_up_sync(0xffffffffu, mine.x, 1);
+        if (lane == 0) before = last_slot;
+        const unsigned starts = __ballot_sync(0xffffffffu, lane < n && mine.x != before);   // bit j: position j opens a segment
+        last_slot = __shfl_sync(0xffffffffu, mine.x, n - 1);
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+            const int j = 2 * jj + sub;
+            const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
+            if (j < n) tt_cp_async16_b(buf + j * 16 + lr, G4 + (size_t)gr * 16 + lr);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        // the pairs of the next batch arrive while the rows are in flight
+        const uint2 cur_pairs = mine;
+        const float cur_w = wmine;
+        if (p0 + 32 < b) {
+            mine = (p0 + 32 + lane < b) ? __ldcs(&w.pairs[p0 + 32 + lane]) : make_uint2(HT_EMPTY, 0u);
+            if (WT) wmine = (p0 + 32 + lane < b) ? __ldcs(&w.wsorted[p0 + 32 + lane]) : 1.f;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+#pragma unroll 8
+        for (int j = 0; j < n; ++j) {
+            if ((starts >> j) & 1u) {
+                close_segment();
+                cur = __shfl_sync(0xffffffffu, cur_pairs.x, j);
+            }
+            float2 x = buf2[j * 32 + lane];
+            if (WT) {
+                const float wj = __shfl_sync(0xffffffffu, cur_w, j);
+                x.x *= wj; x.y *= wj;
+            }
+            acc.x += x.x; acc.y += x.y;
+        }
+        __syncwarp();
+    }
+    {   // last segment of the chunk: tail / head / whole
+        const bool open_start = seg_first && prev == cur;
+        float2* dst = next == cur ? carry2 + 32 : (open_start ? carry2 : E2 + (size_t)cur * 32);
+        dst[lane] = acc;
+    }
+}
+
 template <bool VEC, int CPL>
 static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
 {
@@ -394,6 +492,13 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
     if (grid > 0) {
         const int D4 = h->D / 4;
         const bool wt = h->v.wsorted && (h->v.psw || h->v.pool_mean);
+        if (VEC && h->D == 64) {
+            const size_t smem = (size_t)8 * 32 * 16 * sizeof(float4);
+            cudaError_t e = cudaFuncSetAttribute(wt ? k_dE_stage<true> : k_dE_stage<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            if (wt) k_dE_stage<true><<<grid, 256, smem, s>>>(h->v, grad_out); else k_dE_stage<false><<<grid, 256, smem, s>>>(h->v, grad_out);
+            tt_note_launch();
+        } else
         if (VEC && D4 <= 8) { if (wt) k_dE_fast<8, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<8, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else if (VEC && D4 <= 16) { if (wt) k_dE_fast<16, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<16, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else if (VEC && D4 <= 32) { if (wt) k_dE_fast<32, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<32, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
@@ -1207,11 +1312,6 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 //     Y[m][a]     = sum_c dP_k[m][c] * G_k[a][c]                    (partial over its 4 columns)
 // The Y partials are combined over the TC lanes that share an a-range by a reduce-scatter of warp shuffles and
 // written once per node; k_mid_sum then adds the Y rows of each parent's (contiguous) children.
-__device__ __forceinline__ void tt_cp_async16_b(void* smem_dst, const void* gsrc)
-{
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
 
 template <int NVAL, int W>
 __device__ __forceinline__ int tt_reduce_scatter(float (&v)[NVAL], int lane)

@@ -10,7 +10,7 @@
 #define TT_SCAN_THREADS 256
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
-#define TT_DE_CHUNK 256                                  // sorted lookups per warp in the dE segment reduction
+#define TT_DE_CHUNK 1024                                  // sorted lookups per warp in the dE segment reduction
 #define TT_NUM_STAGES 21                                // 0..8 pipeline stages, 9..14 forward sweep variants, 15..20 backward sweep variants
 #define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
 #define TT_NUM_VARIANTS 5                                // register-tiled shape variants (forward.cu)
