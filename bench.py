@@ -363,6 +363,14 @@ def main():
 
     # ---- forward only (same inputs)
     fwd_ms = timed(lambda: emb.forward(d_idx, d_off, B, out=d_out), args.steps) / args.steps
+    # the same forward replayed from a CUDA graph (fixed buffers): what the launch-latency-bound small batches gain
+    fwd_graph_ms = None
+    if not train and L <= 4_000_000:
+        graph = emb.capture_forward(d_idx, d_off, B, d_out)
+        for _ in range(3):
+            graph.replay()
+        fwd_graph_ms = timed(graph.replay, args.steps) / args.steps
+        del graph
 
     # ---- end to end through host buffers
     e2e = None
@@ -497,7 +505,8 @@ def main():
                    "parallelism": f"dp{world} (batch-sharded replicas" + (", all-reduce of core gradients)" if train else ")"),
                    "l2_policy": "inputs larger than L2 (indices alone are %.0f MB)" % (L * 8 / 1e6)},
         "forward_only": {"value": world * L / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,
-                         "roofline_frac": fwd_roof_t * 1e3 / fwd_ms, "t_roof_ms": fwd_roof_t * 1e3},
+                         "roofline_frac": fwd_roof_t * 1e3 / fwd_ms, "t_roof_ms": fwd_roof_t * 1e3,
+                         "cuda_graph_ms_per_step": fwd_graph_ms},
         "stage_ms": stage_ms, "solo_kernel_ms": solo_ms, "roofline": roofline, "kernel_rooflines": kernel_rooflines, "step_roofline": step_roof,
         "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
                   "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},

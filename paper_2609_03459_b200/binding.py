@@ -244,6 +244,19 @@ class TTEmbeddingBag:
                                   out.data_ptr(), _stream_ptr()), "tt_emb_forward")
         return out
 
+    def capture_forward(self, indices, offsets, batch: int, out):
+        """CUDA graph of one forward on fixed buffers (same batch and number of lookups at every replay; the CONTENTS
+        of `indices` / `offsets` may change between replays: grouping, schedule and all counts are computed on the
+        device).  For launch-latency-bound small batches: replaying the graph saves the per-kernel launch cost of
+        the ~25 small kernels of a forward.  Returns a torch.cuda.CUDAGraph; call .replay()."""
+        torch = self.torch
+        self.forward(indices, offsets, batch, out=out)      # first call outside the capture: creates streams, sets attributes
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.forward(indices, offsets, batch, out=out)
+        return g
+
     def set_pooling(self, mode: str = "sum", per_sample_weights=None):
         """Pooling of the following forward/backward calls: "sum" (default), "mean", or "sum" with per-lookup
         weights (fp32 device tensor [L]).  Needs enable_weighted=True unless plain sum is selected."""

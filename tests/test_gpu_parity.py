@@ -204,6 +204,30 @@ def test_pooling_modes_need_the_config_flag(binding):
         _check(lib.tt_emb_set_pooling(emb2.h, 1, dev(np.ones(4, np.float32)).data_ptr()), "tt_emb_set_pooling")
 
 
+def test_forward_replayed_from_a_cuda_graph(binding):
+    # the forward is capturable (no host synchronisation, fork/join of the side streams inside the capture); a replay
+    # on new contents of the same buffers gives the new result
+    import torch
+    name, tables, B, pooling = MEDIUM[1]
+    wl = workloads.custom(tables, B, 7, seed=31, name=name)
+    wl2 = workloads.custom(tables, B, 7, seed=32, name=name)      # same shapes and lookup count, other rows
+    assert wl.L == wl2.L
+    wl2.cores = wl.cores
+    emb = binding.from_workload(wl)
+    d_idx, d_off = dev(wl.indices), dev(wl.offsets)
+    out = torch.empty((wl.B, wl.T * wl.D), dtype=torch.float32, device="cuda")
+    g = emb.capture_forward(d_idx, d_off, wl.B, out)
+    g.replay()
+    torch.cuda.synchronize()
+    assert_close(out.cpu().numpy(), oracle.forward_workload(wl), "graph replay 1")
+    d_idx.copy_(dev(wl2.indices))
+    d_off.copy_(dev(wl2.offsets))
+    g.replay()
+    torch.cuda.synchronize()
+    assert emb.status() == 0
+    assert_close(out.cpu().numpy(), oracle.forward_workload(wl2), "graph replay 2")
+
+
 def test_forward_only_handle_and_repeat_calls(binding):
     # a forward-only handle (no backward workspace) gives the same output, and calling twice is idempotent
     name, tables, B, pooling = MEDIUM[0]
