@@ -1020,13 +1020,17 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 }
 
 template <int PM, int RB_, int TP, int M, int CPL, bool MMA>
-__device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* gk,
-                                                  float* As, float* Cs, int lane, int wid, int nw)
+__device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDesc& td, uint32_t g1, float* gk,
+                                                  float* As, float* Cs, uint32_t* next, int lane)
 {
     const int K = w.K, km = K - 2;
     const int ra = td.r[km], cols = td.d[km] * RB_;
     const uint32_t nK = (uint32_t)td.n[K - 1];
-    for (uint32_t j = g0 + wid; j < g1; j += nw) {
+    for (;;) {   // groups are handed out through a shared counter: their row counts differ widely
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(next, 1u);
+        j = __shfl_sync(0xffffffffu, j, 0);
+        if (j >= g1) break;
         const uint32_t g = w.tnode[K - 1][j];   // units are cut from the digit-major order (see forward.cu)
         const uint32_t val = w.val[K - 1][g];
         const float* src = tt_left_operand_b(w, td, K - 1, g);
@@ -1076,14 +1080,17 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
         tt_sweep_bwd_generic(w, td, g0, g1, gk, Pl, Cs, dCs, dEs);
         return;
     }
+    __shared__ uint32_t next;
+    if (threadIdx.x == 0) next = g0;
+    __syncthreads();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
-    if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
-    if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g0, g1, gk, As, Cs, lane, wid, 4);
+    if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g1, gk, As, Cs, &next, lane);
 }
 
 // fixed-order sum of the partial copies of the last core's gradient
