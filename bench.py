@@ -428,16 +428,18 @@ def main():
         unit, per = NCU_TRAFFIC[kernel]
         return per * (wl.L if unit == "lookup" else work["U_rows"] * share)
 
+    # (P_{K-1}, r_{K-1}) -> sweep kernel variant (last dim factor 4, at least 3 cores)
+    VARIANT_OF = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4, (8, 32): 5, (8, 16): 6, (8, 8): 7, (4, 32): 8, (4, 16): 9}
     variant_rows = {}   # distinct rows handled by each sweep variant
     for t, s in enumerate(wl.tables):
-        v = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4}.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
+        v = VARIANT_OF.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
             if (s.d[-1] == 4 and K >= 3) else -1
         variant_rows[v] = variant_rows.get(v, 0) + int(counts[t, K - 1])
 
     def variant_slots(v, backward):
         tot = 0
         for t, s in enumerate(wl.tables):
-            vv = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4}.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
+            vv = VARIANT_OF.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
                 if (s.d[-1] == 4 and K >= 3) else -1
             if vv != v:
                 continue

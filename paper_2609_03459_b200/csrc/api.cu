@@ -180,6 +180,12 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (PMv == 16 && Mv == 4 && RBv == 8) td.fast = 2;
             else if (PMv == 32 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 3;
             else if (PMv == 32 && Mv == 8 && RBv == 64 && td.r[K - 2] <= 64) td.fast = 4;
+            // first dim factor 2 (D = 32 as 2x4x4, D = 16 as 2x2x4): FP32-pipe variants
+            else if (PMv == 8 && Mv == 2 && RBv == 32) td.fast = 5;
+            else if (PMv == 8 && Mv == 2 && RBv == 16) td.fast = 6;
+            else if (PMv == 8 && Mv == 2 && RBv == 8) td.fast = 7;
+            else if (PMv == 4 && Mv == 2 && RBv == 32) td.fast = 8;
+            else if (PMv == 4 && Mv == 2 && RBv == 16) td.fast = 9;
         }
         for (int k = 0; k < TT_MAXK; ++k) td.midfast[k] = -1;
         for (int k = 2; k <= K - 1; ++k) {
@@ -188,6 +194,10 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (Mv == 4 && rav == 16 && colsv == 128) td.midfast[k] = 1;
             else if (Mv == 4 && rav == 32 && colsv == 64) td.midfast[k] = 2;
             else if (Mv == 4 && rav == 16 && colsv == 64) td.midfast[k] = 3;
+            else if (Mv == 2 && rav == 32 && colsv == 128) td.midfast[k] = 4;
+            else if (Mv == 2 && rav == 16 && colsv == 64) td.midfast[k] = 5;
+            else if (Mv == 2 && rav == 32 && colsv == 64) td.midfast[k] = 6;
+            else if (Mv == 2 && rav == 16 && colsv == 32) td.midfast[k] = 7;
         }
         td.unit_base = unit_base;
         unit_base += Q;
@@ -483,7 +493,7 @@ extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t*
     v.indices = indices; v.offsets = offsets;
     h->have_forward = false;
     for (int i = 0; i < 4; ++i) h->ev_valid[i] = false;
-    for (int i = 9; i < 15; ++i) h->ev_valid[i] = false;
+    for (int i = 9; i < 9 + TT_NUM_VARIANTS + 1; ++i) h->ev_valid[i] = false;
     TT_STAGE(h, 0, s, tt_launch_grouping(h, s));
     TT_STAGE(h, 1, s, tt_launch_schedule(h, s));
     TT_STAGE(h, 2, s, tt_launch_contraction(h, s));
@@ -524,7 +534,7 @@ extern "C" int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* 
     int r = upload_grads(h, core_grads, s);
     if (r) return r;
     for (int i = 4; i < 8; ++i) h->ev_valid[i] = false;
-    for (int i = 15; i < 21; ++i) h->ev_valid[i] = false;
+    for (int i = 9 + TT_NUM_VARIANTS + 1; i < TT_NUM_STAGES; ++i) h->ev_valid[i] = false;
     TT_STAGE(h, 4, s, tt_launch_bwd_sort(h, s));
     TT_STAGE(h, 5, s, tt_launch_bwd_dE(h, grad_out, s));
     TT_STAGE(h, 6, s, tt_launch_bwd_contraction(h, s));

@@ -667,10 +667,15 @@ __device__ __forceinline__ void tt_warp_mid_b(const float* As, const float* __re
 #pragma unroll
         for (int i = 0; i < CPL; ++i) b[i] = __ldg(B4 + (size_t)a * c4n + ll + i * LA);
         float av[M];
+        if constexpr (M % 4 == 0) {
 #pragma unroll
-        for (int m4 = 0; m4 < M / 4; ++m4) {
-            const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
-            av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+            for (int m4 = 0; m4 < M / 4; ++m4) {
+                const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
+                av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < M; ++m) av[m] = As[a * M + m];
         }
 #pragma unroll
         for (int i = 0; i < CPL; ++i)
@@ -750,9 +755,14 @@ __device__ __forceinline__ void tt_warp_rows_dC(const WsView& w, const TableDesc
     // the lane now holds dc[0..n) = dC values [base, base+n) of its TP rows (value v <-> row v / RB_, column v % RB_)
     constexpr int NF = NV / RW;
     float* dst = dPdst + (TP * q + base / RB_) * RB_ + base % RB_;
+    if constexpr (NF >= 4) {
 #pragma unroll
-    for (int i = 0; i < NF / 4; ++i)
-        *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(dc[4 * i], dc[4 * i + 1], dc[4 * i + 2], dc[4 * i + 3]);
+        for (int i = 0; i < NF / 4; ++i)
+            *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(dc[4 * i], dc[4 * i + 1], dc[4 * i + 2], dc[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NF; ++i) dst[i] = dc[i];
+    }
 }
 
 template <int PM, int RB_, int TP>
@@ -1091,6 +1101,11 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
 }
 
 // fixed-order sum of the partial copies of the last core's gradient
@@ -1118,10 +1133,10 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
                               : (size_t)4 * (max_pl + max_c) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    if ((e = tt_stage_begin(h, 15 + V + 1, s)) != cudaSuccess) return e;
+    if ((e = tt_stage_begin(h, 9 + TT_NUM_VARIANTS + 1 + V + 1, s)) != cudaSuccess) return e;
     k_sweep_bwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
     tt_note_launch();
-    if ((e = tt_stage_end(h, 15 + V + 1, s)) != cudaSuccess) return e;
+    if ((e = tt_stage_end(h, 9 + TT_NUM_VARIANTS + 1 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
@@ -1155,6 +1170,11 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_bwd<2>(h, max_pl, max_c, next_stream(3))) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<3>(h, max_pl, max_c, next_stream(4))) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<4>(h, max_pl, max_c, next_stream(5))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<5>(h, max_pl, max_c, next_stream(6))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<6>(h, max_pl, max_c, next_stream(7))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<7>(h, max_pl, max_c, next_stream(8))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<8>(h, max_pl, max_c, next_stream(9))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<9>(h, max_pl, max_c, next_stream(10))) != cudaSuccess) return e;
     if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
     tt_note_launch();
@@ -1346,10 +1366,11 @@ __device__ __forceinline__ int tt_reduce_scatter(float (&v)[NVAL], int lane)
     return idx;
 }
 
-template <int RA, int COLS>
+template <int M, int RA, int COLS>
 __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
 {
-    constexpr int M = 4, TC = COLS / 4, AG = 128 / TC, APT = RA / AG, NVAL = M * APT;
+    constexpr int TC = COLS / 4, AG = 128 / TC, APT = RA / AG, NVAL = M * APT;
+    static_assert(APT >= 1 && AG * APT == RA && NVAL >= 1, "tile shape");
     constexpr int REP = TC / NVAL > 0 ? TC / NVAL : 1;  // lanes that end up with the same reduced value
     constexpr int ST = 4;   // stages of the node pipeline (cp.async, no staging registers)
     __shared__ __align__(16) float sA[ST][M * RA];
@@ -1467,7 +1488,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
     cudaError_t e;
     for (int k = h->K - 1; k >= 2; --k) {
         int max_n = 1, max_down = 1, max_slice = 1;
-        bool any_generic = false, any_fast[4] = {false, false, false, false};
+        bool any_generic = false, any_fast[8] = {false, false, false, false, false, false, false, false};
         for (int t = 0; t < h->T; ++t) {
             const TableDesc& td = h->tab[t];
             const int kc = k - 1;
@@ -1482,14 +1503,22 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         const dim3 sg(max_n, h->T);
         // the shape variants are independent (different tables): run them side by side so that the tail of one
         // (a few long node lists) overlaps the others
-        const bool fork = (int)any_fast[0] + (int)any_fast[1] + (int)any_fast[2] + (int)any_fast[3] > 1 && !h->serial;
+        int nfast = 0;
+        for (int v = 0; v < 8; ++v) nfast += any_fast[v] ? 1 : 0;
+        const bool fork = nfast > 1 && !h->serial;
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
-        if (any_fast[0]) { k_mid_fused<32, 128><<<sg, 128, 0, fork ? h->side[0] : s>>>(w, k, 0); tt_note_launch(); }
-        if (any_fast[1]) { k_mid_fused<16, 128><<<sg, 128, 0, fork ? h->side[1] : s>>>(w, k, 1); tt_note_launch(); }
-        if (any_fast[2]) { k_mid_fused<32, 64><<<sg, 128, 0, fork ? h->side[2] : s>>>(w, k, 2); tt_note_launch(); }
-        if (any_fast[3]) { k_mid_fused<16, 64><<<sg, 128, 0, fork ? h->side[3] : s>>>(w, k, 3); tt_note_launch(); }
+        int slot = 0;
+        auto st = [&]() { return fork ? h->side[(slot++) & 3] : s; };
+        if (any_fast[0]) { k_mid_fused<4, 32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
+        if (any_fast[1]) { k_mid_fused<4, 16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
+        if (any_fast[2]) { k_mid_fused<4, 32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
+        if (any_fast[3]) { k_mid_fused<4, 16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
+        if (any_fast[4]) { k_mid_fused<2, 32, 128><<<sg, 128, 0, st()>>>(w, k, 4); tt_note_launch(); }
+        if (any_fast[5]) { k_mid_fused<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
+        if (any_fast[6]) { k_mid_fused<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
+        if (any_fast[7]) { k_mid_fused<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
-        if (any_fast[0] || any_fast[1] || any_fast[2] || any_fast[3]) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
+        if (nfast > 0) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {
             if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
             k_mid_slice<<<sg, 256, (size_t)max_slice * sizeof(float), s>>>(w, k);

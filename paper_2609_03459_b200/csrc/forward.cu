@@ -172,10 +172,15 @@ __device__ __forceinline__ void tt_warp_mid(const float* As, const float* __rest
 #pragma unroll
         for (int i = 0; i < CPL; ++i) b[i] = __ldg(B4 + (size_t)a * c4n + ll + i * LA);
         float av[M];
+        if constexpr (M % 4 == 0) {
 #pragma unroll
-        for (int m4 = 0; m4 < M / 4; ++m4) {
-            const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
-            av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+            for (int m4 = 0; m4 < M / 4; ++m4) {
+                const float4 t = *reinterpret_cast<const float4*>(As + a * M + 4 * m4);
+                av[4 * m4] = t.x; av[4 * m4 + 1] = t.y; av[4 * m4 + 2] = t.z; av[4 * m4 + 3] = t.w;
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < M; ++m) av[m] = As[a * M + m];
         }
 #pragma unroll
         for (int i = 0; i < CPL; ++i)
@@ -451,6 +456,11 @@ __global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats, int 
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
     if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 5) tt_sweep_fast<8, 32, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 6) tt_sweep_fast<8, 16, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 7) tt_sweep_fast<8, 8, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 8) tt_sweep_fast<4, 32, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 9) tt_sweep_fast<4, 16, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
 }
 
 // dynamic shared memory of k_sweep_fwd<V> / k_sweep_bwd<V>: four C tiles per warp for the tensor-core variants
@@ -509,6 +519,11 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_fwd<2>(h, max_pl, max_c, next_stream(3))) != cudaSuccess) return e;
     if ((e = launch_sweep_fwd<3>(h, max_pl, max_c, next_stream(4))) != cudaSuccess) return e;
     if ((e = launch_sweep_fwd<4>(h, max_pl, max_c, next_stream(5))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<5>(h, max_pl, max_c, next_stream(6))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<6>(h, max_pl, max_c, next_stream(7))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<7>(h, max_pl, max_c, next_stream(8))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<8>(h, max_pl, max_c, next_stream(9))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<9>(h, max_pl, max_c, next_stream(10))) != cudaSuccess) return e;
     if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     return cudaGetLastError();
 }

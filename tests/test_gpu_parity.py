@@ -146,7 +146,7 @@ def test_medium_forward_backward(binding, case):
             assert_close(grads[t][k], ref[t][k], f"{name} dG[{t}][{k}]")
 
 
-@pytest.mark.parametrize("D,rank", [(16, 8), (16, 32), (32, 16), (32, 32), (64, 8), (64, 32)])
+@pytest.mark.parametrize("D,rank", [(16, 8), (16, 16), (16, 32), (32, 8), (32, 16), (32, 32), (64, 8), (64, 32)])
 def test_sweep_point_shapes(binding, D, rank):
     # the shapes of the dimension / rank sweep (dim factors 2x2x4, 2x4x4, 4x4x4) at a batch the oracle finishes fast
     wl = workloads.sweep_point(D, rank, 96, num_tables=3, with_grad=True)
