@@ -1439,6 +1439,145 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
     for (int i = 0; i < APT; ++i) reinterpret_cast<float4*>(dst + (size_t)(a0 + i) * COLS)[cl] = acc[i];
 }
 
+// ---- tensor-core form of the middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ----
+//
+// Same ownership as k_mid_fused (one CTA of 4 warps per (table, slice i_k), nodes from the digit-major list), but
+// NQ = 4 (r_{k-1} = 32) or 8 (16) nodes per round, staged with cp.async into padded shared-memory tiles (two stages,
+// two barriers per round instead of one per node), and both products as 3xTF32 m16n8k8 tiles (mma.cuh):
+//   dG_k[a][c] += sum_{node, m} P_{k-1}[node][m][a] * dP_k[node][m][c]   M = a, N = c, K = 8 = (2 nodes, 4 rows m);
+//                 a warp owns COLS/4 columns c of the slice, accumulators stay in registers over the whole list
+//   Y[node][m][a] = sum_c dP_k[node][m][c] * G_k[a][c]                   M = 16 = (4 nodes, m), N = 8 values of a,
+//                 K = c; the slice fragments (split into TF32 head and tail once) stay in registers;
+//                 warp -> (n-tile of a, group of four nodes)
+// Row strides RA + 8 and COLS + 8 floats make every fragment load from shared memory conflict-free or 2-way.
+template <int RA, int COLS>
+__global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
+{
+    constexpr int M = 4, NQ = 128 / RA, AP = RA + 8, CP = COLS + 8;
+    constexpr int MT = RA / 16;              // dG: m-tiles over a
+    constexpr int NTW = COLS / 32;           // dG: n-tiles per warp (the warp's COLS/4 columns)
+    constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ / 4 row tiles of four nodes; NTY * NQ / 4 = 4 warps
+    constexpr int KTY = COLS / 8;            // Y: k steps over c
+    __shared__ __align__(16) float sA[2][NQ * M * AP];
+    __shared__ __align__(16) float sD[2][NQ * M * CP];
+    const int t_ = w.vlist[w.T + blockIdx.y];   // largest tables first: their long node lists start early
+    const TableDesc& td = w.tdesc[t_];
+    const int kc = k - 1;
+    if (td.midfast[k] != variant || (int)blockIdx.x >= td.n[kc]) return;
+    const uint32_t ik = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, g = lane >> 2, t = lane & 3;
+    const float* __restrict__ Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
+    // Y: this warp's n-tile of a and its four nodes
+    const int ynt = wid % NTY, yrt = wid / NTY;
+    Tf32Pair bY[KTY][2];
+#pragma unroll
+    for (int kt = 0; kt < KTY; ++kt) {
+        bY[kt][0] = tt_split_tf32(__ldg(Bsl + (size_t)(8 * ynt + g) * COLS + 8 * kt + t));
+        bY[kt][1] = tt_split_tf32(__ldg(Bsl + (size_t)(8 * ynt + g) * COLS + 8 * kt + t + 4));
+    }
+    float acc[MT][NTW][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt) { acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f; }
+    const uint32_t space = td.prefix_space[k - 1];
+    const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
+    const int strideY = w.stride[k - 1];
+    const uint32_t rounds = (j1 - j0 + NQ - 1) / NQ;
+    // stage the NQ nodes of round r (missing nodes of the last round are zero-filled)
+    auto issue = [&](uint32_t r) {
+        const int st = (int)(r & 1u);
+        const uint32_t jb = j0 + r * NQ;
+        for (int i = tid; i < NQ * COLS; i += 128) {            // dP_k rows: M * COLS / 4 float4 per node
+            const int q = i / COLS, rem = i - q * COLS, m = rem / (COLS / 4), c4 = rem - m * (COLS / 4);
+            float4* dst = reinterpret_cast<float4*>(&sD[st][(q * M + m) * CP + 4 * c4]);
+            if (jb + q < j1) {
+                const uint32_t v = w.tnode[k][jb + q];
+                tt_cp_async16_b(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
+            } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int i = tid; i < NQ * RA; i += 128) {              // P_{k-1} of the parent: M * RA / 4 float4 per node
+            const int q = i / RA, rem = i - q * RA, m = rem / (RA / 4), a4 = rem - m * (RA / 4);
+            float4* dst = reinterpret_cast<float4*>(&sA[st][(q * M + m) * AP + 4 * a4]);
+            if (jb + q < j1) {
+                const uint32_t v = w.tnode[k][jb + q];
+                tt_cp_async16_b(dst, reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, v) + m * RA) + a4);
+            } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (rounds > 0) issue(0);
+    for (uint32_t r = 0; r < rounds; ++r) {
+        if (r + 1 < rounds) {
+            issue(r + 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const float* A_ = sA[r & 1u];
+        const float* D_ = sD[r & 1u];
+        // ---- dG: pairs of nodes give k = 8
+#pragma unroll
+        for (int p = 0; p < NQ / 2; ++p) {
+            const float* Aa = A_ + (2 * p * M + t) * AP;         // node 2p,   row m = t
+            const float* Ab = A_ + ((2 * p + 1) * M + t) * AP;   // node 2p+1, row m = t
+            const float* Da = D_ + (2 * p * M + t) * CP + wid * (COLS / 4) + g;
+            const float* Db = D_ + ((2 * p + 1) * M + t) * CP + wid * (COLS / 4) + g;
+            Tf32Pair a[MT][4];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                a[mt][0] = tt_split_tf32(Aa[16 * mt + g]);
+                a[mt][1] = tt_split_tf32(Aa[16 * mt + g + 8]);
+                a[mt][2] = tt_split_tf32(Ab[16 * mt + g]);
+                a[mt][3] = tt_split_tf32(Ab[16 * mt + g + 8]);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) {
+                Tf32Pair b[2];
+                b[0] = tt_split_tf32(Da[8 * nt]);
+                b[1] = tt_split_tf32(Db[8 * nt]);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt][nt], a[mt], b);
+            }
+        }
+        // ---- Y of this warp's four nodes and eight values of a
+        {
+            float y[4] = {0.f, 0.f, 0.f, 0.f};
+            const float* Ra = D_ + ((4 * yrt + (g >> 2)) * M + (g & 3)) * CP;       // row g of the tile: node g / 4, m = g % 4
+            const float* Rb = D_ + ((4 * yrt + 2 + (g >> 2)) * M + (g & 3)) * CP;   // row g + 8
+#pragma unroll
+            for (int kt = 0; kt < KTY; ++kt) {
+                Tf32Pair a[4];
+                a[0] = tt_split_tf32(Ra[8 * kt + t]);
+                a[1] = tt_split_tf32(Rb[8 * kt + t]);
+                a[2] = tt_split_tf32(Ra[8 * kt + t + 4]);
+                a[3] = tt_split_tf32(Rb[8 * kt + t + 4]);
+                tt_mma_3xtf32(y, a, bY[kt]);
+            }
+            const uint32_t ja = j0 + r * NQ + 4 * yrt + (g >> 2), jb2 = ja + 2;
+            if (ja < j1) {
+                const uint32_t v = w.tnode[k][ja];
+                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[0], y[1]);
+            }
+            if (jb2 < j1) {
+                const uint32_t v = w.tnode[k][jb2];
+                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
+            }
+        }
+        __syncthreads();   // everyone is done with this stage before round r + 2 overwrites it
+    }
+    float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt) {
+            const int c = wid * (COLS / 4) + 8 * nt + 2 * t;
+            *reinterpret_cast<float2*>(dst + (size_t)(16 * mt + g) * COLS + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2*>(dst + (size_t)(16 * mt + g + 8) * COLS + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        }
+}
+
 // dP_{k-1}[parent] (k = 2: the first core's gradient slice) = sum of the Y rows of the parent's children,
 // which are contiguous in sorted order; one warp per parent
 __global__ void __launch_bounds__(256) k_mid_sum(WsView w, int k)
@@ -1509,10 +1648,10 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
         auto st = [&]() { return fork ? h->side[(slot++) & 3] : s; };
-        if (any_fast[0]) { k_mid_fused<4, 32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
-        if (any_fast[1]) { k_mid_fused<4, 16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
-        if (any_fast[2]) { k_mid_fused<4, 32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
-        if (any_fast[3]) { k_mid_fused<4, 16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
+        if (any_fast[0]) { k_mid_mma<32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
+        if (any_fast[1]) { k_mid_mma<16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
+        if (any_fast[2]) { k_mid_mma<32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
+        if (any_fast[3]) { k_mid_mma<16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
         if (any_fast[4]) { k_mid_fused<2, 32, 128><<<sg, 128, 0, st()>>>(w, k, 4); tt_note_launch(); }
         if (any_fast[5]) { k_mid_fused<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
         if (any_fast[6]) { k_mid_fused<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
