@@ -160,7 +160,7 @@ class TTEmbeddingBag:
 
     def __del__(self):
         h = getattr(self, "h", None)
-        if h:
+        if h and lib is not None:   # at interpreter shutdown the module globals may already be gone
             lib.tt_emb_destroy(h)
             self.h = None
 
