@@ -1442,8 +1442,8 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
 // ---- tensor-core form of the middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ----
 //
 // Same ownership as k_mid_fused (one CTA of 4 warps per (table, slice i_k), nodes from the digit-major list), but
-// NQ = 4 (r_{k-1} = 32) or 8 (16) nodes per round, staged with cp.async into padded shared-memory tiles (two stages,
-// two barriers per round instead of one per node), and both products as 3xTF32 m16n8k8 tiles (mma.cuh):
+// NQ = 4 (r_{k-1} = 32) or 8 (16) nodes per pass, staged with cp.async into padded shared-memory tiles (two stages,
+// two barriers per pass instead of one per node), and both products as 3xTF32 m16n8k8 tiles (mma.cuh):
 //   dG_k[a][c] += sum_{node, m} P_{k-1}[node][m][a] * dP_k[node][m][c]   M = a, N = c, K = 8 = (2 nodes, 4 rows m);
 //                 a warp owns COLS/4 columns c of the slice, accumulators stay in registers over the whole list
 //   Y[node][m][a] = sum_c dP_k[node][m][c] * G_k[a][c]                   M = 16 = (4 nodes, m), N = 8 values of a,
@@ -1483,8 +1483,8 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
     const uint32_t space = td.prefix_space[k - 1];
     const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
     const int strideY = w.stride[k - 1];
-    const uint32_t rounds = (j1 - j0 + NQ - 1) / NQ;
-    // stage the NQ nodes of round r (missing nodes of the last round are zero-filled)
+    const uint32_t passes = (j1 - j0 + NQ - 1) / NQ;
+    // stage the NQ nodes of pass r (missing nodes of the last pass are zero-filled)
     auto issue = [&](uint32_t r) {
         const int st = (int)(r & 1u);
         const uint32_t jb = j0 + r * NQ;
@@ -1506,9 +1506,9 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    if (rounds > 0) issue(0);
-    for (uint32_t r = 0; r < rounds; ++r) {
-        if (r + 1 < rounds) {
+    if (passes > 0) issue(0);
+    for (uint32_t r = 0; r < passes; ++r) {
+        if (r + 1 < passes) {
             issue(r + 1);
             asm volatile("cp.async.wait_group 1;" ::: "memory");
         } else {
@@ -1565,7 +1565,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
-        __syncthreads();   // everyone is done with this stage before round r + 2 overwrites it
+        __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
     }
     float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
 #pragma unroll
