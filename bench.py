@@ -8,8 +8,9 @@ for the training workload (cfg5, the default: the 60-table configuration with ba
 the backward pass and the SGD update.  Prints ONE JSON line on rank 0.
 
   value      lookups/s of the whole job (all ranks), inputs resident in HBM before the timed region
-  e2e        the same through the public call with HOST (pinned) buffers: H2D of indices/offsets(/grad_out)
-             and D2H of `out` inside the timed region
+  e2e        the same through the public call with HOST (pinned) buffers: every step uploads one batch
+             (indices, offsets, grad_out) and downloads `out` inside the timed region; the upload of step i+1
+             overlaps the compute of step i (double-buffered device inputs, copy streams)
   roofline   the dominant kernel of the step against its own bound (measured peaks)
   step_roofline  the whole step against max(FP32 slots / measured FP32 peak, HBM bytes / measured HBM peak)
   cpu_baseline   the fp64 oracle, as it stands, on a bounded sample of the same workload (rank 0, N = 1)
@@ -295,12 +296,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
+    def timed(fn, steps, after=None):
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
             fn()
+        if after is not None:
+            after()       # e.g. join side streams so that their work falls inside the timed region
         e1.record()
         barrier()
         ms = torch.tensor([e0.elapsed_time(e1)], device=device)
@@ -375,38 +378,59 @@ def main():
     # ---- end to end through host buffers
     e2e = None
     if not args.no_e2e:
-        # the call a user makes with host buffers: indices/offsets go up first, grad_out goes up on a second
-        # stream while the forward runs, `out` comes down while the backward runs
-        copy_stream = torch.cuda.Stream(device)
-        e_idx, e_off = torch.empty_like(d_idx), torch.empty_like(d_off)
-        e_grad = torch.empty_like(d_grad) if train else None
+        # The loop a user runs with host buffers, software-pipelined like a data loader: the inputs of step i+1
+        # (indices, offsets, grad_out) go up on a copy stream while step i computes, `out` of step i comes down on a
+        # third stream while its backward runs.  Every step uploads one batch and downloads one result inside the
+        # timed region; the device buffers are double-buffered, the hazards are ordered with events.
+        up, down = torch.cuda.Stream(device), torch.cuda.Stream(device)
+        e_idx = [torch.empty_like(d_idx) for _ in range(2)]
+        e_off = [torch.empty_like(d_off) for _ in range(2)]
+        e_grad = [torch.empty_like(d_grad) for _ in range(2)] if train else None
+        state = {"i": 0, "ready": [None, None], "free": [None, None], "out_done": None}
+
+        def upload(slot):
+            # batch for buffer `slot`: waits until the step that last used the buffer is over
+            if state["free"][slot] is not None:
+                up.wait_event(state["free"][slot])
+            with torch.cuda.stream(up):
+                e_idx[slot].copy_(h_idx, non_blocking=True)
+                e_off[slot].copy_(h_off, non_blocking=True)
+                if train:
+                    e_grad[slot].copy_(h_grad, non_blocking=True)
+                state["ready"][slot] = up.record_event()
 
         def e2e_step():
             main = torch.cuda.current_stream()
-            e_idx.copy_(h_idx, non_blocking=True)
-            e_off.copy_(h_off, non_blocking=True)
-            ev_in = main.record_event()
-            ev_grad = None
-            if train:
-                copy_stream.wait_event(ev_in)
-                with torch.cuda.stream(copy_stream):
-                    e_grad.copy_(h_grad, non_blocking=True)
-                    ev_grad = copy_stream.record_event()
-            emb.forward(e_idx, e_off, B, out=d_out)
+            i = state["i"]
+            slot = i & 1
+            if state["ready"][slot] is None:
+                upload(slot)                       # first step: nothing was prefetched yet
+            main.wait_event(state["ready"][slot])
+            if state["out_done"] is not None:
+                main.wait_event(state["out_done"])  # the previous result has left d_out
+            upload(slot ^ 1)                       # prefetch the next batch while this one computes
+            emb.forward(e_idx[slot], e_off[slot], B, out=d_out)
             ev_fwd = main.record_event()
-            copy_stream.wait_event(ev_fwd)
-            with torch.cuda.stream(copy_stream):
+            down.wait_event(ev_fwd)
+            with torch.cuda.stream(down):
                 h_out.copy_(d_out, non_blocking=True)
-                ev_out = copy_stream.record_event()
+                state["out_done"] = down.record_event()
             if train:
-                main.wait_event(ev_grad)
-                emb.backward(e_grad)
+                emb.backward(e_grad[slot])
                 ttd.allreduce_core_grads(emb.flat_grads)
                 emb.sgd_step(wl.lr)
-            main.wait_event(ev_out)
+            state["free"][slot] = main.record_event()
+            state["ready"][slot] = None
+            state["i"] = i + 1
+
+        def e2e_drain():
+            main = torch.cuda.current_stream()
+            main.wait_stream(up)
+            main.wait_stream(down)
         for _ in range(2):
             e2e_step()
-        e2e_ms = timed(e2e_step, args.steps) / args.steps
+        e2e_drain()
+        e2e_ms = timed(lambda: e2e_step(), args.steps, after=e2e_drain) / args.steps
         h2d = h_idx.numel() * 8 + h_off.numel() * 8 + (h_grad.numel() * 4 if train else 0)
         e2e = {"value": world * L / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4)}
