@@ -114,6 +114,15 @@ int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, i
                    int64_t num_lookups, float* out, tt_emb_stream_t stream);
 
 /*
+ * The same forward with 32-bit row ids (every N_t is below 2^31 anyway): half the bytes to bring to the device and to
+ * read in the grouping and pooling passes.  indices: device int32[num_lookups]; everything else as tt_emb_forward,
+ * including the rule that indices stay valid until a later tt_emb_backward has completed.  The paper's interface
+ * has 64-bit ids only; this entry point is an addition for callers that hold 32-bit ids.
+ */
+int tt_emb_forward_i32(tt_emb_t h, const int32_t* indices, const int64_t* offsets, int64_t batch,
+                       int64_t num_lookups, float* out, tt_emb_stream_t stream);
+
+/*
  * Pooling mode of the forward / backward calls that follow (default: TT_EMB_POOL_SUM without weights, the paper's
  * pooling [Sec. 3.2]).  The two other forms are extensions that follow the usual embedding-bag operator; the paper
  * has no counterpart.

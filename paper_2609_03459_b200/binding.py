@@ -65,6 +65,7 @@ _SIGS = {
     "tt_emb_dim": (ctypes.c_int, [_vp, ctypes.POINTER(_i32)]),
     "tt_emb_bind": (ctypes.c_int, [_vp, _vp, _vp, ctypes.c_size_t, _vp]),
     "tt_emb_forward": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
+    "tt_emb_forward_i32": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
     "tt_emb_forward_static": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp]),
     "tt_emb_static_workspace_limit": (ctypes.c_size_t, []),
     "tt_emb_backward": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
@@ -234,14 +235,16 @@ class TTEmbeddingBag:
 
     # ---- hot path
     def forward(self, indices, offsets, batch: int, out=None):
-        """indices int64[L] / offsets int64[T*batch+1] device tensors -> out fp32 [batch, T*D] (device)."""
+        """indices int64[L] (or int32[L]) / offsets int64[T*batch+1] device tensors -> out fp32 [batch, T*D] (device)."""
         torch = self.torch
-        assert indices.dtype == torch.int64 and offsets.dtype == torch.int64 and indices.is_cuda and offsets.is_cuda
+        assert indices.dtype in (torch.int64, torch.int32) and offsets.dtype == torch.int64
+        assert indices.is_cuda and offsets.is_cuda
         if out is None:
             out = torch.empty((batch, self.T * self.D), dtype=torch.float32, device=self.device)
         self._keep = (indices, offsets)
-        _check(lib.tt_emb_forward(self.h, indices.data_ptr(), offsets.data_ptr(), int(batch), int(indices.numel()),
-                                  out.data_ptr(), _stream_ptr()), "tt_emb_forward")
+        fn = lib.tt_emb_forward if indices.dtype == torch.int64 else lib.tt_emb_forward_i32   # 32-bit row ids
+        _check(fn(self.h, indices.data_ptr(), offsets.data_ptr(), int(batch), int(indices.numel()),
+                  out.data_ptr(), _stream_ptr()), "tt_emb_forward")
         return out
 
     def capture_forward(self, indices, offsets, batch: int, out):

@@ -481,16 +481,16 @@ extern "C" int tt_emb_stage_ms(tt_emb_t h, int32_t stage, float* ms)
 
 // ------------------------------------------------------------------------------------------------ forward / backward / sgd
 
-extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
-                              int64_t num_lookups, float* out, tt_emb_stream_t stream)
+static int forward_any(tt_emb* h, const void* indices, bool idx32, const int64_t* offsets, int64_t batch, int64_t num_lookups,
+                       float* out, cudaStream_t s)
 {
     if (!h || !offsets || !out || (!indices && num_lookups > 0)) return TT_EMB_ERR_ARG;
     if (!h->bound) return TT_EMB_ERR_STATE;
     if (batch < 1 || batch > h->max_batch || num_lookups < 0 || num_lookups > h->max_lookups) return TT_EMB_ERR_ARG;
-    cudaStream_t s = (cudaStream_t)stream;
     WsView& v = h->v;
     v.B = batch; v.L = num_lookups;
-    v.indices = indices; v.offsets = offsets;
+    v.indices = reinterpret_cast<const int64_t*>(indices); v.offsets = offsets;
+    v.idx32 = idx32 ? 1 : 0;
     h->have_forward = false;
     for (int i = 0; i < 4; ++i) h->ev_valid[i] = false;
     for (int i = 9; i < 9 + TT_NUM_VARIANTS + 1; ++i) h->ev_valid[i] = false;
@@ -500,6 +500,18 @@ extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t*
     TT_STAGE(h, 3, s, tt_launch_pooling(h, out, s));
     h->have_forward = true;
     return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                              int64_t num_lookups, float* out, tt_emb_stream_t stream)
+{
+    return forward_any(h, indices, false, offsets, batch, num_lookups, out, (cudaStream_t)stream);
+}
+
+extern "C" int tt_emb_forward_i32(tt_emb_t h, const int32_t* indices, const int64_t* offsets, int64_t batch,
+                                  int64_t num_lookups, float* out, tt_emb_stream_t stream)
+{
+    return forward_any(h, indices, true, offsets, batch, num_lookups, out, (cudaStream_t)stream);
 }
 
 extern "C" int tt_emb_set_pooling(tt_emb_t h, int32_t mode, const float* per_sample_weights)

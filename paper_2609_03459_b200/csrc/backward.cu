@@ -827,12 +827,18 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
     const uint32_t* __restrict__ rows = w.val[K];
-    float acc[MT][NT][4];
+    // acc: tensor-core accumulators, folded into tot (rounded fp32 adds) every sixteen row pairs: the tensor core adds
+    // with truncation, so a long chain (a group can have hundreds of rows) would drift by chain length * 2^-24
+    float acc[MT][NT][4], tot[MT][NT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f; }
-    for (uint32_t ub = u0; ub < u1; ub += 2) {
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) { acc[mt][nt][x] = 0.f; tot[mt][nt][x] = 0.f; }
+    for (uint32_t ub0 = u0; ub0 < u1; ub0 += 32) {
+    const uint32_t ub1 = min(ub0 + 32u, u1);
+    for (uint32_t ub = ub0; ub < ub1; ub += 2) {
         const bool two = ub + 1 < u1;
         const uint32_t ua = ub, uc = two ? ub + 1 : ub;
         const float* __restrict__ Ea = w.E + (size_t)ua * (PM * 4) + t;
@@ -865,9 +871,16 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) { tot[mt][nt][x] += acc[mt][nt][x]; acc[mt][nt][x] = 0.f; }
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][0], tot[mt][nt][1]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][2], tot[mt][nt][3]);
         }
 }
 
@@ -945,14 +958,18 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
             ct[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g]);
             ct[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g + 8]);
         }
-    float dc[MT][NT][4];
+    float dc[MT][NT][4], dct[MT][NT][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { dc[mt][nt][0] = 0.f; dc[mt][nt][1] = 0.f; dc[mt][nt][2] = 0.f; dc[mt][nt][3] = 0.f; }
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) { dc[mt][nt][x] = 0.f; dct[mt][nt][x] = 0.f; }
     const int rb_ = g >> 2, jb = g & 3;       // dG B fragment: row rb_ of the pair, column jb of dE
     const int rc = t >> 1, jc = 2 * (t & 1);  // dG C fragment: row rc of the pair, columns jc, jc+1
-    for (uint32_t ub = u0; ub < u1; ub += 2) {
+    for (uint32_t ub0 = u0; ub0 < u1; ub0 += 32) {
+    const uint32_t ub1 = min(ub0 + 32u, u1);
+    for (uint32_t ub = ub0; ub < ub1; ub += 2) {
         const bool two = ub + 1 < u1;
         const uint32_t ua = ub, uc = two ? ub + 1 : ub;
         const uint32_t iKa = rows[ua] - row_base, iKc = rows[uc] - row_base;
@@ -1023,9 +1040,16 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) { dct[mt][nt][x] += dc[mt][nt][x]; dc[mt][nt][x] = 0.f; }
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dc[mt][nt][0], dc[mt][nt][1]);
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dc[mt][nt][2], dc[mt][nt][3]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
+            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
         }
 }
 
@@ -1450,6 +1474,10 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
 //                 K = c; the slice fragments (split into TF32 head and tail once) stay in registers;
 //                 warp -> (n-tile of a, group of four nodes)
 // Row strides RA + 8 and COLS + 8 floats make every fragment load from shared memory conflict-free or 2-way.
+// The tensor core adds into its fp32 accumulator with truncation, so an accumulation chain of N products drifts by
+// up to N * 2^-24 of the sum; the dG accumulators are therefore folded into running sums (a rounded fp32
+// add into the CTA's own gradient slice, which stays in L2) every eighth pass, which keeps every chain at 48 or 96
+// products whatever the length of the node list.
 template <int RA, int COLS>
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 {
@@ -1480,6 +1508,26 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) { acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f; }
+    // fold: this CTA is the only writer of its slice of the gradient, so the running sums live there (L2) instead of
+    // in a second register set; each thread adds its accumulators to the elements it owns
+    float* const gdst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
+    bool first_fold = true;
+    auto fold = [&]() {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) {
+                const int c = wid * (COLS / 4) + 8 * nt + 2 * t;
+                float2* p0 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g) * COLS + c);
+                float2* p1 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g + 8) * COLS + c);
+                float2 v0 = first_fold ? make_float2(0.f, 0.f) : *p0;
+                float2 v1 = first_fold ? make_float2(0.f, 0.f) : *p1;
+                v0.x += acc[mt][nt][0]; v0.y += acc[mt][nt][1]; v1.x += acc[mt][nt][2]; v1.y += acc[mt][nt][3];
+                *p0 = v0; *p1 = v1;
+                acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f;
+            }
+        first_fold = false;
+    };
     const uint32_t space = td.prefix_space[k - 1];
     const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
     const int strideY = w.stride[k - 1];
@@ -1565,17 +1613,10 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
+        if ((r & 7u) == 7u) fold();   // rounded running sums every eighth pass
         __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
     }
-    float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < NTW; ++nt) {
-            const int c = wid * (COLS / 4) + 8 * nt + 2 * t;
-            *reinterpret_cast<float2*>(dst + (size_t)(16 * mt + g) * COLS + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
-            *reinterpret_cast<float2*>(dst + (size_t)(16 * mt + g + 8) * COLS + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
-        }
+    fold();   // also writes the zeros of a slice without nodes
 }
 
 // dP_{k-1}[parent] (k = 2: the first core's gradient slice) = sum of the Y rows of the parent's children,

@@ -82,7 +82,19 @@ struct WsView {
     const float* psw;                   // per-lookup weights [L] or null
     float* wsorted;                     // [L] factor of every sorted pair (weight, or 1 / bag length), backward only
     int32_t pool_mean;                  // 1: mean pooling
+    int32_t idx32;                      // 1: `indices` points at int32 row ids (tt_emb_forward_i32)
 };
+
+// row id of lookup l (int64 or int32 storage); STREAM: read-once hint
+template <bool STREAM = false>
+__device__ __forceinline__ int64_t tt_index(const WsView& w, int64_t l)
+{
+    if (w.idx32) {
+        const int32_t* p = reinterpret_cast<const int32_t*>(w.indices) + l;
+        return (int64_t)(STREAM ? __ldcs(p) : __ldg(p));
+    }
+    return STREAM ? __ldcs(w.indices + l) : __ldg(w.indices + l);
+}
 
 enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16 };
 

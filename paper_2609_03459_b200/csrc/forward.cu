@@ -538,7 +538,7 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
 // __shfl_xor at the end.
 __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableDesc& td, int64_t l, uint32_t capK)
 {
-    const int64_t g = __ldcs(w.indices + l);   // streamed once: evict-first, keeps L2 for rows and rank words
+    const int64_t g = tt_index<true>(w, l);    // streamed once: evict-first, keeps L2 for rows and rank words
     uint32_t slot = 0xffffffffu;
     if (g >= 0 && g < td.N) {
         const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
@@ -843,7 +843,7 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
         float* o = out + (size_t)b * w.T * D + (size_t)t * D;
         if (w.upairs)
             for (int64_t l = lo + lane; l < hi; l += 32) {
-                const int64_t g = __ldg(w.indices + l);
+                const int64_t g = tt_index(w, l);
                 uint32_t slot = 0xffffffffu;
                 if (g >= 0 && g < td.N) {
                     const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
@@ -857,7 +857,7 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
 #pragma unroll
             for (int c = 0; c < 8; ++c) acc[c] = 0.f;
             for (int64_t l = lo; l < hi; ++l) {
-                const int64_t g = __ldg(w.indices + l);
+                const int64_t g = tt_index(w, l);
                 if (g < 0 || g >= td.N) continue;
                 const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
                 if (!(e.x >> (g & 31) & 1u)) continue;

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int64_t l = base + (int64_t)j * blockDim.x;
-            g[j] = l < L ? __ldg(w.indices + l) : -1;
+            g[j] = l < L ? tt_index(w, l) : -1;
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -192,7 +192,7 @@ __global__ void k_export_mult(WsView w, int table)
     const TableDesc& td = w.tdesc[table];
     const int64_t lo = w.tl_start[table], hi = w.tl_start[table + 1];
     for (int64_t l = lo + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < hi; l += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t g = w.indices[l];
+        const int64_t g = tt_index(w, l);
         if (g < 0 || g >= td.N) continue;
         const uint2 e = w.bm[td.word_base + ((uint32_t)g >> 5)];
         const uint32_t slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
@@ -236,7 +236,7 @@ __global__ void k_export_inverse(WsView w, int table, int32_t* inv)
     const int64_t lo = w.tl_start[table], hi = w.tl_start[table + 1];
     const uint32_t base = w.tb[w.K][table];
     for (int64_t l = lo + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < hi; l += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t g = w.indices[l];
+        const int64_t g = tt_index(w, l);
         int32_t r = -1;
         if (g >= 0 && g < td.N) {
             const uint2 e = w.bm[td.word_base + ((uint32_t)g >> 5)];

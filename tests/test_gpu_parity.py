@@ -121,6 +121,12 @@ MEDIUM = [
                        # first ranks that are not multiples of 8: the stacked tensor-core product pads its k range
                        TableSpec(9_000, (21, 21, 21), (4, 4, 4), (1, 12, 32, 1), 1.0, "normal", 0.05),
                        TableSpec(7_000, (19, 20, 19), (4, 4, 4), (1, 21, 16, 1), 1.1, "normal", 0.05)], 150, (0, 30)),
+    # long accumulation chains: groups with hundreds of rows (dC summed over a whole group) and middle-core slices
+    # with hundreds of nodes; nearly uniform lookups so that most rows are present.  The tensor core adds into its
+    # accumulator with truncation, which drifts by chain length * 2^-24 unless the chains are kept short.
+    ("long-chains", [TableSpec(72_000, (6, 40, 300), (4, 4, 4), (1, 32, 32, 1), 0.2, "normal", 0.05),
+                     TableSpec(64_000, (200, 8, 40), (4, 4, 4), (1, 16, 32, 1), 0.2, "normal", 0.05),
+                     TableSpec(60_000, (5, 40, 300), (4, 4, 4), (1, 16, 16, 1), 0.2, "normal", 0.05)], 96, (500, 900)),
     ("tiled-d484", [TableSpec(10_000, (20, 25, 20), (4, 8, 4), (1, 32, 32, 1), 1.1, "normal", 0.05)], 100, 20),
     ("tiled-k4-r64", [TableSpec(20_736, (12, 12, 12, 12), (2, 4, 4, 4), (1, 64, 64, 64, 1), 1.2, "normal", 0.02)], 120, 8),
     ("k2", [TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 1.0, "uniform", 0.1)], 257, (1, 9)),
@@ -162,7 +168,7 @@ def test_sweep_point_shapes(binding, D, rank):
             assert_close(grads[t][k], ref[t][k], f"sweep D{D} r{rank} dG[{t}][{k}]")
 
 
-POOLING_CASES = [MEDIUM[0], MEDIUM[1], MEDIUM[2], MEDIUM[4], MEDIUM[6], MEDIUM[7]]   # D = 64 (cp.async pooling), D = 128, K = 2, odd D, wide D
+POOLING_CASES = [MEDIUM[0], MEDIUM[1], MEDIUM[3], MEDIUM[5], MEDIUM[7], MEDIUM[8]]   # D = 64 (cp.async pooling), D = 128, K = 2, odd D, wide D
 
 
 @pytest.mark.parametrize("mode", ["weighted", "mean"])
@@ -202,6 +208,47 @@ def test_pooling_modes_need_the_config_flag(binding):
         import ctypes
         from paper_2609_03459_b200.binding import lib, _check
         _check(lib.tt_emb_set_pooling(emb2.h, 1, dev(np.ones(4, np.float32)).data_ptr()), "tt_emb_set_pooling")
+
+
+def test_long_accumulation_chains_of_one_sign(binding):
+    # all cores and all output gradients positive: every partial sum grows monotonically, the worst case for an
+    # accumulator that truncates (the tensor core's): groups with hundreds of rows, middle-core slices with hundreds of
+    # nodes.  Chains that are not folded into rounded sums miss the tolerance here.
+    name, tables, B, pooling = [c for c in MEDIUM if c[0] == "long-chains"][0]
+    wl = workloads.custom(tables, B, pooling, seed=78, with_grad=True, name=name)
+    wl.cores = [[np.abs(c) for c in tc] for tc in wl.cores]
+    wl.grad_out = np.abs(wl.grad_out)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert_close(out, oracle.forward_workload(wl), "one-sign out")
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        for k in range(3):
+            assert_close(grads[t][k], ref[t][k], f"one-sign dG[{t}][{k}]")
+
+
+def test_int32_row_ids_give_the_same_result(binding):
+    # the 32-bit index entry point: same grouping, same output bit for bit, same gradients; bad ids still flagged
+    import torch
+    name, tables, B, pooling = MEDIUM[0]
+    wl = workloads.custom(tables, B, pooling, seed=41, with_grad=True, name=name)
+    emb = binding.from_workload(wl, enable_backward=True)
+    out64 = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    idx32 = dev(wl.indices.astype(np.int32))
+    out32 = emb.forward(idx32, dev(wl.offsets), wl.B).cpu().numpy()
+    np.testing.assert_array_equal(out32, out64)
+    check_grouping(emb, wl)
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"int32 ids dG[{t}][{k}]")
+    bad = wl.indices.astype(np.int32).copy()
+    bad[3] = -5
+    emb.forward(dev(bad), dev(wl.offsets), wl.B)
+    assert emb.status() & binding.STATUS_INDEX
 
 
 def test_forward_replayed_from_a_cuda_graph(binding):
