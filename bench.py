@@ -383,57 +383,70 @@ def main():
         # third stream while its backward runs.  Every step uploads one batch and downloads one result inside the
         # timed region; the device buffers are double-buffered, the hazards are ordered with events.
         up, down = torch.cuda.Stream(device), torch.cuda.Stream(device)
-        e_idx = [torch.empty_like(d_idx) for _ in range(2)]
-        e_off = [torch.empty_like(d_off) for _ in range(2)]
-        e_grad = [torch.empty_like(d_grad) for _ in range(2)] if train else None
-        state = {"i": 0, "ready": [None, None], "free": [None, None], "out_done": None}
 
-        def upload(slot):
-            # batch for buffer `slot`: waits until the step that last used the buffer is over
-            if state["free"][slot] is not None:
-                up.wait_event(state["free"][slot])
-            with torch.cuda.stream(up):
-                e_idx[slot].copy_(h_idx, non_blocking=True)
-                e_off[slot].copy_(h_off, non_blocking=True)
+        def run_e2e(h_ids):
+            """Pipelined loop with the row ids taken from the pinned host tensor h_ids (int64 or int32)."""
+            e_idx = [torch.empty(h_ids.shape, dtype=h_ids.dtype, device=device) for _ in range(2)]
+            e_off = [torch.empty_like(d_off) for _ in range(2)]
+            e_grad = [torch.empty_like(d_grad) for _ in range(2)] if train else None
+            e_out = [d_out, torch.empty_like(d_out)]     # double-buffered result: its download overlaps the next forward
+            state = {"i": 0, "ready": [None, None], "free": [None, None], "out_done": [None, None]}
+
+            def upload(slot):
+                # batch for buffer `slot`: waits until the step that last used the buffer is over
+                if state["free"][slot] is not None:
+                    up.wait_event(state["free"][slot])
+                with torch.cuda.stream(up):
+                    e_idx[slot].copy_(h_ids, non_blocking=True)
+                    e_off[slot].copy_(h_off, non_blocking=True)
+                    if train:
+                        e_grad[slot].copy_(h_grad, non_blocking=True)
+                    state["ready"][slot] = up.record_event()
+
+            def e2e_step():
+                main = torch.cuda.current_stream()
+                i = state["i"]
+                slot = i & 1
+                if state["ready"][slot] is None:
+                    upload(slot)                       # first step: nothing was prefetched yet
+                main.wait_event(state["ready"][slot])
+                if state["out_done"][slot] is not None:
+                    main.wait_event(state["out_done"][slot])  # the result of two steps ago has left this buffer
+                upload(slot ^ 1)                       # prefetch the next batch while this one computes
+                emb.forward(e_idx[slot], e_off[slot], B, out=e_out[slot])
+                ev_fwd = main.record_event()
+                down.wait_event(ev_fwd)
+                with torch.cuda.stream(down):
+                    h_out.copy_(e_out[slot], non_blocking=True)
+                    state["out_done"][slot] = down.record_event()
                 if train:
-                    e_grad[slot].copy_(h_grad, non_blocking=True)
-                state["ready"][slot] = up.record_event()
+                    emb.backward(e_grad[slot])
+                    ttd.allreduce_core_grads(emb.flat_grads)
+                    emb.sgd_step(wl.lr)
+                state["free"][slot] = main.record_event()
+                state["ready"][slot] = None
+                state["i"] = i + 1
 
-        def e2e_step():
-            main = torch.cuda.current_stream()
-            i = state["i"]
-            slot = i & 1
-            if state["ready"][slot] is None:
-                upload(slot)                       # first step: nothing was prefetched yet
-            main.wait_event(state["ready"][slot])
-            if state["out_done"] is not None:
-                main.wait_event(state["out_done"])  # the previous result has left d_out
-            upload(slot ^ 1)                       # prefetch the next batch while this one computes
-            emb.forward(e_idx[slot], e_off[slot], B, out=d_out)
-            ev_fwd = main.record_event()
-            down.wait_event(ev_fwd)
-            with torch.cuda.stream(down):
-                h_out.copy_(d_out, non_blocking=True)
-                state["out_done"] = down.record_event()
-            if train:
-                emb.backward(e_grad[slot])
-                ttd.allreduce_core_grads(emb.flat_grads)
-                emb.sgd_step(wl.lr)
-            state["free"][slot] = main.record_event()
-            state["ready"][slot] = None
-            state["i"] = i + 1
+            def e2e_drain():
+                main = torch.cuda.current_stream()
+                main.wait_stream(up)
+                main.wait_stream(down)
+            for _ in range(2):
+                e2e_step()
+            e2e_drain()
+            ms = timed(lambda: e2e_step(), args.steps, after=e2e_drain) / args.steps
+            torch.cuda.synchronize()
+            return ms
 
-        def e2e_drain():
-            main = torch.cuda.current_stream()
-            main.wait_stream(up)
-            main.wait_stream(down)
-        for _ in range(2):
-            e2e_step()
-        e2e_drain()
-        e2e_ms = timed(lambda: e2e_step(), args.steps, after=e2e_drain) / args.steps
+        e2e_ms = run_e2e(h_idx)
+        # the same loop with 32-bit row ids (tt_emb_forward_i32): half the index bytes over PCIe
+        h_idx32 = h_idx.to(torch.int32).pin_memory()
+        e2e32_ms = run_e2e(h_idx32)
         h2d = h_idx.numel() * 8 + h_off.numel() * 8 + (h_grad.numel() * 4 if train else 0)
         e2e = {"value": world * L / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4)}
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4),
+               "int32_ids": {"value": world * L / (e2e32_ms * 1e-3), "ms_per_step": e2e32_ms,
+                             "h2d_bytes_per_step": int(h2d - h_idx.numel() * 4)}}
     clocks = sampler.stop()
 
     emb.forward(d_idx, d_off, B, out=d_out)
