@@ -424,10 +424,14 @@ __global__ void __launch_bounds__(256, 3) k_dE_stage(WsView w, const float* __re
     // slot range of the table the chunk is in: positions are sorted, so a batch rarely leaves it
     int tcur = tt_find_table(tbK, w.T, cur);
     uint32_t t_lo = tbK[tcur], t_hi = tbK[tcur + 1];
+    // two-level sum: rows are added into a per-batch partial (at most 32 terms) which is added to the segment's sum at
+    // the end of the batch, so the rounding error of a long segment grows with sqrt(length / 32), not sqrt(length)
+    float2 part = make_float2(0.f, 0.f);
     auto close_segment = [&]() {
         float2* dst = (seg_first && prev == cur) ? carry2 : E2 + (size_t)cur * 32;   // head piece or whole segment
-        dst[lane] = acc;
+        dst[lane] = make_float2(acc.x + part.x, acc.y + part.y);
         acc = make_float2(0.f, 0.f);
+        part = make_float2(0.f, 0.f);
         seg_first = false;
     };
     uint2 mine = (a + lane < b) ? __ldcs(&w.pairs[a + lane]) : make_uint2(HT_EMPTY, 0u);
@@ -473,8 +477,10 @@ __global__ void __launch_bounds__(256, 3) k_dE_stage(WsView w, const float* __re
                 const float wj = __shfl_sync(0xffffffffu, cur_w, j);
                 x.x *= wj; x.y *= wj;
             }
-            acc.x += x.x; acc.y += x.y;
+            part.x += x.x; part.y += x.y;
         }
+        acc.x += part.x; acc.y += part.y;
+        part = make_float2(0.f, 0.f);
         __syncwarp();
     }
     {   // last segment of the chunk: tail / head / whole

@@ -624,6 +624,9 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
             if (l0 + 32 < o_hi) fetch(l0 + 32, o_hi, t);
             else if (has_next) fetch(o_hi, n_hi, tn);
             const int n = (int)min((int64_t)32, o_hi - l0);
+            float4 part[CPL];   // two-level sum: per-batch partial, added to the bag's sum once per batch
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) part[c] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int j0 = 0; j0 < NIT; j0 += NF) {
                 if (j0 * RPI >= n) break;
@@ -646,14 +649,16 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
 #pragma unroll
                     for (int c = 0; c < CPL; ++c) {
                         if (WT) {
-                            acc[c].x = fmaf(wj, v[jj][c].x, acc[c].x); acc[c].y = fmaf(wj, v[jj][c].y, acc[c].y);
-                            acc[c].z = fmaf(wj, v[jj][c].z, acc[c].z); acc[c].w = fmaf(wj, v[jj][c].w, acc[c].w);
+                            part[c].x = fmaf(wj, v[jj][c].x, part[c].x); part[c].y = fmaf(wj, v[jj][c].y, part[c].y);
+                            part[c].z = fmaf(wj, v[jj][c].z, part[c].z); part[c].w = fmaf(wj, v[jj][c].w, part[c].w);
                         } else {
-                            acc[c].x += v[jj][c].x; acc[c].y += v[jj][c].y; acc[c].z += v[jj][c].z; acc[c].w += v[jj][c].w;
+                            part[c].x += v[jj][c].x; part[c].y += v[jj][c].y; part[c].z += v[jj][c].z; part[c].w += v[jj][c].w;
                         }
                     }
                 }
             }
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) { acc[c].x += part[c].x; acc[c].y += part[c].y; acc[c].z += part[c].z; acc[c].w += part[c].w; }
         }
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
@@ -750,6 +755,9 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
             if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));
             const int n = (int)min((int64_t)32, o_hi - l0);
             const unsigned valid = __ballot_sync(0xffffffffu, lane < n && slot != 0xffffffffu);
+            // two-level sum: the batch's rows go into a partial that is added to the bag's sum once per batch, so the
+            // rounding error of a bag with thousands of lookups grows with the number of batches, not of rows
+            float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
             // all rows of the batch in flight
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) {
@@ -769,10 +777,11 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
                 const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
                 if (((valid >> j) & 1u) && lane_on) {
                     const float4 v = buf[j * 16 + lr];
-                    if (WT) { acc.x = fmaf(wj, v.x, acc.x); acc.y = fmaf(wj, v.y, acc.y); acc.z = fmaf(wj, v.z, acc.z); acc.w = fmaf(wj, v.w, acc.w); }
-                    else { acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
+                    if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
+                    else { part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w; }
                 }
             }
+            acc.x += part.x; acc.y += part.y; acc.z += part.z; acc.w += part.w;
             __syncwarp();
         }
         acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
