@@ -436,7 +436,7 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
 // one instantiation per shape variant V so that each gets its own register budget.  blockIdx.y walks the
 // tables of variant V (w.vlist), blockIdx.x the table's equal-cost slices.
 template <int V>
-__global__ void __launch_bounds__(128) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
+__global__ void __launch_bounds__(128, (V == 0 || V == 1) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
     extern __shared__ __align__(16) float sm[];
     __shared__ uint32_t next;

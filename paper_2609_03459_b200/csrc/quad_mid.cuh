@@ -24,18 +24,19 @@ template <int COLS, int MROWS, int KTMAX>
 __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
                                                 const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane)
 {
-    static_assert((MROWS == 4 || MROWS == 8) && KTMAX % 4 == 0, "stacking of 4 or 2 groups");
+    static_assert((MROWS == 4 || MROWS == 8) && KTMAX % 2 == 0, "stacking of 4 or 2 groups");
     const int g = lane >> 2, t = lane & 3, m = g & (MROWS - 1);
     const int kta = (ra + 7) >> 3;
-    Tf32Pair a[KTMAX][4];
+    // the stacked operand stays unsplit in registers (KTMAX * 4) and is split where it is used: half the registers of
+    // pre-split fragments, which buys a resident CTA more per SM
+    float araw[KTMAX][4];
 #pragma unroll
     for (int kt = 0; kt < KTMAX; ++kt) {
         const int k0 = 8 * kt + t, k1 = k0 + 4;
-        const float a0 = (selA && k0 < ra) ? __ldg(srcA + m * ra + k0) : 0.f;
-        const float a1 = (selB && k0 < ra) ? __ldg(srcB + m * ra + k0) : 0.f;
-        const float a2 = (selA && k1 < ra) ? __ldg(srcA + m * ra + k1) : 0.f;
-        const float a3 = (selB && k1 < ra) ? __ldg(srcB + m * ra + k1) : 0.f;
-        a[kt][0] = tt_split_tf32(a0); a[kt][1] = tt_split_tf32(a1); a[kt][2] = tt_split_tf32(a2); a[kt][3] = tt_split_tf32(a3);
+        araw[kt][0] = (selA && k0 < ra) ? __ldg(srcA + m * ra + k0) : 0.f;
+        araw[kt][1] = (selB && k0 < ra) ? __ldg(srcB + m * ra + k0) : 0.f;
+        araw[kt][2] = (selA && k1 < ra) ? __ldg(srcA + m * ra + k1) : 0.f;
+        araw[kt][3] = (selB && k1 < ra) ? __ldg(srcB + m * ra + k1) : 0.f;
     }
     const float4* __restrict__ B4 = reinterpret_cast<const float4*>(B);
     constexpr int C4N = COLS / 4;
@@ -47,17 +48,20 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
 #pragma unroll
         for (int j = 0; j < 4; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
 #pragma unroll
-        for (int kc = 0; kc < KTMAX; kc += 4) {   // four k steps (32 rows of B) in flight at a time
-            float4 f[4][2];
+        for (int kc = 0; kc < KTMAX; kc += 2) {   // two k steps (16 rows of B) in flight at a time
+            float4 f[2][2];
 #pragma unroll
-            for (int kt = 0; kt < 4; ++kt) {
+            for (int kt = 0; kt < 2; ++kt) {
                 const int k0 = 8 * (kc + kt) + t, k1 = k0 + 4;
                 f[kt][0] = k0 < ra ? __ldg(B4 + (size_t)k0 * C4N + 8 * nb + g) : make_float4(0.f, 0.f, 0.f, 0.f);
                 f[kt][1] = k1 < ra ? __ldg(B4 + (size_t)k1 * C4N + 8 * nb + g) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int kt = 0; kt < 4; ++kt) {
+            for (int kt = 0; kt < 2; ++kt) {
                 if (kc + kt < kta) {
+                    Tf32Pair a[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) a[x] = tt_split_tf32(araw[kc + kt][x]);
                     const float v0[4] = {f[kt][0].x, f[kt][0].y, f[kt][0].z, f[kt][0].w};
                     const float v1[4] = {f[kt][1].x, f[kt][1].y, f[kt][1].z, f[kt][1].w};
 #pragma unroll
@@ -65,7 +69,7 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
                         Tf32Pair b[2];
                         b[0] = tt_split_tf32(v0[j]);
                         b[1] = tt_split_tf32(v1[j]);
-                        tt_mma_3xtf32(acc[j], a[kc + kt], b);
+                        tt_mma_3xtf32(acc[j], a, b);
                     }
                 }
             }
