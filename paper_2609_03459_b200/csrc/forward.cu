@@ -281,15 +281,19 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
     const int rb_ = g >> 2, jb = g & 3;   // this lane's B-fragment column: child row rb_ of the pair, output column jb
     const int rc = t >> 1, jc = 2 * (t & 1);  // this lane's C-fragment columns: child row rc, output columns jc, jc+1
     constexpr int NP = 3;   // row pairs in flight
-    uint32_t ids = 0;       // last digits of 32 rows at a time, one per lane (the loop takes them by shuffle)
+    constexpr uint32_t IDC = 32 - 32 % (2 * NP);   // rows per id chunk: a multiple of the rows per iteration
+    uint32_t ids = 0, cb = u0;   // last digits of IDC rows at a time, one per lane (the loop takes them by shuffle)
     for (uint32_t ub = u0; ub < u1; ub += 2 * NP) {
-        if (((ub - u0) & 31u) == 0u) ids = ub + lane < u1 ? rows[ub + lane] - row_base : 0u;
+        if (ub == cb + IDC || ub == u0) {
+            cb = ub;
+            ids = (lane < IDC && ub + lane < u1) ? rows[ub + lane] - row_base : 0u;
+        }
         float bv[NP][KT][2];
 #pragma unroll
         for (int np = 0; np < NP; ++np) {
             // an odd tail (or a missing second pair) repeats the last row; it is computed but not stored
             const uint32_t ul = min(ub + 2 * np + (uint32_t)rb_, u1 - 1);
-            const uint32_t iK = __shfl_sync(0xffffffffu, ids, (ul - u0) & 31u);
+            const uint32_t iK = __shfl_sync(0xffffffffu, ids, ul - cb);
             const float* __restrict__ Dl = GK + (size_t)iK * (RB * 4) + jb;
 #pragma unroll
             for (int kt = 0; kt < KT; ++kt) {
