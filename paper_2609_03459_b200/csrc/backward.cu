@@ -844,6 +844,7 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
             for (int x = 0; x < 4; ++x) { acc[mt][nt][x] = 0.f; tot[mt][nt][x] = 0.f; }
     for (uint32_t ub0 = u0; ub0 < u1; ub0 += 32) {
     const uint32_t ub1 = min(ub0 + 32u, u1);
+#pragma unroll 2
     for (uint32_t ub = ub0; ub < ub1; ub += 2) {
         const bool two = ub + 1 < u1;
         const uint32_t ua = ub, uc = two ? ub + 1 : ub;
@@ -909,6 +910,7 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
         }
     const int rb_ = g >> 2, jb = g & 3;       // B fragment: row rb_ of the pair, column jb of dE
     const int rc = t >> 1, jc = 2 * (t & 1);  // C fragment: row rc of the pair, columns jc, jc+1
+#pragma unroll 2
     for (uint32_t ub = u0; ub < u1; ub += 2) {
         const uint32_t ul = min(ub + (uint32_t)rb_, u1 - 1);
         const bool valid = ub + (uint32_t)rb_ < u1;
