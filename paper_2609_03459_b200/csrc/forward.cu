@@ -280,7 +280,7 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
     const uint32_t* __restrict__ rows = w.val[K];
     const int rb_ = g >> 2, jb = g & 3;   // this lane's B-fragment column: child row rb_ of the pair, output column jb
     const int rc = t >> 1, jc = 2 * (t & 1);  // this lane's C-fragment columns: child row rc, output columns jc, jc+1
-    constexpr int NP = 3;   // row pairs in flight
+    constexpr int NP = MT == 1 ? 3 : 2;   // row pairs in flight (two where C has two row tiles: registers)
     constexpr uint32_t IDC = 32 - 32 % (2 * NP);   // rows per id chunk: a multiple of the rows per iteration
     uint32_t ids = 0, cb = u0;   // last digits of IDC rows at a time, one per lane (the loop takes them by shuffle)
     for (uint32_t ub = u0; ub < u1; ub += 2 * NP) {
