@@ -537,9 +537,16 @@ cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s)
 __device__ __forceinline__ void tt_unit_range_b(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
 {
     const TableDesc& td = w.tdesc[t];
-    const int Q = td.units;
     const int lvl = w.K - 1;
     const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
+    // the host sizes the grid for the largest possible number of groups; with fewer groups in this batch the table is
+    // cut into fewer units (at least 16 groups each) and the surplus CTAs leave at once
+    int Q = td.units;
+    {
+        const int by_groups = (int)((b - a) >> 4);
+        if (Q > by_groups) Q = by_groups < 1 ? 1 : by_groups;
+    }
+    if (q >= Q) { g0 = a; g1 = a; return; }
     const uint64_t ca = w.cost[a], cb = w.cost[b];
     const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
     auto lower = [&](uint64_t target) {

@@ -14,6 +14,8 @@
 #include "mma.cuh"
 #include "quad_mid.cuh"
 
+__device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc);   // defined with the pooling kernels
+
 // ---------------------------------------------------------------------------------------------- schedule
 
 struct CostScan {
@@ -58,9 +60,16 @@ cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s)
 __device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
 {
     const TableDesc& td = w.tdesc[t];
-    const int Q = td.units;
     const int lvl = w.K - 1;
     const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
+    // the host sizes the grid for the largest possible number of groups; with fewer groups in this batch the table is
+    // cut into fewer units (at least 16 groups each) and the surplus CTAs leave at once
+    int Q = td.units;
+    {
+        const int by_groups = (int)((b - a) >> 4);
+        if (Q > by_groups) Q = by_groups < 1 ? 1 : by_groups;
+    }
+    if (q >= Q) { g0 = a; g1 = a; return; }
     const uint64_t ca = w.cost[a], cb = w.cost[b];
     if (w.ablation & 2) {   // study switch: static schedule, equal group counts
         g0 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)q / Q);
@@ -211,7 +220,7 @@ __device__ __forceinline__ void tt_warp_mid(const float* As, const float* __rest
 // E rows u0..u1 of the group whose C (PM x RB, row-major) is in Cs.  d_K = 4.
 template <int PM, int RB, int TP>
 __device__ __forceinline__ void tt_warp_rows(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
-                                             uint32_t row_base, int lane)
+                                             uint32_t row_base, int lane, int part = 0, int nparts = 1)   // this warp takes every nparts-th batch
 {
     constexpr int LR = PM / TP;   // lanes per row
     constexpr int RW = 32 / LR;   // rows per batch
@@ -227,7 +236,7 @@ __device__ __forceinline__ void tt_warp_rows(const float* Cs, const WsView& w, c
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
     const uint32_t* __restrict__ rows = w.val[K];
-    for (uint32_t ub = u0; ub < u1; ub += RW) {
+    for (uint32_t ub = u0 + (uint32_t)(part * RW); ub < u1; ub += (uint32_t)(RW * nparts)) {
         const uint32_t u = ub + slot;
         const bool act = u < u1;
         const uint32_t iK = act ? rows[u] - row_base : 0u;
@@ -398,6 +407,125 @@ __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& 
     }
 }
 
+// Stacked product of two 8-row groups against this warp's 64 columns of the slice B (ra <= 64 rows, COLS columns): the
+// 64 x 64 block is fetched into shared memory in one go (32 cp.async per lane, one L2 round trip instead of one per 16
+// rows and 32 columns), then the 3xTF32 tiles run from shared memory.  Row stride 68 floats: fragment loads 2-way at worst.
+template <int COLS>
+__device__ __forceinline__ void tt_pair_mid_staged(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
+                                                   const float* __restrict__ srcB, bool selA, bool selB, float* Cs2, float* stg,
+                                                   int lane, int wid)
+{
+    constexpr int RS = 68;
+    const int g = lane >> 2, t = lane & 3;
+    const int c0 = 64 * wid;   // first column of this warp's block
+    for (int i = lane; i < 64 * 16; i += 32) {
+        const int k = i >> 4, f = i & 15;
+        if (k < ra) tt_cp_async16(stg + k * RS + 4 * f, B + (size_t)k * COLS + c0 + 4 * f);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    float araw[8][4];   // rows g (first group) and g + 8 (second group) of the stacked operand, unsplit
+#pragma unroll
+    for (int kt = 0; kt < 8; ++kt) {
+        const int k0 = 8 * kt + t, k1 = k0 + 4;
+        araw[kt][0] = (selA && k0 < ra) ? __ldg(srcA + g * ra + k0) : 0.f;
+        araw[kt][1] = (selB && k0 < ra) ? __ldg(srcB + g * ra + k0) : 0.f;
+        araw[kt][2] = (selA && k1 < ra) ? __ldg(srcA + g * ra + k1) : 0.f;
+        araw[kt][3] = (selB && k1 < ra) ? __ldg(srcB + g * ra + k1) : 0.f;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    const int kta = (ra + 7) >> 3;
+    float* dstA = Cs2 + g * COLS + c0 + 8 * t;                  // group 0, row g of P
+    float* dstB = Cs2 + (size_t)8 * COLS + g * COLS + c0 + 8 * t;   // group 1
+#pragma unroll 1
+    for (int nb = 0; nb < 2; ++nb) {
+        float acc[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
+#pragma unroll
+        for (int kt = 0; kt < 8; ++kt) {
+            if (kt < kta) {
+                const int k0 = 8 * kt + t, k1 = k0 + 4;
+                const float4 f0 = k0 < ra ? *reinterpret_cast<const float4*>(stg + k0 * RS + 32 * nb + 4 * g) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 f1 = k1 < ra ? *reinterpret_cast<const float4*>(stg + k1 * RS + 32 * nb + 4 * g) : make_float4(0.f, 0.f, 0.f, 0.f);
+                Tf32Pair a[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) a[x] = tt_split_tf32(araw[kt][x]);
+                const float v0[4] = {f0.x, f0.y, f0.z, f0.w};
+                const float v1[4] = {f1.x, f1.y, f1.z, f1.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    Tf32Pair b[2];
+                    b[0] = tt_split_tf32(v0[j]);
+                    b[1] = tt_split_tf32(v1[j]);
+                    tt_mma_3xtf32(acc[j], a, b);
+                }
+            }
+        }
+        if (selA) {
+            *reinterpret_cast<float4*>(dstA + 32 * nb) = make_float4(acc[0][0], acc[1][0], acc[2][0], acc[3][0]);
+            *reinterpret_cast<float4*>(dstA + 32 * nb + 4) = make_float4(acc[0][1], acc[1][1], acc[2][1], acc[3][1]);
+        }
+        if (selB) {
+            *reinterpret_cast<float4*>(dstB + 32 * nb) = make_float4(acc[0][2], acc[1][2], acc[2][2], acc[3][2]);
+            *reinterpret_cast<float4*>(dstB + 32 * nb + 4) = make_float4(acc[0][3], acc[1][3], acc[2][3], acc[3][3]);
+        }
+    }
+    __syncwarp();   // the block is overwritten by the next call
+}
+
+// Rank-64 four-core shape: the stage K-1 product of one group is 8 x 64 by 64 x 256 and there are few groups (tens of
+// thousands), so the whole CTA works on one pair of groups at a time: the four warps each compute two of the eight
+// column blocks of the stacked 16-row tensor-core product into one shared C buffer (16 KB per CTA instead of per
+// warp), then two warps per group produce its rows.  Four times the parallelism per pair of the warp-per-pair form.
+template <int PM, int RB>
+__device__ __forceinline__ void tt_sweep_pair_cta(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* Cs2,
+                                                  int lane, int wid)
+{
+    constexpr int MROWS = 8, COLS = PM / MROWS * RB;
+    static_assert(COLS == 256, "four warps x 64 columns");
+    __shared__ uint32_t m_val[2], m_im[2], m_u0[2], m_u1[2];
+    __shared__ const float* m_src[2];
+    const int K = w.K, km = K - 2;
+    const int ra = td.r[km];
+    const uint32_t nK = (uint32_t)td.n[K - 1];
+    for (uint32_t base = g0; base < g1; base += 2) {
+        const int cnt = (int)min(2u, g1 - base);
+        if (threadIdx.x < 2) {
+            const int q = threadIdx.x;
+            if (q < cnt) {
+                const uint32_t pos = base + q;
+                const uint32_t gq = (w.ablation & 1) ? pos : w.tnode[K - 1][pos];
+                const uint32_t v = w.val[K - 1][gq];
+                m_val[q] = v;
+                m_im[q] = v % (uint32_t)td.n[km];
+                m_src[q] = tt_left_operand(w, td, K - 1, gq);
+                m_u0[q] = w.cstart[K - 1][gq];
+                m_u1[q] = w.cstart[K - 1][gq + 1];
+            } else {
+                m_val[q] = 0; m_im[q] = 0xffffffffu; m_src[q] = nullptr; m_u0[q] = 0; m_u1[q] = 0;
+            }
+        }
+        __syncthreads();
+        const float* B0 = td.core[km] + (size_t)m_im[0] * td.slice_floats[km];
+        float* stg = Cs2 + 2 * PM * RB + (size_t)wid * (64 * 68);   // this warp's staged 64 x 64 block of the slice
+        if (cnt == 2 && m_im[1] == m_im[0]) {
+            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, true, Cs2, stg, lane, wid);
+        } else {
+            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, false, Cs2, stg, lane, wid);
+            if (cnt == 2)
+                tt_pair_mid_staged<COLS>(td.core[km] + (size_t)m_im[1] * td.slice_floats[km], ra, m_src[0], m_src[1], false, true, Cs2,
+                                         stg, lane, wid);
+        }
+        __syncthreads();
+        {
+            const int q = wid >> 1;   // warps 0,1: first group; warps 2,3: second group
+            if (q < cnt) tt_warp_rows<PM, RB, 2>(Cs2 + (size_t)q * (PM * RB), w, td, m_u0[q], m_u1[q], m_val[q] * nK, lane, wid & 1, 2);
+        }
+        __syncthreads();
+    }
+}
+
 // generic fallback: the whole CTA works on one group at a time (any shape)
 __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1, float* Pl, float* Cs)
 {
@@ -458,7 +586,7 @@ __global__ void __launch_bounds__(128, (V == 0 || V == 1) ? 6 : 1) k_sweep_fwd(W
     if (V == 0) tt_sweep_quad<16, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 32), &next, lane);
     if (V == 1) tt_sweep_quad<16, 16, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 16), &next, lane);
     if (V == 3) tt_sweep_quad<32, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 32 * 32), &next, lane);
-    if (V == 4) tt_sweep_quad<32, 64, 8, 8, 2>(w, td, g1, sm + (size_t)wid * (2 * 32 * 64), &next, lane);
+    if (V == 4) tt_sweep_pair_cta<32, 64>(w, td, g0, g1, sm, lane, wid);
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
     if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1, false>(w, td, g1, As, Cs, &next, lane);
@@ -475,7 +603,7 @@ static size_t tt_sweep_smem(int V, int max_pl, int max_c)
     if (V == 0) return (size_t)4 * 4 * 16 * 32 * sizeof(float);
     if (V == 1) return (size_t)4 * 4 * 16 * 16 * sizeof(float);
     if (V == 3) return (size_t)4 * 4 * 32 * 32 * sizeof(float);
-    if (V == 4) return (size_t)4 * 2 * 32 * 64 * sizeof(float);
+    if (V == 4) return (size_t)(2 * 32 * 64 + 4 * 64 * 68) * sizeof(float);   // one pair of C tiles per CTA + a staged slice block per warp
     return (size_t)4 * (max_pl + max_c) * sizeof(float);
 }
 

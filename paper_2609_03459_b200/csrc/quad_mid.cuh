@@ -22,7 +22,8 @@
 // that a lane ends up with 8 consecutive columns of each of its two rows (two float4 stores per row).
 template <int COLS, int MROWS, int KTMAX>
 __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
-                                                const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane)
+                                                const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane,
+                                                int nb0 = 0, int nb1 = COLS / 32)   // column blocks of 32 this warp computes
 {
     static_assert((MROWS == 4 || MROWS == 8) && KTMAX % 2 == 0, "stacking of 4 or 2 groups");
     const int g = lane >> 2, t = lane & 3, m = g & (MROWS - 1);
@@ -43,7 +44,7 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
     float* dstA = Cs4 + (size_t)(g / MROWS) * (MROWS * COLS) + m * COLS + 8 * t;
     float* dstB = Cs4 + (size_t)((8 + g) / MROWS) * (MROWS * COLS) + m * COLS + 8 * t;
 #pragma unroll 1
-    for (int nb = 0; nb < COLS / 32; ++nb) {
+    for (int nb = nb0; nb < nb1; ++nb) {
         float acc[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) { acc[j][0] = 0.f; acc[j][1] = 0.f; acc[j][2] = 0.f; acc[j][3] = 0.f; }
