@@ -268,7 +268,7 @@ __device__ __forceinline__ void tt_warp_rows(const float* Cs, const WsView& w, c
 // head and tail) stay in PM*RB/8 registers for the whole group; each child's slice is read exactly once per warp
 // (two coalesced 64-byte pieces per load instruction), so the shared-memory / L1 path carries 4x fewer bytes per
 // FMA than the FP32-pipe form and a warp needs ~1/3 of its registers.
-template <int PM, int RB>
+template <int PM, int RB, int CS = RB>   // CS: row stride of C in shared memory
 __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
                                                  uint32_t row_base, int lane)
 {
@@ -279,10 +279,10 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
-            a[mt][kt][0] = tt_split_tf32(Cs[(16 * mt + g) * RB + 8 * kt + t]);
-            a[mt][kt][1] = tt_split_tf32(Cs[(16 * mt + g + 8) * RB + 8 * kt + t]);
-            a[mt][kt][2] = tt_split_tf32(Cs[(16 * mt + g) * RB + 8 * kt + t + 4]);
-            a[mt][kt][3] = tt_split_tf32(Cs[(16 * mt + g + 8) * RB + 8 * kt + t + 4]);
+            a[mt][kt][0] = tt_split_tf32(Cs[(16 * mt + g) * CS + 8 * kt + t]);
+            a[mt][kt][1] = tt_split_tf32(Cs[(16 * mt + g + 8) * CS + 8 * kt + t]);
+            a[mt][kt][2] = tt_split_tf32(Cs[(16 * mt + g) * CS + 8 * kt + t + 4]);
+            a[mt][kt][3] = tt_split_tf32(Cs[(16 * mt + g + 8) * CS + 8 * kt + t + 4]);
         }
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
@@ -395,12 +395,12 @@ __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& 
             u0q = w.cstart[K - 1][gq];
             u1q = w.cstart[K - 1][gq + 1];
         }
-        tt_quad_mid<COLS, MROWS, KTMAX>(td.core[km], td.slice_floats[km], ra, cnt, imq, srcq, Cs4, lane);
+        tt_quad_mid<COLS, MROWS, KTMAX, (TP == 0 ? RB : 0)>(td.core[km], td.slice_floats[km], ra, cnt, imq, srcq, Cs4, lane);
         __syncwarp();
         for (int q = 0; q < cnt; ++q) {
             const uint32_t val = __shfl_sync(0xffffffffu, valq, q);
             const uint32_t u0 = __shfl_sync(0xffffffffu, u0q, q), u1 = __shfl_sync(0xffffffffu, u1q, q);
-            if constexpr (TP == 0) tt_warp_rows_mma<PM, RB>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
+            if constexpr (TP == 0) tt_warp_rows_mma<PM, RB, RB + 4>(Cs4 + (size_t)q * (PM * (RB + 4)), w, td, u0, u1, val * nK, lane);
             else tt_warp_rows<PM, RB, TP>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
         }
         __syncwarp();
@@ -583,9 +583,9 @@ __global__ void __launch_bounds__(128, (V == 0 || V == 1) ? 6 : 1) k_sweep_fwd(W
     if (threadIdx.x == 0) next = g0;
     __syncthreads();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    if (V == 0) tt_sweep_quad<16, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 32), &next, lane);
-    if (V == 1) tt_sweep_quad<16, 16, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 16), &next, lane);
-    if (V == 3) tt_sweep_quad<32, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 32 * 32), &next, lane);
+    if (V == 0) tt_sweep_quad<16, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 36), &next, lane);
+    if (V == 1) tt_sweep_quad<16, 16, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 20), &next, lane);
+    if (V == 3) tt_sweep_quad<32, 32, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 32 * 36), &next, lane);
     if (V == 4) tt_sweep_pair_cta<32, 64>(w, td, g0, g1, sm, lane, wid);
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
@@ -600,9 +600,9 @@ __global__ void __launch_bounds__(128, (V == 0 || V == 1) ? 6 : 1) k_sweep_fwd(W
 // dynamic shared memory of k_sweep_fwd<V> / k_sweep_bwd<V>: four C tiles per warp for the tensor-core variants
 static size_t tt_sweep_smem(int V, int max_pl, int max_c)
 {
-    if (V == 0) return (size_t)4 * 4 * 16 * 32 * sizeof(float);
-    if (V == 1) return (size_t)4 * 4 * 16 * 16 * sizeof(float);
-    if (V == 3) return (size_t)4 * 4 * 32 * 32 * sizeof(float);
+    if (V == 0) return (size_t)4 * 4 * 16 * 36 * sizeof(float);   // C rows padded by four floats (conflict-free fragment loads)
+    if (V == 1) return (size_t)4 * 4 * 16 * 20 * sizeof(float);
+    if (V == 3) return (size_t)4 * 4 * 32 * 36 * sizeof(float);
     if (V == 4) return (size_t)(2 * 32 * 64 + 4 * 64 * 68) * sizeof(float);   // one pair of C tiles per CTA + a staged slice block per warp
     return (size_t)4 * (max_pl + max_c) * sizeof(float);
 }

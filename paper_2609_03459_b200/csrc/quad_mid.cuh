@@ -20,7 +20,9 @@
 // Column mapping: a block of 32 columns is one float4 load per lane and k row (8 lanes x 16 bytes = 128 bytes per
 // row); tile j of the block takes component j, i.e. tile column n' stands for slice column 32 * block + 4 n' + j, so
 // that a lane ends up with 8 consecutive columns of each of its two rows (two float4 stores per row).
-template <int COLS, int MROWS, int KTMAX>
+// RBP > 0: C tiles are stored as [PM][RBP + 4] (rows of r_{K-1} = RBP values padded by four floats), which makes the
+// row stage's fragment loads from shared memory conflict-free; RBP = 0: plain [MROWS][COLS] tiles.
+template <int COLS, int MROWS, int KTMAX, int RBP = 0>
 __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
                                                 const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane,
                                                 int nb0 = 0, int nb1 = COLS / 32)   // column blocks of 32 this warp computes
@@ -41,8 +43,18 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
     }
     const float4* __restrict__ B4 = reinterpret_cast<const float4*>(B);
     constexpr int C4N = COLS / 4;
-    float* dstA = Cs4 + (size_t)(g / MROWS) * (MROWS * COLS) + m * COLS + 8 * t;
-    float* dstB = Cs4 + (size_t)((8 + g) / MROWS) * (MROWS * COLS) + m * COLS + 8 * t;
+    constexpr int DSUB = RBP > 0 ? COLS / RBP : 1;              // d_{K-1}: rows of C per row of P
+    constexpr int TILE = RBP > 0 ? MROWS * DSUB * (RBP + 4) : MROWS * COLS;
+    float* dstA = Cs4 + (size_t)(g / MROWS) * TILE + (RBP > 0 ? 0 : m * COLS + 8 * t);
+    float* dstB = Cs4 + (size_t)((8 + g) / MROWS) * TILE + (RBP > 0 ? 0 : m * COLS + 8 * t);
+    // offset of columns [32 nb + 8 t, + 8) of row m inside a tile
+    auto coff = [&](int nb) {
+        if (RBP > 0) {
+            const int col = 32 * nb + 8 * t;
+            return (m * DSUB + col / RBP) * (RBP + 4) + col % RBP;
+        }
+        return 32 * nb;
+    };
 #pragma unroll 1
     for (int nb = nb0; nb < nb1; ++nb) {
         float acc[4][4];
@@ -76,19 +88,19 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
             }
         }
         if (selA) {
-            *reinterpret_cast<float4*>(dstA + 32 * nb) = make_float4(acc[0][0], acc[1][0], acc[2][0], acc[3][0]);
-            *reinterpret_cast<float4*>(dstA + 32 * nb + 4) = make_float4(acc[0][1], acc[1][1], acc[2][1], acc[3][1]);
+            *reinterpret_cast<float4*>(dstA + coff(nb)) = make_float4(acc[0][0], acc[1][0], acc[2][0], acc[3][0]);
+            *reinterpret_cast<float4*>(dstA + coff(nb) + 4) = make_float4(acc[0][1], acc[1][1], acc[2][1], acc[3][1]);
         }
         if (selB) {
-            *reinterpret_cast<float4*>(dstB + 32 * nb) = make_float4(acc[0][2], acc[1][2], acc[2][2], acc[3][2]);
-            *reinterpret_cast<float4*>(dstB + 32 * nb + 4) = make_float4(acc[0][3], acc[1][3], acc[2][3], acc[3][3]);
+            *reinterpret_cast<float4*>(dstB + coff(nb)) = make_float4(acc[0][2], acc[1][2], acc[2][2], acc[3][2]);
+            *reinterpret_cast<float4*>(dstB + coff(nb) + 4) = make_float4(acc[0][3], acc[1][3], acc[2][3], acc[3][3]);
         }
     }
 }
 
 // All passes of one batch of cnt <= 16 / MROWS groups.  Lane q < cnt holds group q's slice index (imq) and operand
 // pointer (srcq).
-template <int COLS, int MROWS, int KTMAX>
+template <int COLS, int MROWS, int KTMAX, int RBP = 0>
 __device__ __forceinline__ void tt_quad_mid(const float* __restrict__ core_mid, size_t slice_floats, int ra, int cnt, uint32_t imq,
                                             const float* srcq, float* Cs4, int lane)
 {
@@ -103,7 +115,7 @@ __device__ __forceinline__ void tt_quad_mid(const float* __restrict__ core_mid, 
         const uint32_t im = __shfl_sync(0xffffffffu, imq, first);
         const unsigned sel = __ballot_sync(0xffffffffu, lane < 4 && ((remaining >> lane) & 1u) && imq == im) & 0xfu;
         const bool selA = (sel >> qA) & 1u, selB = (sel >> qB) & 1u;
-        tt_quad_mid_mma<COLS, MROWS, KTMAX>(core_mid + (size_t)im * slice_floats, ra, srcA, srcB, selA, selB, Cs4, lane);
+        tt_quad_mid_mma<COLS, MROWS, KTMAX, RBP>(core_mid + (size_t)im * slice_floats, ra, srcA, srcB, selA, selB, Cs4, lane);
         remaining &= ~sel;
     }
 }
