@@ -661,7 +661,9 @@ __device__ __forceinline__ void tt_red_v4(float* p, float x, float y, float z, f
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(wv) : "memory");
 }
 
-template <int M, int CPL>
+// RBP > 0: C is stored as [P][RBP + 8] (rows of r_{K-1} = RBP values, stride RBP + 8 floats), the layout whose transposed
+// fragment loads in the tensor-core dG pass are free of bank conflicts; RBP = 0: plain [M][cols].
+template <int M, int CPL, int RBP = 0>
 __device__ __forceinline__ void tt_warp_mid_b(const float* As, const float* __restrict__ Bsl, float* Cs, int ra, int cols, int lane)
 {
     const int c4n = cols >> 2;
@@ -711,8 +713,12 @@ __device__ __forceinline__ void tt_warp_mid_b(const float* As, const float* __re
 #pragma unroll
         for (int i = 0; i < CPL; ++i)
 #pragma unroll
-            for (int m = 0; m < M; ++m)
-                *reinterpret_cast<float4*>(Cs + m * cols + 4 * (ll + i * LA)) = make_float4(acc[i][m][0], acc[i][m][1], acc[i][m][2], acc[i][m][3]);
+            for (int m = 0; m < M; ++m) {
+                const int col = 4 * (ll + i * LA);
+                float* dst = RBP > 0 ? Cs + (m * (cols / (RBP > 0 ? RBP : 1)) + col / (RBP > 0 ? RBP : 1)) * (RBP + 8) + col % (RBP > 0 ? RBP : 1)
+                                     : Cs + m * cols + col;
+                *reinterpret_cast<float4*>(dst) = make_float4(acc[i][m][0], acc[i][m][1], acc[i][m][2], acc[i][m][3]);
+            }
     }
 }
 
@@ -910,10 +916,10 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
-            a[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g]);
-            a[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g + 8]);
-            a[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g]);
-            a[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g + 8]);
+            a[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
+            a[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
+            a[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
+            a[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     const int rb_ = g >> 2, jb = g & 3;       // B fragment: row rb_ of the pair, column jb of dE
     const int rc = t >> 1, jc = 2 * (t & 1);  // C fragment: row rc of the pair, columns jc, jc+1
@@ -968,10 +974,10 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
     for (int mt = 0; mt < MT2; ++mt)
 #pragma unroll
         for (int kt = 0; kt < KT2; ++kt) {
-            ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g]);
-            ct[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * RB_ + 16 * mt + g + 8]);
-            ct[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g]);
-            ct[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * RB_ + 16 * mt + g + 8]);
+            ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
+            ct[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
+            ct[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
+            ct[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     float dc[MT][NT][4], dct[MT][NT][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
 #pragma unroll
@@ -1089,7 +1095,7 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
         }
         __syncwarp();
         const uint32_t im = val % (uint32_t)td.n[km];
-        tt_warp_mid_b<M, CPL>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
+        tt_warp_mid_b<M, CPL, (MMA ? RB_ : 0)>(As, td.core[km] + (size_t)im * td.slice_floats[km], Cs, ra, cols, lane);
         __syncwarp();
         const uint32_t u0 = w.cstart[K - 1][g], u1 = w.cstart[K - 1][g + 1];
         if constexpr (MMA) {
@@ -1168,6 +1174,10 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
 {
     const int n = h->vcount[V + 1];
     if (n == 0) return cudaSuccess;
+    // tensor-core variants keep C with padded rows (stride r_{K-1} + 8 floats)
+    if (V == 0) max_c = 16 * (32 + 8);
+    if (V == 1) max_c = 16 * (16 + 8);
+    if (V == 3) max_c = 32 * (32 + 8);
     const size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
                               : (size_t)4 * (max_pl + max_c) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
