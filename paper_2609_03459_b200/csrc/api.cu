@@ -124,7 +124,11 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             td.slice_floats[k] = td.r[k] * td.d[k] * td.r[k + 1];
             td.core_floats[k] = (int64_t)td.n[k] * td.slice_floats[k];
             if (td.P[k + 1] * td.r[k + 1] > 4096) return fail(TT_EMB_ERR_ARG);
-            if (td.P[k + 1] * td.r[k + 1] > stride[k + 1]) stride[k + 1] = td.P[k + 1] * td.r[k + 1];
+            // node pitch of the level buffers (partial products, dP, Y): the largest P_k * r_k over the tables, rounded
+            // up to four floats -- tables of the register-tiled variants read their nodes with 16-byte accesses, and a
+            // generic table of the same handle may have the larger, odd P_k * r_k
+            const int pr = (td.P[k + 1] * td.r[k + 1] + 3) / 4 * 4;
+            if (pr > stride[k + 1]) stride[k + 1] = pr;
         }
         sumN += td.N;
         td.word_base = (uint32_t)words;
