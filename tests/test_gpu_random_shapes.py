@@ -79,3 +79,25 @@ def test_random_shape_forward_backward(binding, seed):
     for t in range(wl.T):
         for k in range(wl.tables[t].K):
             close(grads[t][k], ref[t][k], f"random {seed} dG[{t}][{k}] (d={tables[t].d}, r={tables[t].r}, n={tables[t].n})")
+
+
+@pytest.mark.parametrize("seed", range(24, 40))
+def test_random_shape_weighted_mean_int32(binding, seed):
+    # the same draw of shapes under the other pooling laws, ids handed over as int32 on the even seeds
+    tables, B, pooling = random_case(seed)
+    wl = workloads.custom(tables, B, pooling, seed=500 + seed, with_grad=True, name=f"random-{seed}")
+    weighted = seed % 4 < 2
+    wts = np.random.default_rng(seed).normal(size=wl.L).astype(np.float32) if weighted else None
+    mode = "sum" if weighted else "mean"
+    emb = binding.from_workload(wl, enable_backward=True, enable_weighted=True)
+    emb.set_pooling(mode, None if wts is None else dev(wts))
+    ids = wl.indices.astype(np.int32) if seed % 2 == 0 else wl.indices
+    out = emb.forward(dev(ids), dev(wl.offsets), wl.B).cpu().numpy()
+    assert emb.status() == 0
+    close(out, oracle.forward_workload(wl, weights=wts, mode=mode), f"random {seed} {mode} out")
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl, weights=wts, mode=mode)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            close(grads[t][k], ref[t][k], f"random {seed} {mode} dG[{t}][{k}] (d={tables[t].d}, r={tables[t].r}, n={tables[t].n})")
