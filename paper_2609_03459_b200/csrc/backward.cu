@@ -2,8 +2,8 @@
 //
 //   1. sort:  the forward left one (slot, bag) pair per lookup; a counting sort by slot (counts -> exclusive
 //             scan -> scatter) groups the lookups of every distinct row.  Hot rows would serialise global
-//             atomics, so each CTA first aggregates its tile in a shared-memory hash table and issues one
-//             global atomic per distinct row per tile.
+//             atomics, so each CTA first aggregates the duplicates of its tile in shared memory (owner tags) and
+//             issues one global atomic per aggregated row per tile.
 //   2. dE:    segmented sum of grad_out rows over the sorted pairs.  Fixed-size chunks of sorted positions per
 //             warp (skew-proof); segments that cross chunk borders leave partial sums which a second kernel
 //             adds in position order.
@@ -48,20 +48,45 @@ __global__ void k_zero_grads(WsView w)
 // ---------------------------------------------------------------------------------------------- 1. sort by slot
 
 // MODE 0: cnt[slot] += occurrences.  MODE 1: pairs[seg_start[slot] + claimed position] = (slot, bag).
+//
+// Aggregation of a tile's duplicates without a probing hash table (two shared-memory atomics per pair made the
+// shared-memory atomic unit the limit of both passes): every pair stores a tag (low key bits, its number in the tile)
+// into bucket h(key) with a plain store; after a barrier the bucket holds the tag of one of its writers.  That pair
+// owns the bucket.  A pair with the owner's key is a duplicate: it counts itself in extra[h] (the only shared-memory
+// atomic left, and only duplicates issue it) and the owner makes one global atomic for all of them.  A pair with another
+// key lost the bucket and goes to the global counter by itself.  h takes the key bits above bit 19 as they are, so that
+// bucket and the 20 low bits together identify the key and a 32-bit tag is enough.
+#define HT_LOW_BITS 20
+#define HT_ID_BITS 11
 template <int MODE>
 __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 {
+    static_assert(HT_TILE == (1 << HT_ID_BITS) && HT_SIZE == (1 << (32 - HT_LOW_BITS)) && HT_LOW_BITS + HT_ID_BITS <= 32, "tag layout");
     const uint2* __restrict__ upairs = w.upairs;
     const uint32_t capK = w.cap[w.K];
-    __shared__ uint32_t keys[HT_SIZE];
-    __shared__ uint32_t vals[HT_SIZE];
+    __shared__ uint32_t tag[HT_SIZE];
+    __shared__ uint32_t extra[HT_SIZE];   // duplicates of the owner's key; MODE 1: then the claimed base position
     const int64_t L = w.L;
     const int64_t ntiles = (L + HT_TILE - 1) / HT_TILE;
+    const bool weighted = MODE == 1 && w.wsorted && (w.psw || w.pool_mean);
+    for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) extra[i] = 0u;
+    // the first barrier of the tile loop orders this before the first atomic on extra
+    auto emit = [&](uint32_t pos, const uint2& pr, int64_t l) {
+        w.pairs[pos] = pr;
+        if (weighted) {   // weighted / mean pooling: the pair's factor travels with it
+            float a = w.psw ? __ldg(w.psw + l) : 1.f;
+            if (w.pool_mean) {
+                const int64_t gb = (int64_t)tt_find_table(w.tb[w.K], w.T, pr.x) * w.B + pr.y;
+                const int64_t len = __ldg(w.offsets + gb + 1) - __ldg(w.offsets + gb);
+                a /= (float)(len > 0 ? len : 1);
+            }
+            w.wsorted[pos] = a;
+        }
+    };
+    enum { ROLE_NONE = 0, ROLE_OWNER = 1, ROLE_DUP = 2 };
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) { keys[i] = HT_EMPTY; vals[i] = 0u; }
-        __syncthreads();
         uint2 pr[HT_TILE / 256];
-        uint32_t hh[HT_TILE / 256], rk[HT_TILE / 256];
+        uint32_t st[HT_TILE / 256];   // bucket (12 bits) | rank among the duplicates (12 bits) << 12 | role << 24
 #pragma unroll
         for (int j = 0; j < HT_TILE / 256; ++j) {
             const int64_t l = tile * HT_TILE + j * 256 + threadIdx.x;
@@ -71,44 +96,56 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 #pragma unroll
         for (int j = 0; j < HT_TILE / 256; ++j) {
             if (pr[j].x == HT_EMPTY) continue;
-            uint32_t p = (pr[j].x * 2654435761u) >> 20;
-            for (int probe = 0; probe < HT_SIZE; ++probe) {
-                const uint32_t old = atomicCAS(&keys[p], HT_EMPTY, pr[j].x);
-                if (old == HT_EMPTY || old == pr[j].x) break;
-                p = (p + 1) & (HT_SIZE - 1);
-            }
-            hh[j] = p;
-            rk[j] = atomicAdd(&vals[p], 1u);
+            const uint32_t low = pr[j].x & ((1u << HT_LOW_BITS) - 1u);
+            const uint32_t h = ((pr[j].x >> HT_LOW_BITS) ^ ((low * 2654435761u) >> HT_LOW_BITS)) & (HT_SIZE - 1);
+            st[j] = h;
+            tag[h] = (low << HT_ID_BITS) | (uint32_t)(j * 256 + threadIdx.x);
         }
         __syncthreads();
-        // one global atomic per distinct row of the tile.  MODE 1 claims a run of positions directly on the scanned
-        // count array: cnt[slot] starts as the segment start and ends as the segment end (= next segment's start)
-        for (int i = threadIdx.x; i < HT_SIZE; i += blockDim.x) {
-            if (keys[i] != HT_EMPTY) {
-                if (MODE == 0) atomicAdd(&w.cnt[keys[i]], vals[i]);
-                else vals[i] = atomicAdd(&w.cnt[keys[i]], vals[i]);
+#pragma unroll
+        for (int j = 0; j < HT_TILE / 256; ++j) {
+            if (pr[j].x == HT_EMPTY) continue;
+            const uint32_t low = pr[j].x & ((1u << HT_LOW_BITS) - 1u);
+            const uint32_t h = st[j];
+            const uint32_t tg = tag[h];
+            if ((tg >> HT_ID_BITS) == low) {
+                if ((tg & (HT_TILE - 1)) == (uint32_t)(j * 256 + threadIdx.x)) st[j] = h | (ROLE_OWNER << 24);
+                else if (MODE == 0) { atomicAdd(&extra[h], 1u); st[j] = h | (ROLE_DUP << 24); }
+                else st[j] = h | ((atomicAdd(&extra[h], 1u) + 1u) << 12) | (ROLE_DUP << 24);
+            } else {   // another key holds the bucket
+                if (MODE == 0) atomicAdd(&w.cnt[pr[j].x], 1u);
+                else emit(atomicAdd(&w.cnt[pr[j].x], 1u), pr[j], tile * HT_TILE + j * 256 + threadIdx.x);
+            }
+        }
+        __syncthreads();
+        // one global atomic per owner.  MODE 1 claims a run of positions directly on the scanned count array:
+        // cnt[slot] starts as the segment start and ends as the segment end (= next segment's start)
+#pragma unroll
+        for (int j = 0; j < HT_TILE / 256; ++j) {
+            if (pr[j].x == HT_EMPTY || (st[j] >> 24) != ROLE_OWNER) continue;
+            const uint32_t h = st[j] & (HT_SIZE - 1);
+            const uint32_t n = 1u + extra[h];
+            if (MODE == 0) {
+                atomicAdd(&w.cnt[pr[j].x], n);
+                extra[h] = 0u;
+            } else {
+                const uint32_t base = atomicAdd(&w.cnt[pr[j].x], n);
+                extra[h] = base;
+                emit(base, pr[j], tile * HT_TILE + j * 256 + threadIdx.x);
             }
         }
         if (MODE == 1) {
             __syncthreads();
 #pragma unroll
             for (int j = 0; j < HT_TILE / 256; ++j) {
-                if (pr[j].x == HT_EMPTY) continue;
-                const uint32_t pos = vals[hh[j]] + rk[j];
-                w.pairs[pos] = pr[j];
-                if (w.wsorted && (w.psw || w.pool_mean)) {   // weighted / mean pooling: the pair's factor travels with it
-                    const int64_t l = tile * HT_TILE + j * 256 + threadIdx.x;
-                    float a = w.psw ? __ldg(w.psw + l) : 1.f;
-                    if (w.pool_mean) {
-                        const int64_t gb = (int64_t)tt_find_table(w.tb[w.K], w.T, pr[j].x) * w.B + pr[j].y;
-                        const int64_t len = __ldg(w.offsets + gb + 1) - __ldg(w.offsets + gb);
-                        a /= (float)(len > 0 ? len : 1);
-                    }
-                    w.wsorted[pos] = a;
-                }
+                if (pr[j].x == HT_EMPTY || (st[j] >> 24) != ROLE_DUP) continue;
+                emit(extra[st[j] & (HT_SIZE - 1)] + ((st[j] >> 12) & 0xfffu), pr[j], tile * HT_TILE + j * 256 + threadIdx.x);
             }
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < HT_TILE / 256; ++j)
+                if (pr[j].x != HT_EMPTY && (st[j] >> 24) == ROLE_OWNER) extra[st[j] & (HT_SIZE - 1)] = 0u;
         }
-        __syncthreads();
     }
 }
 
