@@ -298,7 +298,9 @@ def main():
 
     def step(idx, off, grad):
         emb.forward(idx, off, B, out=d_out)
-        if train:
+        if train and world == 1:
+            emb.backward_sgd(grad, wl.lr)              # the update rides on the kernels that finalise each gradient
+        elif train:
             emb.backward(grad)
             ttd.allreduce_core_grads(emb.flat_grads)   # the one exchange of the data-parallel path
             emb.sgd_step(wl.lr)
@@ -431,7 +433,9 @@ def main():
                 with torch.cuda.stream(down):
                     h_out.copy_(e_out[slot], non_blocking=True)
                     state["out_done"][slot] = down.record_event()
-                if train:
+                if train and world == 1:
+                    emb.backward_sgd(e_grad[slot], wl.lr)
+                elif train:
                     emb.backward(e_grad[slot])
                     ttd.allreduce_core_grads(emb.flat_grads)
                     emb.sgd_step(wl.lr)

@@ -168,6 +168,19 @@ size_t tt_emb_static_workspace_limit(void);
 int tt_emb_sgd_step(tt_emb_t h, float* const* core_grads, float lr, tt_emb_stream_t stream);
 
 /*
+ * tt_emb_backward followed by tt_emb_sgd_step(lr) as one call, with the update fused into the backward
+ *   [Sec. 3.2 backward; the paper mentions a fused update and leaves it switched off]:
+ * every core's gradient has a kernel that writes its final value (the fixed-order sum of the last core's partial
+ * copies, the owner CTA of a middle-core slice, the sum over the children of a first digit); with lr != 0 that
+ * kernel also applies G <- G - lr * dG to the elements it has just finished, so the gradient is not read again.
+ * Cores whose gradient is finalised by a kernel that other blocks still read the core in (generic shape path,
+ * K = 2 first core) are updated by the plain kernel at the end of the call.  core_grads is still fully written
+ * (gradients at the pre-update cores), the result equals the two separate calls up to the rounding of identical
+ * expressions.  Arguments and errors as tt_emb_backward; lr = 0 is tt_emb_backward.  Asynchronous.
+ */
+int tt_emb_backward_sgd(tt_emb_t h, const float* grad_out, float* const* core_grads, float lr, tt_emb_stream_t stream);
+
+/*
  * Copy the device status word (OR of tt_emb_status_bits since the last forward began) to *status_host.
  * SYNCHRONISES `stream`.
  */

@@ -70,6 +70,7 @@ _SIGS = {
     "tt_emb_static_workspace_limit": (ctypes.c_size_t, []),
     "tt_emb_backward": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "tt_emb_sgd_step": (ctypes.c_int, [_vp, _vp, _f32, _vp]),
+    "tt_emb_backward_sgd": (ctypes.c_int, [_vp, _vp, _vp, _f32, _vp]),
     "tt_emb_status": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), _vp]),
     "tt_emb_grouping_counts": (ctypes.c_int, [_vp, _vp, _vp]),
     "tt_emb_export_level": (ctypes.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _vp]),
@@ -290,6 +291,14 @@ class TTEmbeddingBag:
         assert grad_out.dtype == torch.float32 and grad_out.is_cuda and grad_out.is_contiguous()
         ptrs = (ctypes.c_void_p * (self.T * self.K))(*[g.data_ptr() for row in self.grads for g in row])
         _check(lib.tt_emb_backward(self.h, grad_out.data_ptr(), ptrs, _stream_ptr()), "tt_emb_backward")
+        return self.grads
+
+    def backward_sgd(self, grad_out, lr: float):
+        """Backward and SGD update in one call, the update fused into the kernels that finalise each gradient."""
+        torch = self.torch
+        assert grad_out.dtype == torch.float32 and grad_out.is_cuda and grad_out.is_contiguous()
+        ptrs = (ctypes.c_void_p * (self.T * self.K))(*[g.data_ptr() for row in self.grads for g in row])
+        _check(lib.tt_emb_backward_sgd(self.h, grad_out.data_ptr(), ptrs, float(lr), _stream_ptr()), "tt_emb_backward_sgd")
         return self.grads
 
     def sgd_step(self, lr: float):

@@ -231,6 +231,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     WsView& v = h->v;
     v.T = T; v.K = K; v.D = D;
     v.ablation = h->ablation;
+    v.fused_lr = 0.f;
     v.capU = h->capU;
     for (int k = 1; k <= K; ++k) {
         uint64_t c = level_space[k] < (uint64_t)h->capU ? level_space[k] : (uint64_t)h->capU;
@@ -542,21 +543,47 @@ static int upload_grads(tt_emb* h, float* const* core_grads, cudaStream_t s)
     return TT_EMB_OK;
 }
 
-extern "C" int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads, tt_emb_stream_t stream)
+// fused_lr != 0: the kernels that finalise a core's gradient also apply the SGD update (cores in sgd_mask); the
+// remaining cores get the plain update kernel afterwards
+static int backward_any(tt_emb* h, const float* grad_out, float* const* core_grads, float fused_lr, cudaStream_t s)
 {
     if (!h || !grad_out || !core_grads) return TT_EMB_ERR_ARG;
     if (!h->bound || !h->have_forward || !h->enable_backward) return TT_EMB_ERR_STATE;
-    cudaStream_t s = (cudaStream_t)stream;
+    const int K = h->K;
+    bool rest = false;
+    for (int t = 0; t < h->T; ++t) {
+        TableDesc& td = h->tab[t];
+        int mask = 1 << (K - 1);                     // last core: the fixed-order sum of the stripes
+        for (int k = 2; k <= K - 1; ++k)
+            if (td.midfast[k] >= 0) mask |= 1 << (k - 1);   // middle cores: the slice's owner CTA
+        if (K >= 3 && td.midfast[2] >= 0) mask |= 1;        // first core: the sum over the children of a first digit
+        td.sgd_mask = mask;
+        if (mask != (1 << K) - 1) rest = true;
+    }
     int r = upload_grads(h, core_grads, s);
     if (r) return r;
-    for (int i = 4; i < 8; ++i) h->ev_valid[i] = false;
+    for (int i = 4; i < 9; ++i) h->ev_valid[i] = false;
     for (int i = 9 + TT_NUM_VARIANTS + 1; i < TT_NUM_STAGES; ++i) h->ev_valid[i] = false;
+    h->v.fused_lr = fused_lr;
+    struct Reset { tt_emb* h; ~Reset() { h->v.fused_lr = 0.f; } } reset{h};
     TT_STAGE(h, 4, s, tt_launch_bwd_sort(h, s));
     TT_STAGE(h, 5, s, tt_launch_bwd_dE(h, grad_out, s));
     TT_STAGE(h, 6, s, tt_launch_bwd_contraction(h, s));
     TT_STAGE(h, 7, s, tt_launch_bwd_middle(h, s));
     h->have_forward = false;  // dE overwrote the rows; a second backward needs a new forward
+    if (fused_lr != 0.f && rest) TT_STAGE(h, 8, s, tt_launch_sgd(h, fused_lr, true, s));
     return TT_EMB_OK;
+}
+
+extern "C" int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads, tt_emb_stream_t stream)
+{
+    return backward_any(h, grad_out, core_grads, 0.f, (cudaStream_t)stream);
+}
+
+extern "C" int tt_emb_backward_sgd(tt_emb_t h, const float* grad_out, float* const* core_grads, float lr, tt_emb_stream_t stream)
+{
+    if (lr == 0.f) return backward_any(h, grad_out, core_grads, 0.f, (cudaStream_t)stream);
+    return backward_any(h, grad_out, core_grads, lr, (cudaStream_t)stream);
 }
 
 extern "C" int tt_emb_sgd_step(tt_emb_t h, float* const* core_grads, float lr, tt_emb_stream_t stream)
@@ -567,7 +594,7 @@ extern "C" int tt_emb_sgd_step(tt_emb_t h, float* const* core_grads, float lr, t
     int r = upload_grads(h, core_grads, s);
     if (r) return r;
     h->ev_valid[8] = false;
-    TT_STAGE(h, 8, s, tt_launch_sgd(h, lr, s));
+    TT_STAGE(h, 8, s, tt_launch_sgd(h, lr, false, s));
     return TT_EMB_OK;
 }
 

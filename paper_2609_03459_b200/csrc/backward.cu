@@ -1203,6 +1203,7 @@ __global__ void __launch_bounds__(256) k_reduce_gpart(WsView w)
 #pragma unroll
         for (int q = 0; q < TT_STRIPES; ++q) s += src[(size_t)q * w.gpart_stride + i];
         td.grad[kl][i] = s;
+        if (w.fused_lr != 0.f) td.core[kl][i] = td.core[kl][i] - w.fused_lr * s;   // nothing reads the last core after the sweeps
     }
 }
 
@@ -1523,6 +1524,16 @@ __global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
     float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
 #pragma unroll
     for (int i = 0; i < APT; ++i) reinterpret_cast<float4*>(dst + (size_t)(a0 + i) * COLS)[cl] = acc[i];
+    if (w.fused_lr != 0.f) {   // fused update of the CTA's own slice (held in breg since the start; nobody else reads it)
+        float* cdst = td.core[kc] + (size_t)ik * td.slice_floats[kc];
+#pragma unroll
+        for (int i = 0; i < APT; ++i) {
+            float4 u = breg[i];
+            u.x = u.x - w.fused_lr * acc[i].x; u.y = u.y - w.fused_lr * acc[i].y;
+            u.z = u.z - w.fused_lr * acc[i].z; u.w = u.w - w.fused_lr * acc[i].w;
+            reinterpret_cast<float4*>(cdst + (size_t)(a0 + i) * COLS)[cl] = u;
+        }
+    }
 }
 
 // ---- tensor-core form of the middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ----
@@ -1574,7 +1585,10 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
     // in a second register set; each thread adds its accumulators to the elements it owns
     float* const gdst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
     bool first_fold = true;
-    auto fold = [&]() {
+    // last: the sums are final; the fused update of this CTA's slice goes with them (its fragments were read at the start,
+    // and no other CTA or later kernel of the backward reads this slice)
+    float* const cdst = td.core[kc] + (size_t)ik * td.slice_floats[kc];
+    auto fold = [&](bool last) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -1586,6 +1600,14 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 float2 v1 = first_fold ? make_float2(0.f, 0.f) : *p1;
                 v0.x += acc[mt][nt][0]; v0.y += acc[mt][nt][1]; v1.x += acc[mt][nt][2]; v1.y += acc[mt][nt][3];
                 *p0 = v0; *p1 = v1;
+                if (last && w.fused_lr != 0.f) {
+                    float2* c0 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g) * COLS + c);
+                    float2* c1 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g + 8) * COLS + c);
+                    float2 u0 = *c0, u1 = *c1;
+                    u0.x = u0.x - w.fused_lr * v0.x; u0.y = u0.y - w.fused_lr * v0.y;
+                    u1.x = u1.x - w.fused_lr * v1.x; u1.y = u1.y - w.fused_lr * v1.y;
+                    *c0 = u0; *c1 = u1;
+                }
                 acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f;
             }
         first_fold = false;
@@ -1675,10 +1697,10 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
-        if ((r & 7u) == 7u) fold();   // rounded running sums every eighth pass
+        if ((r & 7u) == 7u) fold(false);   // rounded running sums every eighth pass
         __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
     }
-    fold();   // also writes the zeros of a slice without nodes
+    fold(true);   // also writes the zeros of a slice without nodes
 }
 
 // dP_{k-1}[parent] (k = 2: the first core's gradient slice) = sum of the Y rows of the parent's children,
@@ -1703,6 +1725,12 @@ __global__ void __launch_bounds__(256) k_mid_sum(WsView w, int k)
                 s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
             }
             reinterpret_cast<float4*>(dst)[f] = s;
+            if (k == 2 && w.fused_lr != 0.f) {   // first core: the slices of present first digits are final here
+                float4* c4 = reinterpret_cast<float4*>(td.core[0] + (size_t)w.val[1][pn] * td.slice_floats[0]) + f;
+                float4 u = *c4;
+                u.x = u.x - w.fused_lr * s.x; u.y = u.y - w.fused_lr * s.y; u.z = u.z - w.fused_lr * s.z; u.w = u.w - w.fused_lr * s.w;
+                *c4 = u;
+            }
         }
     }
 }
@@ -1775,10 +1803,11 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
 
 // ---------------------------------------------------------------------------------------------- SGD
 
-__global__ void __launch_bounds__(256) k_sgd(WsView w, float lr)
+__global__ void __launch_bounds__(256) k_sgd(WsView w, float lr, int only_unfused)
 {
     const int t = blockIdx.y / w.K, k = blockIdx.y % w.K;
     const TableDesc& td = w.tdesc[t];
+    if (only_unfused && ((td.sgd_mask >> k) & 1)) return;   // updated by the kernel that finalised its gradient
     float* __restrict__ G = td.core[k];
     const float* __restrict__ dG = td.grad[k];
     const int64_t n = td.core_floats[k];
@@ -1786,9 +1815,9 @@ __global__ void __launch_bounds__(256) k_sgd(WsView w, float lr)
         G[i] = G[i] - lr * dG[i];
 }
 
-cudaError_t tt_launch_sgd(tt_emb* h, float lr, cudaStream_t s)
+cudaError_t tt_launch_sgd(tt_emb* h, float lr, bool only_unfused, cudaStream_t s)
 {
-    k_sgd<<<dim3(64, h->T * h->K), 256, 0, s>>>(h->v, lr);
+    k_sgd<<<dim3(64, h->T * h->K), 256, 0, s>>>(h->v, lr, only_unfused ? 1 : 0);
     tt_note_launch();
     return cudaGetLastError();
 }

@@ -34,7 +34,7 @@ struct TableDesc {
     int64_t gpart_off;                  // float offset of this table's last core inside one stripe
     int32_t units;                      // work units (CTAs) this table is cut into
     int32_t unit_base;                  // first global unit id
-    int32_t pad0;
+    int32_t sgd_mask;                   // bit k: the fused backward + SGD call updates core k inside the kernel that finalises its gradient
     int32_t fast;                       // register-tiled kernel variant for this table's shapes, -1 = generic path
     int32_t midfast[TT_MAXK];           // same for the middle-core backward of level k (index k), -1 = generic
 };
@@ -43,6 +43,7 @@ struct TableDesc {
 struct WsView {
     int32_t T, K, D;
     int32_t ablation;                   // study switches: bit 0 no prefix reuse, bit 1 static (equal-count) schedule
+    float fused_lr;                     // != 0: the kernels that finalise a gradient also apply G -= fused_lr * dG (cores in sgd_mask)
     int32_t stride[TT_MAXK + 1];        // floats per node of the level-k partial-product buffers (max over tables)
     int64_t B, L;                       // current batch / lookups
     int64_t capU;                       // capacity in distinct rows
@@ -155,7 +156,7 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s);
 cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s);
 cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s);
 cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s);
-cudaError_t tt_launch_sgd(tt_emb* h, float lr, cudaStream_t s);
+cudaError_t tt_launch_sgd(tt_emb* h, float lr, bool only_unfused, cudaStream_t s);
 cudaError_t tt_launch_export_level(tt_emb* h, int table, int level, int64_t* vals, int32_t* rc, int32_t* lc, cudaStream_t s);
 cudaError_t tt_launch_export_inverse(tt_emb* h, int table, int32_t* inv, cudaStream_t s);
 cudaError_t tt_launch_pack(const TableDesc& td, int core, const float* src, float* dst, bool to_canonical, cudaStream_t s);

@@ -104,6 +104,32 @@ def test_tiny_configs_backward_and_sgd(binding, cfg):
     assert emb.status() == 0
 
 
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_tiny_configs_fused_backward_sgd(binding, cfg):
+    # backward and update in one call: gradients at the pre-update cores, cores after the step
+    wl = workloads.make(cfg, tiny=True)
+    rng = np.random.default_rng(cfg)
+    go = wl.grad_out if wl.grad_out is not None else rng.standard_normal((wl.B, wl.T * wl.D)).astype(np.float32)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    emb.backward_sgd(dev(go), 0.01)
+    grads = emb.get_grads()
+    cores = emb.get_cores()
+    ref = oracle.backward_workload(wl, grad_out=go)
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref[t], 0.01)
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"cfg{cfg}-tiny fused dG[{t}][{k}]")
+            assert_close(cores[t][k], want[k], f"cfg{cfg}-tiny core[{t}][{k}] after the fused step")
+    assert emb.status() == 0
+    # the handle is back to the plain backward afterwards: cores stay as they are
+    out2 = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    emb.backward(dev(go))
+    after = emb.get_cores()
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert np.array_equal(after[t][k], cores[t][k]), "a plain backward after a fused one must not touch the cores"
+
+
 # ------------------------------------------------------------------------------------------ medium cases: several tiles, ragged tails
 
 MEDIUM = [

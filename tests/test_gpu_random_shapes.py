@@ -101,3 +101,29 @@ def test_random_shape_weighted_mean_int32(binding, seed):
     for t in range(wl.T):
         for k in range(wl.tables[t].K):
             close(grads[t][k], ref[t][k], f"random {seed} {mode} dG[{t}][{k}] (d={tables[t].d}, r={tables[t].r}, n={tables[t].n})")
+
+
+@pytest.mark.parametrize("seed", range(40, 64))
+def test_random_shape_fused_backward_sgd(binding, seed):
+    # every shape class finalises its gradients in another kernel: the fused update must reach each core exactly once
+    tables, B, pooling = random_case(seed)
+    wl = workloads.custom(tables, B, pooling, seed=500 + seed, with_grad=True, name=f"random-{seed}")
+    lr = 0.05
+    emb = binding.from_workload(wl, enable_backward=True)
+    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    emb.backward_sgd(dev(wl.grad_out), lr)
+    assert emb.status() == 0
+    grads = emb.get_grads()
+    cores = emb.get_cores()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref[t], lr)
+        for k in range(wl.tables[t].K):
+            what = f"(d={tables[t].d}, r={tables[t].r}, n={tables[t].n})"
+            close(grads[t][k], ref[t][k], f"random {seed} fused dG[{t}][{k}] {what}")
+            # the update itself is exact in the gradient: compare the applied step with lr * gradient
+            step = (np.asarray(wl.cores[t][k], np.float64) - np.asarray(cores[t][k], np.float64))
+            want_step = lr * np.asarray(ref[t][k], np.float64)
+            slack = TOL * np.abs(want_step).max() + 2.0 ** -23 * np.abs(np.asarray(wl.cores[t][k])).max()   # + the rounding of the fp32 core
+            assert np.abs(step - want_step).max() <= slack, f"random {seed} fused step[{t}][{k}] {what}"
+            close(cores[t][k], want[k], f"random {seed} core[{t}][{k}] after the fused step {what}")
