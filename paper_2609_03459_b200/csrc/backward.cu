@@ -434,10 +434,11 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
 // order owning two of the 64 columns: one shared-memory load and two adds per row, a coalesced 256-byte store when a
 // segment ends, and no shuffles to combine partial sums.  About half the instructions per lookup of k_dE_fast, which
 // was bound by instruction issue.  Chunks, carries and the fix-up pass are those of k_dE / k_dE_fast.
+#define DE_WARPS 9   // 3 CTAs x 9 warps x 8 KB of staging per SM
 template <bool WT>
-__global__ void __launch_bounds__(256, 3) k_dE_stage(WsView w, const float* __restrict__ grad_out)
+__global__ void __launch_bounds__(32 * DE_WARPS, 3) k_dE_stage(WsView w, const float* __restrict__ grad_out)
 {
-    extern __shared__ __align__(16) float4 de_buf[];   // [8 warps][32 rows][16 float4]
+    extern __shared__ __align__(16) float4 de_buf[];   // [DE_WARPS][32 rows][16 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane >> 4, lr = lane & 15;
     float4* buf = de_buf + (size_t)wid * 32 * 16;
     const float2* buf2 = reinterpret_cast<const float2*>(buf);
@@ -536,10 +537,11 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
         const int D4 = h->D / 4;
         const bool wt = h->v.wsorted && (h->v.psw || h->v.pool_mean);
         if (VEC && h->D == 64) {
-            const size_t smem = (size_t)8 * 32 * 16 * sizeof(float4);
+            const size_t smem = (size_t)DE_WARPS * 32 * 16 * sizeof(float4);
             cudaError_t e = cudaFuncSetAttribute(wt ? k_dE_stage<true> : k_dE_stage<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            if (wt) k_dE_stage<true><<<grid, 256, smem, s>>>(h->v, grad_out); else k_dE_stage<false><<<grid, 256, smem, s>>>(h->v, grad_out);
+            const int sgrid = (int)((chunks + DE_WARPS - 1) / DE_WARPS);
+            if (wt) k_dE_stage<true><<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out); else k_dE_stage<false><<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out);
             tt_note_launch();
         } else
         if (VEC && D4 <= 8) { if (wt) k_dE_fast<8, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<8, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }

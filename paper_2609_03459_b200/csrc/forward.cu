@@ -831,10 +831,11 @@ __device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
 
+#define POOL_WARPS 9   // 3 CTAs x 9 warps x 8 KB = 216 KB of the SM's shared memory: one more gather in flight per CTA than 8
 template <bool WT>
-__global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restrict__ out)
+__global__ void __launch_bounds__(32 * POOL_WARPS, 3) k_pool_async(WsView w, float* __restrict__ out)
 {
-    extern __shared__ __align__(16) float4 pool_buf[];   // [8 warps][32 rows][16 float4]
+    extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][16 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int sub = lane >> 4, lr = lane & 15;
     float4* buf = pool_buf + (size_t)wid * 32 * 16;
@@ -935,18 +936,18 @@ __global__ void __launch_bounds__(256, 3) k_pool_async(WsView w, float* __restri
 template <bool WT>
 static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
 {
-    const size_t smem = (size_t)8 * 32 * 16 * sizeof(float4);
+    const size_t smem = (size_t)POOL_WARPS * 32 * 16 * sizeof(float4);
     cudaError_t e = cudaFuncSetAttribute(k_pool_async<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async<WT>, 256, smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async<WT>, 32 * POOL_WARPS, smem)) != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const int64_t nb = (int64_t)h->v.T * h->v.B;
     int64_t grid = (int64_t)per_sm * h->sm_count;
-    const int64_t need = (nb + 7) / 8;
+    const int64_t need = (nb + POOL_WARPS - 1) / POOL_WARPS;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_async<WT><<<(int)grid, 256, smem, s>>>(h->v, out);
+    k_pool_async<WT><<<(int)grid, 32 * POOL_WARPS, smem, s>>>(h->v, out);
     tt_note_launch();
     return cudaGetLastError();
 }
