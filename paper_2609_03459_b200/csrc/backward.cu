@@ -434,9 +434,9 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
 // order owning two of the 64 columns: one shared-memory load and two adds per row, a coalesced 256-byte store when a
 // segment ends, and no shuffles to combine partial sums.  About half the instructions per lookup of k_dE_fast, which
 // was bound by instruction issue.  Chunks, carries and the fix-up pass are those of k_dE / k_dE_fast.
-#define DE_WARPS 9   // 3 CTAs x 9 warps x 8 KB of staging per SM
+#define DE_WARPS 7   // 4 CTAs x 7 warps x 8 KB of staging per SM
 template <bool WT>
-__global__ void __launch_bounds__(32 * DE_WARPS, 3) k_dE_stage(WsView w, const float* __restrict__ grad_out)
+__global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const float* __restrict__ grad_out)
 {
     extern __shared__ __align__(16) float4 de_buf[];   // [DE_WARPS][32 rows][16 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane >> 4, lr = lane & 15;

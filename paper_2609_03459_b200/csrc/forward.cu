@@ -831,9 +831,9 @@ __device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
 
-#define POOL_WARPS 9   // 3 CTAs x 9 warps x 8 KB = 216 KB of the SM's shared memory: one more gather in flight per CTA than 8
+#define POOL_WARPS 7   // 4 CTAs x 7 warps x 8 KB = 224 KB of the SM's shared memory
 template <bool WT>
-__global__ void __launch_bounds__(32 * POOL_WARPS, 3) k_pool_async(WsView w, float* __restrict__ out)
+__global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, float* __restrict__ out)
 {
     extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][16 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
