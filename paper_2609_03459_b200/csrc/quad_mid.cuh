@@ -2,7 +2,7 @@
 // tensor cores.
 //
 // Groups are walked in digit-major order, so neighbours share the slice B = G_{K-1}[i_{K-1}] (r_a x cols).  With
-// P_{K-2} of MROWS = 4 (or 8) rows per group, NG = 16 / MROWS = 4 (or 2) groups stack into one 16 x r_a operand, and
+// P_{K-2} of MROWS = 4 (or 2, 8) rows per group, NG = 16 / MROWS = 4 (or 8, 2) groups stack into one 16 x r_a operand, and
 //     [C_0; ..; C_{NG-1}] = [P_0; ..; P_{NG-1}] . B
 // is a 16 x cols product of m16n8k8 tiles in 3xTF32 (see mma.cuh).  The slice then enters the SM once per NG
 // groups instead of once per group (the FP32-pipe form of this product was bound by the L1 operand path), and the
@@ -27,7 +27,7 @@ __device__ __forceinline__ void tt_quad_mid_mma(const float* __restrict__ B, int
                                                 const float* __restrict__ srcB, bool selA, bool selB, float* Cs4, int lane,
                                                 int nb0 = 0, int nb1 = COLS / 32)   // column blocks of 32 this warp computes
 {
-    static_assert((MROWS == 4 || MROWS == 8) && KTMAX % 2 == 0, "stacking of 4 or 2 groups");
+    static_assert((MROWS == 2 || MROWS == 4 || MROWS == 8) && KTMAX % 2 == 0, "stacking of 8, 4 or 2 groups");
     const int g = lane >> 2, t = lane & 3, m = g & (MROWS - 1);
     const int kta = (ra + 7) >> 3;
     // the stacked operand stays unsplit in registers (KTMAX * 4) and is split where it is used: half the registers of
@@ -113,7 +113,7 @@ __device__ __forceinline__ void tt_quad_mid(const float* __restrict__ core_mid, 
     while (remaining) {
         const int first = __ffs(remaining) - 1;
         const uint32_t im = __shfl_sync(0xffffffffu, imq, first);
-        const unsigned sel = __ballot_sync(0xffffffffu, lane < 4 && ((remaining >> lane) & 1u) && imq == im) & 0xfu;
+        const unsigned sel = __ballot_sync(0xffffffffu, lane < 16 / MROWS && ((remaining >> lane) & 1u) && imq == im) & ((1u << (16 / MROWS)) - 1u);
         const bool selA = (sel >> qA) & 1u, selB = (sel >> qB) & 1u;
         tt_quad_mid_mma<COLS, MROWS, KTMAX, RBP>(core_mid + (size_t)im * slice_floats, ra, srcA, srcB, selA, selB, Cs4, lane);
         remaining &= ~sel;
