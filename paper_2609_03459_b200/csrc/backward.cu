@@ -880,7 +880,9 @@ template <int PM, int RB_>
 __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1, uint32_t row_base,
                                                     float* dPdst, int lane)
 {
-    constexpr int MT = PM / 16, NT = RB_ / 8;
+    static_assert(PM == 8 || PM % 16 == 0, "8 rows of dC fill the upper half of one row tile, else whole tiles");
+    constexpr bool HALF = PM == 8;   // rows 8..15 of the tile stay zero and are not stored
+    constexpr int MT = HALF ? 1 : PM / 16, NT = RB_ / 8;
     const int g = lane >> 2, t = lane & 3;
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
@@ -908,9 +910,9 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             a[mt][0] = tt_split_tf32(__ldg(Ea + (16 * mt + g) * 4));
-            a[mt][1] = tt_split_tf32(__ldg(Ea + (16 * mt + g + 8) * 4));
+            a[mt][1] = tt_split_tf32(HALF ? 0.f : __ldg(Ea + (16 * mt + g + 8) * 4));
             a[mt][2] = tt_split_tf32(two ? __ldg(Ec + (16 * mt + g) * 4) : 0.f);
-            a[mt][3] = tt_split_tf32(two ? __ldg(Ec + (16 * mt + g + 8) * 4) : 0.f);
+            a[mt][3] = tt_split_tf32(two && !HALF ? __ldg(Ec + (16 * mt + g + 8) * 4) : 0.f);
         }
         float bv[NT][2];
 #pragma unroll
@@ -939,7 +941,7 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][0], tot[mt][nt][1]);
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][2], tot[mt][nt][3]);
+            if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][2], tot[mt][nt][3]);
         }
 }
 
@@ -1002,7 +1004,9 @@ template <int PM, int RB_>
 __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
                                                      uint32_t row_base, float* dPdst, float* gk, int lane)
 {
-    constexpr int MT = PM / 16, NT = RB_ / 8;     // dC tiles: rows p, columns b
+    static_assert(PM == 8 || PM % 16 == 0, "8 rows of dC fill the upper half of one row tile, else whole tiles");
+    constexpr bool HALF = PM == 8;                // rows 8..15 of the dC tile stay zero and are not stored
+    constexpr int MT = HALF ? 1 : PM / 16, NT = RB_ / 8;     // dC tiles: rows p, columns b
     constexpr int MT2 = RB_ / 16, KT2 = PM / 8;   // dG tiles: rows b, k = p
     const int g = lane >> 2, t = lane & 3;
     const int K = w.K;
@@ -1040,9 +1044,9 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             av[mt][0] = __ldg(Ea + (16 * mt + g) * 4 + t);
-            av[mt][1] = __ldg(Ea + (16 * mt + g + 8) * 4 + t);
+            av[mt][1] = HALF ? 0.f : __ldg(Ea + (16 * mt + g + 8) * 4 + t);
             av[mt][2] = two ? __ldg(Ec + (16 * mt + g) * 4 + t) : 0.f;
-            av[mt][3] = two ? __ldg(Ec + (16 * mt + g + 8) * 4 + t) : 0.f;
+            av[mt][3] = two && !HALF ? __ldg(Ec + (16 * mt + g + 8) * 4 + t) : 0.f;
         }
         const float* __restrict__ Da = GK + (size_t)iKa * (RB_ * 4) + t;
         const float* __restrict__ Dc = GK + (size_t)iKc * (RB_ * 4) + t;
@@ -1109,7 +1113,7 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
+            if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
         }
 }
 
@@ -1185,8 +1189,8 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
@@ -1218,6 +1222,8 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     if (V == 0) max_c = 16 * (32 + 8);
     if (V == 1) max_c = 16 * (16 + 8);
     if (V == 3) max_c = 32 * (32 + 8);
+    if (V == 5) max_c = 8 * (32 + 8);
+    if (V == 6) max_c = 8 * (16 + 8);
     const size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
                               : (size_t)4 * (max_pl + max_c) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
