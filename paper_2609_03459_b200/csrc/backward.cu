@@ -435,13 +435,17 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
 // segment ends, and no shuffles to combine partial sums.  About half the instructions per lookup of k_dE_fast, which
 // was bound by instruction issue.  Chunks, carries and the fix-up pass are those of k_dE / k_dE_fast.
 #define DE_WARPS 7   // 4 CTAs x 7 warps x 8 KB of staging per SM
-template <bool WT>
+template <int DD, bool WT>   // DD = D: 64 (two columns per lane) or 32 (one)
 __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const float* __restrict__ grad_out)
 {
-    extern __shared__ __align__(16) float4 de_buf[];   // [DE_WARPS][32 rows][16 float4]
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane >> 4, lr = lane & 15;
-    float4* buf = de_buf + (size_t)wid * 32 * 16;
-    const float2* buf2 = reinterpret_cast<const float2*>(buf);
+    static_assert(DD == 64 || DD == 32, "a lane owns DD / 32 columns");
+    constexpr int R4 = DD / 4;          // float4 pieces per row
+    constexpr int RPI = 32 / R4;        // rows per cp.async instruction
+    constexpr int VPL = DD / 32;        // columns per lane
+    extern __shared__ __align__(16) float4 de_buf[];   // [DE_WARPS][32 rows][R4 float4]
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane / R4, lr = lane % R4;
+    float4* buf = de_buf + (size_t)wid * 32 * R4;
+    const float* bufv = reinterpret_cast<const float*>(buf);
     const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
     const uint32_t Ltot = w.cnt[U];
@@ -452,10 +456,11 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
     const uint32_t prev = a > 0 ? w.pairs[a - 1].x : HT_EMPTY;
     const uint32_t next = b < Ltot ? w.pairs[b].x : HT_EMPTY;
     const float4* __restrict__ G4 = reinterpret_cast<const float4*>(grad_out);
-    float2* __restrict__ E2 = reinterpret_cast<float2*>(w.E);
-    float2* carry2 = reinterpret_cast<float2*>(w.carry + (size_t)chunk * 2 * 64);
+    float* carry = w.carry + (size_t)chunk * 2 * DD;
     const uint32_t* __restrict__ tbK = w.tb[w.K];
-    float2 acc = make_float2(0.f, 0.f);
+    float acc[VPL], part[VPL];
+#pragma unroll
+    for (int x = 0; x < VPL; ++x) { acc[x] = 0.f; part[x] = 0.f; }
     uint32_t cur = w.pairs[a].x;
     bool seg_first = true;
     uint32_t last_slot = cur;
@@ -464,12 +469,14 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
     uint32_t t_lo = tbK[tcur], t_hi = tbK[tcur + 1];
     // two-level sum: rows are added into a per-batch partial (at most 32 terms) which is added to the segment's sum at
     // the end of the batch, so the rounding error of a long segment grows with sqrt(length / 32), not sqrt(length)
-    float2 part = make_float2(0.f, 0.f);
+    auto store_row = [&](float* dst, bool with_part) {
+        if (VPL == 2) reinterpret_cast<float2*>(dst)[lane] = make_float2(acc[0] + (with_part ? part[0] : 0.f), acc[VPL - 1] + (with_part ? part[VPL - 1] : 0.f));
+        else dst[lane] = acc[0] + (with_part ? part[0] : 0.f);
+    };
     auto close_segment = [&]() {
-        float2* dst = (seg_first && prev == cur) ? carry2 : E2 + (size_t)cur * 32;   // head piece or whole segment
-        dst[lane] = make_float2(acc.x + part.x, acc.y + part.y);
-        acc = make_float2(0.f, 0.f);
-        part = make_float2(0.f, 0.f);
+        store_row((seg_first && prev == cur) ? carry : w.E + (size_t)cur * DD, true);   // head piece or whole segment
+#pragma unroll
+        for (int x = 0; x < VPL; ++x) { acc[x] = 0.f; part[x] = 0.f; }
         seg_first = false;
     };
     uint2 mine = (a + lane < b) ? __ldcs(&w.pairs[a + lane]) : make_uint2(HT_EMPTY, 0u);
@@ -483,16 +490,16 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
             t_lo = tbK[tcur];
             t_hi = tbK[tcur + 1];
         }
-        const uint32_t grow = mine.y * (uint32_t)w.T + (uint32_t)tl;   // row of grad_out viewed as [B*T][64]
+        const uint32_t grow = mine.y * (uint32_t)w.T + (uint32_t)tl;   // row of grad_out viewed as [B*T][DD]
         uint32_t before = __shfl_up_sync(0xffffffffu, mine.x, 1);
         if (lane == 0) before = last_slot;
         const unsigned starts = __ballot_sync(0xffffffffu, lane < n && mine.x != before);   // bit j: position j opens a segment
         last_slot = __shfl_sync(0xffffffffu, mine.x, n - 1);
 #pragma unroll
-        for (int jj = 0; jj < 16; ++jj) {
-            const int j = 2 * jj + sub;
+        for (int jj = 0; jj < 32 / RPI; ++jj) {
+            const int j = RPI * jj + sub;
             const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
-            if (j < n) tt_cp_async16_b(buf + j * 16 + lr, G4 + (size_t)gr * 16 + lr);
+            if (j < n) tt_cp_async16_b(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         // the pairs of the next batch arrive while the rows are in flight
@@ -510,21 +517,26 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
                 close_segment();
                 cur = __shfl_sync(0xffffffffu, cur_pairs.x, j);
             }
-            float2 x = buf2[j * 32 + lane];
+            float x[VPL];
+            if (VPL == 2) {
+                const float2 v = reinterpret_cast<const float2*>(bufv)[j * 32 + lane];
+                x[0] = v.x; x[VPL - 1] = v.y;
+            } else x[0] = bufv[j * 32 + lane];
             if (WT) {
                 const float wj = __shfl_sync(0xffffffffu, cur_w, j);
-                x.x *= wj; x.y *= wj;
+#pragma unroll
+                for (int c = 0; c < VPL; ++c) x[c] *= wj;
             }
-            part.x += x.x; part.y += x.y;
+#pragma unroll
+            for (int c = 0; c < VPL; ++c) part[c] += x[c];
         }
-        acc.x += part.x; acc.y += part.y;
-        part = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < VPL; ++c) { acc[c] += part[c]; part[c] = 0.f; }
         __syncwarp();
     }
     {   // last segment of the chunk: tail / head / whole
         const bool open_start = seg_first && prev == cur;
-        float2* dst = next == cur ? carry2 + 32 : (open_start ? carry2 : E2 + (size_t)cur * 32);
-        dst[lane] = acc;
+        store_row(next == cur ? carry + DD : (open_start ? carry : w.E + (size_t)cur * DD), false);
     }
 }
 
@@ -536,12 +548,13 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
     if (grid > 0) {
         const int D4 = h->D / 4;
         const bool wt = h->v.wsorted && (h->v.psw || h->v.pool_mean);
-        if (VEC && h->D == 64) {
-            const size_t smem = (size_t)DE_WARPS * 32 * 16 * sizeof(float4);
-            cudaError_t e = cudaFuncSetAttribute(wt ? k_dE_stage<true> : k_dE_stage<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (VEC && (h->D == 64 || h->D == 32)) {
+            const size_t smem = (size_t)DE_WARPS * 32 * (h->D / 4) * sizeof(float4);
+            auto kern = h->D == 64 ? (wt ? k_dE_stage<64, true> : k_dE_stage<64, false>) : (wt ? k_dE_stage<32, true> : k_dE_stage<32, false>);
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             const int sgrid = (int)((chunks + DE_WARPS - 1) / DE_WARPS);
-            if (wt) k_dE_stage<true><<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out); else k_dE_stage<false><<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out);
+            kern<<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out);
             tt_note_launch();
         } else
         if (VEC && D4 <= 8) { if (wt) k_dE_fast<8, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<8, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }

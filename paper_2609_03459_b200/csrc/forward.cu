@@ -840,13 +840,15 @@ __device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
 }
 
 #define POOL_WARPS 7   // 4 CTAs x 7 warps x 8 KB = 224 KB of the SM's shared memory
-template <bool WT>
+template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, float* __restrict__ out)
 {
-    extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][16 float4]
+    static_assert(R4 == 16 || R4 == 8, "two or four rows per cp.async instruction");
+    constexpr int RPI = 32 / R4;
+    extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][R4 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int sub = lane >> 4, lr = lane & 15;
-    float4* buf = pool_buf + (size_t)wid * 32 * 16;
+    const int sub = lane / R4, lr = lane % R4;
+    float4* buf = pool_buf + (size_t)wid * 32 * R4;
     const int D4 = w.D >> 2;
     const bool lane_on = lr < D4;
     const int64_t nb = (int64_t)w.T * w.B;
@@ -903,10 +905,10 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
             // all rows of the batch in flight
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-                const int j = 2 * jj + sub;
+            for (int jj = 0; jj < 32 / RPI; ++jj) {
+                const int j = RPI * jj + sub;
                 const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
-                if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * 16 + lr, E4 + (size_t)sl * D4 + lr);
+                if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * D4 + lr);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             // the rank look-ups of the next batch (or of the next bag) overlap the gather
@@ -915,11 +917,11 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-                const int j = 2 * jj + sub;
+            for (int jj = 0; jj < 32 / RPI; ++jj) {
+                const int j = RPI * jj + sub;
                 const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
                 if (((valid >> j) & 1u) && lane_on) {
-                    const float4 v = buf[j * 16 + lr];
+                    const float4 v = buf[j * R4 + lr];
                     if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
                     else { part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w; }
                 }
@@ -927,8 +929,11 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             acc.x += part.x; acc.y += part.y; acc.z += part.z; acc.w += part.w;
             __syncwarp();
         }
-        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
-        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+#pragma unroll
+        for (int o = R4; o < 32; o <<= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+        }
         if (WT && w.pool_mean && o_hi > o_lo) {
             const float inv = 1.f / (float)(o_hi - o_lo);
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
@@ -941,21 +946,21 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     }
 }
 
-template <bool WT>
+template <int R4, bool WT>
 static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
 {
-    const size_t smem = (size_t)POOL_WARPS * 32 * 16 * sizeof(float4);
-    cudaError_t e = cudaFuncSetAttribute(k_pool_async<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = (size_t)POOL_WARPS * 32 * R4 * sizeof(float4);
+    cudaError_t e = cudaFuncSetAttribute(k_pool_async<R4, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async<WT>, 32 * POOL_WARPS, smem)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_pool_async<R4, WT>, 32 * POOL_WARPS, smem)) != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const int64_t nb = (int64_t)h->v.T * h->v.B;
     int64_t grid = (int64_t)per_sm * h->sm_count;
     const int64_t need = (nb + POOL_WARPS - 1) / POOL_WARPS;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_async<WT><<<(int)grid, 32 * POOL_WARPS, smem, s>>>(h->v, out);
+    k_pool_async<R4, WT><<<(int)grid, 32 * POOL_WARPS, smem, s>>>(h->v, out);
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -1036,7 +1041,8 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
 template <bool WT>
 static cudaError_t launch_pool_sized(tt_emb* h, int D4, float* out, cudaStream_t s)
 {
-    if (D4 > 8 && D4 <= 16) return launch_pool_async<WT>(h, out, s);
+    if (D4 > 8 && D4 <= 16) return launch_pool_async<16, WT>(h, out, s);
+    if (D4 > 4 && D4 <= 8) return launch_pool_async<8, WT>(h, out, s);
     if (D4 <= 4) return launch_pool_vec<4, 1, WT>(h, out, s);
     if (D4 <= 8) return launch_pool_vec<8, 1, WT>(h, out, s);
     if (D4 <= 16) return launch_pool_vec<16, 1, WT>(h, out, s);
