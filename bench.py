@@ -475,7 +475,7 @@ def main():
     # (8 tables; profiles/ncu_full_cfg5_reduced.md), scaled to this launch by the units it processes.
     NCU_TRAFFIC = {"k_pool": ("lookup", 98.1), "k_dE": ("lookup", 73.9),
                    "k_sweep_fwd": ("row", 232.0), "k_sweep_bwd": ("row", 335.4)}
-    pool_kernel = "k_pool_async" if 32 < D <= 64 and D % 4 == 0 else "k_pool_vec"
+    pool_kernel = "k_pool_async" if 16 < D <= 64 and D % 4 == 0 else "k_pool_vec"
 
     def traffic_of(kernel, share=1.0):
         unit, per = NCU_TRAFFIC[kernel]
@@ -518,7 +518,7 @@ def main():
     if train and "bwd_dE" in stage_ms:
         ms = stage_ms["bwd_dE"]
         ach = work["dE_kernel_bytes"] / (ms * 1e-3) / 1e9
-        de_kernel = "k_dE_stage" if D == 64 else "k_dE_fast"
+        de_kernel = "k_dE_stage" if D in (16, 32, 64) else "k_dE_fast"
         kernels[de_kernel] = (ms, {"kernel": de_kernel + " (+k_dE_fix)", "bound": "hbm", "achieved": ach, "peak": hbm_gbs,
                                      "unit": "GB/s", "frac": ach / hbm_gbs, "traffic": traffic_of("k_dE"),
                                      "peak_source": peak_src})

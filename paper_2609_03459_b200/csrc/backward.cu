@@ -435,13 +435,13 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
 // segment ends, and no shuffles to combine partial sums.  About half the instructions per lookup of k_dE_fast, which
 // was bound by instruction issue.  Chunks, carries and the fix-up pass are those of k_dE / k_dE_fast.
 #define DE_WARPS 7   // 4 CTAs x 7 warps x 8 KB of staging per SM
-template <int DD, bool WT>   // DD = D: 64 (two columns per lane) or 32 (one)
+template <int DD, bool WT>   // DD = D: 64 (two columns per lane), 32 (one) or 16 (one, lanes 0..15)
 __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const float* __restrict__ grad_out)
 {
-    static_assert(DD == 64 || DD == 32, "a lane owns DD / 32 columns");
+    static_assert(DD == 64 || DD == 32 || DD == 16, "a lane owns DD / 32 columns (one column on the first DD lanes below 32)");
     constexpr int R4 = DD / 4;          // float4 pieces per row
     constexpr int RPI = 32 / R4;        // rows per cp.async instruction
-    constexpr int VPL = DD / 32;        // columns per lane
+    constexpr int VPL = DD >= 32 ? DD / 32 : 1;   // columns per lane
     extern __shared__ __align__(16) float4 de_buf[];   // [DE_WARPS][32 rows][R4 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, sub = lane / R4, lr = lane % R4;
     float4* buf = de_buf + (size_t)wid * 32 * R4;
@@ -471,7 +471,7 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
     // the end of the batch, so the rounding error of a long segment grows with sqrt(length / 32), not sqrt(length)
     auto store_row = [&](float* dst, bool with_part) {
         if (VPL == 2) reinterpret_cast<float2*>(dst)[lane] = make_float2(acc[0] + (with_part ? part[0] : 0.f), acc[VPL - 1] + (with_part ? part[VPL - 1] : 0.f));
-        else dst[lane] = acc[0] + (with_part ? part[0] : 0.f);
+        else if (lane < DD) dst[lane] = acc[0] + (with_part ? part[0] : 0.f);
     };
     auto close_segment = [&]() {
         store_row((seg_first && prev == cur) ? carry : w.E + (size_t)cur * DD, true);   // head piece or whole segment
@@ -521,7 +521,7 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
             if (VPL == 2) {
                 const float2 v = reinterpret_cast<const float2*>(bufv)[j * 32 + lane];
                 x[0] = v.x; x[VPL - 1] = v.y;
-            } else x[0] = bufv[j * 32 + lane];
+            } else x[0] = bufv[j * DD + (lane & (DD - 1))];
             if (WT) {
                 const float wj = __shfl_sync(0xffffffffu, cur_w, j);
 #pragma unroll
@@ -548,9 +548,10 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
     if (grid > 0) {
         const int D4 = h->D / 4;
         const bool wt = h->v.wsorted && (h->v.psw || h->v.pool_mean);
-        if (VEC && (h->D == 64 || h->D == 32)) {
+        if (VEC && (h->D == 64 || h->D == 32 || h->D == 16)) {
             const size_t smem = (size_t)DE_WARPS * 32 * (h->D / 4) * sizeof(float4);
-            auto kern = h->D == 64 ? (wt ? k_dE_stage<64, true> : k_dE_stage<64, false>) : (wt ? k_dE_stage<32, true> : k_dE_stage<32, false>);
+            auto kern = h->D == 64 ? (wt ? k_dE_stage<64, true> : k_dE_stage<64, false>)
+                      : h->D == 32 ? (wt ? k_dE_stage<32, true> : k_dE_stage<32, false>) : (wt ? k_dE_stage<16, true> : k_dE_stage<16, false>);
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             const int sgrid = (int)((chunks + DE_WARPS - 1) / DE_WARPS);

@@ -42,8 +42,7 @@ def time_point(D: int, rank: int, batch: int, train: bool, steps: int, warmup: i
     def step():
         fwd()
         if train:
-            emb.backward(d_grad)
-            emb.sgd_step(wl.lr)
+            emb.backward_sgd(d_grad, wl.lr)
 
     def timed(fn):
         ms = []
