@@ -185,12 +185,12 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (PMv == 32 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 3;
             else if (PMv == 32 && Mv == 8 && RBv == 64 && td.r[K - 2] <= 64) td.fast = 4;
             // first dim factor 2 (D = 32 as 2x4x4): eight groups of two rows stack into the 16-row product, C has 8 rows
-            // (the upper half of one row tile); D = 16 as 2x2x4 and rank 8: FP32-pipe variants
+            // (the first rows of one row tile), D = 16 as 2x2x4: 4 rows; rank 8: FP32-pipe variants
             else if (PMv == 8 && Mv == 2 && RBv == 32 && quad_ok) td.fast = 5;
             else if (PMv == 8 && Mv == 2 && RBv == 16 && quad_ok) td.fast = 6;
             else if (PMv == 8 && Mv == 2 && RBv == 8) td.fast = 7;
-            else if (PMv == 4 && Mv == 2 && RBv == 32) td.fast = 8;
-            else if (PMv == 4 && Mv == 2 && RBv == 16) td.fast = 9;
+            else if (PMv == 4 && Mv == 2 && RBv == 32 && quad_ok) td.fast = 8;
+            else if (PMv == 4 && Mv == 2 && RBv == 16 && quad_ok) td.fast = 9;
         }
         for (int k = 0; k < TT_MAXK; ++k) td.midfast[k] = -1;
         for (int k = 2; k <= K - 1; ++k) {

@@ -894,10 +894,11 @@ template <int PM, int RB_>
 __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1, uint32_t row_base,
                                                     float* dPdst, int lane)
 {
-    static_assert(PM == 8 || PM % 16 == 0, "8 rows of dC fill the upper half of one row tile, else whole tiles");
-    constexpr bool HALF = PM == 8;   // rows 8..15 of the tile stay zero and are not stored
+    static_assert(PM == 4 || PM == 8 || PM % 16 == 0, "4 or 8 rows of dC fill the first rows of one row tile, else whole tiles");
+    constexpr bool HALF = PM < 16;   // rows PM..15 of the tile stay zero and are not stored
     constexpr int MT = HALF ? 1 : PM / 16, NT = RB_ / 8;
     const int g = lane >> 2, t = lane & 3;
+    const bool rowok = !HALF || g < PM;
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
     const uint32_t* __restrict__ rows = w.val[K];
@@ -923,9 +924,9 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
         Tf32Pair a[MT][4];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-            a[mt][0] = tt_split_tf32(__ldg(Ea + (16 * mt + g) * 4));
+            a[mt][0] = tt_split_tf32(rowok ? __ldg(Ea + (16 * mt + g) * 4) : 0.f);
             a[mt][1] = tt_split_tf32(HALF ? 0.f : __ldg(Ea + (16 * mt + g + 8) * 4));
-            a[mt][2] = tt_split_tf32(two ? __ldg(Ec + (16 * mt + g) * 4) : 0.f);
+            a[mt][2] = tt_split_tf32(two && rowok ? __ldg(Ec + (16 * mt + g) * 4) : 0.f);
             a[mt][3] = tt_split_tf32(two && !HALF ? __ldg(Ec + (16 * mt + g + 8) * 4) : 0.f);
         }
         float bv[NT][2];
@@ -954,7 +955,7 @@ __device__ __forceinline__ void tt_warp_rows_dC_mma(const WsView& w, const Table
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][0], tot[mt][nt][1]);
+            if (rowok) *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][0], tot[mt][nt][1]);
             if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(tot[mt][nt][2], tot[mt][nt][3]);
         }
 }
@@ -963,7 +964,8 @@ template <int PM, int RB_>
 __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsView& w, uint32_t u0, uint32_t u1, uint32_t row_base,
                                                     float* gk, int lane)
 {
-    constexpr int MT = RB_ / 16, KT = PM / 8;
+    constexpr bool KHALF = PM == 4;   // p = 4..7 of the one k step do not exist: zero operands
+    constexpr int MT = RB_ / 16, KT = KHALF ? 1 : PM / 8;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t* __restrict__ rows = w.val[w.K];
     Tf32Pair a[MT][KT][4];   // A[m = b][k = p] = C[p][b]
@@ -973,8 +975,8 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
         for (int kt = 0; kt < KT; ++kt) {
             a[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
             a[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
-            a[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
-            a[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
+            a[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
+            a[mt][kt][3] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     const int rb_ = g >> 2, jb = g & 3;       // B fragment: row rb_ of the pair, column jb of dE
     const int rc = t >> 1, jc = 2 * (t & 1);  // C fragment: row rc of the pair, columns jc, jc+1
@@ -990,7 +992,7 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
             bv[kt][0] = valid ? __ldg(El + (8 * kt + t) * 4) : 0.f;
-            bv[kt][1] = valid ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
+            bv[kt][1] = valid && !KHALF ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
         }
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
@@ -1018,11 +1020,13 @@ template <int PM, int RB_>
 __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
                                                      uint32_t row_base, float* dPdst, float* gk, int lane)
 {
-    static_assert(PM == 8 || PM % 16 == 0, "8 rows of dC fill the upper half of one row tile, else whole tiles");
-    constexpr bool HALF = PM == 8;                // rows 8..15 of the dC tile stay zero and are not stored
+    static_assert(PM == 4 || PM == 8 || PM % 16 == 0, "4 or 8 rows of dC fill the first rows of one row tile, else whole tiles");
+    constexpr bool HALF = PM < 16;                // rows PM..15 of the dC tile stay zero and are not stored
+    constexpr bool KHALF = PM == 4;               // p = 4..7 of the one dG k step do not exist: zero operands
     constexpr int MT = HALF ? 1 : PM / 16, NT = RB_ / 8;     // dC tiles: rows p, columns b
-    constexpr int MT2 = RB_ / 16, KT2 = PM / 8;   // dG tiles: rows b, k = p
+    constexpr int MT2 = RB_ / 16, KT2 = KHALF ? 1 : PM / 8;   // dG tiles: rows b, k = p
     const int g = lane >> 2, t = lane & 3;
+    const bool rowok = !HALF || g < PM;
     const int K = w.K;
     const float* __restrict__ GK = td.core[K - 1];
     const uint32_t* __restrict__ rows = w.val[K];
@@ -1033,8 +1037,8 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
         for (int kt = 0; kt < KT2; ++kt) {
             ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
             ct[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
-            ct[mt][kt][2] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
-            ct[mt][kt][3] = tt_split_tf32(Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
+            ct[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
+            ct[mt][kt][3] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     float dc[MT][NT][4], dct[MT][NT][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
 #pragma unroll
@@ -1057,9 +1061,9 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
         float av[MT][4], bv[NT][2], ev[KT2][2];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-            av[mt][0] = __ldg(Ea + (16 * mt + g) * 4 + t);
+            av[mt][0] = rowok ? __ldg(Ea + (16 * mt + g) * 4 + t) : 0.f;
             av[mt][1] = HALF ? 0.f : __ldg(Ea + (16 * mt + g + 8) * 4 + t);
-            av[mt][2] = two ? __ldg(Ec + (16 * mt + g) * 4 + t) : 0.f;
+            av[mt][2] = two && rowok ? __ldg(Ec + (16 * mt + g) * 4 + t) : 0.f;
             av[mt][3] = two && !HALF ? __ldg(Ec + (16 * mt + g + 8) * 4 + t) : 0.f;
         }
         const float* __restrict__ Da = GK + (size_t)iKa * (RB_ * 4) + t;
@@ -1074,7 +1078,7 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
         for (int kt = 0; kt < KT2; ++kt) {
             ev[kt][0] = valid ? __ldg(El + (8 * kt + t) * 4) : 0.f;
-            ev[kt][1] = valid ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
+            ev[kt][1] = valid && !KHALF ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
         }
         // ---- dC += dE . D^T
         {
@@ -1126,7 +1130,7 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
+            if (rowok) *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
             if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
         }
 }
@@ -1206,8 +1210,8 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
 }
 
 // fixed-order sum of the partial copies of the last core's gradient
@@ -1238,6 +1242,8 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     if (V == 3) max_c = 32 * (32 + 8);
     if (V == 5) max_c = 8 * (32 + 8);
     if (V == 6) max_c = 8 * (16 + 8);
+    if (V == 8) max_c = 4 * (32 + 8);
+    if (V == 9) max_c = 4 * (16 + 8);
     const size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
                               : (size_t)4 * (max_pl + max_c) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -272,17 +272,18 @@ template <int PM, int RB, int CS = RB>   // CS: row stride of C in shared memory
 __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
                                                  uint32_t row_base, int lane)
 {
-    static_assert(PM == 8 || PM % 16 == 0, "C of 8 rows fills the upper half of one row tile, else whole tiles");
-    constexpr bool HALF = PM == 8;          // rows 8..15 of the tile are zero and are not stored
+    static_assert(PM == 4 || PM == 8 || PM % 16 == 0, "C of 4 or 8 rows fills the first rows of one row tile, else whole tiles");
+    constexpr bool HALF = PM < 16;          // rows PM..15 of the tile are zero and are not stored
     constexpr int MT = HALF ? 1 : PM / 16, KT = RB / 8;
     const int g = lane >> 2, t = lane & 3;
+    const bool rowok = !HALF || g < PM;     // this lane's first row exists
     Tf32Pair a[MT][KT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
-            a[mt][kt][0] = tt_split_tf32(Cs[(16 * mt + g) * CS + 8 * kt + t]);
-            a[mt][kt][2] = tt_split_tf32(Cs[(16 * mt + g) * CS + 8 * kt + t + 4]);
+            a[mt][kt][0] = tt_split_tf32(rowok ? Cs[(16 * mt + g) * CS + 8 * kt + t] : 0.f);
+            a[mt][kt][2] = tt_split_tf32(rowok ? Cs[(16 * mt + g) * CS + 8 * kt + t + 4] : 0.f);
             if (HALF) {
                 a[mt][kt][1].hi = 0u; a[mt][kt][1].lo = 0u; a[mt][kt][3].hi = 0u; a[mt][kt][3].lo = 0u;
             } else {
@@ -334,7 +335,7 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
                 float* e = w.E + (size_t)us * (PM * 4) + jc;
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
-                    __stcs(reinterpret_cast<float2*>(e + (16 * mt + g) * 4), make_float2(acc[mt][0], acc[mt][1]));
+                    if (rowok) __stcs(reinterpret_cast<float2*>(e + (16 * mt + g) * 4), make_float2(acc[mt][0], acc[mt][1]));
                     if (!HALF) __stcs(reinterpret_cast<float2*>(e + (16 * mt + g + 8) * 4), make_float2(acc[mt][2], acc[mt][3]));
                 }
             }
@@ -574,7 +575,7 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
 // one instantiation per shape variant V so that each gets its own register budget.  blockIdx.y walks the
 // tables of variant V (w.vlist), blockIdx.x the table's equal-cost slices.
 template <int V>
-__global__ void __launch_bounds__(128, (V == 0 || V == 1 || V == 5 || V == 6) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
+__global__ void __launch_bounds__(128, (V == 0 || V == 1 || V == 5 || V == 6 || V == 8 || V == 9) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
     extern __shared__ __align__(16) float sm[];
     __shared__ uint32_t next;
@@ -599,8 +600,8 @@ __global__ void __launch_bounds__(128, (V == 0 || V == 1 || V == 5 || V == 6) ? 
     if (V == 5) tt_sweep_quad<8, 32, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 36), &next, lane);
     if (V == 6) tt_sweep_quad<8, 16, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 20), &next, lane);
     if (V == 7) tt_sweep_fast<8, 8, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
-    if (V == 8) tt_sweep_fast<4, 32, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
-    if (V == 9) tt_sweep_fast<4, 16, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 8) tt_sweep_quad<4, 32, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 36), &next, lane);
+    if (V == 9) tt_sweep_quad<4, 16, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 20), &next, lane);
 }
 
 // dynamic shared memory of k_sweep_fwd<V> / k_sweep_bwd<V>: four C tiles per warp for the tensor-core variants
@@ -611,6 +612,8 @@ static size_t tt_sweep_smem(int V, int max_pl, int max_c)
     if (V == 3) return (size_t)4 * 4 * 32 * 36 * sizeof(float);
     if (V == 5) return (size_t)4 * 8 * 8 * 36 * sizeof(float);    // eight C tiles of 8 rows per warp
     if (V == 6) return (size_t)4 * 8 * 8 * 20 * sizeof(float);
+    if (V == 8) return (size_t)4 * 8 * 4 * 36 * sizeof(float);
+    if (V == 9) return (size_t)4 * 8 * 4 * 20 * sizeof(float);
     if (V == 4) return (size_t)(2 * 32 * 64 + 4 * 64 * 68) * sizeof(float);   // one pair of C tiles per CTA + a staged slice block per warp
     return (size_t)4 * (max_pl + max_c) * sizeof(float);
 }
