@@ -1351,7 +1351,7 @@ __global__ void __launch_bounds__(256) k_mid_down(WsView w, int k)
     for (uint32_t pn = blockIdx.x; pn < count; pn += gridDim.x) {
         const int t = tt_find_table(w.tb[k - 1], w.T, pn);
         const TableDesc& td = w.tdesc[t];
-        if (td.midfast[k] >= 0) continue;  // handled by k_mid_fused + k_mid_sum
+        if (td.midfast[k] >= 0) continue;  // handled by k_mid_mma + k_mid_sum
         const int kc = k - 1;
         const int M = td.P[kc], ra = td.r[kc], cols = td.d[kc] * td.r[kc + 1];
         const int ld = cols + 1;
@@ -1444,145 +1444,27 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
     }
 }
 
-// ---- register-tiled middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ------
+// ---- tensor-core middle-core backward (P_{k-1} = 4 or 2 rows, r_{k-1} in {16,32}, d_k * r_k in {32,64,128}) ----
 //
-// One CTA of 128 threads per (table, slice i_k).  The slice G_k[i_k] (RA x COLS) never changes inside the CTA,
-// so each thread keeps its APT x 4 tile of it in registers.  The nodes with digit i_k arrive in ascending parent
-// order from the digit-major list; per node the CTA stages dP_k (4 x COLS) and the parent's P_{k-1} (4 x RA)
-// in shared memory (a 4-stage cp.async pipeline, one barrier per node) and every thread does, for its tile,
-//     dG_k[a][c] += sum_m P_{k-1}[m][a] * dP_k[m][c]               (accumulated in registers over all nodes)
-//     Y[m][a]     = sum_c dP_k[m][c] * G_k[a][c]                    (partial over its 4 columns)
-// The Y partials are combined over the TC lanes that share an a-range by a reduce-scatter of warp shuffles and
-// written once per node; k_mid_sum then adds the Y rows of each parent's (contiguous) children.
-
-template <int NVAL, int W>
-__device__ __forceinline__ int tt_reduce_scatter(float (&v)[NVAL], int lane)
-{
-    int idx = 0;
-    int n = NVAL;
-#pragma unroll
-    for (int o = W / 2; o >= 1; o >>= 1) {
-        if (n > 1) {
-            n >>= 1;
-            const bool hi = (lane & o) != 0;
-#pragma unroll
-            for (int i = 0; i < NVAL / 2; ++i) {
-                if (i < n) {
-                    const float send = hi ? v[i] : v[i + n];
-                    const float recv = __shfl_xor_sync(0xffffffffu, send, o);
-                    v[i] = (hi ? v[i + n] : v[i]) + recv;
-                }
-            }
-            idx += hi ? n : 0;
-        } else {
-            v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
-        }
-    }
-    return idx;
-}
-
-template <int M, int RA, int COLS>
-__global__ void __launch_bounds__(128) k_mid_fused(WsView w, int k, int variant)
-{
-    constexpr int TC = COLS / 4, AG = 128 / TC, APT = RA / AG, NVAL = M * APT;
-    static_assert(APT >= 1 && AG * APT == RA && NVAL >= 1, "tile shape");
-    constexpr int REP = TC / NVAL > 0 ? TC / NVAL : 1;  // lanes that end up with the same reduced value
-    constexpr int ST = 4;   // stages of the node pipeline (cp.async, no staging registers)
-    __shared__ __align__(16) float sA[ST][M * RA];
-    __shared__ __align__(16) float sD[ST][M * COLS];
-    const int t = w.vlist[w.T + blockIdx.y];   // largest tables first: their long node lists start early
-    const TableDesc& td = w.tdesc[t];
-    const int kc = k - 1;
-    if (td.midfast[k] != variant || (int)blockIdx.x >= td.n[kc]) return;
-    const uint32_t ik = blockIdx.x;
-    const int tid = threadIdx.x, cl = tid % TC, ag = tid / TC, a0 = ag * APT;
-    const float* __restrict__ Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
-    float4 breg[APT], acc[APT];
-#pragma unroll
-    for (int i = 0; i < APT; ++i) {
-        breg[i] = __ldg(reinterpret_cast<const float4*>(Bsl + (size_t)(a0 + i) * COLS) + cl);
-        acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    const uint32_t space = td.prefix_space[k - 1];
-    const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
-    const int strideY = w.stride[k - 1];
-    // node jn of the list -> stage jn % ST (always commits a group so that the group count stays in step)
-    auto issue = [&](uint32_t jn) {
-        if (jn < j1) {
-            const uint32_t v = w.tnode[k][jn];
-            const int buf = (int)((jn - j0) % ST);
-            if (tid < M * COLS / 4)
-                tt_cp_async16_b(reinterpret_cast<float4*>(sD[buf]) + tid,
-                                reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k]) + tid);
-            if (tid < M * RA / 4)
-                tt_cp_async16_b(reinterpret_cast<float4*>(sA[buf]) + tid,
-                                reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, v)) + tid);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-#pragma unroll
-    for (int i = 0; i < ST - 1; ++i) issue(j0 + i);
-    for (uint32_t jn = j0; jn < j1; ++jn) {
-        const int cur = (int)((jn - j0) % ST);
-        asm volatile("cp.async.wait_group %0;" ::"n"(ST - 2) : "memory");
-        __syncthreads();            // node jn has landed for everyone; everyone is done with node jn-1
-        issue(jn + ST - 1);         // refills the stage node jn-1 used
-        const uint32_t vcur = w.tnode[k][jn];
-        float y[NVAL];
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            const float4 d = reinterpret_cast<const float4*>(sD[cur])[m * TC + cl];
-#pragma unroll
-            for (int i = 0; i < APT; ++i) {
-                const float av = sA[cur][m * RA + a0 + i];
-                acc[i].x = fmaf(av, d.x, acc[i].x); acc[i].y = fmaf(av, d.y, acc[i].y);
-                acc[i].z = fmaf(av, d.z, acc[i].z); acc[i].w = fmaf(av, d.w, acc[i].w);
-                float yy = d.x * breg[i].x;
-                yy = fmaf(d.y, breg[i].y, yy); yy = fmaf(d.z, breg[i].z, yy); yy = fmaf(d.w, breg[i].w, yy);
-                y[m * APT + i] = yy;
-            }
-        }
-        const int idx = tt_reduce_scatter<NVAL, TC>(y, cl);
-        if ((cl % REP) == 0) {
-            const int m = idx / APT, i = idx - m * APT;
-            w.Y[k][(size_t)vcur * strideY + m * RA + a0 + i] = y[0];
-        }
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    float* dst = td.grad[kc] + (size_t)ik * td.slice_floats[kc];
-#pragma unroll
-    for (int i = 0; i < APT; ++i) reinterpret_cast<float4*>(dst + (size_t)(a0 + i) * COLS)[cl] = acc[i];
-    if (w.fused_lr != 0.f) {   // fused update of the CTA's own slice (held in breg since the start; nobody else reads it)
-        float* cdst = td.core[kc] + (size_t)ik * td.slice_floats[kc];
-#pragma unroll
-        for (int i = 0; i < APT; ++i) {
-            float4 u = breg[i];
-            u.x = u.x - w.fused_lr * acc[i].x; u.y = u.y - w.fused_lr * acc[i].y;
-            u.z = u.z - w.fused_lr * acc[i].z; u.w = u.w - w.fused_lr * acc[i].w;
-            reinterpret_cast<float4*>(cdst + (size_t)(a0 + i) * COLS)[cl] = u;
-        }
-    }
-}
-
-// ---- tensor-core form of the middle-core backward (P_{k-1} = 4 rows, r_{k-1} in {16,32}, d_k * r_k in {64,128}) ----
-//
-// Same ownership as k_mid_fused (one CTA of 4 warps per (table, slice i_k), nodes from the digit-major list), but
-// NQ = 4 (r_{k-1} = 32) or 8 (16) nodes per pass, staged with cp.async into padded shared-memory tiles (two stages,
-// two barriers per pass instead of one per node), and both products as 3xTF32 m16n8k8 tiles (mma.cuh):
-//   dG_k[a][c] += sum_{node, m} P_{k-1}[node][m][a] * dP_k[node][m][c]   M = a, N = c, K = 8 = (2 nodes, 4 rows m);
+// One CTA of 4 warps per (table, slice i_k).  The nodes with digit i_k arrive in ascending parent order from the
+// digit-major list, 16 or 32 stacked rows (node, m) per pass: NQ = 4..16 nodes, staged with cp.async into padded
+// shared-memory tiles (two stages, two barriers per pass), and both products run as 3xTF32 m16n8k8 tiles (mma.cuh):
+//   dG_k[a][c] += sum_{node, m} P_{k-1}[node][m][a] * dP_k[node][m][c]   M = a, N = c, K = 8 stacked rows (node, m);
 //                 a warp owns COLS/4 columns c of the slice, accumulators stay in registers over the whole list
-//   Y[node][m][a] = sum_c dP_k[node][m][c] * G_k[a][c]                   M = 16 = (4 nodes, m), N = 8 values of a,
+//   Y[node][m][a] = sum_c dP_k[node][m][c] * G_k[a][c]                   M = 16 stacked rows, N = 8 values of a,
 //                 K = c; the slice fragments (split into TF32 head and tail once) stay in registers;
-//                 warp -> (n-tile of a, group of four nodes)
+//                 warp -> (n-tile of a, tile of sixteen stacked rows)
+// k_mid_sum then adds the Y rows of each parent's (contiguous) children.
 // Row strides RA + 8 and COLS + 8 floats make every fragment load from shared memory conflict-free or 2-way.
 // The tensor core adds into its fp32 accumulator with truncation, so an accumulation chain of N products drifts by
 // up to N * 2^-24 of the sum; the dG accumulators are therefore folded into running sums (a rounded fp32
 // add into the CTA's own gradient slice, which stays in L2) every eighth pass, which keeps every chain at 48 or 96
 // products whatever the length of the node list.
-template <int RA, int COLS>
+template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 {
-    constexpr int M = 4, NQ = 128 / RA, AP = RA + 8, CP = COLS + 8;
+    static_assert(M == 4 || M == 2, "rows per node");
+    constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16 or 32 stacked rows per pass
     constexpr int MT = RA / 16;              // dG: m-tiles over a
     constexpr int NTW = COLS / 32;           // dG: n-tiles per warp (the warp's COLS/4 columns)
     constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ / 4 row tiles of four nodes; NTY * NQ / 4 = 4 warps
@@ -1648,16 +1530,16 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
     auto issue = [&](uint32_t r) {
         const int st = (int)(r & 1u);
         const uint32_t jb = j0 + r * NQ;
-        for (int i = tid; i < NQ * COLS; i += 128) {            // dP_k rows: M * COLS / 4 float4 per node
-            const int q = i / COLS, rem = i - q * COLS, m = rem / (COLS / 4), c4 = rem - m * (COLS / 4);
+        for (int i = tid; i < NQ * M * (COLS / 4); i += 128) {   // dP_k rows: M * COLS / 4 float4 per node
+            const int q = i / (M * (COLS / 4)), rem = i - q * (M * (COLS / 4)), m = rem / (COLS / 4), c4 = rem - m * (COLS / 4);
             float4* dst = reinterpret_cast<float4*>(&sD[st][(q * M + m) * CP + 4 * c4]);
             if (jb + q < j1) {
                 const uint32_t v = w.tnode[k][jb + q];
                 tt_cp_async16_b(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
             } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        for (int i = tid; i < NQ * RA; i += 128) {              // P_{k-1} of the parent: M * RA / 4 float4 per node
-            const int q = i / RA, rem = i - q * RA, m = rem / (RA / 4), a4 = rem - m * (RA / 4);
+        for (int i = tid; i < NQ * M * (RA / 4); i += 128) {     // P_{k-1} of the parent: M * RA / 4 float4 per node
+            const int q = i / (M * (RA / 4)), rem = i - q * (M * (RA / 4)), m = rem / (RA / 4), a4 = rem - m * (RA / 4);
             float4* dst = reinterpret_cast<float4*>(&sA[st][(q * M + m) * AP + 4 * a4]);
             if (jb + q < j1) {
                 const uint32_t v = w.tnode[k][jb + q];
@@ -1677,13 +1559,13 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
         __syncthreads();
         const float* A_ = sA[r & 1u];
         const float* D_ = sD[r & 1u];
-        // ---- dG: pairs of nodes give k = 8
+        // ---- dG: eight stacked rows (node, m) give k = 8
 #pragma unroll
-        for (int p = 0; p < NQ / 2; ++p) {
-            const float* Aa = A_ + (2 * p * M + t) * AP;         // node 2p,   row m = t
-            const float* Ab = A_ + ((2 * p + 1) * M + t) * AP;   // node 2p+1, row m = t
-            const float* Da = D_ + (2 * p * M + t) * CP + wid * (COLS / 4) + g;
-            const float* Db = D_ + ((2 * p + 1) * M + t) * CP + wid * (COLS / 4) + g;
+        for (int p = 0; p < NQ * M / 8; ++p) {
+            const float* Aa = A_ + (8 * p + t) * AP;       // stacked row 8p + t:     node (8p + t) / M, row (8p + t) % M
+            const float* Ab = A_ + (8 * p + t + 4) * AP;   // stacked row 8p + t + 4
+            const float* Da = D_ + (8 * p + t) * CP + wid * (COLS / 4) + g;
+            const float* Db = D_ + (8 * p + t + 4) * CP + wid * (COLS / 4) + g;
             Tf32Pair a[MT][4];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
@@ -1701,11 +1583,11 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt][nt], a[mt], b);
             }
         }
-        // ---- Y of this warp's four nodes and eight values of a
+        // ---- Y of this warp's sixteen stacked rows and eight values of a
         {
             float y[4] = {0.f, 0.f, 0.f, 0.f};
-            const float* Ra = D_ + ((4 * yrt + (g >> 2)) * M + (g & 3)) * CP;       // row g of the tile: node g / 4, m = g % 4
-            const float* Rb = D_ + ((4 * yrt + 2 + (g >> 2)) * M + (g & 3)) * CP;   // row g + 8
+            const float* Ra = D_ + (16 * yrt + g) * CP;       // row g of the tile: stacked row 16 yrt + g
+            const float* Rb = D_ + (16 * yrt + g + 8) * CP;   // row g + 8
 #pragma unroll
             for (int kt = 0; kt < KTY; ++kt) {
                 Tf32Pair a[4];
@@ -1715,14 +1597,15 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 a[3] = tt_split_tf32(Rb[8 * kt + t + 4]);
                 tt_mma_3xtf32(y, a, bY[kt]);
             }
-            const uint32_t ja = j0 + r * NQ + 4 * yrt + (g >> 2), jb2 = ja + 2;
+            const uint32_t ja = j0 + r * NQ + (16 * yrt + g) / M, jb2 = j0 + r * NQ + (16 * yrt + g + 8) / M;
+            const int ma = (16 * yrt + g) % M;   // the same row of P for g and g + 8 (M divides 8)
             if (ja < j1) {
                 const uint32_t v = w.tnode[k][ja];
-                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[0], y[1]);
+                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + ma * RA + 8 * ynt + 2 * t]) = make_float2(y[0], y[1]);
             }
             if (jb2 < j1) {
                 const uint32_t v = w.tnode[k][jb2];
-                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + (g & 3) * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
+                *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + ma * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
         if ((r & 7u) == 7u) fold(false);   // rounded running sums every eighth pass
@@ -1807,14 +1690,14 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
         auto st = [&]() { return fork ? h->side[(slot++) & 3] : s; };
-        if (any_fast[0]) { k_mid_mma<32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
-        if (any_fast[1]) { k_mid_mma<16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
-        if (any_fast[2]) { k_mid_mma<32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
-        if (any_fast[3]) { k_mid_mma<16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
-        if (any_fast[4]) { k_mid_fused<2, 32, 128><<<sg, 128, 0, st()>>>(w, k, 4); tt_note_launch(); }
-        if (any_fast[5]) { k_mid_fused<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
-        if (any_fast[6]) { k_mid_fused<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
-        if (any_fast[7]) { k_mid_fused<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
+        if (any_fast[0]) { k_mid_mma<4, 32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
+        if (any_fast[1]) { k_mid_mma<4, 16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
+        if (any_fast[2]) { k_mid_mma<4, 32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
+        if (any_fast[3]) { k_mid_mma<4, 16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
+        if (any_fast[4]) { k_mid_mma<2, 32, 128><<<sg, 128, 0, st()>>>(w, k, 4); tt_note_launch(); }
+        if (any_fast[5]) { k_mid_mma<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
+        if (any_fast[6]) { k_mid_mma<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
+        if (any_fast[7]) { k_mid_mma<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (nfast > 0) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {
