@@ -203,6 +203,8 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (Mv == 2 && rav == 16 && colsv == 64) td.midfast[k] = 5;
             else if (Mv == 2 && rav == 32 && colsv == 64) td.midfast[k] = 6;
             else if (Mv == 2 && rav == 16 && colsv == 32) td.midfast[k] = 7;
+            else if (Mv == 4 && rav == 8 && colsv == 32) td.midfast[k] = 8;
+            else if (Mv == 2 && rav == 8 && colsv == 32) td.midfast[k] = 9;
         }
         td.unit_base = unit_base;
         unit_base += Q;

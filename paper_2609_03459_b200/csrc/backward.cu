@@ -1463,9 +1463,10 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 {
-    static_assert(M == 4 || M == 2, "rows per node");
-    constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16 or 32 stacked rows per pass
-    constexpr int MT = RA / 16;              // dG: m-tiles over a
+    static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && COLS % 32 == 0, "rows per node; r_{k-1}; columns per warp");
+    constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16, 32 or 64 stacked rows per pass
+    constexpr bool AHALF = RA == 8;          // dG: a = 8..15 of the one m-tile do not exist: zero operands, not stored
+    constexpr int MT = AHALF ? 1 : RA / 16;  // dG: m-tiles over a
     constexpr int NTW = COLS / 32;           // dG: n-tiles per warp (the warp's COLS/4 columns)
     constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ / 4 row tiles of four nodes; NTY * NQ / 4 = 4 warps
     constexpr int KTY = COLS / 8;            // Y: k steps over c
@@ -1507,16 +1508,21 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
                 float2* p0 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g) * COLS + c);
                 float2* p1 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g + 8) * COLS + c);
                 float2 v0 = first_fold ? make_float2(0.f, 0.f) : *p0;
-                float2 v1 = first_fold ? make_float2(0.f, 0.f) : *p1;
+                float2 v1 = (first_fold || AHALF) ? make_float2(0.f, 0.f) : *p1;
                 v0.x += acc[mt][nt][0]; v0.y += acc[mt][nt][1]; v1.x += acc[mt][nt][2]; v1.y += acc[mt][nt][3];
-                *p0 = v0; *p1 = v1;
+                *p0 = v0;
+                if (!AHALF) *p1 = v1;
                 if (last && w.fused_lr != 0.f) {
                     float2* c0 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g) * COLS + c);
-                    float2* c1 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g + 8) * COLS + c);
-                    float2 u0 = *c0, u1 = *c1;
+                    float2 u0 = *c0;
                     u0.x = u0.x - w.fused_lr * v0.x; u0.y = u0.y - w.fused_lr * v0.y;
-                    u1.x = u1.x - w.fused_lr * v1.x; u1.y = u1.y - w.fused_lr * v1.y;
-                    *c0 = u0; *c1 = u1;
+                    *c0 = u0;
+                    if (!AHALF) {
+                        float2* c1 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g + 8) * COLS + c);
+                        float2 u1 = *c1;
+                        u1.x = u1.x - w.fused_lr * v1.x; u1.y = u1.y - w.fused_lr * v1.y;
+                        *c1 = u1;
+                    }
                 }
                 acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f;
             }
@@ -1570,9 +1576,9 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 a[mt][0] = tt_split_tf32(Aa[16 * mt + g]);
-                a[mt][1] = tt_split_tf32(Aa[16 * mt + g + 8]);
+                a[mt][1] = tt_split_tf32(AHALF ? 0.f : Aa[16 * mt + g + 8]);
                 a[mt][2] = tt_split_tf32(Ab[16 * mt + g]);
-                a[mt][3] = tt_split_tf32(Ab[16 * mt + g + 8]);
+                a[mt][3] = tt_split_tf32(AHALF ? 0.f : Ab[16 * mt + g + 8]);
             }
 #pragma unroll
             for (int nt = 0; nt < NTW; ++nt) {
@@ -1669,7 +1675,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
     cudaError_t e;
     for (int k = h->K - 1; k >= 2; --k) {
         int max_n = 1, max_down = 1, max_slice = 1;
-        bool any_generic = false, any_fast[8] = {false, false, false, false, false, false, false, false};
+        bool any_generic = false, any_fast[10] = {false, false, false, false, false, false, false, false, false, false};
         for (int t = 0; t < h->T; ++t) {
             const TableDesc& td = h->tab[t];
             const int kc = k - 1;
@@ -1685,7 +1691,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // the shape variants are independent (different tables): run them side by side so that the tail of one
         // (a few long node lists) overlaps the others
         int nfast = 0;
-        for (int v = 0; v < 8; ++v) nfast += any_fast[v] ? 1 : 0;
+        for (int v = 0; v < 10; ++v) nfast += any_fast[v] ? 1 : 0;
         const bool fork = nfast > 1 && !h->serial;
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
@@ -1698,6 +1704,8 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (any_fast[5]) { k_mid_mma<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
         if (any_fast[6]) { k_mid_mma<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
         if (any_fast[7]) { k_mid_mma<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
+        if (any_fast[8]) { k_mid_mma<4, 8, 32><<<sg, 128, 0, st()>>>(w, k, 8); tt_note_launch(); }
+        if (any_fast[9]) { k_mid_mma<2, 8, 32><<<sg, 128, 0, st()>>>(w, k, 9); tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (nfast > 0) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {
