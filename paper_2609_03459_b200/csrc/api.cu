@@ -181,14 +181,14 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             const bool quad_ok = td.r[K - 2] <= 32;
             if (PMv == 16 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 0;
             else if (PMv == 16 && Mv == 4 && RBv == 16 && quad_ok) td.fast = 1;
-            else if (PMv == 16 && Mv == 4 && RBv == 8) td.fast = 2;
+            else if (PMv == 16 && Mv == 4 && RBv == 8 && quad_ok) td.fast = 2;
             else if (PMv == 32 && Mv == 4 && RBv == 32 && quad_ok) td.fast = 3;
             else if (PMv == 32 && Mv == 8 && RBv == 64 && td.r[K - 2] <= 64) td.fast = 4;
             // first dim factor 2 (D = 32 as 2x4x4): eight groups of two rows stack into the 16-row product, C has 8 rows
             // (the first rows of one row tile), D = 16 as 2x2x4: 4 rows; rank 8: FP32-pipe variants
             else if (PMv == 8 && Mv == 2 && RBv == 32 && quad_ok) td.fast = 5;
             else if (PMv == 8 && Mv == 2 && RBv == 16 && quad_ok) td.fast = 6;
-            else if (PMv == 8 && Mv == 2 && RBv == 8) td.fast = 7;
+            else if (PMv == 8 && Mv == 2 && RBv == 8 && quad_ok) td.fast = 7;
             else if (PMv == 4 && Mv == 2 && RBv == 32 && quad_ok) td.fast = 8;
             else if (PMv == 4 && Mv == 2 && RBv == 16 && quad_ok) td.fast = 9;
         }

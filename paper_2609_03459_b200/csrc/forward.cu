@@ -575,7 +575,7 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
 // one instantiation per shape variant V so that each gets its own register budget.  blockIdx.y walks the
 // tables of variant V (w.vlist), blockIdx.x the table's equal-cost slices.
 template <int V>
-__global__ void __launch_bounds__(128, (V == 0 || V == 1 || V == 5 || V == 6 || V == 8 || V == 9) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
+__global__ void __launch_bounds__(128, (V >= 0 && V != 3 && V != 4) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
     extern __shared__ __align__(16) float sm[];
     __shared__ uint32_t next;
@@ -596,10 +596,10 @@ __global__ void __launch_bounds__(128, (V == 0 || V == 1 || V == 5 || V == 6 || 
     if (V == 4) tt_sweep_pair_cta<32, 64>(w, td, g0, g1, sm, lane, wid);
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
-    if (V == 2) tt_sweep_fast<16, 8, 4, 4, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 2) tt_sweep_quad<16, 8, 4, 4, 0>(w, td, g1, sm + (size_t)wid * (4 * 16 * 12), &next, lane);
     if (V == 5) tt_sweep_quad<8, 32, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 36), &next, lane);
     if (V == 6) tt_sweep_quad<8, 16, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 20), &next, lane);
-    if (V == 7) tt_sweep_fast<8, 8, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
+    if (V == 7) tt_sweep_quad<8, 8, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 12), &next, lane);
     if (V == 8) tt_sweep_quad<4, 32, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 36), &next, lane);
     if (V == 9) tt_sweep_quad<4, 16, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 20), &next, lane);
 }
@@ -612,6 +612,8 @@ static size_t tt_sweep_smem(int V, int max_pl, int max_c)
     if (V == 3) return (size_t)4 * 4 * 32 * 36 * sizeof(float);
     if (V == 5) return (size_t)4 * 8 * 8 * 36 * sizeof(float);    // eight C tiles of 8 rows per warp
     if (V == 6) return (size_t)4 * 8 * 8 * 20 * sizeof(float);
+    if (V == 2) return (size_t)4 * 4 * 16 * 12 * sizeof(float);
+    if (V == 7) return (size_t)4 * 8 * 8 * 12 * sizeof(float);
     if (V == 8) return (size_t)4 * 8 * 4 * 36 * sizeof(float);
     if (V == 9) return (size_t)4 * 8 * 4 * 20 * sizeof(float);
     if (V == 4) return (size_t)(2 * 32 * 64 + 4 * 64 * 68) * sizeof(float);   // one pair of C tiles per CTA + a staged slice block per warp
