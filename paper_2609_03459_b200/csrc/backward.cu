@@ -965,7 +965,8 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
                                                     float* gk, int lane)
 {
     constexpr bool KHALF = PM == 4;   // p = 4..7 of the one k step do not exist: zero operands
-    constexpr int MT = RB_ / 16, KT = KHALF ? 1 : PM / 8;
+    constexpr bool BHALF = RB_ == 8;  // b = 8..15 of the one row tile do not exist: zero operands, not reduced
+    constexpr int MT = BHALF ? 1 : RB_ / 16, KT = KHALF ? 1 : PM / 8;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t* __restrict__ rows = w.val[w.K];
     Tf32Pair a[MT][KT][4];   // A[m = b][k = p] = C[p][b]
@@ -974,9 +975,9 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
             a[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
-            a[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
+            a[mt][kt][1] = tt_split_tf32(BHALF ? 0.f : Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
             a[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
-            a[mt][kt][3] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
+            a[mt][kt][3] = tt_split_tf32(KHALF || BHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     const int rb_ = g >> 2, jb = g & 3;       // B fragment: row rb_ of the pair, column jb of dE
     const int rc = t >> 1, jc = 2 * (t & 1);  // C fragment: row rc of the pair, columns jc, jc+1
@@ -1008,7 +1009,7 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 tt_red_v2(dst + (16 * mt + g) * 4, acc[mt][0], acc[mt][1]);
-                tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
+                if (!BHALF) tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
             }
         }
     }
@@ -1024,7 +1025,8 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
     constexpr bool HALF = PM < 16;                // rows PM..15 of the dC tile stay zero and are not stored
     constexpr bool KHALF = PM == 4;               // p = 4..7 of the one dG k step do not exist: zero operands
     constexpr int MT = HALF ? 1 : PM / 16, NT = RB_ / 8;     // dC tiles: rows p, columns b
-    constexpr int MT2 = RB_ / 16, KT2 = KHALF ? 1 : PM / 8;   // dG tiles: rows b, k = p
+    constexpr bool BHALF = RB_ == 8;              // b = 8..15 of the one dG row tile do not exist: zero operands, not reduced
+    constexpr int MT2 = BHALF ? 1 : RB_ / 16, KT2 = KHALF ? 1 : PM / 8;   // dG tiles: rows b, k = p
     const int g = lane >> 2, t = lane & 3;
     const bool rowok = !HALF || g < PM;
     const int K = w.K;
@@ -1036,9 +1038,9 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
         for (int kt = 0; kt < KT2; ++kt) {
             ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
-            ct[mt][kt][1] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
+            ct[mt][kt][1] = tt_split_tf32(BHALF ? 0.f : Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
             ct[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
-            ct[mt][kt][3] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
+            ct[mt][kt][3] = tt_split_tf32(KHALF || BHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
     float dc[MT][NT][4], dct[MT][NT][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
 #pragma unroll
@@ -1114,7 +1116,7 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
 #pragma unroll
                 for (int mt = 0; mt < MT2; ++mt) {
                     tt_red_v2(dst + (16 * mt + g) * 4, acc[mt][0], acc[mt][1]);
-                    tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
+                    if (!BHALF) tt_red_v2(dst + (16 * mt + g + 8) * 4, acc[mt][2], acc[mt][3]);
                 }
             }
         }
@@ -1204,12 +1206,12 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     float* Cs = As + pl_floats;
     if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);   // 8 x 8: the FP32 pipe wins (0.39 against 0.41 ms)
     if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
 }
@@ -1239,6 +1241,7 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     // tensor-core variants keep C with padded rows (stride r_{K-1} + 8 floats)
     if (V == 0) max_c = 16 * (32 + 8);
     if (V == 1) max_c = 16 * (16 + 8);
+    if (V == 2) max_c = 16 * (8 + 8);
     if (V == 3) max_c = 32 * (32 + 8);
     if (V == 5) max_c = 8 * (32 + 8);
     if (V == 6) max_c = 8 * (16 + 8);
