@@ -178,7 +178,7 @@ def test_medium_forward_backward(binding, case):
             assert_close(grads[t][k], ref[t][k], f"{name} dG[{t}][{k}]")
 
 
-@pytest.mark.parametrize("D,rank", [(16, 8), (16, 16), (16, 32), (32, 8), (32, 16), (32, 32), (64, 8), (64, 32)])
+@pytest.mark.parametrize("D,rank", [(16, 8), (16, 16), (16, 32), (32, 8), (32, 16), (32, 32), (64, 8), (64, 16), (64, 32)])
 def test_sweep_point_shapes(binding, D, rank):
     # the shapes of the dimension / rank sweep (dim factors 2x2x4, 2x4x4, 4x4x4) at a batch the oracle finishes fast
     wl = workloads.sweep_point(D, rank, 96, num_tables=3, with_grad=True)
@@ -192,6 +192,25 @@ def test_sweep_point_shapes(binding, D, rank):
     for t in range(wl.T):
         for k in range(3):
             assert_close(grads[t][k], ref[t][k], f"sweep D{D} r{rank} dG[{t}][{k}]")
+
+
+@pytest.mark.parametrize("D,rank", [(16, 16), (16, 32), (32, 8), (32, 32), (64, 8)])
+def test_sweep_point_shapes_many_groups(binding, D, rank):
+    # the same shape classes with thousands of prefix groups per table (several work units per table, long node lists
+    # for the middle cores, rows of 64 / 128 / 256 bytes through the staged pooling and dE kernels), fused update
+    wl = workloads.sweep_point(D, rank, 2048, num_tables=2, with_grad=True)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"sweep-large D{D} r{rank} out")
+    emb.backward_sgd(dev(wl.grad_out), 0.01)
+    grads = emb.get_grads()
+    cores = emb.get_cores()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref[t], 0.01)
+        for k in range(3):
+            assert_close(grads[t][k], ref[t][k], f"sweep-large D{D} r{rank} dG[{t}][{k}]")
+            assert_close(cores[t][k], want[k], f"sweep-large D{D} r{rank} core[{t}][{k}]")
 
 
 POOLING_CASES = [MEDIUM[0], MEDIUM[1], MEDIUM[3], MEDIUM[5], MEDIUM[7], MEDIUM[8]]   # D = 64 (cp.async pooling), D = 128, K = 2, odd D, wide D
