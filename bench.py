@@ -482,7 +482,7 @@ def main():
         return per * (wl.L if unit == "lookup" else work["U_rows"] * share)
 
     # (P_{K-1}, r_{K-1}) -> sweep kernel variant (last dim factor 4, at least 3 cores)
-    VARIANT_OF = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4, (8, 32): 5, (8, 16): 6, (8, 8): 7, (4, 32): 8, (4, 16): 9}
+    VARIANT_OF = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4, (8, 32): 5, (8, 16): 6, (8, 8): 7, (4, 32): 8, (4, 16): 9, (4, 8): 10}
     variant_rows = {}   # distinct rows handled by each sweep variant
     for t, s in enumerate(wl.tables):
         v = VARIANT_OF.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \

@@ -221,8 +221,8 @@ int tt_emb_unpack_core(tt_emb_t h, int32_t table, int32_t core, const float* can
  * Device events: time of stage `stage` of the most recent call, in milliseconds, measured with CUDA
  * events recorded on the call's stream when timing is enabled.  SYNCHRONISES on the stage's end event.
  * Stages: 0 grouping, 1 schedule, 2 contraction, 3 pooling, 4 backward sort, 5 backward dE,
- * 6 backward contraction, 7 backward middle cores + reductions, 8 sgd; 9..19 the forward sweep kernel of shape
- * variant -1 (generic), 0..9; 20..30 the backward sweep kernel of the same variants (TT_EMB_ERR_STATE for a
+ * 6 backward contraction, 7 backward middle cores + reductions, 8 sgd; 9..20 the forward sweep kernel of shape
+ * variant -1 (generic), 0..10; 21..32 the backward sweep kernel of the same variants (TT_EMB_ERR_STATE for a
  * variant no table uses).
  * on = 0: no events; 1: events, normal execution; 2: events, and kernels of different shape variants, which
  * normally run side by side on forked streams, run one after the other, so that a per-kernel duration is that

@@ -22,7 +22,7 @@ from . import build as _build
 _HERE = os.path.dirname(os.path.abspath(__file__))
 
 STAGES = ["grouping", "schedule", "contraction", "pooling", "bwd_sort", "bwd_dE", "bwd_contraction",
-          "bwd_middle", "sgd"] + [f"k_sweep_fwd<{v}>" for v in range(-1, 10)] + [f"k_sweep_bwd<{v}>" for v in range(-1, 10)]
+          "bwd_middle", "sgd"] + [f"k_sweep_fwd<{v}>" for v in range(-1, 11)] + [f"k_sweep_bwd<{v}>" for v in range(-1, 11)]
 
 TT_EMB_OK = 0
 TT_EMB_ERR_ARG, TT_EMB_ERR_WORKSPACE, TT_EMB_ERR_ARCH, TT_EMB_ERR_STATE, TT_EMB_ERR_CUDA = -1, -2, -3, -4, -5

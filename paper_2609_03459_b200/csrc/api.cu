@@ -191,6 +191,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (PMv == 8 && Mv == 2 && RBv == 8 && quad_ok) td.fast = 7;
             else if (PMv == 4 && Mv == 2 && RBv == 32 && quad_ok) td.fast = 8;
             else if (PMv == 4 && Mv == 2 && RBv == 16 && quad_ok) td.fast = 9;
+            else if (PMv == 4 && Mv == 2 && RBv == 8) td.fast = 10;   // D = 16 with rank 8: FP32 pipe (slices of 16 columns)
         }
         for (int k = 0; k < TT_MAXK; ++k) td.midfast[k] = -1;
         for (int k = 2; k <= K - 1; ++k) {
@@ -205,6 +206,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             else if (Mv == 2 && rav == 16 && colsv == 32) td.midfast[k] = 7;
             else if (Mv == 4 && rav == 8 && colsv == 32) td.midfast[k] = 8;
             else if (Mv == 2 && rav == 8 && colsv == 32) td.midfast[k] = 9;
+            else if (Mv == 2 && rav == 8 && colsv == 16) td.midfast[k] = 10;
         }
         td.unit_base = unit_base;
         unit_base += Q;

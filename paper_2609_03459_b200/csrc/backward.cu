@@ -1214,6 +1214,7 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);   // 8 x 8: the FP32 pipe wins (0.39 against 0.41 ms)
     if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 10) tt_sweep_bwd_fast<4, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
 }
 
 // fixed-order sum of the partial copies of the last core's gradient
@@ -1293,6 +1294,7 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_bwd<7>(h, max_pl, max_c, next_stream(8))) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<8>(h, max_pl, max_c, next_stream(9))) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<9>(h, max_pl, max_c, next_stream(10))) != cudaSuccess) return e;
+    if ((e = launch_sweep_bwd<10>(h, max_pl, max_c, next_stream(11))) != cudaSuccess) return e;
     if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
     tt_note_launch();
@@ -1466,11 +1468,12 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 {
-    static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && COLS % 32 == 0, "rows per node; r_{k-1}; columns per warp");
+    static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && (COLS % 32 == 0 || COLS == 16), "rows per node; r_{k-1}; columns per warp");
     constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16, 32 or 64 stacked rows per pass
     constexpr bool AHALF = RA == 8;          // dG: a = 8..15 of the one m-tile do not exist: zero operands, not stored
     constexpr int MT = AHALF ? 1 : RA / 16;  // dG: m-tiles over a
-    constexpr int NTW = COLS / 32;           // dG: n-tiles per warp (the warp's COLS/4 columns)
+    constexpr int CW = COLS >= 32 ? COLS / 4 : 8;   // dG: columns per warp (16 columns: warps 0 and 1 only)
+    constexpr int NTW = CW / 8;              // dG: n-tiles per warp
     constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ / 4 row tiles of four nodes; NTY * NQ / 4 = 4 warps
     constexpr int KTY = COLS / 8;            // Y: k steps over c
     __shared__ __align__(16) float sA[2][NQ * M * AP];
@@ -1507,7 +1510,8 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int nt = 0; nt < NTW; ++nt) {
-                const int c = wid * (COLS / 4) + 8 * nt + 2 * t;
+                const int c = wid * CW + 8 * nt + 2 * t;
+                if (c >= COLS) continue;     // this warp owns no columns of the slice gradient
                 float2* p0 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g) * COLS + c);
                 float2* p1 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g + 8) * COLS + c);
                 float2 v0 = first_fold ? make_float2(0.f, 0.f) : *p0;
@@ -1573,8 +1577,9 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
         for (int p = 0; p < NQ * M / 8; ++p) {
             const float* Aa = A_ + (8 * p + t) * AP;       // stacked row 8p + t:     node (8p + t) / M, row (8p + t) % M
             const float* Ab = A_ + (8 * p + t + 4) * AP;   // stacked row 8p + t + 4
-            const float* Da = D_ + (8 * p + t) * CP + wid * (COLS / 4) + g;
-            const float* Db = D_ + (8 * p + t + 4) * CP + wid * (COLS / 4) + g;
+            if (wid * CW >= COLS) break;     // this warp owns no columns of the slice gradient
+            const float* Da = D_ + (8 * p + t) * CP + wid * CW + g;
+            const float* Db = D_ + (8 * p + t + 4) * CP + wid * CW + g;
             Tf32Pair a[MT][4];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
@@ -1678,7 +1683,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
     cudaError_t e;
     for (int k = h->K - 1; k >= 2; --k) {
         int max_n = 1, max_down = 1, max_slice = 1;
-        bool any_generic = false, any_fast[10] = {false, false, false, false, false, false, false, false, false, false};
+        bool any_generic = false, any_fast[11] = {false, false, false, false, false, false, false, false, false, false, false};
         for (int t = 0; t < h->T; ++t) {
             const TableDesc& td = h->tab[t];
             const int kc = k - 1;
@@ -1694,7 +1699,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // the shape variants are independent (different tables): run them side by side so that the tail of one
         // (a few long node lists) overlaps the others
         int nfast = 0;
-        for (int v = 0; v < 10; ++v) nfast += any_fast[v] ? 1 : 0;
+        for (int v = 0; v < 11; ++v) nfast += any_fast[v] ? 1 : 0;
         const bool fork = nfast > 1 && !h->serial;
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
@@ -1709,6 +1714,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (any_fast[7]) { k_mid_mma<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
         if (any_fast[8]) { k_mid_mma<4, 8, 32><<<sg, 128, 0, st()>>>(w, k, 8); tt_note_launch(); }
         if (any_fast[9]) { k_mid_mma<2, 8, 32><<<sg, 128, 0, st()>>>(w, k, 9); tt_note_launch(); }
+        if (any_fast[10]) { k_mid_mma<2, 8, 16><<<sg, 128, 0, st()>>>(w, k, 10); tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (nfast > 0) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
         if (any_generic) {

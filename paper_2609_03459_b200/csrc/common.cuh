@@ -11,9 +11,9 @@
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
 #define TT_DE_CHUNK 1024                                  // sorted lookups per warp in the dE segment reduction
-#define TT_NUM_STAGES 31                                // 0..8 pipeline stages, 9..19 forward sweep variants -1..9, 20..30 backward sweep variants
+#define TT_NUM_STAGES 33                                // 0..8 pipeline stages, 9..20 forward sweep variants -1..10, 21..32 backward sweep variants
 #define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
-#define TT_NUM_VARIANTS 10                               // register-tiled shape variants (forward.cu)
+#define TT_NUM_VARIANTS 11                               // register-tiled shape variants (forward.cu)
 
 // Per-table descriptor, resident in the workspace.  k below is 0-based (core k+1 of the paper).
 struct TableDesc {

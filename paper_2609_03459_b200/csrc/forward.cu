@@ -602,6 +602,7 @@ __global__ void __launch_bounds__(128, (V >= 0 && V != 3 && V != 4) ? 6 : 1) k_s
     if (V == 7) tt_sweep_quad<8, 8, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 8 * 12), &next, lane);
     if (V == 8) tt_sweep_quad<4, 32, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 36), &next, lane);
     if (V == 9) tt_sweep_quad<4, 16, 2, 4, 0>(w, td, g1, sm + (size_t)wid * (8 * 4 * 20), &next, lane);
+    if (V == 10) tt_sweep_fast<4, 8, 2, 2, 1, false>(w, td, g1, As, Cs, &next, lane);
 }
 
 // dynamic shared memory of k_sweep_fwd<V> / k_sweep_bwd<V>: four C tiles per warp for the tensor-core variants
@@ -671,6 +672,7 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_fwd<7>(h, max_pl, max_c, next_stream(8))) != cudaSuccess) return e;
     if ((e = launch_sweep_fwd<8>(h, max_pl, max_c, next_stream(9))) != cudaSuccess) return e;
     if ((e = launch_sweep_fwd<9>(h, max_pl, max_c, next_stream(10))) != cudaSuccess) return e;
+    if ((e = launch_sweep_fwd<10>(h, max_pl, max_c, next_stream(11))) != cudaSuccess) return e;
     if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
