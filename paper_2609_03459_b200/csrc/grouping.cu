@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
             const uint32_t row = (uint32_t)g[j];
             unsigned* word = &w.bm[td.word_base + (row >> 5)].x;
             const unsigned m = 1u << (row & 31);
-            if (!(__ldcg(word) & m)) atomicOr(word, m);
+            if (!(__ldca(word) & m)) atomicOr(word, m);   // L1 may hold a stale word: at worst a redundant atomic
         }
     }
     if (bad) atomicOr(w.status, TT_EMB_STATUS_INDEX);
