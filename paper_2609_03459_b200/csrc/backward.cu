@@ -511,12 +511,7 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
-#pragma unroll 8
-        for (int j = 0; j < n; ++j) {
-            if ((starts >> j) & 1u) {
-                close_segment();
-                cur = __shfl_sync(0xffffffffu, cur_pairs.x, j);
-            }
+        auto add_row = [&](int j) {
             float x[VPL];
             if (VPL == 2) {
                 const float2 v = reinterpret_cast<const float2*>(bufv)[j * 32 + lane];
@@ -529,6 +524,23 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
             }
 #pragma unroll
             for (int c = 0; c < VPL; ++c) part[c] += x[c];
+        };
+        // eight rows at a time; a run of eight without a segment start (popular rows: most lookups sit in segments far
+        // longer than a batch) is added without looking at the start bits
+        for (int j0 = 0; j0 < n; j0 += 8) {
+            if (j0 + 8 <= n && ((starts >> j0) & 0xffu) == 0u) {
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) add_row(j0 + jj);
+            } else {
+                const int j1 = min(j0 + 8, n);
+                for (int j = j0; j < j1; ++j) {
+                    if ((starts >> j) & 1u) {
+                        close_segment();
+                        cur = __shfl_sync(0xffffffffu, cur_pairs.x, j);
+                    }
+                    add_row(j);
+                }
+            }
         }
 #pragma unroll
         for (int c = 0; c < VPL; ++c) { acc[c] += part[c]; part[c] = 0.f; }
