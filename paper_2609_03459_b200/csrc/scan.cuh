@@ -45,10 +45,12 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
     const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
     if (base >= n) return;
     uint32_t s = 0;
-    const uint64_t i0 = base + (uint64_t)threadIdx.x * TT_SCAN_ITEMS;
+    // a sum has no order: neighbouring threads take neighbouring elements (coalesced)
 #pragma unroll 4
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j)
-        if (i0 + j < n) s += f.value((uint32_t)(i0 + j));
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+        const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
+        if (i < n) s += f.value((uint32_t)i);
+    }
     uint32_t tot;
     tt_block_excl_scan(s, sm, tot);
     if (threadIdx.x == 0) tile_sums[blockIdx.x] = tot;
@@ -72,27 +74,46 @@ __global__ void __launch_bounds__(1024) tt_scan_spine(F f, uint32_t* __restrict_
     if (threadIdx.x == 0) f.total(carry);
 }
 
+// Elements are read and emitted striped (thread t takes elements t, t + 256, ...: coalesced for the functor's loads and
+// stores), scanned blocked (thread t owns elements 16 t .. 16 t + 15); the two orders meet in shared memory, padded by
+// one word per 32 so that both access patterns are free of bank conflicts.
+__device__ __forceinline__ int tt_scan_pad(int i) { return i + (i >> 5); }
+
 template <class F>
 __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
 {
     __shared__ uint32_t sm[34];
+    __shared__ uint32_t sv[TT_SCAN_TILE + TT_SCAN_TILE / 32];
     const uint32_t n = f.size();
     const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
     if (base >= n) return;
     uint32_t v[TT_SCAN_ITEMS];
-    uint32_t s = 0;
-    const uint64_t i0 = base + (uint64_t)threadIdx.x * TT_SCAN_ITEMS;
 #pragma unroll
     for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
-        v[j] = (i0 + j < n) ? f.value((uint32_t)(i0 + j)) : 0u;
-        s += v[j];
+        const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
+        v[j] = i < n ? f.value((uint32_t)i) : 0u;
+        sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)] = v[j];
+    }
+    __syncthreads();
+    uint32_t s = 0;
+    uint32_t mine[TT_SCAN_ITEMS];
+#pragma unroll
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+        mine[j] = sv[tt_scan_pad(threadIdx.x * TT_SCAN_ITEMS + j)];
+        s += mine[j];
     }
     uint32_t tot;
     uint32_t ex = tile_sums[blockIdx.x] + tt_block_excl_scan(s, sm, tot);
 #pragma unroll
     for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
-        if (i0 + j < n) f.emit((uint32_t)(i0 + j), ex, v[j]);
-        ex += v[j];
+        sv[tt_scan_pad(threadIdx.x * TT_SCAN_ITEMS + j)] = ex;   // exclusive prefix of element 16 t + j
+        ex += mine[j];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+        const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
+        if (i < n) f.emit((uint32_t)i, sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)], v[j]);
     }
 }
 
