@@ -97,7 +97,7 @@ __device__ __forceinline__ int64_t tt_index(const WsView& w, int64_t l)
     return STREAM ? __ldcs(w.indices + l) : __ldg(w.indices + l);
 }
 
-enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16 };
+enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16, CTR_SCAN_TICKET = 32 /* tiles of the running scan that have reported */ };
 
 struct tt_emb {
     int T, K, D;

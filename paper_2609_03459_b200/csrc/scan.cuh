@@ -1,11 +1,12 @@
-// Device-wide exclusive scan of uint32 values produced by a functor, as three kernels
-// (tile sums -> scan of tile sums by one CTA -> per-tile scan + apply).  No inter-CTA waiting.
+// Device-wide exclusive scan of uint32 values produced by a functor, as two kernels: tile sums, where the CTA that
+// reports last (a ticket counter; nobody waits) also scans the tile sums, then per-tile scan + apply.
 //
 // Functor F:
 //   __device__ uint32_t size() const;                       number of elements (may read device memory)
 //   __device__ uint32_t value(uint32_t i) const;            input i
 //   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v) const;   called once per element in the apply pass
 //   __device__ void total(uint32_t tot) const;              called by one thread with the grand total
+//   WsView w;                                               w.counters[CTR_SCAN_TICKET] is the ticket (zero between scans)
 #pragma once
 #include "common.cuh"
 
@@ -37,13 +38,35 @@ __device__ __forceinline__ uint32_t tt_block_excl_scan(uint32_t x, uint32_t* sm 
     return res;
 }
 
+// exclusive scan of the tile sums in place (one CTA), grand total to the functor
 template <class F>
-__global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t* __restrict__ tile_sums)
+__device__ __forceinline__ void tt_scan_spine_cta(const F& f, uint32_t* tile_sums, uint32_t ntiles, uint32_t* sm)
+{
+    uint32_t carry = 0;
+    for (uint32_t b0 = 0; b0 < ntiles; b0 += blockDim.x) {
+        const uint32_t i = b0 + threadIdx.x;
+        const uint32_t x = i < ntiles ? __ldcg(tile_sums + i) : 0u;   // written by other CTAs: read past L1
+        uint32_t tot;
+        const uint32_t ex = tt_block_excl_scan(x, sm, tot);
+        if (i < ntiles) tile_sums[i] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) f.total(carry);
+}
+
+template <class F>
+__global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t* tile_sums)
 {
     __shared__ uint32_t sm[34];
+    __shared__ uint32_t ticket;
     const uint32_t n = f.size();
+    const uint32_t ntiles = (uint32_t)(((uint64_t)n + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
+    if (ntiles == 0) {   // nothing to scan: the first CTA still reports the total
+        if (blockIdx.x == 0 && threadIdx.x == 0) f.total(0u);
+        return;
+    }
+    if (blockIdx.x >= ntiles) return;
     const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
-    if (base >= n) return;
     uint32_t s = 0;
     // a sum has no order: neighbouring threads take neighbouring elements (coalesced)
 #pragma unroll 4
@@ -53,25 +76,17 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
     }
     uint32_t tot;
     tt_block_excl_scan(s, sm, tot);
-    if (threadIdx.x == 0) tile_sums[blockIdx.x] = tot;
-}
-
-template <class F>
-__global__ void __launch_bounds__(1024) tt_scan_spine(F f, uint32_t* __restrict__ tile_sums)
-{
-    __shared__ uint32_t sm[34];
-    const uint32_t n = f.size();
-    const uint32_t ntiles = (uint32_t)(((uint64_t)n + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
-    uint32_t carry = 0;
-    for (uint32_t b0 = 0; b0 < ntiles; b0 += blockDim.x) {
-        uint32_t i = b0 + threadIdx.x;
-        uint32_t x = i < ntiles ? tile_sums[i] : 0u;
-        uint32_t tot;
-        uint32_t ex = tt_block_excl_scan(x, sm, tot);
-        if (i < ntiles) tile_sums[i] = carry + ex;
-        carry += tot;
+    if (threadIdx.x == 0) {
+        tile_sums[blockIdx.x] = tot;
+        __threadfence();                                   // the sum is visible before the ticket is
+        ticket = atomicAdd(f.w.counters + CTR_SCAN_TICKET, 1u);
     }
-    if (threadIdx.x == 0) f.total(carry);
+    __syncthreads();
+    if (ticket != ntiles - 1) return;
+    // every tile has reported: this CTA scans the sums and leaves the ticket at zero for the next scan
+    __threadfence();
+    tt_scan_spine_cta(f, tile_sums, ntiles, sm);
+    if (threadIdx.x == 0) f.w.counters[CTR_SCAN_TICKET] = 0u;
 }
 
 // Elements are read and emitted striped (thread t takes elements t, t + 256, ...: coalesced for the functor's loads and
@@ -124,8 +139,6 @@ static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, 
     unsigned tiles = (unsigned)((capacity + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
     if (tiles == 0) tiles = 1;
     tt_scan_reduce<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
-    tt_note_launch();
-    tt_scan_spine<F><<<1, 1024, 0, s>>>(f, tmp);
     tt_note_launch();
     tt_scan_apply<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
     tt_note_launch();
