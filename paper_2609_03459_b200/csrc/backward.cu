@@ -1324,6 +1324,7 @@ __device__ __forceinline__ uint32_t tt_tkey(const TableDesc& td, int k, uint32_t
 
 __global__ void k_tmark(WsView w, int k)
 {
+    tt_pdl_enter();
     const uint32_t count = w.counters[CTR_LEVEL0 + k];
     for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < count; v += gridDim.x * blockDim.x) {
         const int t = tt_find_table(w.tb[k], w.T, v);
@@ -1350,6 +1351,7 @@ __device__ __forceinline__ uint32_t tt_trank(const WsView& w, const TableDesc& t
 
 __global__ void k_tfill(WsView w, int k)
 {
+    tt_pdl_enter();
     const uint32_t count = w.counters[CTR_LEVEL0 + k];
     for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < count; v += gridDim.x * blockDim.x) {
         const int t = tt_find_table(w.tb[k], w.T, v);
@@ -1680,11 +1682,11 @@ cudaError_t tt_launch_tlist(tt_emb* h, int k, cudaStream_t s)
     cudaError_t e;
     if ((e = cudaMemsetAsync(w.tbm[k], 0, (size_t)w.ttotal_words[k] * sizeof(uint2), s)) != cudaSuccess) return e;
     const int g = h->sm_count * 8;
-    k_tmark<<<g, 256, 0, s>>>(w, k);
+    if ((e = tt_launch_pdl(k_tmark, dim3(g), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
     tt_note_launch();
     TPopScan tp{w, k};
     if ((e = tt_scan(tp, w.ttotal_words[k], w.scan_tmp, s)) != cudaSuccess) return e;
-    k_tfill<<<g, 256, 0, s>>>(w, k);
+    if ((e = tt_launch_pdl(k_tfill, dim3(g), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }

@@ -161,6 +161,33 @@ cudaError_t tt_launch_export_level(tt_emb* h, int table, int level, int64_t* val
 cudaError_t tt_launch_export_inverse(tt_emb* h, int table, int32_t* inv, cudaStream_t s);
 cudaError_t tt_launch_pack(const TableDesc& td, int core, const float* src, float* dst, bool to_canonical, cudaStream_t s);
 
+// ---- programmatic dependent launch: the kernels of the forward chain are launched with the attribute below and
+// begin with tt_pdl_enter().  A kernel's CTAs may then become resident while its predecessor in the stream is still
+// running and wait (griddepcontrol.wait) until that grid has completed and its writes are visible, so the launch
+// latency of a chain of short kernels overlaps the previous kernel instead of following it.  Without the attribute
+// (or after a non-kernel operation in the stream) the wait returns at once.
+__device__ __forceinline__ void tt_pdl_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <class... KArgs, class... Args>
+static inline cudaError_t tt_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // ---- small device helpers ----
 __device__ __forceinline__ int tt_find_table(const uint32_t* __restrict__ tb, int T, uint32_t v)
 {

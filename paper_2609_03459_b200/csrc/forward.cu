@@ -133,6 +133,7 @@ __device__ __forceinline__ const float* tt_left_operand(const WsView& w, const T
 // P_k for every level-k node, 2 <= k <= K-2 (only K = 4 has such a level); one CTA per node, grid-stride
 __global__ void __launch_bounds__(128) k_mid_level(WsView w, int k)
 {
+    tt_pdl_enter();
     extern __shared__ float sm[];
     const uint32_t count = w.counters[CTR_LEVEL0 + k];
     for (uint32_t v = blockIdx.x; v < count; v += gridDim.x) {
@@ -577,6 +578,7 @@ __device__ __forceinline__ void tt_sweep_generic(const WsView& w, const TableDes
 template <int V>
 __global__ void __launch_bounds__(128, (V >= 0 && V != 3 && V != 4) ? 6 : 1) k_sweep_fwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
+    tt_pdl_enter();
     extern __shared__ __align__(16) float sm[];
     __shared__ uint32_t next;
     const int t = w.vlist[vbase + blockIdx.y];
@@ -630,7 +632,7 @@ static cudaError_t launch_sweep_fwd(tt_emb* h, int max_pl, int max_c, cudaStream
     cudaError_t e = cudaFuncSetAttribute(k_sweep_fwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if ((e = tt_stage_begin(h, 9 + V + 1, s)) != cudaSuccess) return e;
-    k_sweep_fwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    if ((e = tt_launch_pdl(k_sweep_fwd<V>, dim3(h->units_per_table, n), dim3(128), smem, s, h->v, max_pl, max_c, h->vbase[V + 1])) != cudaSuccess) return e;
     tt_note_launch();
     if ((e = tt_stage_end(h, 9 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
@@ -650,7 +652,8 @@ cudaError_t tt_launch_contraction(tt_emb* h, cudaStream_t s)
     }
     for (int k = 2; k <= h->K - 2; ++k) {
         int grid = h->sm_count * 16;
-        k_mid_level<<<grid, 128, (size_t)max_pl * sizeof(float), s>>>(w, k);
+        cudaError_t e0 = tt_launch_pdl(k_mid_level, dim3(grid), dim3(128), (size_t)max_pl * sizeof(float), s, w, k);
+        if (e0 != cudaSuccess) return e0;
         tt_note_launch();
     }
     cudaError_t e;
@@ -712,6 +715,7 @@ __device__ __forceinline__ int64_t tt_pool_chunks(int64_t L, int64_t W)
 template <int LPR, int CPL, bool WT>  // lanes per row, float4 chunks per lane, weighted / mean pooling
 __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_pool_vec(WsView w, float* __restrict__ out)
 {
+    tt_pdl_enter();
     const int lane = threadIdx.x & 31;
     const int sub = lane / LPR, lr = lane % LPR;
     constexpr int RPI = 32 / LPR;                       // rows per load instruction
@@ -850,6 +854,7 @@ __device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
 template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, float* __restrict__ out)
 {
+    tt_pdl_enter();
     static_assert(R4 == 16 || R4 == 8, "two or four rows per cp.async instruction");
     constexpr int RPI = 32 / R4;
     extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][R4 float4]
@@ -967,7 +972,7 @@ static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
     const int64_t need = (nb + POOL_WARPS - 1) / POOL_WARPS;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_async<R4, WT><<<(int)grid, 32 * POOL_WARPS, smem, s>>>(h->v, out);
+    if ((e = tt_launch_pdl(k_pool_async<R4, WT>, dim3((int)grid), dim3(32 * POOL_WARPS), smem, s, h->v, out)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -984,7 +989,7 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
     const int64_t need = (nb + 7) / 8;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    k_pool_vec<LPR, CPL, WT><<<(int)grid, 256, 0, s>>>(h->v, out);
+    if ((e = tt_launch_pdl(k_pool_vec<LPR, CPL, WT>, dim3((int)grid), dim3(256), 0, s, h->v, out)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -992,6 +997,7 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
 // any D (scalar path): lane handles elements lane, lane+32, ...
 __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict__ out)
 {
+    tt_pdl_enter();
     const int lane = threadIdx.x & 31;
     const int D = w.D;
     const int64_t nb = (int64_t)w.T * w.B;
@@ -1070,7 +1076,8 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0);
     if (!vec_ok) {
         int pgrid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
-        k_pool_scalar<<<pgrid < 1 ? 1 : pgrid, 256, 0, s>>>(w, out);
+        cudaError_t e0 = tt_launch_pdl(k_pool_scalar, dim3(pgrid < 1 ? 1 : pgrid), dim3(256), 0, s, w, out);
+        if (e0 != cudaSuccess) return e0;
         tt_note_launch();
         return cudaGetLastError();
     }

@@ -14,6 +14,7 @@
 
 __global__ void k_check_offsets(WsView w)
 {
+    tt_pdl_enter();
     const int64_t nb = (int64_t)w.T * w.B;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     bool bad = false;
@@ -35,6 +36,7 @@ __global__ void k_check_offsets(WsView w)
 
 __global__ void __launch_bounds__(256) k_mark(WsView w)
 {
+    tt_pdl_enter();
     const int64_t L = w.L;
     const int64_t step = (int64_t)gridDim.x * blockDim.x * 4;
     int t = 0;
@@ -142,6 +144,7 @@ struct LevelUp {
 // tables without any node at level k+1 never had tb[k][t] written: inherit from the next table
 __global__ void k_fix_tb(WsView w, int k)
 {
+    tt_pdl_enter();
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (int t = w.T - 1; t >= 0; --t)
             if (w.tb[k + 1][t] == w.tb[k + 1][t + 1]) w.tb[k][t] = w.tb[k][t + 1];
@@ -158,12 +161,12 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
     const int64_t nb = (int64_t)w.T * w.B + 1;
     int g0 = (int)((nb + 255) / 256);
     if (g0 > h->sm_count * 8) g0 = h->sm_count * 8;
-    k_check_offsets<<<g0, 256, 0, s>>>(w);
+    if ((e = tt_launch_pdl(k_check_offsets, dim3(g0), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     if (w.L > 0) {
         int64_t want = (w.L + 1023) / 1024;
         int g1 = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
-        k_mark<<<g1, 256, 0, s>>>(w);
+        if ((e = tt_launch_pdl(k_mark, dim3(g1), dim3(256), 0, s, w)) != cudaSuccess) return e;
         tt_note_launch();
     }
     PopScan ps{w};
@@ -171,7 +174,7 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
     for (int k = w.K - 1; k >= 1; --k) {
         LevelUp lu{w, k};
         if ((e = tt_scan(lu, w.cap[k + 1], w.scan_tmp, s)) != cudaSuccess) return e;
-        k_fix_tb<<<1, 32, 0, s>>>(w, k);
+        if ((e = tt_launch_pdl(k_fix_tb, dim3(1), dim3(32), 0, s, w, k)) != cudaSuccess) return e;
         tt_note_launch();
     }
     return cudaGetLastError();

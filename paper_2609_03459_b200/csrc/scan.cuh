@@ -57,6 +57,7 @@ __device__ __forceinline__ void tt_scan_spine_cta(const F& f, uint32_t* tile_sum
 template <class F>
 __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t* tile_sums)
 {
+    tt_pdl_enter();
     __shared__ uint32_t sm[34];
     __shared__ uint32_t ticket;
     const uint32_t n = f.size();
@@ -97,6 +98,7 @@ __device__ __forceinline__ int tt_scan_pad(int i) { return i + (i >> 5); }
 template <class F>
 __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
 {
+    tt_pdl_enter();
     __shared__ uint32_t sm[34];
     __shared__ uint32_t sv[TT_SCAN_TILE + TT_SCAN_TILE / 32];
     const uint32_t n = f.size();
@@ -138,9 +140,10 @@ static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, 
 {
     unsigned tiles = (unsigned)((capacity + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
     if (tiles == 0) tiles = 1;
-    tt_scan_reduce<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    cudaError_t e = tt_launch_pdl(tt_scan_reduce<F>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, tmp);
+    if (e != cudaSuccess) return e;
     tt_note_launch();
-    tt_scan_apply<F><<<tiles, TT_SCAN_THREADS, 0, s>>>(f, tmp);
+    if ((e = tt_launch_pdl(tt_scan_apply<F>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, (const uint32_t*)tmp)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
