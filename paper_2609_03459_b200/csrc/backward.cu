@@ -29,6 +29,7 @@
 
 __global__ void k_zero_u32_dev(uint32_t* p, const uint32_t* count, uint32_t extra)
 {
+    tt_pdl_enter();
     const uint32_t n = *count + extra;
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0u;
 }
@@ -37,6 +38,7 @@ __global__ void k_zero_u32_dev(uint32_t* p, const uint32_t* count, uint32_t extr
 // first digits are written later)
 __global__ void k_zero_grads(WsView w)
 {
+    tt_pdl_enter();
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
     const int K = w.K;
@@ -61,6 +63,7 @@ __global__ void k_zero_grads(WsView w)
 template <int MODE>
 __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 {
+    tt_pdl_enter();
     static_assert(HT_TILE == (1 << HT_ID_BITS) && HT_SIZE == (1 << (32 - HT_LOW_BITS)) && HT_LOW_BITS + HT_ID_BITS <= 32, "tag layout");
     const uint2* __restrict__ upairs = w.upairs;
     const uint32_t capK = w.cap[w.K];
@@ -161,10 +164,10 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
     const int zgrid = h->sm_count * 8;
-    k_zero_u32_dev<<<zgrid, 256, 0, s>>>(w.cnt, w.counters + CTR_LEVEL0 + w.K, 1u);
+    cudaError_t e;
+    if ((e = tt_launch_pdl(k_zero_u32_dev, dim3(zgrid), dim3(256), 0, s, w.cnt, (const uint32_t*)(w.counters + CTR_LEVEL0 + w.K), 1u)) != cudaSuccess) return e;
     tt_note_launch();
     const int64_t ntiles = (w.L + HT_TILE - 1) / HT_TILE;
-    cudaError_t e;
     int per_sm0 = 0, per_sm1 = 0;   // persistent grids sized to what is actually resident (no partial second wave)
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm0, k_sort_pass<0>, 256, 0)) != cudaSuccess) return e;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm1, k_sort_pass<1>, 256, 0)) != cudaSuccess) return e;
@@ -173,11 +176,11 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
         if (g > ntiles) g = ntiles;
         return (int)(g < 1 ? 1 : g);
     };
-    k_sort_pass<0><<<grid_of(per_sm0), 256, 0, s>>>(w);
+    if ((e = tt_launch_pdl(k_sort_pass<0>, dim3(grid_of(per_sm0)), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     CntScan cs{w};
     if ((e = tt_scan(cs, w.cap[w.K], w.scan_tmp, s)) != cudaSuccess) return e;
-    k_sort_pass<1><<<grid_of(per_sm1), 256, 0, s>>>(w);
+    if ((e = tt_launch_pdl(k_sort_pass<1>, dim3(grid_of(per_sm1)), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -243,6 +246,7 @@ struct RowAcc {
 template <bool VEC, int CPL>
 __global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ grad_out)
 {
+    tt_pdl_enter();
     const int lane = threadIdx.x & 31;
     const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
@@ -293,6 +297,7 @@ __global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ 
 template <bool VEC, int CPL>
 __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
 {
+    tt_pdl_enter();
     const int lane = threadIdx.x & 31;
     const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t U = w.counters[CTR_LEVEL0 + w.K];
@@ -344,6 +349,7 @@ __global__ void __launch_bounds__(256) k_dE_fix(WsView w)
 template <int LPR, bool WT>
 __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __restrict__ grad_out)
 {
+    tt_pdl_enter();
     constexpr int RPI = 32 / LPR, NF = 4;
     const int lane = threadIdx.x & 31, sub = lane / LPR, lr = lane % LPR;
     const int64_t chunk = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -438,6 +444,7 @@ __global__ void __launch_bounds__(256, 5) k_dE_fast(WsView w, const float* __res
 template <int DD, bool WT>   // DD = D: 64 (two columns per lane), 32 (one) or 16 (one, lanes 0..15)
 __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const float* __restrict__ grad_out)
 {
+    tt_pdl_enter();
     static_assert(DD == 64 || DD == 32 || DD == 16, "a lane owns DD / 32 columns (one column on the first DD lanes below 32)");
     constexpr int R4 = DD / 4;          // float4 pieces per row
     constexpr int RPI = 32 / R4;        // rows per cp.async instruction
@@ -567,14 +574,15 @@ static cudaError_t launch_dE_t(tt_emb* h, const float* grad_out, cudaStream_t s)
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             const int sgrid = (int)((chunks + DE_WARPS - 1) / DE_WARPS);
-            kern<<<sgrid, 32 * DE_WARPS, smem, s>>>(h->v, grad_out);
+            if ((e = tt_launch_pdl(kern, dim3(sgrid), dim3(32 * DE_WARPS), smem, s, h->v, grad_out)) != cudaSuccess) return e;
             tt_note_launch();
         } else
         if (VEC && D4 <= 8) { if (wt) k_dE_fast<8, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<8, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else if (VEC && D4 <= 16) { if (wt) k_dE_fast<16, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<16, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else if (VEC && D4 <= 32) { if (wt) k_dE_fast<32, true><<<grid, 256, 0, s>>>(h->v, grad_out); else k_dE_fast<32, false><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
         else { k_dE<VEC, CPL><<<grid, 256, 0, s>>>(h->v, grad_out); tt_note_launch(); }
-        k_dE_fix<VEC, CPL><<<grid, 256, 0, s>>>(h->v);
+        cudaError_t ef = tt_launch_pdl(k_dE_fix<VEC, CPL>, dim3(grid), dim3(256), 0, s, h->v);
+        if (ef != cudaSuccess) return ef;
         tt_note_launch();
     }
     return cudaGetLastError();
@@ -1195,6 +1203,7 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
 template <int V>
 __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
+    tt_pdl_enter();
     extern __shared__ __align__(16) float sm[];
     const int t = w.vlist[vbase + blockIdx.y], q = blockIdx.x;
     uint32_t g0, g1;
@@ -1232,6 +1241,7 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
 // fixed-order sum of the partial copies of the last core's gradient
 __global__ void __launch_bounds__(256) k_reduce_gpart(WsView w)
 {
+    tt_pdl_enter();
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
     const int kl = w.K - 1;
@@ -1265,7 +1275,7 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if ((e = tt_stage_begin(h, 9 + TT_NUM_VARIANTS + 1 + V + 1, s)) != cudaSuccess) return e;
-    k_sweep_bwd<V><<<dim3(h->units_per_table, n), 128, smem, s>>>(h->v, max_pl, max_c, h->vbase[V + 1]);
+    if ((e = tt_launch_pdl(k_sweep_bwd<V>, dim3(h->units_per_table, n), dim3(128), smem, s, h->v, max_pl, max_c, h->vbase[V + 1])) != cudaSuccess) return e;
     tt_note_launch();
     if ((e = tt_stage_end(h, 9 + TT_NUM_VARIANTS + 1 + V + 1, s)) != cudaSuccess) return e;
     return cudaGetLastError();
@@ -1308,7 +1318,7 @@ cudaError_t tt_launch_bwd_contraction(tt_emb* h, cudaStream_t s)
     if ((e = launch_sweep_bwd<9>(h, max_pl, max_c, next_stream(10))) != cudaSuccess) return e;
     if ((e = launch_sweep_bwd<10>(h, max_pl, max_c, next_stream(11))) != cudaSuccess) return e;
     if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
-    k_reduce_gpart<<<dim3(32, h->T), 256, 0, s>>>(w);
+    if ((e = tt_launch_pdl(k_reduce_gpart, dim3(32, h->T), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
@@ -1365,6 +1375,7 @@ __global__ void k_tfill(WsView w, int k)
 // one CTA per parent, children in sorted order; the slice is staged in shared memory (padded rows)
 __global__ void __launch_bounds__(256) k_mid_down(WsView w, int k)
 {
+    tt_pdl_enter();
     extern __shared__ float sm[];
     const uint32_t count = w.counters[CTR_LEVEL0 + k - 1];
     for (uint32_t pn = blockIdx.x; pn < count; pn += gridDim.x) {
@@ -1419,6 +1430,7 @@ __global__ void __launch_bounds__(256) k_mid_down(WsView w, int k)
 // one CTA per (table, slice); nodes come from the digit-major list, i.e. in ascending parent order
 __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 {
+    tt_pdl_enter();
     extern __shared__ float sm[];
     const int t = blockIdx.y;
     const TableDesc& td = w.tdesc[t];
@@ -1482,6 +1494,7 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 {
+    tt_pdl_enter();
     static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && (COLS % 32 == 0 || COLS == 16), "rows per node; r_{k-1}; columns per warp");
     constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16, 32 or 64 stacked rows per pass
     constexpr bool AHALF = RA == 8;          // dG: a = 8..15 of the one m-tile do not exist: zero operands, not stored
@@ -1646,6 +1659,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
 // which are contiguous in sorted order; one warp per parent
 __global__ void __launch_bounds__(256) k_mid_sum(WsView w, int k)
 {
+    tt_pdl_enter();
     const int lane = threadIdx.x & 31;
     const uint32_t count = w.counters[CTR_LEVEL0 + k - 1];
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -1718,19 +1732,22 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
         auto st = [&]() { return fork ? h->side[(slot++) & 3] : s; };
-        if (any_fast[0]) { k_mid_mma<4, 32, 128><<<sg, 128, 0, st()>>>(w, k, 0); tt_note_launch(); }
-        if (any_fast[1]) { k_mid_mma<4, 16, 128><<<sg, 128, 0, st()>>>(w, k, 1); tt_note_launch(); }
-        if (any_fast[2]) { k_mid_mma<4, 32, 64><<<sg, 128, 0, st()>>>(w, k, 2); tt_note_launch(); }
-        if (any_fast[3]) { k_mid_mma<4, 16, 64><<<sg, 128, 0, st()>>>(w, k, 3); tt_note_launch(); }
-        if (any_fast[4]) { k_mid_mma<2, 32, 128><<<sg, 128, 0, st()>>>(w, k, 4); tt_note_launch(); }
-        if (any_fast[5]) { k_mid_mma<2, 16, 64><<<sg, 128, 0, st()>>>(w, k, 5); tt_note_launch(); }
-        if (any_fast[6]) { k_mid_mma<2, 32, 64><<<sg, 128, 0, st()>>>(w, k, 6); tt_note_launch(); }
-        if (any_fast[7]) { k_mid_mma<2, 16, 32><<<sg, 128, 0, st()>>>(w, k, 7); tt_note_launch(); }
-        if (any_fast[8]) { k_mid_mma<4, 8, 32><<<sg, 128, 0, st()>>>(w, k, 8); tt_note_launch(); }
-        if (any_fast[9]) { k_mid_mma<2, 8, 32><<<sg, 128, 0, st()>>>(w, k, 9); tt_note_launch(); }
-        if (any_fast[10]) { k_mid_mma<2, 8, 16><<<sg, 128, 0, st()>>>(w, k, 10); tt_note_launch(); }
+        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128>, sg, dim3(128), 0, st(), w, k, 0)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[1]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 128>, sg, dim3(128), 0, st(), w, k, 1)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64>, sg, dim3(128), 0, st(), w, k, 2)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[3]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 64>, sg, dim3(128), 0, st(), w, k, 3)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[4]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 128>, sg, dim3(128), 0, st(), w, k, 4)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[5]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 64>, sg, dim3(128), 0, st(), w, k, 5)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[6]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 64>, sg, dim3(128), 0, st(), w, k, 6)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[7]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 32>, sg, dim3(128), 0, st(), w, k, 7)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[8]) { if ((e = tt_launch_pdl(k_mid_mma<4, 8, 32>, sg, dim3(128), 0, st(), w, k, 8)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[9]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 32>, sg, dim3(128), 0, st(), w, k, 9)) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[10]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 16>, sg, dim3(128), 0, st(), w, k, 10)) != cudaSuccess) return e; tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
-        if (nfast > 0) { k_mid_sum<<<h->sm_count * 8, 256, 0, s>>>(w, k); tt_note_launch(); }
+        if (nfast > 0) {
+            if ((e = tt_launch_pdl(k_mid_sum, dim3(h->sm_count * 8), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
+            tt_note_launch();
+        }
         if (any_generic) {
             if ((e = cudaFuncSetAttribute(k_mid_slice, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(max_slice * sizeof(float)))) != cudaSuccess) return e;
             k_mid_slice<<<sg, 256, (size_t)max_slice * sizeof(float), s>>>(w, k);
@@ -1747,6 +1764,7 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
 
 __global__ void __launch_bounds__(256) k_sgd(WsView w, float lr, int only_unfused)
 {
+    tt_pdl_enter();
     const int t = blockIdx.y / w.K, k = blockIdx.y % w.K;
     const TableDesc& td = w.tdesc[t];
     if (only_unfused && ((td.sgd_mask >> k) & 1)) return;   // updated by the kernel that finalised its gradient
