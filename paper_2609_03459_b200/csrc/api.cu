@@ -217,7 +217,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->units_per_table = Q;
     // vlist[0..T): table ids grouped by kernel variant; vlist[T..2T): all tables.  Inside each list the tables come
     // largest first (rows N_t): CTAs of big tables run long, so they should start first and the small ones fill the tail
-    h->vlist_host = (int32_t*)calloc((size_t)2 * T, sizeof(int32_t));
+    h->vlist_host = (int32_t*)calloc((size_t)(2 + TT_MAXK + 1) * T, sizeof(int32_t));
     if (!h->vlist_host) return fail(TT_EMB_ERR_ARG);
     {
         int32_t* all = h->vlist_host + T;
@@ -229,6 +229,21 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
             for (int i = 0; i < T; ++i)
                 if (h->tab[all[i]].fast == vi - 1) h->vlist_host[pos++] = all[i];
             h->vcount[vi] = pos - h->vbase[vi];
+        }
+        // the same grouping by the variant of each middle level's backward kernel
+        for (int k = 2; k <= K - 1; ++k) {
+            int32_t* ml = h->vlist_host + (size_t)(2 + k) * T;
+            int mpos = 0;
+            for (int vi = 0; vi <= TT_NUM_MIDFAST; ++vi) {
+                h->mbase[k][vi] = mpos;
+                h->mmaxn[k][vi] = 1;
+                for (int i = 0; i < T; ++i)
+                    if (h->tab[all[i]].midfast[k] == vi - 1) {
+                        ml[mpos++] = all[i];
+                        if (h->tab[all[i]].n[k - 1] > h->mmaxn[k][vi]) h->mmaxn[k][vi] = h->tab[all[i]].n[k - 1];
+                    }
+                h->mcount[k][vi] = mpos - h->mbase[k][vi];
+            }
         }
     }
     h->gpart_floats = gpart;
@@ -264,7 +279,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->off_counters = h->off_status + 16 * sizeof(uint32_t);
     h->off_tdesc = take((size_t)T * sizeof(TableDesc));
     h->off_tlstart = take((size_t)(T + 1) * sizeof(int64_t));
-    h->off_vlist = take((size_t)2 * T * sizeof(int32_t));
+    h->off_vlist = take((size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t));
     h->off_bm = take((size_t)words * sizeof(uint2));
     uint64_t scan_max = words;
     for (int k = 1; k <= K; ++k) if (v.cap[k] > scan_max) scan_max = v.cap[k];
@@ -395,7 +410,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     }
     // pageable source: the runtime stages it before returning, so h->tab may change afterwards
     TT_CUDA(cudaMemcpyAsync(v.tdesc, h->tab, (size_t)T * sizeof(TableDesc), cudaMemcpyHostToDevice, s));
-    TT_CUDA(cudaMemcpyAsync(v.vlist, h->vlist_host, (size_t)2 * T * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    TT_CUDA(cudaMemcpyAsync(v.vlist, h->vlist_host, (size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     TT_CUDA(cudaMemsetAsync(v.status, 0, (16 + 64) * sizeof(uint32_t), s));
     h->bound = true;
     h->have_forward = false;

@@ -1492,7 +1492,7 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 // add into the CTA's own gradient slice, which stays in L2) every eighth pass, which keeps every chain at 48 or 96
 // products whatever the length of the node list.
 template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
-__global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
+__global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, int lbase)
 {
     tt_pdl_enter();
     static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && (COLS % 32 == 0 || COLS == 16), "rows per node; r_{k-1}; columns per warp");
@@ -1505,7 +1505,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant)
     constexpr int KTY = COLS / 8;            // Y: k steps over c
     __shared__ __align__(16) float sA[2][NQ * M * AP];
     __shared__ __align__(16) float sD[2][NQ * M * CP];
-    const int t_ = w.vlist[w.T + blockIdx.y];   // largest tables first: their long node lists start early
+    const int t_ = w.vlist[lbase + blockIdx.y];   // the tables of this variant, largest first: their long node lists start early
     const TableDesc& td = w.tdesc[t_];
     const int kc = k - 1;
     if (td.midfast[k] != variant || (int)blockIdx.x >= td.n[kc]) return;
@@ -1732,17 +1732,20 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         if (fork && (e = tt_fork(h, s, 4)) != cudaSuccess) return e;
         int slot = 0;
         auto st = [&]() { return fork ? h->side[(slot++) & 3] : s; };
-        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128>, sg, dim3(128), 0, st(), w, k, 0)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[1]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 128>, sg, dim3(128), 0, st(), w, k, 1)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64>, sg, dim3(128), 0, st(), w, k, 2)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[3]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 64>, sg, dim3(128), 0, st(), w, k, 3)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[4]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 128>, sg, dim3(128), 0, st(), w, k, 4)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[5]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 64>, sg, dim3(128), 0, st(), w, k, 5)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[6]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 64>, sg, dim3(128), 0, st(), w, k, 6)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[7]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 32>, sg, dim3(128), 0, st(), w, k, 7)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[8]) { if ((e = tt_launch_pdl(k_mid_mma<4, 8, 32>, sg, dim3(128), 0, st(), w, k, 8)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[9]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 32>, sg, dim3(128), 0, st(), w, k, 9)) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[10]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 16>, sg, dim3(128), 0, st(), w, k, 10)) != cudaSuccess) return e; tt_note_launch(); }
+        // grid of variant v: its own tables only, slices up to the largest n_k among them
+        auto mgrid = [&](int v) { return dim3(h->mmaxn[k][v + 1], h->mcount[k][v + 1]); };
+        auto mlist = [&](int v) { return (2 + k) * h->T + h->mbase[k][v + 1]; };
+        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128>, mgrid(0), dim3(128), 0, st(), w, k, 0, mlist(0))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[1]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 128>, mgrid(1), dim3(128), 0, st(), w, k, 1, mlist(1))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64>, mgrid(2), dim3(128), 0, st(), w, k, 2, mlist(2))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[3]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 64>, mgrid(3), dim3(128), 0, st(), w, k, 3, mlist(3))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[4]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 128>, mgrid(4), dim3(128), 0, st(), w, k, 4, mlist(4))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[5]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 64>, mgrid(5), dim3(128), 0, st(), w, k, 5, mlist(5))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[6]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 64>, mgrid(6), dim3(128), 0, st(), w, k, 6, mlist(6))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[7]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 32>, mgrid(7), dim3(128), 0, st(), w, k, 7, mlist(7))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[8]) { if ((e = tt_launch_pdl(k_mid_mma<4, 8, 32>, mgrid(8), dim3(128), 0, st(), w, k, 8, mlist(8))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[9]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 32>, mgrid(9), dim3(128), 0, st(), w, k, 9, mlist(9))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[10]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 16>, mgrid(10), dim3(128), 0, st(), w, k, 10, mlist(10))) != cudaSuccess) return e; tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (nfast > 0) {
             if ((e = tt_launch_pdl(k_mid_sum, dim3(h->sm_count * 8), dim3(256), 0, s, w, k)) != cudaSuccess) return e;

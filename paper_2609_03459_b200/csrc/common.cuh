@@ -13,6 +13,7 @@
 #define TT_DE_CHUNK 1024                                  // sorted lookups per warp in the dE segment reduction
 #define TT_NUM_STAGES 33                                // 0..8 pipeline stages, 9..20 forward sweep variants -1..10, 21..32 backward sweep variants
 #define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
+#define TT_NUM_MIDFAST 11                                // tensor-core instances of the middle-core backward (backward.cu)
 #define TT_NUM_VARIANTS 11                               // register-tiled shape variants (forward.cu)
 
 // Per-table descriptor, resident in the workspace.  k below is 0-based (core k+1 of the paper).
@@ -110,6 +111,9 @@ struct tt_emb {
     int units_per_table;
     int vcount[TT_NUM_VARIANTS + 1];   // tables per variant, index 0 = generic (-1)
     int vbase[TT_NUM_VARIANTS + 1];    // first entry of each variant in vlist
+    // middle-core kernels of level k: tables grouped by their variant (index 0 = generic), largest first, in
+    // vlist[(2 + k) * T ..); first entry, count and largest n_k of each group
+    int mbase[TT_MAXK + 1][TT_NUM_MIDFAST + 1], mcount[TT_MAXK + 1][TT_NUM_MIDFAST + 1], mmaxn[TT_MAXK + 1][TT_NUM_MIDFAST + 1];
     int32_t* vlist_host;
     size_t off_vlist;
     int cost_shift;       // cost unit of the schedule = 2^cost_shift FMAs
