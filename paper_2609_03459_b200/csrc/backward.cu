@@ -155,8 +155,9 @@ __global__ void __launch_bounds__(256) k_sort_pass(WsView w)
 struct CntScan {
     WsView w;
     __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + w.K]; }
-    __device__ uint32_t value(uint32_t i) const { return w.cnt[i]; }
-    __device__ void emit(uint32_t i, uint32_t excl, uint32_t) const { w.cnt[i] = excl; }
+    __device__ int locate(uint32_t) const { return 0; }
+    __device__ uint32_t value(uint32_t i, int) const { return w.cnt[i]; }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t, int) const { w.cnt[i] = excl; }
     __device__ void total(uint32_t tot) const { w.cnt[size()] = tot; }
 };
 
@@ -1348,8 +1349,9 @@ struct TPopScan {
     WsView w;
     int k;
     __device__ uint32_t size() const { return w.ttotal_words[k]; }
-    __device__ uint32_t value(uint32_t i) const { return __popc(w.tbm[k][i].x); }
-    __device__ void emit(uint32_t i, uint32_t excl, uint32_t) const { w.tbm[k][i].y = excl; }
+    __device__ int locate(uint32_t) const { return 0; }
+    __device__ uint32_t value(uint32_t i, int) const { return __popc(w.tbm[k][i].x); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t, int) const { w.tbm[k][i].y = excl; }
     __device__ void total(uint32_t) const {}
 };
 

@@ -204,6 +204,14 @@ __device__ __forceinline__ int tt_find_table(const uint32_t* __restrict__ tb, in
     return lo;
 }
 
+// the same, starting from a table known not to lie after v's (elements of a tile are ascending: the table of the
+// tile's first element); usually no step at all
+__device__ __forceinline__ int tt_find_table_from(const uint32_t* __restrict__ tb, int T, uint32_t v, int t)
+{
+    while (t + 1 < T && tb[t + 1] <= v) ++t;
+    return t;
+}
+
 __device__ __forceinline__ int tt_find_table64(const int64_t* __restrict__ tb, int T, int64_t v)
 {
     int lo = 0, hi = T;

@@ -22,12 +22,13 @@ struct CostScan {
     WsView w;
     int shift;
     __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + w.K - 1]; }
-    __device__ uint32_t value(uint32_t j) const
+    __device__ int locate(uint32_t j0) const { return tt_find_table(w.tb[w.K - 1], w.T, j0); }
+    __device__ uint32_t value(uint32_t j, int hint) const
     {
         // position j of the sweep order: digit-major for K >= 3 (groups that share the big slice of core K-1 are
         // neighbours, so that slice is fetched from L2 once per run instead of once per group), natural for K = 2
         const int K = w.K;
-        const int t = tt_find_table(w.tb[K - 1], w.T, j);
+        const int t = tt_find_table_from(w.tb[K - 1], w.T, j, hint);
         const uint32_t g = (K >= 3 && !(w.ablation & 1)) ? w.tnode[K - 1][j] : j;
         const TableDesc& td = w.tdesc[t];
         const uint32_t nchild = w.cstart[K - 1][g + 1] - w.cstart[K - 1][g];
@@ -37,7 +38,7 @@ struct CostScan {
         uint64_t c = ((c_mid + (uint64_t)nchild * c_last) >> shift) + 1;
         return (uint32_t)c;
     }
-    __device__ void emit(uint32_t g, uint32_t excl, uint32_t) const { w.cost[g] = excl; }
+    __device__ void emit(uint32_t g, uint32_t excl, uint32_t, int) const { w.cost[g] = excl; }
     __device__ void total(uint32_t tot) const
     {
         w.cost[size()] = tot;

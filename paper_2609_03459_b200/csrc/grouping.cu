@@ -69,21 +69,21 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
 struct PopScan {
     WsView w;
     __device__ uint32_t size() const { return w.total_words; }
-    __device__ uint32_t value(uint32_t i) const { return __popc(w.bm[i].x); }
-    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v) const
+    // every table starts on a scan-tile boundary: the table of a tile's first word is the table of all its words
+    __device__ int locate(uint32_t i0) const
+    {
+        int lo = 0, hi = w.T;
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (w.tdesc[mid].word_base <= i0) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+    __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bm[i].x); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
     {
         w.bm[i].y = excl;
         const int K = w.K;
-        // every table starts on a scan-tile boundary, so this search is uniform within a CTA
-        int t = 0;
-        {
-            int lo = 0, hi = w.T;
-            while (hi - lo > 1) {
-                int mid = (lo + hi) >> 1;
-                if (w.tdesc[mid].word_base <= i) lo = mid; else hi = mid;
-            }
-            t = lo;
-        }
         const uint32_t wb = w.tdesc[t].word_base;
         if (i == wb) w.tb[K][t] = excl < w.cap[K] ? excl : w.cap[K];
         if (v) {
@@ -113,19 +113,20 @@ struct LevelUp {
     WsView w;
     int k;  // level being produced (1..K-1); reads level k+1
     __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + k + 1]; }
-    __device__ uint32_t value(uint32_t v) const
+    __device__ int locate(uint32_t v0) const { return tt_find_table(w.tb[k + 1], w.T, v0); }
+    __device__ uint32_t value(uint32_t v, int hint) const
     {
         const uint32_t* tbc = w.tb[k + 1];
-        const int t = tt_find_table(tbc, w.T, v);
+        const int t = tt_find_table_from(tbc, w.T, v, hint);
         const uint32_t nk = (uint32_t)w.tdesc[t].n[k];  // radix of digit k+1 (0-based core index k)
         if (v == tbc[t]) return 1u;
         if ((w.ablation & 1) && k == w.K - 1) return 1u;   // study switch: no prefix reuse, every row opens a group
         return (w.val[k + 1][v] / nk != w.val[k + 1][v - 1] / nk) ? 1u : 0u;
     }
-    __device__ void emit(uint32_t v, uint32_t excl, uint32_t flag) const
+    __device__ void emit(uint32_t v, uint32_t excl, uint32_t flag, int hint) const
     {
         const uint32_t* tbc = w.tb[k + 1];
-        const int t = tt_find_table(tbc, w.T, v);
+        const int t = tt_find_table_from(tbc, w.T, v, hint);
         w.parent[k + 1][v] = excl + flag - 1u;
         if (flag) {
             w.val[k][excl] = w.val[k + 1][v] / (uint32_t)w.tdesc[t].n[k];

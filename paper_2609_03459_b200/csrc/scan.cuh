@@ -3,8 +3,10 @@
 //
 // Functor F:
 //   __device__ uint32_t size() const;                       number of elements (may read device memory)
-//   __device__ uint32_t value(uint32_t i) const;            input i
-//   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v) const;   called once per element in the apply pass
+//   __device__ int locate(uint32_t i0) const;               once per tile, for its first element: a hint handed to value / emit
+//                                                           (e.g. the table the tile starts in, so that elements need no search)
+//   __device__ uint32_t value(uint32_t i, int hint) const;  input i
+//   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int hint) const;   called once per element in the apply pass
 //   __device__ void total(uint32_t tot) const;              called by one thread with the grand total
 //   WsView w;                                               w.counters[CTR_SCAN_TICKET] is the ticket (zero between scans)
 #pragma once
@@ -69,11 +71,12 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
     if (blockIdx.x >= ntiles) return;
     const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
     uint32_t s = 0;
+    const int hint = f.locate((uint32_t)base);
     // a sum has no order: neighbouring threads take neighbouring elements (coalesced)
 #pragma unroll 4
     for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
-        if (i < n) s += f.value((uint32_t)i);
+        if (i < n) s += f.value((uint32_t)i, hint);
     }
     uint32_t tot;
     tt_block_excl_scan(s, sm, tot);
@@ -105,10 +108,11 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint
     const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
     if (base >= n) return;
     uint32_t v[TT_SCAN_ITEMS];
+    const int hint = f.locate((uint32_t)base);
 #pragma unroll
     for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
-        v[j] = i < n ? f.value((uint32_t)i) : 0u;
+        v[j] = i < n ? f.value((uint32_t)i, hint) : 0u;
         sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)] = v[j];
     }
     __syncthreads();
@@ -130,7 +134,7 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint
 #pragma unroll
     for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
-        if (i < n) f.emit((uint32_t)i, sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)], v[j]);
+        if (i < n) f.emit((uint32_t)i, sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)], v[j], hint);
     }
 }
 
