@@ -41,6 +41,9 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
     const int64_t step = (int64_t)gridDim.x * blockDim.x * 4;
     int t = 0;
     bool bad = false;
+    // the table of the last lookup, kept in registers: lookup range, row count, first presence word
+    int64_t l_lo = 0, l_hi = 0, tN = 0;
+    uint32_t twb = 0;
     for (int64_t base = (int64_t)blockIdx.x * blockDim.x * 4 + threadIdx.x; base < L; base += step) {
         int64_t g[4];
 #pragma unroll
@@ -52,11 +55,16 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
         for (int j = 0; j < 4; ++j) {
             const int64_t l = base + (int64_t)j * blockDim.x;
             if (l >= L) continue;
-            if (!(w.tl_start[t] <= l && l < w.tl_start[t + 1])) t = tt_find_table64(w.tl_start, w.T, l);
-            const TableDesc& td = w.tdesc[t];
-            if (g[j] < 0 || g[j] >= td.N) { bad = true; continue; }
+            if (!(l_lo <= l && l < l_hi)) {
+                t = tt_find_table64(w.tl_start, w.T, l);
+                l_lo = w.tl_start[t];
+                l_hi = w.tl_start[t + 1];
+                tN = w.tdesc[t].N;
+                twb = w.tdesc[t].word_base;
+            }
+            if (g[j] < 0 || g[j] >= tN) { bad = true; continue; }
             const uint32_t row = (uint32_t)g[j];
-            unsigned* word = &w.bm[td.word_base + (row >> 5)].x;
+            unsigned* word = &w.bm[twb + (row >> 5)].x;
             const unsigned m = 1u << (row & 31);
             if (!(__ldca(word) & m)) atomicOr(word, m);   // L1 may hold a stale word: at worst a redundant atomic
         }
