@@ -474,7 +474,7 @@ def main():
     # DRAM traffic per lookup / per distinct row of the top kernels, from the ncu capture of the reduced case
     # (8 tables; profiles/ncu_full_cfg5_reduced.md), scaled to this launch by the units it processes.
     NCU_TRAFFIC = {"k_pool": ("lookup", 98.2), "k_dE": ("lookup", 78.1),
-                   "k_sweep_fwd": ("row", 230.4), "k_sweep_bwd": ("row", 335.4)}
+                   "k_sweep_fwd": ("row", 231.0), "k_sweep_bwd": ("row", 335.6)}
     pool_kernel = "k_pool_async" if 16 < D <= 64 and D % 4 == 0 else "k_pool_vec"
 
     def traffic_of(kernel, share=1.0):
