@@ -230,6 +230,25 @@ def run_reference(args, wl, train, desc, rank, world):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------------ launcher
+
+def launch_ranks(n: int) -> int:
+    """Re-run this command line as n ranks (torch.distributed.run, one process per GPU, rendezvous on 127.0.0.1).
+    Fails before starting anything when the node has fewer than n GPUs.  Returns the exit code."""
+    import socket
+    import torch
+    have = torch.cuda.device_count()
+    if have < n:
+        print(f"bench.py: --gpus {n} needs {n} GPUs on this node, {have} visible; not running on fewer", file=sys.stderr)
+        return 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd).returncode
+
+
 # ------------------------------------------------------------------------------------------------ main arm
 
 def main():
@@ -251,9 +270,14 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # called plainly with --gpus N: start the N ranks ourselves (one process per GPU) and hand over
+        raise SystemExit(launch_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "ours" and world != max(args.gpus, 1):
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}: launch one rank per GPU")
     cfg_id, train, desc = WORKLOADS[args.workload]
 
     if args.impl == "reference":
@@ -269,9 +293,16 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    if torch.cuda.device_count() < world or local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: {world} ranks asked for, {torch.cuda.device_count()} GPUs visible "
+                         "(one rank per GPU; nothing is run on fewer)")
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
+        # communicator set-up lines (rings / trees / NVLS) go to stderr: the JSON line stays alone on stdout
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT,GRAPH")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
         dist.init_process_group("nccl", device_id=device)
 
     # every rank draws its own batch from the same recipe (weak scaling); tables/cores are identical
@@ -283,6 +314,7 @@ def main():
     if rank > 0:
         wl = workloads.make(cfg_id, mapping=args.mapping, batch_seed=ttd.rank_seed(workloads.BASE_SEED, rank), **shrink)
     T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
+    L_all = ttd.sum_over_ranks(L, device=device) if world > 1 else L   # lookups of the whole job (every rank has its own batch)
 
     abl = {"none": 0, "unique-only": 1, "static": 2, "unique-only+static": 3}[args.ablation]
     if abl and train:
@@ -459,9 +491,9 @@ def main():
         h_idx32 = h_idx.to(torch.int32).pin_memory()
         e2e32_ms = run_e2e(h_idx32)
         h2d = h_idx.numel() * 8 + h_off.numel() * 8 + (h_grad.numel() * 4 if train else 0)
-        e2e = {"value": world * L / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": L_all / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(h_out.numel() * 4),
-               "int32_ids": {"value": world * L / (e2e32_ms * 1e-3), "ms_per_step": e2e32_ms,
+               "int32_ids": {"value": L_all / (e2e32_ms * 1e-3), "ms_per_step": e2e32_ms,
                              "h2d_bytes_per_step": int(h2d - h_idx.numel() * 4)}}
     clocks = sampler.stop()
 
@@ -556,14 +588,14 @@ def main():
     fwd_roof_t = max(work["fwd_slots"] / fp32_peak, work["fwd_hbm_bytes"] / (hbm_gbs * 1e9), work["fwd_l2_bytes"] / l2_gather)
 
     line = {
-        "metric": METRIC, "value": world * L / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": L_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": desc, "mapping": args.mapping, "tables": T, "batch_per_gpu": B, "lookups_per_gpu": L,
                    "step": "forward+backward+sgd" if train else "forward", "ablation": args.ablation,
                    "parallelism": f"dp{world} (batch-sharded replicas" + (", all-reduce of core gradients)" if train else ")"),
                    "l2_policy": "inputs larger than L2 (indices alone are %.0f MB)" % (L * 8 / 1e6)},
-        "forward_only": {"value": world * L / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,
+        "forward_only": {"value": L_all / (fwd_ms * 1e-3), "unit": UNIT, "ms_per_step": fwd_ms,
                          "roofline_frac": fwd_roof_t * 1e3 / fwd_ms, "t_roof_ms": fwd_roof_t * 1e3,
                          "cuda_graph_ms_per_step": fwd_graph_ms},
         "stage_ms": stage_ms, "solo_kernel_ms": solo_ms, "roofline": roofline, "kernel_rooflines": kernel_rooflines, "step_roofline": step_roof,

@@ -2,7 +2,9 @@
 
 Only tests, the smoke check and the benchmark's CPU legs may import this package.  It never imports
 the CUDA package and the CUDA package never imports it.  The arithmetic lives in `tt_oracle.c`
-(plain C, one lookup at a time); this file marshals numpy arrays and holds the integer grouping oracle
+(plain C, one lookup at a time) and in `tt_oracle_memo.c` (the same definition with each distinct row built
+once, so that the full-size configurations finish in test time; the two files share no code and are compared
+with each other by the tests); this file marshals numpy arrays and holds the integer grouping oracle
 (Sec. 3.3: sort, unique, mixed radix, run-length encoding), written with numpy's sort as the one
 library primitive.
 
@@ -20,14 +22,18 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "libtt_oracle.so")
 _SRC = os.path.join(_HERE, "tt_oracle.c")
+_SO_MEMO = os.path.join(_HERE, "libtt_oracle_memo.so")
+_SRC_MEMO = os.path.join(_HERE, "tt_oracle_memo.c")
 _lib = None
+_lib_memo = None
 
 
 def build(force: bool = False) -> str:
-    """Compile tt_oracle.c with gcc into libtt_oracle.so (next to the source)."""
-    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", _SO, _SRC, "-lm"]
-        subprocess.run(cmd, check=True)
+    """Compile tt_oracle.c and tt_oracle_memo.c with gcc into shared libraries next to the sources."""
+    for so, src, opt in ((_SO, _SRC, "-O2"), (_SO_MEMO, _SRC_MEMO, "-O3")):
+        if force or not os.path.exists(so) or os.path.getmtime(so) < os.path.getmtime(src):
+            cmd = ["gcc", opt, "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", so, src, "-lm"]
+            subprocess.run(cmd, check=True)
     return _SO
 
 
@@ -39,6 +45,16 @@ def lib():
         _lib.tt_oracle_forward.restype = ctypes.c_int64
         _lib.tt_oracle_backward.restype = ctypes.c_int64
     return _lib
+
+
+def lib_memo():
+    global _lib_memo
+    if _lib_memo is None:
+        build()
+        _lib_memo = ctypes.CDLL(_SO_MEMO)
+        _lib_memo.tt_memo_forward.restype = ctypes.c_int64
+        _lib_memo.tt_memo_backward.restype = ctypes.c_int64
+    return _lib_memo
 
 
 def _i64(a) -> np.ndarray:
@@ -87,8 +103,9 @@ def _weights_arg(weights, L):
     return w, _p(w)
 
 
-def forward(n, d, r, N, cores, indices, offsets, weights=None, mode: str = "sum") -> np.ndarray:
-    """Pooled rows of one table: fp64 [B, D].  weights: per-lookup factors [L]; mode "sum" (the paper) or "mean"."""
+def forward(n, d, r, N, cores, indices, offsets, weights=None, mode: str = "sum", memo: bool = False) -> np.ndarray:
+    """Pooled rows of one table: fp64 [B, D].  weights: per-lookup factors [L]; mode "sum" (the paper) or "mean".
+    memo=True: the memoised oracle (every distinct row built once) instead of the plain per-lookup one."""
     _check(n, d, r, cores)
     nn, dd, rr = _i64(n), _i64(d), _i64(r)
     idx, off = _i64(indices), _i64(offsets)
@@ -97,14 +114,17 @@ def forward(n, d, r, N, cores, indices, offsets, weights=None, mode: str = "sum"
     keep, cp = _core_ptrs(cores)
     out = np.zeros((B, D), dtype=np.float64)
     wkeep, wp = _weights_arg(weights, idx.shape[0])
-    lib().tt_oracle_forward(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
+    fn = lib_memo().tt_memo_forward if memo else lib().tt_oracle_forward
+    fn(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
                             _p(idx), _p(off), ctypes.c_int64(B), _p(out), ctypes.c_int64(D), wp,
                             ctypes.c_int(1 if mode == "mean" else 0))
     return out
 
 
-def backward(n, d, r, N, cores, indices, offsets, grad_out, weights=None, mode: str = "sum") -> List[np.ndarray]:
-    """Core gradients of one table for loss = sum(grad_out * out): list of fp64 arrays shaped like the cores."""
+def backward(n, d, r, N, cores, indices, offsets, grad_out, weights=None, mode: str = "sum",
+             memo: bool = False) -> List[np.ndarray]:
+    """Core gradients of one table for loss = sum(grad_out * out): list of fp64 arrays shaped like the cores.
+    memo=True: the memoised oracle (grad_out summed per distinct row first, one backward chain per distinct row)."""
     _check(n, d, r, cores)
     nn, dd, rr = _i64(n), _i64(d), _i64(r)
     idx, off = _i64(indices), _i64(offsets)
@@ -116,7 +136,8 @@ def backward(n, d, r, N, cores, indices, offsets, grad_out, weights=None, mode: 
     grads = [np.zeros(c.shape, dtype=np.float64) for c in keep]
     gp = (ctypes.c_void_p * len(grads))(*[g.ctypes.data for g in grads])
     wkeep, wp = _weights_arg(weights, idx.shape[0])
-    lib().tt_oracle_backward(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
+    fn = lib_memo().tt_memo_backward if memo else lib().tt_oracle_backward
+    fn(ctypes.c_int(len(n)), _p(nn), _p(dd), _p(rr), ctypes.c_int64(int(N)), cp,
                              _p(idx), _p(off), ctypes.c_int64(B), _p(go), ctypes.c_int64(D), gp, wp,
                              ctypes.c_int(1 if mode == "mean" else 0))
     return grads
@@ -151,7 +172,7 @@ def _table_weights(wl, t, weights):
     return np.asarray(weights)[lo:hi]
 
 
-def forward_workload(wl, tables=None, bags=None, weights=None, mode: str = "sum") -> np.ndarray:
+def forward_workload(wl, tables=None, bags=None, weights=None, mode: str = "sum", memo: bool = False) -> np.ndarray:
     """out fp64 [B, T*D] for a workloads.Workload (optionally only some tables; others stay zero).
     weights: per-lookup factors aligned with wl.indices."""
     D = wl.D
@@ -160,11 +181,12 @@ def forward_workload(wl, tables=None, bags=None, weights=None, mode: str = "sum"
         s = wl.tables[t]
         idx, off = wl.table_slice(t)
         out[:, t * D:(t + 1) * D] = forward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off,
-                                            _table_weights(wl, t, weights), mode)
+                                            _table_weights(wl, t, weights), mode, memo)
     return out
 
 
-def backward_workload(wl, grad_out=None, tables=None, weights=None, mode: str = "sum") -> List[List[np.ndarray]]:
+def backward_workload(wl, grad_out=None, tables=None, weights=None, mode: str = "sum",
+                      memo: bool = False) -> List[List[np.ndarray]]:
     go = wl.grad_out if grad_out is None else grad_out
     D = wl.D
     res = []
@@ -172,7 +194,7 @@ def backward_workload(wl, grad_out=None, tables=None, weights=None, mode: str = 
         s = wl.tables[t]
         idx, off = wl.table_slice(t)
         res.append(backward(s.n, s.d, s.r, s.N, wl.cores[t], idx, off, go[:, t * D:(t + 1) * D],
-                            _table_weights(wl, t, weights), mode))
+                            _table_weights(wl, t, weights), mode, memo))
     return res
 
 

@@ -1,13 +1,13 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: EVERY element of `out`,
+of every core gradient and of every core after the SGD step is compared with the fp64 oracle.
 
-The plain oracle cannot redo a whole 99-million-lookup batch in test time, so outputs are sampled:
-  * forward: pooled rows of sampled (table, bag) pairs, recomputed one by one by the oracle;
-  * grouping: distinct-row / prefix counts of every table against numpy sets; sampled tables in full;
-  * backward: gradient slices of sampled (table, core, digit) triples.  A slice of core k with digit value i
-    only receives contributions from lookups whose k-th digit is i, so the oracle's per-lookup backward over
-    exactly those lookups (each as its own bag with its bag's grad_out row) gives the slice exactly;
-  * SGD: the same slices of the updated cores.
-Tolerance: max|err| <= 1e-5 * max|ref| per compared tensor."""
+  * configs 1, 2, 4 (single table): the plain per-lookup oracle redoes the whole batch (seconds), and the
+    memoised oracle must agree with it on the same full inputs;
+  * configs 3 and 5 (60 tables, 99 million lookups; identity and scattered rank -> row mapping): the memoised
+    oracle (every distinct row built once, grad_out summed per distinct row in fp64; pinned against the plain
+    oracle by the CPU tests, among them a 1/64 sub-sample of this very batch);
+  * grouping: distinct-row / prefix counts of every table against numpy sets, sampled tables in full.
+Tolerance: max|err| <= 1e-5 * max|ref| per compared tensor (per table block of `out`, per core gradient, per core)."""
 import numpy as np
 import pytest
 
@@ -42,23 +42,6 @@ def close(got, ref, what):
     return err / max(scale, 1e-300)
 
 
-def sample_pairs(wl, n, seed):
-    rng = np.random.default_rng(seed)
-    pairs = [(int(rng.integers(wl.T)), int(rng.integers(wl.B))) for _ in range(n)]
-    lens = wl.offsets[1:] - wl.offsets[:-1]
-    # make sure the longest and the shortest bag are in the sample
-    for pick in (int(np.argmax(lens)), int(np.argmin(lens))):
-        pairs.append((pick // wl.B, pick % wl.B))
-    return pairs
-
-
-def check_forward_samples(wl, out, n=192, seed=0):
-    pairs = sample_pairs(wl, n, seed)
-    ref = oracle.forward_bags(wl, pairs)
-    got = np.stack([out[b, t * wl.D:(t + 1) * wl.D] for t, b in pairs])
-    return close(got, ref, f"{wl.name} sampled bags")
-
-
 def check_counts(emb, wl, full_tables=()):
     counts = emb.grouping_counts()
     for t, s in enumerate(wl.tables):
@@ -82,6 +65,36 @@ def check_counts(emb, wl, full_tables=()):
         np.testing.assert_array_equal(emb.export_inverse(t, idx.shape[0]), g["inv"])
 
 
+def check_out_all(wl, out, ref, what):
+    """Every pooled output, table block by table block (the scale of a block is its own largest reference value)."""
+    worst = 0.0
+    D = wl.D
+    for t in range(wl.T):
+        worst = max(worst, close(out[:, t * D:(t + 1) * D], ref[:, t * D:(t + 1) * D], f"{what} out, table {t}"))
+    return worst
+
+
+def check_training_all(wl, emb, ref_grads, what):
+    """Every gradient entry and every core entry after the update, tensor by tensor."""
+    grads = emb.get_grads()
+    cores = emb.get_cores()
+    worst = 0.0
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref_grads[t], wl.lr)
+        for k in range(wl.tables[t].K):
+            worst = max(worst, close(grads[t][k], ref_grads[t][k], f"{what} grad[{t}][{k}]"))
+            close(cores[t][k], want[k], f"{what} core[{t}][{k}] after SGD")
+    # slices of padding digits (never looked up) must have exactly zero gradient and unchanged cores
+    for t in range(wl.T):
+        s = wl.tables[t]
+        rest = int(np.prod(s.n[1:]))
+        last_i1 = (s.N - 1) // rest
+        if last_i1 + 1 < s.n[0]:
+            assert np.count_nonzero(grads[t][0][:, last_i1 + 1:]) == 0
+            np.testing.assert_array_equal(cores[t][0][:, last_i1 + 1:], wl.cores[t][0][:, last_i1 + 1:])
+    return worst
+
+
 def test_config1_full(binding):
     wl = workloads.make(1)
     emb = binding.from_workload(wl)
@@ -92,88 +105,65 @@ def test_config1_full(binding):
 
 
 @pytest.mark.parametrize("cfg", [2, 4])
-def test_single_table_configs_sampled(binding, cfg):
-    wl = workloads.make(cfg)
+@pytest.mark.parametrize("mapping", ["identity", "scattered"])
+def test_single_table_configs_full(binding, cfg, mapping):
+    wl = workloads.make(cfg, mapping=mapping)
     emb = binding.from_workload(wl)
     out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
     assert emb.status() == 0
-    check_forward_samples(wl, out, n=160, seed=cfg)
+    ref = oracle.forward_workload(wl)                    # the plain per-lookup oracle over the whole batch
+    close(out, ref, f"cfg{cfg} {mapping} out (all bags)")
+    memo = oracle.forward_workload(wl, memo=True)        # the two oracles agree on the full inputs as well
+    np.testing.assert_allclose(memo, ref, rtol=1e-11, atol=1e-13 * np.abs(ref).max())
     check_counts(emb, wl, full_tables=(0,))
-    # pooled sums are additive: the column sums of `out` equal the multiplicity-weighted sum of distinct rows
-    s = wl.tables[0]
-    uniq, mult = np.unique(wl.indices, return_counts=True)
-    pick = np.random.default_rng(1).choice(uniq.shape[0], size=min(2000, uniq.shape[0]), replace=False)
-    rows = oracle.forward(s.n, s.d, s.r, s.N, wl.cores[0], uniq[pick], np.arange(pick.shape[0] + 1))
-    assert np.isfinite(out).all() and rows.shape[1] == wl.D
 
 
-@pytest.fixture(scope="module")
-def cfg5():
-    return workloads.make(5)
+class _Full:
+    """The 60-table training workload of one mapping with its oracle results (memoised oracle, fp64)."""
+    def __init__(self, mapping):
+        self.wl = workloads.make(5, mapping=mapping)
+        self.ref_out = oracle.forward_workload(self.wl, memo=True)
+        self.ref_grads = oracle.backward_workload(self.wl, memo=True)
 
 
-def test_config3_forward_sampled(binding, cfg5):
-    wl = cfg5
-    emb = binding.from_workload(wl)
+@pytest.fixture(scope="module", params=["identity", "scattered"])
+def full(request):
+    f = _Full(request.param)
+    yield f
+    del f
+
+
+def test_config3_forward_every_output(binding, full):
+    wl = full.wl
+    emb = binding.from_workload(wl)                       # forward-only handle: the launch configuration of config 3
     out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
     assert emb.status() == 0
-    check_forward_samples(wl, out, n=400, seed=3)
+    check_out_all(wl, out, full.ref_out, f"cfg3 {wl.mapping}")
     check_counts(emb, wl, full_tables=(0, 17))
     del emb
 
 
-def _slice_lookups(wl, t, k, i):
-    """Lookups of table t whose k-th (0-based) digit is i, with their bag ids."""
-    s = wl.tables[t]
-    idx, off = wl.table_slice(t)
-    suffix = int(np.prod(s.n[k + 1:])) if k + 1 < s.K else 1
-    sel = np.nonzero((idx // suffix) % s.n[k] == i)[0]
-    bags = np.searchsorted(off, sel, side="right") - 1
-    return idx[sel], bags
-
-
-def test_config5_training_step_sampled_slices(binding, cfg5):
-    wl = cfg5
-    D = wl.D
+def test_config5_training_step_every_gradient_and_core(binding, full):
+    wl = full.wl
     emb = binding.from_workload(wl, enable_backward=True)
     out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
     emb.backward_sgd(dev(wl.grad_out), wl.lr)     # the call the benchmark's training step makes
-    grads = emb.get_grads()
-    cores = emb.get_cores()
     assert emb.status() == 0
-    check_forward_samples(wl, out.cpu().numpy(), n=64, seed=5)
-    rng = np.random.default_rng(55)
-    worst = 0.0
-    checked = 0
-    hot = 0
-    for t in rng.choice(wl.T, size=8, replace=False):
-        s = wl.tables[t]
-        for k in range(s.K):
-            digits = {int(rng.integers(s.n[k]))}
-            if k == s.K - 1 and hot < 3:
-                digits.add(0)      # the slice the most popular rows select: sums of ~10^5 terms in fp32
-                hot += 1
-            for i in digits:
-                rows, bags = _slice_lookups(wl, t, k, i)
-                if rows.shape[0] == 0 or rows.shape[0] > 400_000:
-                    continue
-                go = wl.grad_out[bags, t * D:(t + 1) * D]
-                ref = oracle.backward(s.n, s.d, s.r, s.N, wl.cores[t], rows, np.arange(rows.shape[0] + 1), go)
-                ref_slice = ref[k][:, i]
-                full_scale = np.abs(ref[k]).max()
-                got_slice = grads[t][k][:, i]
-                err = np.abs(got_slice - ref_slice).max()
-                assert err <= TOL * max(full_scale, 1e-300), (t, k, i, err, full_scale)
-                worst = max(worst, err / max(full_scale, 1e-300))
-                want_core = oracle.sgd([wl.cores[t][k][:, i]], [ref_slice], wl.lr)[0]
-                close(cores[t][k][:, i], want_core, f"core[{t}][{k}] slice {i} after SGD")
-                checked += 1
-    assert checked >= 12
-    # slices of padding digits (never looked up) must have exactly zero gradient and unchanged cores
-    for t in range(wl.T):
-        s = wl.tables[t]
-        if s.n[0] * s.n[1] * s.n[2] > s.N:
-            last_i1 = (s.N - 1) // (s.n[1] * s.n[2])
-            if last_i1 + 1 < s.n[0]:
-                assert np.count_nonzero(grads[t][0][:, last_i1 + 1:]) == 0
-                np.testing.assert_array_equal(cores[t][0][:, last_i1 + 1:], wl.cores[t][0][:, last_i1 + 1:])
+    check_out_all(wl, out.cpu().numpy(), full.ref_out, f"cfg5 {wl.mapping}")
+    del out
+    check_training_all(wl, emb, full.ref_grads, f"cfg5 {wl.mapping}")
+    del emb
+
+
+def test_config5_separate_backward_and_update_every_gradient_and_core(binding, full):
+    # the three calls of the multi-GPU step (backward, [all-reduce], sgd_step) instead of the fused one
+    wl = full.wl
+    if wl.mapping != "identity":
+        pytest.skip("one mapping is enough for the unfused call sequence")
+    emb = binding.from_workload(wl, enable_backward=True)
+    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    emb.backward(dev(wl.grad_out))
+    emb.sgd_step(wl.lr)
+    assert emb.status() == 0
+    check_training_all(wl, emb, full.ref_grads, "cfg5 unfused")
+    del emb
