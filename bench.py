@@ -44,7 +44,34 @@ WORKLOADS = {
     "cfg3": (3, False, "config 3: 60 tables N~logU[1e4,4e7], D=64, ranks {16,32}, batch 32768, pooling U[1,100], Zipf U[0.8,1.2], forward"),
     "cfg4": (4, False, "config 4: 1 table 64^4, D=128, ranks [1,64,64,64,1], batch 65536, pooling 8, Zipf 1.2, forward"),
     "cfg5": (5, True, "config 5: config-3 tables and indices, forward + backward (grad_out N(0,1)) + SGD lr 0.01"),
+    # a shape outside the register-tiled kernel variants: what a user of the any-shape path gets
+    "generic": (0, True, "generic path: 8 tables of the config-3 recipe with dim factors 3x3x5 (D=45), ranks [1,6,4,1], "
+                         "batch 32768, pooling U[1,100], forward + backward + SGD"),
 }
+
+
+def make_workload(cfg_id, mapping, num_tables=None, batch=None, batch_seed=None):
+    if cfg_id == 0:
+        if batch_seed is not None:
+            raise SystemExit("the generic workload is a single-GPU measurement")
+        return workloads.generic_point(batch or 32768, num_tables=num_tables or 8, mapping=mapping)
+    return workloads.make(cfg_id, mapping=mapping, num_tables=num_tables, batch=batch, batch_seed=batch_seed)
+
+
+def dram_traffic_per_unit():
+    """DRAM bytes per lookup / per distinct row of the gather and sweep kernels from the tracked ncu summary
+    (profiles/dram_traffic_per_unit.txt: `kernel unit bytes` lines plus the shape the capture was taken on)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic_per_unit.txt")
+    res, shape = {}, {}
+    if not os.path.exists(path):
+        return res, shape
+    for ln in open(path):
+        f = ln.split("#")[0].split()
+        if len(f) == 3 and f[1] in ("lookup", "row"):
+            res[f[0]] = (f[1], float(f[2]))
+        elif len(f) == 2 and f[0].startswith("capture_"):
+            shape[f[0]] = f[1]
+    return res, shape
 
 
 # ------------------------------------------------------------------------------------------------ helpers
@@ -262,8 +289,8 @@ def main():
     ap.add_argument("--cpu-stride", type=int, default=0, help="bag stride of the oracle sample (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--ablation", default="none", choices=["none", "unique-only", "static", "unique-only+static"],
-                    help="study switches (forward workloads only): no prefix reuse / equal-count schedule")
+    ap.add_argument("--ablation", default="none", choices=["none", "unique-only", "static", "unique-only+static", "no-dedup"],
+                    help="study switches (forward workloads only): no prefix reuse / equal-count schedule / no de-duplication")
     ap.add_argument("--num-tables", type=int, default=0, help="reduced case for profiler captures: fewer tables (cfg3/cfg5)")
     ap.add_argument("--batch", type=int, default=0, help="reduced case for profiler captures: smaller batch")
     args = ap.parse_args()
@@ -283,7 +310,7 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        wl = workloads.make(cfg_id, mapping=args.mapping)
+        wl = make_workload(cfg_id, args.mapping)
         run_reference(args, wl, train, desc, rank, world)
         return
 
@@ -307,19 +334,23 @@ def main():
 
     # every rank draws its own batch from the same recipe (weak scaling); tables/cores are identical
     shrink = dict(num_tables=args.num_tables or None, batch=args.batch or None)
-    wl = workloads.make(cfg_id, mapping=args.mapping, **shrink) if rank == 0 else None
+    wl = make_workload(cfg_id, args.mapping, **shrink) if rank == 0 else None
     if shrink["num_tables"] or shrink["batch"]:
         desc += f" [REDUCED: tables={shrink['num_tables'] or 'all'}, batch={shrink['batch'] or 'full'}]"
     from paper_2609_03459_b200 import dist as ttd
     if rank > 0:
-        wl = workloads.make(cfg_id, mapping=args.mapping, batch_seed=ttd.rank_seed(workloads.BASE_SEED, rank), **shrink)
+        wl = make_workload(cfg_id, args.mapping, batch_seed=ttd.rank_seed(workloads.BASE_SEED, rank), **shrink)
     T, K, D, B, L = wl.T, wl.tables[0].K, wl.D, wl.B, wl.L
     L_all = ttd.sum_over_ranks(L, device=device) if world > 1 else L   # lookups of the whole job (every rank has its own batch)
 
-    abl = {"none": 0, "unique-only": 1, "static": 2, "unique-only+static": 3}[args.ablation]
+    abl = {"none": 0, "unique-only": 1, "static": 2, "unique-only+static": 3, "no-dedup": 4}[args.ablation]
     if abl and train:
         raise SystemExit("--ablation needs a forward workload (cfg1..cfg4)")
-    emb = binding.from_workload(wl, enable_backward=train, ablation=abl, device=device)
+    # Room for distinct rows: the safe bound min(L, sum N) would size the row buffer for 99 M rows (25 GB) on the 60-table
+    # workload, whose batches hold about 0.2 L distinct rows.  Large batches get L / 4 rows; a batch with more would set the
+    # overflow status bit, which is checked below.
+    mur = 0 if (abl & 4) else max(L // 4, min(L, 1 << 22))
+    emb = binding.from_workload(wl, enable_backward=train, ablation=abl, max_unique_rows=mur, device=device)
     h_idx = torch.from_numpy(wl.indices).pin_memory()
     h_off = torch.from_numpy(wl.offsets).pin_memory()
     h_grad = torch.from_numpy(wl.grad_out).pin_memory() if train else None
@@ -367,6 +398,8 @@ def main():
         step(d_idx, d_off, d_grad)
     torch.cuda.synchronize()
     status = emb.status()
+    if status & binding.STATUS_OVERFLOW:
+        raise SystemExit("bench.py: more distinct rows than max_unique_rows; the timed work would be incomplete")
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -503,30 +536,28 @@ def main():
     work = algorithmic_work(wl, counts, train)
 
     # ---- roofline of the dominant kernel and of the whole step
-    # DRAM traffic per lookup / per distinct row of the top kernels, from the ncu capture of the reduced case
-    # (8 tables; profiles/ncu_full_cfg5_reduced.md), scaled to this launch by the units it processes.
-    NCU_TRAFFIC = {"k_pool": ("lookup", 98.2), "k_dE": ("lookup", 78.1),
-                   "k_sweep_fwd": ("row", 231.0), "k_sweep_bwd": ("row", 335.6)}
-    pool_kernel = "k_pool_async" if 16 < D <= 64 and D % 4 == 0 else "k_pool_vec"
+    # DRAM traffic per lookup / per distinct row of the top kernels comes from the tracked ncu summary of a reduced case
+    # and is scaled by the units this launch processes; it is reported only for the shape the capture was taken on.
+    ncu_traffic, capture = dram_traffic_per_unit()
+    pool_kernel = "k_pool_async" if 16 < D <= 64 and D % 4 == 0 else ("k_pool_vec" if D % 4 == 0 else "k_pool_scalar")
+    same_shape = capture.get("capture_D") == str(D) and capture.get("capture_recipe") in ("cfg3", "cfg5") and cfg_id in (3, 5)
 
     def traffic_of(kernel, share=1.0):
-        unit, per = NCU_TRAFFIC[kernel]
+        if not same_shape or kernel not in ncu_traffic:
+            return None
+        unit, per = ncu_traffic[kernel]
         return per * (wl.L if unit == "lookup" else work["U_rows"] * share)
 
-    # (P_{K-1}, r_{K-1}) -> sweep kernel variant (last dim factor 4, at least 3 cores)
-    VARIANT_OF = {(16, 32): 0, (16, 16): 1, (16, 8): 2, (32, 32): 3, (32, 64): 4, (8, 32): 5, (8, 16): 6, (8, 8): 7, (4, 32): 8, (4, 16): 9, (4, 8): 10}
+    # sweep kernel variant of every table, as the library assigned it
+    table_variant = [emb.table_variant(t) for t in range(T)]
     variant_rows = {}   # distinct rows handled by each sweep variant
-    for t, s in enumerate(wl.tables):
-        v = VARIANT_OF.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
-            if (s.d[-1] == 4 and K >= 3) else -1
-        variant_rows[v] = variant_rows.get(v, 0) + int(counts[t, K - 1])
+    for t in range(T):
+        variant_rows[table_variant[t]] = variant_rows.get(table_variant[t], 0) + int(counts[t, K - 1])
 
     def variant_slots(v, backward):
         tot = 0
         for t, s in enumerate(wl.tables):
-            vv = VARIANT_OF.get((int(np.prod(s.d[:-1])), s.r[-2]), -1) \
-                if (s.d[-1] == 4 and K >= 3) else -1
-            if vv != v:
+            if table_variant[t] != v:
                 continue
             P = int(np.prod(s.d[:K - 2])) if K >= 3 else 1
             c_mid = P * s.r[K - 2] * s.d[K - 2] * s.r[K - 1] if K >= 3 else 0
@@ -544,7 +575,9 @@ def main():
                                       "note": "algorithmic bytes: indices + offsets + every distinct row once + out "
                                               "(+ one (slot,bag) pair per lookup when the backward is enabled); the "
                                               "per-lookup row gather (L*D*4 bytes) is on-chip / re-read traffic and is "
-                                              "not counted; traffic scaled from the reduced-case ncu capture",
+                                              "not counted; traffic scaled from the reduced-case ncu capture named in "
+                                              "profiles/dram_traffic_per_unit.txt (null for other shapes)",
+                                      "frac_without_row_buffer": (8 * L + 8 * (T * B + 1) + 4 * B * T * D) / (ms * 1e-3) / 1e9 / hbm_gbs,
                                       "row_gather_GBs": wl.L * D * 4 / (ms * 1e-3) / 1e9,
                                       "row_gather_peak_l2_GBs": l2_gather / 1e9, "row_gather_peak_hbm_GBs": hbm_gather / 1e9})
     if train and "bwd_dE" in stage_ms:

@@ -71,11 +71,13 @@ typedef struct {
     int64_t max_lookups;        /* upper bound on `num_lookups` (all tables together) */
     int64_t max_unique_rows;    /* upper bound on distinct (table,row) pairs per call; 0 = min(max_lookups, sum N_t) */
     int32_t enable_backward;    /* 0: forward only (smaller workspace); 1: tt_emb_backward may be called */
-    int32_t ablation;           /* 0 = the full method.  Study switches (forward only, tt_emb_backward returns
-                                   TT_EMB_ERR_STATE): bit 0 = no prefix reuse, every distinct row forms its own group and
-                                   rebuilds its prefix product ("unique only", cf. the paper's reuse ablation);
+    int32_t ablation;           /* 0 = the full method.  Study switches (forward only; tt_emb_create rejects them together
+                                   with enable_backward): bit 0 = no prefix reuse, every distinct row forms its own group
+                                   and rebuilds its prefix product ("unique only", cf. the paper's reuse ablation);
                                    bit 1 = static schedule, every table cut into units of equal group COUNT instead of
-                                   equal cost (cf. the paper's scheduling ablation) */
+                                   equal cost (cf. the paper's scheduling ablation); bit 2 = no de-duplication, every
+                                   lookup is a row and a group of its own ("no dedup", the first arm of the reuse
+                                   ablation; sizes the row buffer for max_lookups rows; implies bit 0) */
     int32_t enable_weighted;    /* 1: tt_emb_set_pooling may select mean pooling or per-lookup weights (with the
                                    backward enabled the workspace grows by 4 bytes per lookup) */
 } tt_emb_config_t;
@@ -106,18 +108,21 @@ int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace, size_t wor
  * indices  device int64[num_lookups], table-major: all bags of table 0, then table 1, ...
  * offsets  device int64[T*batch + 1], CSR over (table, bag): bag (t,b) owns
  *          indices[offsets[t*batch+b] .. offsets[t*batch+b+1]); offsets[0] = 0, last = num_lookups
- * out      device fp32[batch][T*D], row-major, fully overwritten
- * indices and offsets must stay valid and unchanged until a later tt_emb_backward for this forward
- * has completed (the backward re-reads them).  Asynchronous.
+ * out      device fp32[batch][T*D], row-major, fully overwritten (also when a status bit reports malformed
+ *          offsets: every bag is then summed over its offsets clamped to [0, num_lookups], an inverted pair
+ *          counting as an empty bag)
+ * The forward keeps what the backward needs (one (row slot, bag) pair per lookup) in the workspace: `indices` may be
+ * freed or overwritten once the forward has completed.  `offsets` must stay valid and unchanged until the backward
+ * has completed if mean pooling is selected (the bag lengths are re-read); the inspection calls
+ * tt_emb_export_level (with lookup_counts) and tt_emb_export_inverse re-read both arrays.  Asynchronous.
  */
 int tt_emb_forward(tt_emb_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
                    int64_t num_lookups, float* out, tt_emb_stream_t stream);
 
 /*
  * The same forward with 32-bit row ids (every N_t is below 2^31 anyway): half the bytes to bring to the device and to
- * read in the grouping and pooling passes.  indices: device int32[num_lookups]; everything else as tt_emb_forward,
- * including the rule that indices stay valid until a later tt_emb_backward has completed.  The paper's interface
- * has 64-bit ids only; this entry point is an addition for callers that hold 32-bit ids.
+ * read in the grouping and pooling passes.  indices: device int32[num_lookups]; everything else as tt_emb_forward.
+ * The paper's interface has 64-bit ids only; this entry point is an addition for callers that hold 32-bit ids.
  */
 int tt_emb_forward_i32(tt_emb_t h, const int32_t* indices, const int64_t* offsets, int64_t batch,
                        int64_t num_lookups, float* out, tt_emb_stream_t stream);
@@ -154,10 +159,14 @@ int tt_emb_backward(tt_emb_t h, const float* grad_out, float* const* core_grads,
  * Same result as tt_emb_bind(core_ptrs, <workspace>) followed by tt_emb_forward(...), but the workspace is a
  * fixed 32 MiB array inside the library (tt_emb_static_workspace_limit()); nothing is allocated.
  *   - returns TT_EMB_ERR_WORKSPACE, launching nothing, if tt_emb_workspace_bytes(h) exceeds that limit;
- *   - the first call on a device looks up the array's address: make it outside any stream capture;
+ *   - the first call on a device looks up the array's address, and the first forward of a handle creates the
+ *     handle's side streams and events and sets kernel attributes (host-side objects, no device memory): make those
+ *     first calls outside any stream capture;
  *   - all calls on a device share the array (it keeps the previous call's contents; what must start at zero is
  *     cleared by the call); calls whose GPU work overlaps (other streams, other handles) race: serialise them;
- *   - afterwards the handle is bound to the array.
+ *   - afterwards the handle is bound to the array; a call on a handle that already is, with the same core
+ *     pointers, enqueues nothing but the forward itself.
+ * TT_EMB_ERR_ARCH without a compute-capability-10 device; TT_EMB_ERR_ARG if the current device's index is 64 or more.
  * core_ptrs as in tt_emb_bind; the remaining arguments as in tt_emb_forward.  Asynchronous.
  */
 int tt_emb_forward_static(tt_emb_t h, float* const* core_ptrs, const int64_t* indices, const int64_t* offsets,
@@ -208,6 +217,18 @@ int tt_emb_export_level(tt_emb_t h, int32_t table, int32_t level, int64_t* vals,
  * ascending distinct rows (-1 for an out-of-range row id).
  */
 int tt_emb_export_inverse(tt_emb_t h, int32_t table, int32_t* inv, tt_emb_stream_t stream);
+
+/* Register-tiled kernel variant that serves the last two levels of `table` (-1: the generic any-shape path). */
+int tt_emb_table_variant(tt_emb_t h, int32_t table, int32_t* sweep_variant);
+
+/*
+ * Debug aid, a stand-in for a memory checker: tt_emb_bind writes guard bytes behind every region of the workspace
+ * (status, bitmap, level arrays, row buffer, ...); this call reports in *first_bad the index of the first region whose
+ * guard bytes no longer hold the pattern, i.e. that some kernel wrote past (-1: all intact), and
+ * tt_emb_region_name(h, index) names it.  The paper has no counterpart.  SYNCHRONISES.
+ */
+int tt_emb_check_guards(tt_emb_t h, int32_t* first_bad, tt_emb_stream_t stream);
+const char* tt_emb_region_name(tt_emb_t h, int32_t index);
 
 /* Layout conversion, device to device.  rndr = [r_{k-1}][n_k][d_k][r_k], canonical = slice-major. */
 int tt_emb_pack_core(tt_emb_t h, int32_t table, int32_t core, const float* rndr, float* canonical,

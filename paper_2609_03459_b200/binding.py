@@ -83,6 +83,9 @@ _SIGS = {
     "tt_emb_probe_fp32": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_probe_gather": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp, _i64, ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_launch_count": (ctypes.c_int, [ctypes.POINTER(_i64), _i32]),
+    "tt_emb_table_variant": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i32)]),
+    "tt_emb_check_guards": (ctypes.c_int, [_vp, ctypes.POINTER(_i32), _vp]),
+    "tt_emb_region_name": (ctypes.c_char_p, [_vp, _i32]),
     "tt_emb_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "tt_emb_last_cuda_error": (ctypes.c_int, []),
 }
@@ -342,6 +345,18 @@ class TTEmbeddingBag:
         inv = torch.empty(max(num_lookups, 1), dtype=torch.int32, device=self.device)
         _check(lib.tt_emb_export_inverse(self.h, table, inv.data_ptr(), _stream_ptr()), "tt_emb_export_inverse")
         return inv.cpu().numpy()[:num_lookups]
+
+    def table_variant(self, table: int) -> int:
+        """Register-tiled sweep kernel variant of a table (-1: generic path)."""
+        v = ctypes.c_int32()
+        _check(lib.tt_emb_table_variant(self.h, table, ctypes.byref(v)), "tt_emb_table_variant")
+        return int(v.value)
+
+    def check_guards(self):
+        """None if the guard bytes behind every workspace region are intact, else the name of the first damaged region."""
+        bad = ctypes.c_int32()
+        _check(lib.tt_emb_check_guards(self.h, ctypes.byref(bad), _stream_ptr()), "tt_emb_check_guards")
+        return None if bad.value < 0 else lib.tt_emb_region_name(self.h, bad.value).decode()
 
     def enable_timing(self, on=True):
         """False/0: off; True/1: stage events; 2: stage events with the shape-variant kernels serialised."""

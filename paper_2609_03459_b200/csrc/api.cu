@@ -10,6 +10,7 @@ static thread_local int g_last_cuda_error = 0;
 static thread_local long long g_launches = 0;
 
 void tt_note_launch(int n) { g_launches += n; }
+void tt_set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 
 extern "C" int tt_emb_launch_count(int64_t* count, int32_t reset)
 {
@@ -30,7 +31,7 @@ extern "C" int tt_emb_launch_count(int64_t* count, int32_t reset)
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-static int device_ok(int* sm_count)
+int tt_device_ok(int* sm_count)
 {
     int n = 0;
     if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return 0; }
@@ -80,11 +81,12 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->T = T; h->K = K;
     h->max_batch = cfg->max_batch; h->max_lookups = cfg->max_lookups;
     h->enable_backward = cfg->enable_backward ? 1 : 0;
-    h->ablation = cfg->ablation & 3;
+    h->ablation = cfg->ablation & 7;
+    if (h->ablation & 4) h->ablation |= 1;   // without de-duplication there is nothing to share a prefix with either
     h->enable_weighted = cfg->enable_weighted != 0;
     if (h->ablation && h->enable_backward) return fail(TT_EMB_ERR_ARG);   // the study switches are forward only
     h->sm_count = 148;
-    { int sms = 0; if (device_ok(&sms) && sms > 0) h->sm_count = sms; }
+    { int sms = 0; if (tt_device_ok(&sms) && sms > 0) h->sm_count = sms; }
 
     int D = -1;
     int64_t sumN = 0;
@@ -156,6 +158,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     int64_t bound = cfg->max_lookups < sumN ? cfg->max_lookups : sumN;
     if (bound < 1) bound = 1;
     h->capU = (cfg->max_unique_rows > 0 && cfg->max_unique_rows < bound) ? cfg->max_unique_rows : bound;
+    if (h->ablation & 4) h->capU = cfg->max_lookups > 0 ? cfg->max_lookups : 1;   // one row slot per lookup
 
     // work units: every table is cut into `units` equal-cost slices, one CTA each
     // about 8 waves of 8 resident CTAs per SM: fine enough that the last wave and table-size differences do not matter
@@ -256,6 +259,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     for (int k = 1; k <= K; ++k) {
         uint64_t c = level_space[k] < (uint64_t)h->capU ? level_space[k] : (uint64_t)h->capU;
         if ((h->ablation & 1) && k == K - 1) c = (uint64_t)h->capU;   // one group per distinct row
+        if (h->ablation & 4) c = (uint64_t)h->capU;                   // one node per lookup at every level
         v.cap[k] = (uint32_t)c;
         v.stride[k] = stride[k];
     }
@@ -273,44 +277,60 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->cost_shift = shift;
 
     // ---- workspace plan
+    // every region is followed by at least 64 guard bytes (written at bind, checked on demand by tt_emb_check_guards)
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    h->off_status = take((16 + 64) * sizeof(uint32_t));
+    h->num_regions = 0;
+    const char* rname = "";
+    auto take = [&](size_t bytes) {
+        const size_t o = off, end = off + bytes;
+        off = align_up(end + 64, 256);
+        if (h->num_regions < 96) {
+            h->guard_off[h->num_regions] = end;
+            h->guard_len[h->num_regions] = off - end;
+            h->region_name[h->num_regions] = rname;
+            ++h->num_regions;
+        }
+        return o;
+    };
+#define TAKE(name, bytes) (rname = name, take(bytes))
+    h->off_status = TAKE("status", (16 + 64) * sizeof(uint32_t));
     h->off_counters = h->off_status + 16 * sizeof(uint32_t);
-    h->off_tdesc = take((size_t)T * sizeof(TableDesc));
-    h->off_tlstart = take((size_t)(T + 1) * sizeof(int64_t));
-    h->off_vlist = take((size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t));
-    h->off_bm = take((size_t)words * sizeof(uint2));
+    h->off_tdesc = TAKE("tdesc", (size_t)T * sizeof(TableDesc));
+    h->off_tlstart = TAKE("tlstart", (size_t)(T + 1) * sizeof(int64_t));
+    h->off_vlist = TAKE("vlist", (size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t));
+    h->off_bm = TAKE("bm", (size_t)words * sizeof(uint2));
     uint64_t scan_max = words;
     for (int k = 1; k <= K; ++k) if (v.cap[k] > scan_max) scan_max = v.cap[k];
     for (int k = 2; k <= K - 1; ++k) if (twords[k] > scan_max) scan_max = twords[k];
     h->scan_tmp_elems = (size_t)(scan_max / TT_SCAN_TILE + 4);
-    h->off_scan = take(h->scan_tmp_elems * sizeof(uint32_t));
+    h->off_scan = TAKE("scan", h->scan_tmp_elems * sizeof(uint32_t));
     for (int k = 1; k <= K; ++k) {
-        h->off_val[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
-        h->off_tb[k] = take((size_t)(T + 1) * sizeof(uint32_t));
-        if (k < K) h->off_cstart[k] = take(((size_t)v.cap[k] + 1) * sizeof(uint32_t));
-        if (k >= 2) h->off_parent[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+        h->off_val[k] = TAKE("val", (size_t)v.cap[k] * sizeof(uint32_t));
+        h->off_tb[k] = TAKE("tb", (size_t)(T + 1) * sizeof(uint32_t));
+        if (k < K) h->off_cstart[k] = TAKE("cstart", ((size_t)v.cap[k] + 1) * sizeof(uint32_t));
+        if (k >= 2) h->off_parent[k] = TAKE("parent", (size_t)v.cap[k] * sizeof(uint32_t));
     }
-    h->off_cost = take(((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
-    for (int k = 2; k <= K - 2; ++k) h->off_pbuf[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
-    h->off_E = take((size_t)h->capU * D * sizeof(float));
+    h->off_cost = TAKE("cost", ((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
+    for (int k = 2; k <= K - 2; ++k) h->off_pbuf[k] = TAKE("pbuf", (size_t)v.cap[k] * stride[k] * sizeof(float));
+    h->off_E = TAKE("E", (size_t)h->capU * D * sizeof(float));
     for (int k = 2; k <= K - 1; ++k) {   // digit-major node lists: level K-1 orders the sweeps, the others serve the backward
-        h->off_tbm[k] = take((size_t)twords[k] * sizeof(uint2));
-        h->off_tnode[k] = take((size_t)v.cap[k] * sizeof(uint32_t));
+        h->off_tbm[k] = TAKE("tbm", (size_t)twords[k] * sizeof(uint2));
+        h->off_tnode[k] = TAKE("tnode", (size_t)v.cap[k] * sizeof(uint32_t));
     }
     if (h->enable_backward) {
-        h->off_cnt = take(((size_t)h->capU + 1) * sizeof(uint32_t));
-        h->off_cursor = take((size_t)h->capU * sizeof(uint32_t));
-        h->off_pairs = take((size_t)2 * (size_t)(h->max_lookups + 1) * sizeof(uint2));
-        h->off_wsorted = h->enable_weighted ? take((size_t)(h->max_lookups + 1) * sizeof(float)) : 0;
+        h->off_cnt = TAKE("cnt", ((size_t)h->capU + 1) * sizeof(uint32_t));
+        h->off_cursor = TAKE("cursor", (size_t)h->capU * sizeof(uint32_t));
+        h->off_pairs = TAKE("pairs", (size_t)2 * (size_t)(h->max_lookups + 1) * sizeof(uint2));
+        h->off_wsorted = h->enable_weighted ? TAKE("wsorted", (size_t)(h->max_lookups + 1) * sizeof(float)) : 0;
         for (int k = 2; k <= K - 1; ++k) {
-            h->off_dP[k] = take((size_t)v.cap[k] * stride[k] * sizeof(float));
-            h->off_Y[k] = take((size_t)v.cap[k] * stride[k - 1] * sizeof(float));
+            h->off_dP[k] = TAKE("dP", (size_t)v.cap[k] * stride[k] * sizeof(float));
+            h->off_Y[k] = TAKE("Y", (size_t)v.cap[k] * stride[k - 1] * sizeof(float));
         }
-        h->off_carry = take(((size_t)(h->max_lookups / TT_DE_CHUNK) + 2) * 2 * D * sizeof(float));
-        h->off_gpart = take((size_t)TT_STRIPES * (size_t)(gpart > 0 ? gpart : 4) * sizeof(float));
+        h->off_carry = TAKE("carry", ((size_t)(h->max_lookups / TT_DE_CHUNK) + 2) * 2 * D * sizeof(float));
+        h->off_gpart = TAKE("gpart", (size_t)TT_STRIPES * (size_t)(gpart > 0 ? gpart : 4) * sizeof(float));
     }
+    h->off_guard_list = TAKE("guard_list", (size_t)(2 * 96 + 2) * sizeof(uint64_t));
+#undef TAKE
     h->ws_bytes = off;
     *out_handle = h;
     return TT_EMB_OK;
@@ -360,7 +380,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     if (!h || !core_ptrs) return TT_EMB_ERR_ARG;
     if (!workspace || workspace_bytes < h->ws_bytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return TT_EMB_ERR_WORKSPACE;
     int sms = 0;
-    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    if (!tt_device_ok(&sms)) return TT_EMB_ERR_ARCH;
     cudaStream_t s = (cudaStream_t)stream;
     const int T = h->T, K = h->K;
     for (int t = 0; t < T; ++t)
@@ -412,6 +432,19 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     TT_CUDA(cudaMemcpyAsync(v.tdesc, h->tab, (size_t)T * sizeof(TableDesc), cudaMemcpyHostToDevice, s));
     TT_CUDA(cudaMemcpyAsync(v.vlist, h->vlist_host, (size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     TT_CUDA(cudaMemsetAsync(v.status, 0, (16 + 64) * sizeof(uint32_t), s));
+    // guard bytes behind every region, and their list for the check kernel
+    h->ws_base = workspace;
+    {
+        uint64_t list[2 * 96 + 2];
+        for (int i = 0; i < h->num_regions; ++i) {
+            TT_CUDA(cudaMemsetAsync(base + h->guard_off[i], 0xA5, h->guard_len[i], s));
+            list[2 * i] = (uint64_t)h->guard_off[i];
+            list[2 * i + 1] = (uint64_t)h->guard_len[i];
+        }
+        list[2 * 96] = 0; list[2 * 96 + 1] = 0;
+        // the list's own guard was just written; the list itself is uploaded after it (pageable source: staged before return)
+        TT_CUDA(cudaMemcpyAsync(base + h->off_guard_list, list, sizeof(list), cudaMemcpyHostToDevice, s));
+    }
     h->bound = true;
     h->have_forward = false;
     return TT_EMB_OK;
@@ -674,7 +707,7 @@ extern "C" int tt_emb_pack_core(tt_emb_t h, int32_t table, int32_t core, const f
                                 tt_emb_stream_t stream)
 {
     if (!h || !rndr || !canonical || table < 0 || table >= h->T || core < 0 || core >= h->K) return TT_EMB_ERR_ARG;
-    if (!device_ok(nullptr)) return TT_EMB_ERR_ARCH;
+    if (!tt_device_ok(nullptr)) return TT_EMB_ERR_ARCH;
     TT_CUDA(tt_launch_pack(h->tab[table], core, rndr, canonical, true, (cudaStream_t)stream));
     return TT_EMB_OK;
 }
@@ -683,7 +716,7 @@ extern "C" int tt_emb_unpack_core(tt_emb_t h, int32_t table, int32_t core, const
                                   tt_emb_stream_t stream)
 {
     if (!h || !rndr || !canonical || table < 0 || table >= h->T || core < 0 || core >= h->K) return TT_EMB_ERR_ARG;
-    if (!device_ok(nullptr)) return TT_EMB_ERR_ARCH;
+    if (!tt_device_ok(nullptr)) return TT_EMB_ERR_ARCH;
     TT_CUDA(tt_launch_pack(h->tab[table], core, canonical, rndr, false, (cudaStream_t)stream));
     return TT_EMB_OK;
 }
@@ -707,7 +740,7 @@ extern "C" int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t strea
 {
     if (!slots_per_second) return TT_EMB_ERR_ARG;
     int sms = 0;
-    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    if (!tt_device_ok(&sms)) return TT_EMB_ERR_ARCH;
     cudaStream_t s = (cudaStream_t)stream;
     float* dsink = nullptr;
     TT_CUDA(cudaGetSymbolAddress((void**)&dsink, g_probe_sink));
@@ -769,7 +802,7 @@ extern "C" int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* sc
     if (!buffer || !scratch_idx || !bytes_per_second || bytes < 256 || num_rows_read < 1) return TT_EMB_ERR_ARG;
     if (reinterpret_cast<uintptr_t>(buffer) & 15) return TT_EMB_ERR_ARG;
     int sms = 0;
-    if (!device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    if (!tt_device_ok(&sms)) return TT_EMB_ERR_ARCH;
     cudaStream_t s = (cudaStream_t)stream;
     float* dsink = nullptr;
     TT_CUDA(cudaGetSymbolAddress((void**)&dsink, g_probe_sink));
@@ -796,5 +829,50 @@ extern "C" int tt_emb_probe_gather(const void* buffer, size_t bytes, int32_t* sc
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     *bytes_per_second = best;
+    return TT_EMB_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ guards / variants
+
+__global__ void k_check_guards(const unsigned char* base, const uint64_t* list, int n, int* first_bad)
+{
+    for (int i = 0; i < n; ++i) {
+        const uint64_t off = list[2 * i], len = list[2 * i + 1];
+        bool bad = false;
+        for (uint64_t b = threadIdx.x; b < len; b += blockDim.x)
+            if (base[off + b] != 0xA5) bad = true;
+        if (bad) atomicMin(first_bad, i);
+    }
+}
+
+extern "C" int tt_emb_check_guards(tt_emb_t h, int32_t* first_bad, tt_emb_stream_t stream)
+{
+    if (!h || !first_bad) return TT_EMB_ERR_ARG;
+    if (!h->bound) return TT_EMB_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    unsigned char* base = (unsigned char*)h->ws_base;
+    uint64_t* list = (uint64_t*)(base + h->off_guard_list);
+    int* res = (int*)(list + 2 * 96);
+    const int big = 1 << 30;
+    TT_CUDA(cudaMemcpyAsync(res, &big, sizeof(int), cudaMemcpyHostToDevice, s));
+    k_check_guards<<<1, 256, 0, s>>>(base, list, h->num_regions, res);
+    tt_note_launch();
+    int got = 0;
+    TT_CUDA(cudaMemcpyAsync(&got, res, sizeof(int), cudaMemcpyDeviceToHost, s));
+    TT_CUDA(cudaStreamSynchronize(s));
+    *first_bad = got == big ? -1 : got;
+    return TT_EMB_OK;
+}
+
+extern "C" const char* tt_emb_region_name(tt_emb_t h, int32_t index)
+{
+    if (!h || index < 0 || index >= h->num_regions) return "";
+    return h->region_name[index];
+}
+
+extern "C" int tt_emb_table_variant(tt_emb_t h, int32_t table, int32_t* sweep_variant)
+{
+    if (!h || !sweep_variant || table < 0 || table >= h->T) return TT_EMB_ERR_ARG;
+    *sweep_variant = h->tab[table].fast;
     return TT_EMB_OK;
 }

@@ -188,12 +188,6 @@ cudaError_t tt_launch_bwd_sort(tt_emb* h, cudaStream_t s)
 
 // ---------------------------------------------------------------------------------------------- 2. dE
 
-__device__ __forceinline__ void tt_cp_async16_b(void* smem_dst, const void* gsrc)
-{
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
-
 // lane l of the warp owns float4 chunks l, l+32, ... of a row (VEC) or floats l, l+32, ... (!VEC)
 template <bool VEC, int CPL>
 struct RowAcc {
@@ -507,7 +501,7 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
         for (int jj = 0; jj < 32 / RPI; ++jj) {
             const int j = RPI * jj + sub;
             const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
-            if (j < n) tt_cp_async16_b(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
+            if (j < n) tt_cp_async16(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         // the pairs of the next batch arrive while the rows are in flight
@@ -607,57 +601,6 @@ cudaError_t tt_launch_bwd_dE(tt_emb* h, const float* grad_out, cudaStream_t s)
 
 // ---------------------------------------------------------------------------------------------- 3. last level
 
-// same cost-balanced units as the forward sweep (forward.cu)
-__device__ __forceinline__ void tt_unit_range_b(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
-{
-    const TableDesc& td = w.tdesc[t];
-    const int lvl = w.K - 1;
-    const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
-    // the host sizes the grid for the largest possible number of groups; with fewer groups in this batch the table is
-    // cut into fewer units (at least 16 groups each) and the surplus CTAs leave at once
-    int Q = td.units;
-    {
-        const int by_groups = (int)((b - a) >> 4);
-        if (Q > by_groups) Q = by_groups < 1 ? 1 : by_groups;
-    }
-    if (q >= Q) { g0 = a; g1 = a; return; }
-    const uint64_t ca = w.cost[a], cb = w.cost[b];
-    const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
-    auto lower = [&](uint64_t target) {
-        uint32_t lo = a, hi = b;
-        while (lo < hi) {
-            uint32_t mid = lo + ((hi - lo) >> 1);
-            if ((uint64_t)w.cost[mid] < target) lo = mid + 1; else hi = mid;
-        }
-        return lo;
-    };
-    const bool odd = (threadIdx.x & 1) != 0;
-    const uint32_t mine = lower(odd ? hi_c : lo_c);
-    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
-    g0 = q == 0 ? a : (odd ? other : mine);
-    g1 = q == Q - 1 ? b : (odd ? mine : other);
-}
-
-__device__ __forceinline__ void tt_mid_product_b(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
-                                                 int M, int ra, int cols)
-{
-    for (int c = threadIdx.x; c < cols; c += blockDim.x)
-        for (int m = 0; m < M; ++m) {
-            float acc = 0.f;
-            for (int a = 0; a < ra; ++a) acc = fmaf(Pl[m * ra + a], __ldg(Bsl + (size_t)a * cols + c), acc);
-            out[(size_t)m * cols + c] = acc;
-        }
-}
-
-__device__ __forceinline__ const float* tt_left_operand_b(const WsView& w, const TableDesc& td, int k, uint32_t v)
-{
-    if (k == 2) {
-        const uint32_t i1 = w.val[2][v] / (uint32_t)td.n[1];
-        return td.core[0] + (size_t)i1 * td.slice_floats[0];
-    }
-    return w.pbuf[k - 1] + (size_t)w.parent[k][v] * w.stride[k - 1];
-}
-
 // generic fallback (any shape): the whole CTA works on one group at a time
 __device__ __forceinline__ void tt_sweep_bwd_generic(const WsView& w, const TableDesc& td, uint32_t g0, uint32_t g1,
                                                      float* gk, float* Pl, float* Cs, float* dCs, float* dEs)
@@ -673,11 +616,11 @@ __device__ __forceinline__ void tt_sweep_bwd_generic(const WsView& w, const Tabl
         const uint32_t val = w.val[K - 1][g];
         if (K >= 3) {
             const int M = td.P[km], ra = td.r[km], cols = td.d[km] * rb;
-            const float* src = tt_left_operand_b(w, td, K - 1, g);
+            const float* src = tt_left_operand(w, td, K - 1, g);
             for (int i = threadIdx.x; i < M * ra; i += blockDim.x) Pl[i] = src[i];
             __syncthreads();
             const uint32_t im = val % (uint32_t)td.n[km];
-            tt_mid_product_b(Pl, td.core[km] + (size_t)im * td.slice_floats[km], Cs, M, ra, cols);
+            tt_mid_product(Pl, td.core[km] + (size_t)im * td.slice_floats[km], Cs, M, ra, cols);
         } else {
             const float* src = td.core[0] + (size_t)val * td.slice_floats[0];
             for (int i = threadIdx.x; i < Pm * rb; i += blockDim.x) Cs[i] = src[i];
@@ -1172,7 +1115,7 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
         if (j >= g1) break;
         const uint32_t g = w.tnode[K - 1][j];   // units are cut from the digit-major order (see forward.cu)
         const uint32_t val = w.val[K - 1][g];
-        const float* src = tt_left_operand_b(w, td, K - 1, g);
+        const float* src = tt_left_operand(w, td, K - 1, g);
         for (int i = lane; i < M * ra; i += 32) {
             const int m = i / ra, a = i - m * ra;
             As[a * M + m] = __ldg(src + i);
@@ -1208,7 +1151,7 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     extern __shared__ __align__(16) float sm[];
     const int t = w.vlist[vbase + blockIdx.y], q = blockIdx.x;
     uint32_t g0, g1;
-    tt_unit_range_b(w, t, q, g0, g1);
+    tt_unit_range(w, t, q, g0, g1);
     const TableDesc& td = w.tdesc[t];
     const int stripe = (blockIdx.x + blockIdx.y) % TT_STRIPES;
     float* gk = w.gpart + (size_t)stripe * w.gpart_stride + td.gpart_off;
@@ -1452,7 +1395,7 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
         for (int i = 0; i < 16; ++i) acc[i] = 0.f;
         for (uint32_t jn = j0; jn < j1; ++jn) {
             const uint32_t v = w.tnode[k][jn];
-            const float* pl = tt_left_operand_b(w, td, k, v);
+            const float* pl = tt_left_operand(w, td, k, v);
             for (int i = threadIdx.x; i < M * ra; i += blockDim.x) Pls[i] = pl[i];
             const float* dp = w.dP[k] + (size_t)v * w.stride[k];
             for (int i = threadIdx.x; i < M * cols; i += blockDim.x) dPs[i] = dp[i];
@@ -1577,7 +1520,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
             float4* dst = reinterpret_cast<float4*>(&sD[st][(q * M + m) * CP + 4 * c4]);
             if (jb + q < j1) {
                 const uint32_t v = w.tnode[k][jb + q];
-                tt_cp_async16_b(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
+                tt_cp_async16(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
             } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         for (int i = tid; i < NQ * M * (RA / 4); i += 128) {     // P_{k-1} of the parent: M * RA / 4 float4 per node
@@ -1585,7 +1528,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
             float4* dst = reinterpret_cast<float4*>(&sA[st][(q * M + m) * AP + 4 * a4]);
             if (jb + q < j1) {
                 const uint32_t v = w.tnode[k][jb + q];
-                tt_cp_async16_b(dst, reinterpret_cast<const float4*>(tt_left_operand_b(w, td, k, v) + m * RA) + a4);
+                tt_cp_async16(dst, reinterpret_cast<const float4*>(tt_left_operand(w, td, k, v) + m * RA) + a4);
             } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");

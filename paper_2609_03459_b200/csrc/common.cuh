@@ -43,7 +43,8 @@ struct TableDesc {
 // Device-side view of the workspace handed to kernels by value.
 struct WsView {
     int32_t T, K, D;
-    int32_t ablation;                   // study switches: bit 0 no prefix reuse, bit 1 static (equal-count) schedule
+    int32_t ablation;                   // study switches: bit 0 no prefix reuse, bit 1 static (equal-count) schedule,
+                                        // bit 2 no de-duplication (every lookup is its own row and its own group; implies bit 0)
     float fused_lr;                     // != 0: the kernels that finalise a gradient also apply G -= fused_lr * dG (cores in sgd_mask)
     int32_t stride[TT_MAXK + 1];        // floats per node of the level-k partial-product buffers (max over tables)
     int64_t B, L;                       // current batch / lookups
@@ -124,6 +125,12 @@ struct tt_emb {
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
     size_t off_Y[TT_MAXK + 1];
     size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted;
+    // guard bytes after every workspace region (tt_emb_check_guards): [guard_off[i], guard_off[i] + guard_len[i])
+    int num_regions;
+    size_t guard_off[96], guard_len[96];
+    const char* region_name[96];
+    size_t off_guard_list;      // device copy of the (offset, length) pairs + the check's result word
+    void* ws_base;
     size_t scan_tmp_elems;
     int64_t gpart_floats;
     WsView v;             // filled at bind
@@ -141,6 +148,10 @@ struct tt_emb {
 
 // every kernel launch of the library is noted here (api.cu); read with tt_emb_launch_count
 void tt_note_launch(int n = 1);
+// remember a failing CUDA call for tt_emb_last_cuda_error (api.cu)
+void tt_set_last_cuda_error(cudaError_t e);
+// compute capability 10.x device current? (api.cu)
+int tt_device_ok(int* sm_count);
 
 // fork/join helpers (api.cu): side streams wait for everything enqueued on `s` so far / `s` waits for the side streams
 cudaError_t tt_fork(tt_emb* h, cudaStream_t s, int n);
@@ -210,6 +221,84 @@ __device__ __forceinline__ int tt_find_table_from(const uint32_t* __restrict__ t
 {
     while (t + 1 < T && tb[t + 1] <= v) ++t;
     return t;
+}
+
+// out[m*cols + c] = sum_a Pl[m*ra + a] * Bsl[a*cols + c]   (Pl in shared memory, Bsl in global, out anywhere)
+__device__ __forceinline__ void tt_mid_product(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
+                                               int M, int ra, int cols)
+{
+    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
+        for (int m0 = 0; m0 < M; m0 += 8) {
+            float acc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+            const int mm = min(8, M - m0);
+            for (int a = 0; a < ra; ++a) {
+                const float b = __ldg(Bsl + (size_t)a * cols + c);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i < mm) acc[i] = fmaf(Pl[(m0 + i) * ra + a], b, acc[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i < mm) out[(size_t)(m0 + i) * cols + c] = acc[i];
+        }
+    }
+}
+
+// 16-byte asynchronous copy global -> shared, past L1
+__device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
+// left operand of level k (2..K-1) for node v: P_{k-1} of its parent (k = 2: the slice of the first core)
+__device__ __forceinline__ const float* tt_left_operand(const WsView& w, const TableDesc& td, int k, uint32_t v)
+{
+    if (k == 2) {
+        const uint32_t i1 = w.val[2][v] / (uint32_t)td.n[1];
+        return td.core[0] + (size_t)i1 * td.slice_floats[0];
+    }
+    return w.pbuf[k - 1] + (size_t)w.parent[k][v] * w.stride[k - 1];
+}
+
+// group range [g0, g1) of work unit q of table t: an equal-cost slice of the table's level-(K-1) groups in sweep order
+__device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
+{
+    const TableDesc& td = w.tdesc[t];
+    const int lvl = w.K - 1;
+    const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
+    // the host sizes the grid for the largest possible number of groups; with fewer groups in this batch the table is
+    // cut into fewer units (at least 16 groups each) and the surplus CTAs leave at once
+    int Q = td.units;
+    {
+        const int by_groups = (int)((b - a) >> 4);
+        if (Q > by_groups) Q = by_groups < 1 ? 1 : by_groups;
+    }
+    if (q >= Q) { g0 = a; g1 = a; return; }
+    const uint64_t ca = w.cost[a], cb = w.cost[b];
+    if (w.ablation & 2) {   // study switch: static schedule, equal group counts
+        g0 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)q / Q);
+        g1 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)(q + 1) / Q);
+        return;
+    }
+    const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
+    // first group whose exclusive cost >= target
+    auto lower = [&](uint64_t target) {
+        uint32_t lo = a, hi = b;
+        while (lo < hi) {
+            uint32_t mid = lo + ((hi - lo) >> 1);
+            if ((uint64_t)w.cost[mid] < target) lo = mid + 1; else hi = mid;
+        }
+        return lo;
+    };
+    // every thread needs both bounds; even and odd lanes each search one and exchange it
+    const bool odd = (threadIdx.x & 1) != 0;
+    const uint32_t mine = lower(odd ? hi_c : lo_c);
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
+    g0 = q == 0 ? a : (odd ? other : mine);
+    g1 = q == Q - 1 ? b : (odd ? mine : other);
 }
 
 __device__ __forceinline__ int tt_find_table64(const int64_t* __restrict__ tb, int T, int64_t v)

@@ -14,8 +14,6 @@
 #include "mma.cuh"
 #include "quad_mid.cuh"
 
-__device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc);   // defined with the pooling kernels
-
 // ---------------------------------------------------------------------------------------------- schedule
 
 struct CostScan {
@@ -57,79 +55,7 @@ cudaError_t tt_launch_schedule(tt_emb* h, cudaStream_t s)
     return tt_scan(cs, h->v.cap[h->v.K - 1], h->v.scan_tmp, s);
 }
 
-// group range [g0, g1) of work unit `unit` (global id) -- equal-cost slice of its table
-__device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
-{
-    const TableDesc& td = w.tdesc[t];
-    const int lvl = w.K - 1;
-    const uint32_t a = w.tb[lvl][t], b = w.tb[lvl][t + 1];
-    // the host sizes the grid for the largest possible number of groups; with fewer groups in this batch the table is
-    // cut into fewer units (at least 16 groups each) and the surplus CTAs leave at once
-    int Q = td.units;
-    {
-        const int by_groups = (int)((b - a) >> 4);
-        if (Q > by_groups) Q = by_groups < 1 ? 1 : by_groups;
-    }
-    if (q >= Q) { g0 = a; g1 = a; return; }
-    const uint64_t ca = w.cost[a], cb = w.cost[b];
-    if (w.ablation & 2) {   // study switch: static schedule, equal group counts
-        g0 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)q / Q);
-        g1 = a + (uint32_t)((uint64_t)(b - a) * (uint64_t)(q + 1) / Q);
-        return;
-    }
-    const uint64_t lo_c = ca + (cb - ca) * (uint64_t)q / Q, hi_c = ca + (cb - ca) * (uint64_t)(q + 1) / Q;
-    // first group whose exclusive cost >= target
-    auto lower = [&](uint64_t target) {
-        uint32_t lo = a, hi = b;
-        while (lo < hi) {
-            uint32_t mid = lo + ((hi - lo) >> 1);
-            if ((uint64_t)w.cost[mid] < target) lo = mid + 1; else hi = mid;
-        }
-        return lo;
-    };
-    // every thread needs both bounds; even and odd lanes each search one and exchange it
-    const bool odd = (threadIdx.x & 1) != 0;
-    const uint32_t mine = lower(odd ? hi_c : lo_c);
-    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
-    g0 = q == 0 ? a : (odd ? other : mine);
-    g1 = q == Q - 1 ? b : (odd ? mine : other);
-}
-
 // ---------------------------------------------------------------------------------------------- products
-
-// out[m*cols + c] = sum_a Pl[m*ra + a] * Bsl[a*cols + c]   (Pl in shared memory, Bsl in global, out anywhere)
-__device__ __forceinline__ void tt_mid_product(const float* __restrict__ Pl, const float* __restrict__ Bsl, float* out,
-                                               int M, int ra, int cols)
-{
-    for (int c = threadIdx.x; c < cols; c += blockDim.x) {
-        for (int m0 = 0; m0 < M; m0 += 8) {
-            float acc[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-            const int mm = min(8, M - m0);
-            for (int a = 0; a < ra; ++a) {
-                const float b = __ldg(Bsl + (size_t)a * cols + c);
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i < mm) acc[i] = fmaf(Pl[(m0 + i) * ra + a], b, acc[i]);
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i < mm) out[(size_t)(m0 + i) * cols + c] = acc[i];
-        }
-    }
-}
-
-// left operand of level k (0-based core index kc = k-1 >= 1) for node v: P_{k-1} of its parent
-__device__ __forceinline__ const float* tt_left_operand(const WsView& w, const TableDesc& td, int k, uint32_t v)
-{
-    // k = level of the node being produced (2..K-1)
-    if (k == 2) {
-        const uint32_t i1 = w.val[2][v] / (uint32_t)td.n[1];
-        return td.core[0] + (size_t)i1 * td.slice_floats[0];
-    }
-    return w.pbuf[k - 1] + (size_t)w.parent[k][v] * w.stride[k - 1];
-}
 
 // P_k for every level-k node, 2 <= k <= K-2 (only K = 4 has such a level); one CTA per node, grid-stride
 __global__ void __launch_bounds__(128) k_mid_level(WsView w, int k)
@@ -693,6 +619,7 @@ __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableD
 {
     const int64_t g = tt_index<true>(w, l);    // streamed once: evict-first, keeps L2 for rows and rank words
     uint32_t slot = 0xffffffffu;
+    if (w.ablation & 4) return (g >= 0 && g < td.N && l < (int64_t)capK) ? (uint32_t)l : slot;   // no de-duplication: lookup l is row slot l
     if (g >= 0 && g < td.N) {
         const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
         if (e.x >> (g & 31) & 1u) {
@@ -732,12 +659,12 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
     const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
     auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
-    int64_t b_prev = 0;
     for (int64_t ci = wi; ci < C; ci += W) {
     int64_t b0, b1;
     {
         const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
-        int64_t lo = b_prev, hi = nb;                   // first bag with offsets[bag] >= target
+        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target; the same search for
+                                                        // both neighbours of a boundary, whatever the offsets hold
         if (lane < 2)
             while (lo < hi) {
                 const int64_t mid = (lo + hi) >> 1;
@@ -747,11 +674,12 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
         b1 = __shfl_sync(0xffffffffu, lo, 1);
         if (ci == 0) b0 = 0;
         if (ci == C - 1) b1 = nb;
-        b_prev = b1;
     }
     if (b0 >= b1) continue;
-    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
-    if (o_hi < o_lo) o_hi = o_lo;
+    // every bag is summed over its own (offsets[bag], offsets[bag + 1]) pair, clamped to [0, L]; an inverted pair (malformed
+    // offsets) is an empty bag.  o_next: start of the next bag = this bag's end as stored, before the inversion fix
+    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = clampL(__ldg(w.offsets + b0 + 1));
+    int64_t o_hi = o_next < o_lo ? o_lo : o_next;
     int t = (int)(b0 / w.B);
     uint32_t slot_next;
     float wt_next = 1.f;
@@ -764,19 +692,20 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
         const int64_t b = bag - (int64_t)t * w.B;
         // next bag (for the prefetch of its first 32 rank look-ups)
         const bool has_next = bag + 1 < b1;
-        int64_t n_hi = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_hi;
-        if (n_hi < o_hi) n_hi = o_hi;
+        const int64_t n_lo = o_next;
+        const int64_t n_next = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_next;
+        const int64_t n_hi = n_next < n_lo ? n_lo : n_next;
         const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
         float4 acc[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (o_lo >= o_hi && has_next) fetch(o_hi, n_hi, tn);
+        if (o_lo >= o_hi && has_next) fetch(n_lo, n_hi, tn);
         for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
             const float wt = wt_next;
             if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));  // kept for the backward sort
             if (l0 + 32 < o_hi) fetch(l0 + 32, o_hi, t);
-            else if (has_next) fetch(o_hi, n_hi, tn);
+            else if (has_next) fetch(n_lo, n_hi, tn);
             const int n = (int)min((int64_t)32, o_hi - l0);
             float4 part[CPL];   // two-level sum: per-batch partial, added to the bag's sum once per batch
 #pragma unroll
@@ -834,8 +763,9 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
                 if (ch < D4) __stcs(o4 + ch, acc[c]);
             }
         }
-        o_lo = o_hi;
+        o_lo = n_lo;
         o_hi = n_hi;
+        o_next = n_next;
         t = tn;
     }
     }
@@ -845,12 +775,6 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
 // flight.  Here every warp owns an 8 KB shared-memory buffer and fills it with cp.async (16 bytes per lane, two
 // rows per instruction, no staging registers): the 32 rows of a batch are all in flight at once.  Same bag
 // partition (equal shares of the lookups per warp), same prefetch of the next batch's rank look-ups.
-__device__ __forceinline__ void tt_cp_async16(void* smem_dst, const void* gsrc)
-{
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
-
 #define POOL_WARPS 7   // 4 CTAs x 7 warps x 8 KB = 224 KB of the SM's shared memory
 template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, float* __restrict__ out)
@@ -871,12 +795,12 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
     auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
-    int64_t b_prev = 0;
     for (int64_t ci = wi; ci < C; ci += W) {
     int64_t b0, b1;
     {
         const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
-        int64_t lo = b_prev, hi = nb;                   // first bag with offsets[bag] >= target
+        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target; the same search for
+                                                        // both neighbours of a boundary, whatever the offsets hold
         if (lane < 2)
             while (lo < hi) {
                 const int64_t mid = (lo + hi) >> 1;
@@ -886,11 +810,12 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
         b1 = __shfl_sync(0xffffffffu, lo, 1);
         if (ci == 0) b0 = 0;
         if (ci == C - 1) b1 = nb;
-        b_prev = b1;
     }
     if (b0 >= b1) continue;
-    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_hi = clampL(__ldg(w.offsets + b0 + 1));
-    if (o_hi < o_lo) o_hi = o_lo;
+    // every bag is summed over its own (offsets[bag], offsets[bag + 1]) pair, clamped to [0, L]; an inverted pair (malformed
+    // offsets) is an empty bag.  o_next: start of the next bag = this bag's end as stored, before the inversion fix
+    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = clampL(__ldg(w.offsets + b0 + 1));
+    int64_t o_hi = o_next < o_lo ? o_lo : o_next;
     int t = (int)(b0 / w.B);
     uint32_t slot_next;
     float wt_next = 1.f;
@@ -902,11 +827,12 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     for (int64_t bag = b0; bag < b1; ++bag) {
         const int64_t b = bag - (int64_t)t * w.B;
         const bool has_next = bag + 1 < b1;
-        int64_t n_hi = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_hi;
-        if (n_hi < o_hi) n_hi = o_hi;
+        const int64_t n_lo = o_next;
+        const int64_t n_next = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_next;
+        const int64_t n_hi = n_next < n_lo ? n_lo : n_next;
         const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (o_lo >= o_hi && has_next) fetch(o_hi, n_hi, tn);
+        if (o_lo >= o_hi && has_next) fetch(n_lo, n_hi, tn);
         for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
             const float wt = wt_next;
@@ -926,7 +852,7 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             asm volatile("cp.async.commit_group;" ::: "memory");
             // the rank look-ups of the next batch (or of the next bag) overlap the gather
             if (l0 + 32 < o_hi) fetch(l0 + 32, o_hi, t);
-            else if (has_next) fetch(o_hi, n_hi, tn);
+            else if (has_next) fetch(n_lo, n_hi, tn);
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
 #pragma unroll
@@ -952,8 +878,9 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
         if (sub == 0 && lane_on) __stcs(reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr, acc);
-        o_lo = o_hi;
+        o_lo = n_lo;
         o_hi = n_hi;
+        o_next = n_next;
         t = tn;
     }
     }
@@ -1013,27 +940,14 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
         hi = hi < lo ? lo : (hi > w.L ? w.L : hi);
         float* o = out + (size_t)b * w.T * D + (size_t)t * D;
         if (w.upairs)
-            for (int64_t l = lo + lane; l < hi; l += 32) {
-                const int64_t g = tt_index(w, l);
-                uint32_t slot = 0xffffffffu;
-                if (g >= 0 && g < td.N) {
-                    const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
-                    if (e.x >> (g & 31) & 1u) slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
-                    if (slot >= capK) slot = 0xffffffffu;
-                }
-                w.upairs[l] = make_uint2(slot, (uint32_t)b);
-            }
+            for (int64_t l = lo + lane; l < hi; l += 32) w.upairs[l] = make_uint2(tt_lookup_slot(w, td, l, capK), (uint32_t)b);
         for (int e0 = 0; e0 < D; e0 += 32 * 8) {
             float acc[8];
 #pragma unroll
             for (int c = 0; c < 8; ++c) acc[c] = 0.f;
             for (int64_t l = lo; l < hi; ++l) {
-                const int64_t g = tt_index(w, l);
-                if (g < 0 || g >= td.N) continue;
-                const uint2 e = __ldg(&w.bm[td.word_base + ((uint32_t)g >> 5)]);
-                if (!(e.x >> (g & 31) & 1u)) continue;
-                const uint32_t slot = e.y + __popc(e.x & ((1u << (g & 31)) - 1u));
-                if (slot >= capK) continue;
+                const uint32_t slot = tt_lookup_slot(w, td, l, capK);
+                if (slot == 0xffffffffu) continue;
                 const float* row = w.E + (size_t)slot * D;
                 const float a = w.psw ? __ldg(w.psw + l) : 1.f;
 #pragma unroll

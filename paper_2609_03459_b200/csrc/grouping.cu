@@ -160,16 +160,60 @@ __global__ void k_fix_tb(WsView w, int k)
     }
 }
 
+// Study switch "no de-duplication" (the first arm of the paper's reuse ablation): lookup l is row slot l and a group of
+// its own at every prefix level, so nothing is shared: every lookup rebuilds its whole chain of products.
+// Lookups with a row id outside the table keep the row 0 (the pooling pass skips them by their id).
+__global__ void __launch_bounds__(256) k_nodedup_levels(WsView w)
+{
+    tt_pdl_enter();
+    const int K = w.K;
+    const int64_t L = w.L < (int64_t)w.cap[K] ? w.L : (int64_t)w.cap[K];
+    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (first == 0) {
+        if (w.L > (int64_t)w.cap[K]) atomicOr(w.status, TT_EMB_STATUS_OVERFLOW);
+        for (int k = 1; k <= K; ++k) {
+            w.counters[CTR_LEVEL0 + k] = (uint32_t)L;
+            if (k < K) w.cstart[k][L] = (uint32_t)L;
+        }
+    }
+    if (first <= w.T)
+        for (int k = 1; k <= K; ++k) {
+            const int64_t v = w.tl_start[first];
+            w.tb[k][first] = (uint32_t)(v < L ? v : L);
+        }
+    int t = 0;
+    for (int64_t l = first; l < L; l += (int64_t)gridDim.x * blockDim.x) {
+        if (!(w.tl_start[t] <= l && l < w.tl_start[t + 1])) t = tt_find_table64(w.tl_start, w.T, l);
+        const TableDesc& td = w.tdesc[t];
+        const int64_t g = tt_index(w, l);
+        if (g < 0 || g >= td.N) atomicOr(w.status, TT_EMB_STATUS_INDEX);
+        uint32_t v = (g >= 0 && g < td.N) ? (uint32_t)g : 0u;
+        for (int k = K; k >= 1; --k) {
+            w.val[k][l] = v;
+            if (k < K) w.cstart[k][l] = (uint32_t)l;
+            if (k >= 2) w.parent[k][l] = (uint32_t)l;
+            v /= (uint32_t)td.n[k - 1];
+        }
+    }
+}
+
 cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
     cudaError_t e;
     // status word + counters are adjacent; bitmap follows its own region
     if ((e = cudaMemsetAsync(w.status, 0, (16 + 64) * sizeof(uint32_t), s)) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(w.bm, 0, (size_t)w.total_words * sizeof(uint2), s)) != cudaSuccess) return e;
     const int64_t nb = (int64_t)w.T * w.B + 1;
     int g0 = (int)((nb + 255) / 256);
     if (g0 > h->sm_count * 8) g0 = h->sm_count * 8;
+    if (w.ablation & 4) {
+        if ((e = tt_launch_pdl(k_check_offsets, dim3(g0), dim3(256), 0, s, w)) != cudaSuccess) return e;
+        tt_note_launch();
+        if ((e = tt_launch_pdl(k_nodedup_levels, dim3(h->sm_count * 8), dim3(256), 0, s, w)) != cudaSuccess) return e;
+        tt_note_launch();
+        return cudaGetLastError();
+    }
+    if ((e = cudaMemsetAsync(w.bm, 0, (size_t)w.total_words * sizeof(uint2), s)) != cudaSuccess) return e;
     if ((e = tt_launch_pdl(k_check_offsets, dim3(g0), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     if (w.L > 0) {
@@ -252,7 +296,7 @@ __global__ void k_export_inverse(WsView w, int table, int32_t* inv)
         int32_t r = -1;
         if (g >= 0 && g < td.N) {
             const uint2 e = w.bm[td.word_base + ((uint32_t)g >> 5)];
-            r = (int32_t)(e.y + __popc(e.x & ((1u << (g & 31)) - 1u)) - base);
+            r = (w.ablation & 4) ? (int32_t)(l - lo) : (int32_t)(e.y + __popc(e.x & ((1u << (g & 31)) - 1u)) - base);
         }
         inv[l - lo] = r;
     }

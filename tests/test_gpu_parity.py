@@ -336,9 +336,9 @@ def test_forward_only_handle_and_repeat_calls(binding):
     assert_close(out3, oracle.forward_workload(wl2), "second batch out")
 
 
-@pytest.mark.parametrize("flags", [1, 2, 3])
+@pytest.mark.parametrize("flags", [1, 2, 3, 4, 6])
 def test_ablation_switches_keep_the_result(binding, flags):
-    # the study switches (no prefix reuse / static schedule) change cost, never values
+    # the study switches (no prefix reuse / static schedule / no de-duplication) change cost, never values
     name, tables, B, pooling = MEDIUM[1]
     wl = workloads.custom(tables, B, pooling, seed=21)
     emb = binding.from_workload(wl, ablation=flags)
@@ -348,6 +348,10 @@ def test_ablation_switches_keep_the_result(binding, flags):
     counts = emb.grouping_counts()
     if flags & 1:   # every distinct row is its own group
         assert np.array_equal(counts[:, 1], counts[:, 2])
+    if flags & 4:   # every lookup is a row, a group and a first-level node of its own
+        per_table = wl.offsets[np.arange(1, wl.T + 1) * wl.B] - wl.offsets[np.arange(wl.T) * wl.B]
+        for k in range(counts.shape[1]):
+            assert np.array_equal(counts[:, k], per_table)
     with pytest.raises(binding.TTEmbError):
         binding.from_workload(wl, ablation=flags, enable_backward=True)
 
@@ -407,14 +411,53 @@ def test_out_of_range_indices_are_flagged_and_ignored(binding):
         assert_close(grads[0][k], ref[0][k], f"oob dG[{k}]")
 
 
-def test_bad_offsets_are_flagged(binding):
-    spec = TableSpec(997, (10, 10, 10), (4, 4, 4), (1, 4, 4, 1), 1.0, "normal", 0.1)
-    wl = workloads.custom([spec], 20, 3, seed=2)
+@pytest.mark.parametrize("d", [(4, 4, 4), (4, 8, 4), (2, 4, 4), (3, 3, 5)])
+def test_bad_offsets_are_flagged_and_out_is_still_fully_written(binding, d):
+    # malformed offsets set the status bit; `out` is still defined everywhere: every bag is the sum over its own
+    # (offsets[b], offsets[b+1]) range, an inverted pair being an empty bag -- which is what the oracle's loop does too
+    spec = TableSpec(997, (10, 10, 10), d, (1, 4, 4, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec], 700, 3, seed=2)
     off = wl.offsets.copy()
-    off[5], off[6] = off[6], off[5] - 1
+    for b in (5, 77, 300, 301, 650):
+        off[b], off[b + 1] = off[b + 1], off[b] - 1
     emb = binding.from_workload(wl)
-    emb.forward(dev(wl.indices), dev(off), wl.B)
+    out = torch_full((wl.B, wl.D), float("nan"))
+    emb.forward(dev(wl.indices), dev(off), wl.B, out=out)
     assert emb.status() & binding.STATUS_OFFSETS
+    s = wl.tables[0]
+    ref = oracle.forward(s.n, s.d, s.r, s.N, wl.cores[0], wl.indices, off)
+    assert_close(out.cpu().numpy(), ref, "out with malformed offsets")
+
+
+def torch_full(shape, value):
+    import torch
+    return torch.full(shape, value, dtype=torch.float32, device="cuda")
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_no_kernel_writes_past_its_workspace_region(binding, cfg):
+    # guard bytes behind every workspace region (the stand-in for a memory checker) after a whole step
+    wl = workloads.make(cfg, tiny=True)
+    emb = binding.from_workload(wl, enable_backward=True, enable_weighted=True)
+    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    go = wl.grad_out if wl.grad_out is not None else np.ones((wl.B, wl.T * wl.D), np.float32)
+    emb.backward_sgd(dev(go), 0.01)
+    assert emb.status() == 0
+    assert emb.check_guards() is None
+
+
+def test_guard_check_medium_shapes_and_detection(binding):
+    for name, tables, B, pooling in MEDIUM:
+        wl = workloads.custom(tables, B, pooling, seed=5, with_grad=True)
+        emb = binding.from_workload(wl, enable_backward=True)
+        emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+        emb.backward(dev(wl.grad_out))
+        emb.sgd_step(0.01)
+        assert emb.check_guards() is None, name
+    # the check does see damage: the last byte of the workspace is a guard byte of the last region
+    base_off = (-emb.workspace.data_ptr()) % 256
+    emb.workspace[base_off + emb.workspace_bytes - 1] = 0
+    assert emb.check_guards() == "guard_list"
 
 
 def test_unique_row_capacity_overflow_is_flagged(binding):

@@ -11,6 +11,7 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 import workloads
 from workloads import TableSpec
 
@@ -56,6 +57,11 @@ def test_static_workspace_forward_matches_regular_forward_twice(binding):
     for got, ref, what in ((out1, ref_a, "first call"), (out2, ref_b, "second call"), (out3, ref_a, "third call")):
         err = np.abs(got.astype(np.float64) - ref.astype(np.float64)).max()
         assert err <= 1e-5 * np.abs(ref).max(), (what, err)
+    # and against the fp64 oracle, like every other forward
+    for got, wl, what in ((out1, wl_a, "first call"), (out2, wl_b, "second call"), (out3, wl_a, "third call")):
+        want = oracle.forward_workload(wl)
+        assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max(), (what, "vs oracle")
+    assert emb_s.check_guards() is None
 
 
 def test_static_workspace_rejects_configurations_that_do_not_fit(binding):

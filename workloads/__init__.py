@@ -259,3 +259,15 @@ def sweep_point(D: int, rank: int, batch: int, *, num_tables: int = 8, with_grad
                         core_dist="normal", core_scale=0.05) for s in base]
     return _assemble(f"sweep-D{D}-r{rank}-B{batch}", tables, batch, (1, 100), seed3 + 7 * D + rank, mapping,
                      with_grad=with_grad)
+
+
+def generic_point(batch: int = 32768, *, num_tables: int = 8, with_grad: bool = True, mapping: str = "identity",
+                  seed: Optional[int] = None) -> Workload:
+    """A shape that none of the register-tiled kernel variants covers: dim factors (3, 3, 5) (D = 45, not a multiple
+    of four) and ranks (1, 6, 4, 1), on the first `num_tables` row counts and Zipf exponents of the config-3 stream,
+    pooling factor uniform in [1, 100].  It exercises the any-shape path end to end (scalar pooling and dE included)."""
+    seed3 = (BASE_SEED if seed is None else seed) + 1000 * 3
+    base = _cfg3_tables(np.random.default_rng(seed3 + 500), num_tables)
+    tables = [TableSpec(N=s.N, n=s.n, d=(3, 3, 5), r=(1, 6, 4, 1), alpha=s.alpha, core_dist="normal", core_scale=0.05)
+              for s in base]
+    return _assemble(f"generic-d3x3x5-r6x4-B{batch}", tables, batch, (1, 100), seed3 + 4500, mapping, with_grad=with_grad)
