@@ -782,6 +782,8 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     tt_pdl_enter();
     static_assert(R4 == 16 || R4 == 8, "two or four rows per cp.async instruction");
     constexpr int RPI = 32 / R4;
+    constexpr int PGRP = 4;              // load instructions per group: a window is cut short and tested for validity per group
+                                         // (half of all windows end a bag and are short; groups of two measured slower)
     extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][R4 float4]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int sub = lane / R4, lr = lane % R4;
@@ -843,11 +845,27 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             // rounding error of a bag with thousands of lookups grows with the number of batches, not of rows
             float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
             // all rows of the batch in flight
+            // (groups of four instructions; a short window -- half of all windows end a bag -- leaves early)
+            // a group whose rows are all valid (the usual case) needs no per-row test
+            const bool plain = valid == (n == 32 ? 0xffffffffu : (1u << n) - 1u) && D4 == R4;
 #pragma unroll
-            for (int jj = 0; jj < 32 / RPI; ++jj) {
-                const int j = RPI * jj + sub;
-                const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
-                if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * D4 + lr);
+            for (int jq = 0; jq < 32 / RPI; jq += PGRP) {
+                if (RPI * jq >= n) break;
+                if (plain && RPI * (jq + PGRP) <= n) {
+#pragma unroll
+                    for (int jj = jq; jj < jq + PGRP; ++jj) {
+                        const int j = RPI * jj + sub;
+                        const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
+                        tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * R4 + lr);
+                    }
+                } else {
+#pragma unroll
+                    for (int jj = jq; jj < jq + PGRP; ++jj) {
+                        const int j = RPI * jj + sub;
+                        const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
+                        if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * D4 + lr);
+                    }
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             // the rank look-ups of the next batch (or of the next bag) overlap the gather
@@ -856,13 +874,25 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
 #pragma unroll
-            for (int jj = 0; jj < 32 / RPI; ++jj) {
-                const int j = RPI * jj + sub;
-                const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
-                if (((valid >> j) & 1u) && lane_on) {
-                    const float4 v = buf[j * R4 + lr];
-                    if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
-                    else { part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w; }
+            for (int jq = 0; jq < 32 / RPI; jq += PGRP) {
+                if (RPI * jq >= n) break;
+                if (!WT && plain && RPI * (jq + PGRP) <= n) {
+#pragma unroll
+                    for (int jj = jq; jj < jq + PGRP; ++jj) {
+                        const float4 v = buf[(RPI * jj + sub) * R4 + lr];
+                        part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int jj = jq; jj < jq + PGRP; ++jj) {
+                        const int j = RPI * jj + sub;
+                        const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
+                        if (((valid >> j) & 1u) && lane_on) {
+                            const float4 v = buf[j * R4 + lr];
+                            if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
+                            else { part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w; }
+                        }
+                    }
                 }
             }
             acc.x += part.x; acc.y += part.y; acc.z += part.z; acc.w += part.w;
