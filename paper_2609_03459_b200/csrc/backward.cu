@@ -497,11 +497,20 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
         if (lane == 0) before = last_slot;
         const unsigned starts = __ballot_sync(0xffffffffu, lane < n && mine.x != before);   // bit j: position j opens a segment
         last_slot = __shfl_sync(0xffffffffu, mine.x, n - 1);
+        if (n == 32) {   // all windows of a chunk but its last: no per-row test
 #pragma unroll
-        for (int jj = 0; jj < 32 / RPI; ++jj) {
-            const int j = RPI * jj + sub;
-            const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
-            if (j < n) tt_cp_async16(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
+            for (int jj = 0; jj < 32 / RPI; ++jj) {
+                const int j = RPI * jj + sub;
+                const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
+                tt_cp_async16(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
+            }
+        } else {
+#pragma unroll
+            for (int jj = 0; jj < 32 / RPI; ++jj) {
+                const int j = RPI * jj + sub;
+                const uint32_t gr = __shfl_sync(0xffffffffu, grow, j);
+                if (j < n) tt_cp_async16(buf + j * R4 + lr, G4 + (size_t)gr * R4 + lr);
+            }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         // the pairs of the next batch arrive while the rows are in flight
@@ -533,6 +542,22 @@ __global__ void __launch_bounds__(32 * DE_WARPS, 4) k_dE_stage(WsView w, const f
             if (j0 + 8 <= n && ((starts >> j0) & 0xffu) == 0u) {
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) add_row(j0 + jj);
+            } else if (j0 + 8 <= n && ((starts >> j0) & 0xffu) == 0xffu) {
+                // eight starts in a row (rows looked up once: most distinct rows): the first closes the running segment,
+                // the next seven rows are whole segments of one row each and are copied out, the eighth opens a new one
+                close_segment();
+#pragma unroll
+                for (int jj = 0; jj < 7; ++jj) {
+                    const uint32_t sj = __shfl_sync(0xffffffffu, cur_pairs.x, j0 + jj);
+                    add_row(j0 + jj);
+                    float* dst = w.E + (size_t)sj * DD;
+                    if (VPL == 2) reinterpret_cast<float2*>(dst)[lane] = make_float2(part[0], part[VPL - 1]);
+                    else if (lane < DD) dst[lane] = part[0];
+#pragma unroll
+                    for (int c = 0; c < VPL; ++c) part[c] = 0.f;
+                }
+                cur = __shfl_sync(0xffffffffu, cur_pairs.x, j0 + 7);
+                add_row(j0 + 7);
             } else {
                 const int j1 = min(j0 + 8, n);
                 for (int j = j0; j < j1; ++j) {

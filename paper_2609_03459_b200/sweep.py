@@ -3,7 +3,7 @@
     python -m paper_2609_03459_b200.sweep [--dims 16,32,64] [--ranks 8,16,32] [--batches 1024,...,131072]
                                           [--train] [--steps 10] [--out table.md]
 
-The axes follow the paper's sensitivity study (Sec. 5, embedding dimension d in {16,32,64}, TT-rank in
+The axes follow the paper's sensitivity study (Sec. 4.1, embedding dimension d in {16,32,64}, TT-rank in
 {8,16,32}, throughput against batch size) plus the paper's own operating point (d=32, rank 32, 3 cores).
 Inputs come from `workloads.sweep_point`: 8 tables of the multi-table recipe, the same tables at every
 point.  Every timed iteration is bracketed by CUDA events on the launching stream; an L2-sized buffer is

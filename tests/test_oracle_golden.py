@@ -43,3 +43,7 @@ def test_frozen_snapshot_of_tiny_configs():
         out = oracle.forward_workload(wl)
         vals = np.array([out.sum(), (out ** 2).sum(), *out[0, :4]])
         np.testing.assert_allclose(vals, g[f"cfg{cfg}"], rtol=1e-12, atol=1e-14)
+        if wl.grad_out is not None:   # per table: the sum of all its core-gradient entries (plain and memoised oracle)
+            for memo in (False, True):
+                sums = [sum(float(c.sum()) for c in tg) for tg in oracle.backward_workload(wl, memo=memo)]
+                np.testing.assert_allclose(sums, g[f"cfg{cfg}_grad_sums"], rtol=1e-10, atol=1e-13)
