@@ -1175,8 +1175,8 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     tt_pdl_enter();
     extern __shared__ __align__(16) float sm[];
     const int t = w.vlist[vbase + blockIdx.y], q = blockIdx.x;
-    uint32_t g0, g1;
-    tt_unit_range(w, t, q, g0, g1);
+    const uint2 rng = w.unit_rng[t * w.units_per_table + q];
+    const uint32_t g0 = rng.x, g1 = rng.y;
     const TableDesc& td = w.tdesc[t];
     const int stripe = (blockIdx.x + blockIdx.y) % TT_STRIPES;
     float* gk = w.gpart + (size_t)stripe * w.gpart_stride + td.gpart_off;

@@ -65,6 +65,8 @@ struct WsView {
     uint32_t* parent[TT_MAXK + 1];      // level k >= 2: parent node at level k-1
     uint32_t* tb[TT_MAXK + 1];          // [T+1] node range of each table at level k
     uint32_t* cost;                     // [cap_{K-1}+1] exclusive scan of per-group cost (+ total)
+    uint2* unit_rng;                    // [T * units per table] group range of every work unit (k_unit_ranges)
+    int32_t units_per_table;
     float* pbuf[TT_MAXK + 1];           // partial products P_k of level-k nodes, 2 <= k <= K-2
     float* E;                           // [capU][D] rows (forward) / dE (backward)
     // backward
@@ -124,7 +126,7 @@ struct tt_emb {
     size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
     size_t off_Y[TT_MAXK + 1];
-    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted;
+    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted, off_unit_rng;
     // guard bytes after every workspace region (tt_emb_check_guards): [guard_off[i], guard_off[i] + guard_len[i])
     int num_regions;
     size_t guard_off[96], guard_len[96];
@@ -264,6 +266,7 @@ __device__ __forceinline__ const float* tt_left_operand(const WsView& w, const T
 }
 
 // group range [g0, g1) of work unit q of table t: an equal-cost slice of the table's level-(K-1) groups in sweep order
+// (called by one thread per unit, once per forward: k_unit_ranges)
 __device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uint32_t& g0, uint32_t& g1)
 {
     const TableDesc& td = w.tdesc[t];
@@ -293,12 +296,8 @@ __device__ __forceinline__ void tt_unit_range(const WsView& w, int t, int q, uin
         }
         return lo;
     };
-    // every thread needs both bounds; even and odd lanes each search one and exchange it
-    const bool odd = (threadIdx.x & 1) != 0;
-    const uint32_t mine = lower(odd ? hi_c : lo_c);
-    const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
-    g0 = q == 0 ? a : (odd ? other : mine);
-    g1 = q == Q - 1 ? b : (odd ? mine : other);
+    g0 = q == 0 ? a : lower(lo_c);
+    g1 = q == Q - 1 ? b : lower(hi_c);
 }
 
 __device__ __forceinline__ int tt_find_table64(const int64_t* __restrict__ tb, int T, int64_t v)
