@@ -1536,30 +1536,52 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
     const uint32_t j0 = tt_trank(w, td, k, ik * space), j1 = tt_trank(w, td, k, (ik + 1) * space);
     const int strideY = w.stride[k - 1];
     const uint32_t passes = (j1 - j0 + NQ - 1) / NQ;
+    // The node ids of a pass and the addresses of the nodes' left operands are looked up two passes ahead by NQ threads
+    // (digit-major list -> node -> prefix value or parent -> operand: a chain of dependent loads) and handed to the
+    // CTA through a ring in shared memory, so that staging a pass starts with its cp.async instructions.
+    __shared__ uint32_t s_node[3][NQ];
+    __shared__ const float* s_left[3][NQ];
+    uint32_t pre_node = 0xffffffffu;
+    const float* pre_left = nullptr;
+    auto lookup_ids = [&](uint32_t r) {          // into registers (threads 0..NQ-1)
+        pre_node = 0xffffffffu;
+        pre_left = nullptr;
+        if (tid < NQ && j0 + r * NQ + tid < j1) {
+            pre_node = w.tnode[k][j0 + r * NQ + tid];
+            pre_left = tt_left_operand(w, td, k, pre_node);
+        }
+    };
+    auto publish_ids = [&](uint32_t r) {         // registers -> ring slot of pass r
+        if (tid < NQ) { s_node[r % 3u][tid] = pre_node; s_left[r % 3u][tid] = pre_left; }
+    };
     // stage the NQ nodes of pass r (missing nodes of the last pass are zero-filled)
     auto issue = [&](uint32_t r) {
         const int st = (int)(r & 1u);
-        const uint32_t jb = j0 + r * NQ;
+        const uint32_t* ids = s_node[r % 3u];
+        const float* const* lefts = s_left[r % 3u];
         for (int i = tid; i < NQ * M * (COLS / 4); i += 128) {   // dP_k rows: M * COLS / 4 float4 per node
             const int q = i / (M * (COLS / 4)), rem = i - q * (M * (COLS / 4)), m = rem / (COLS / 4), c4 = rem - m * (COLS / 4);
             float4* dst = reinterpret_cast<float4*>(&sD[st][(q * M + m) * CP + 4 * c4]);
-            if (jb + q < j1) {
-                const uint32_t v = w.tnode[k][jb + q];
-                tt_cp_async16(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
-            } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
+            const uint32_t v = ids[q];
+            if (v != 0xffffffffu) tt_cp_async16(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
+            else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         for (int i = tid; i < NQ * M * (RA / 4); i += 128) {     // P_{k-1} of the parent: M * RA / 4 float4 per node
             const int q = i / (M * (RA / 4)), rem = i - q * (M * (RA / 4)), m = rem / (RA / 4), a4 = rem - m * (RA / 4);
             float4* dst = reinterpret_cast<float4*>(&sA[st][(q * M + m) * AP + 4 * a4]);
-            if (jb + q < j1) {
-                const uint32_t v = w.tnode[k][jb + q];
-                tt_cp_async16(dst, reinterpret_cast<const float4*>(tt_left_operand(w, td, k, v) + m * RA) + a4);
-            } else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (ids[q] != 0xffffffffu) tt_cp_async16(dst, reinterpret_cast<const float4*>(lefts[q] + m * RA) + a4);
+            else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
+    lookup_ids(0);
+    publish_ids(0);
+    lookup_ids(1);
+    publish_ids(1);
+    __syncthreads();
     if (passes > 0) issue(0);
     for (uint32_t r = 0; r < passes; ++r) {
+        lookup_ids(r + 2);          // in flight while this pass is staged and computed; published at the end of the iteration
         if (r + 1 < passes) {
             issue(r + 1);
             asm volatile("cp.async.wait_group 1;" ::: "memory");
@@ -1611,15 +1633,16 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
             const uint32_t ja = j0 + r * NQ + (16 * yrt + g) / M, jb2 = j0 + r * NQ + (16 * yrt + g + 8) / M;
             const int ma = (16 * yrt + g) % M;   // the same row of P for g and g + 8 (M divides 8)
             if (ja < j1) {
-                const uint32_t v = w.tnode[k][ja];
+                const uint32_t v = s_node[r % 3u][(16 * yrt + g) / M];
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + ma * RA + 8 * ynt + 2 * t]) = make_float2(y[0], y[1]);
             }
             if (jb2 < j1) {
-                const uint32_t v = w.tnode[k][jb2];
+                const uint32_t v = s_node[r % 3u][(16 * yrt + g + 8) / M];
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + ma * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
         if ((r & 7u) == 7u) fold(false);   // rounded running sums every eighth pass
+        publish_ids(r + 2);   // its ring slot held pass r - 1
         __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
     }
     fold(true);   // also writes the zeros of a slice without nodes
