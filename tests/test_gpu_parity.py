@@ -490,3 +490,32 @@ def test_invariants_index_order_and_bag_additivity(binding):
     merged_off = wl.offsets[::2].copy()
     out_m = emb.forward(dev(wl.indices), dev(merged_off), 32).cpu().numpy()
     assert np.abs(out_m - (out[0::2] + out[1::2])).max() <= 2e-6 * np.abs(out).max()
+
+
+def test_forward_and_grouping_are_bit_reproducible(binding):
+    # two runs of the same training step on fresh handles: `out` and the grouping are identical bit for bit (nothing in
+    # the forward depends on timing).  The gradients agree to rounding only: the backward sort claims positions with
+    # atomics and the last core's slices are accumulated with vector reductions, so their summation order varies.
+    name, tables, B, pooling = MEDIUM[1]
+    wl = workloads.custom(tables, B, pooling, seed=33, with_grad=True)
+    runs = []
+    for _ in range(2):
+        emb = binding.from_workload(wl, enable_backward=True)
+        out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+        counts = emb.grouping_counts()
+        levels = [emb.export_level(t, k, int(counts[t, k - 1])) for t in range(wl.T) for k in range(1, wl.tables[t].K + 1)]
+        inv = [emb.export_inverse(t, wl.table_slice(t)[0].shape[0]) for t in range(wl.T)]
+        emb.backward(dev(wl.grad_out))
+        runs.append((out, counts, levels, inv, emb.get_grads()))
+    a, b = runs
+    assert np.array_equal(a[0], b[0])
+    assert np.array_equal(a[1], b[1])
+    for la, lb in zip(a[2], b[2]):
+        for x, y in zip(la, lb):
+            assert np.array_equal(x, y)
+    for x, y in zip(a[3], b[3]):
+        assert np.array_equal(x, y)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            scale = max(np.abs(a[4][t][k]).max(), 1e-30)
+            assert np.abs(a[4][t][k] - b[4][t][k]).max() <= 2e-6 * scale
