@@ -265,21 +265,38 @@ __global__ void __launch_bounds__(256) k_dE(WsView w, const float* __restrict__ 
         const bool weighted = w.wsorted && (w.psw || w.pool_mean);
         const float wmine = (weighted && p0 + lane < b) ? __ldg(&w.wsorted[p0 + lane]) : 1.f;
         const int n = (int)min(32u, b - p0);
-        for (int j = 0; j < n; ++j) {
-            const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j);
-            const uint32_t bag = __shfl_sync(0xffffffffu, mine.y, j);
-            const float wj = __shfl_sync(0xffffffffu, wmine, j);
-            if (sl != cur) {
-                const bool open_start = seg_first && prev == cur;
-                if (open_start) acc.store(carry, D, lane);  // head: started in an earlier chunk, ends here
-                else acc.store(w.E + (size_t)cur * D, D, lane);
-                acc.clear();
-                cur = sl;
-                tcur = tt_find_table(w.tb[w.K], w.T, cur);
-                seg_first = false;
+        // four rows of grad_out in flight at a time (their addresses need the table of each pair's slot; positions are
+        // sorted, so the table changes rarely), then the rows are folded in position order
+        const int tmine = lane < n ? tt_find_table_from(w.tb[w.K], w.T, mine.x, tcur) : tcur;
+        for (int j0 = 0; j0 < n; j0 += 4) {
+            RowAcc<VEC, CPL> rowv[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = min(j0 + jj, n - 1);
+                const uint32_t bag = __shfl_sync(0xffffffffu, mine.y, j);
+                const int tj = __shfl_sync(0xffffffffu, tmine, j);
+                rowv[jj].clear();
+                if (j0 + jj < n) rowv[jj].add_row(grad_out + (size_t)bag * gstride + (size_t)tj * D, D, lane, 1.f);
             }
-            acc.add_row(grad_out + (size_t)bag * gstride + (size_t)tcur * D, D, lane, wj);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = j0 + jj;
+                if (j >= n) break;
+                const uint32_t sl = __shfl_sync(0xffffffffu, mine.x, j);
+                const float wj = __shfl_sync(0xffffffffu, wmine, j);
+                if (sl != cur) {
+                    const bool open_start = seg_first && prev == cur;
+                    if (open_start) acc.store(carry, D, lane);  // head: started in an earlier chunk, ends here
+                    else acc.store(w.E + (size_t)cur * D, D, lane);
+                    acc.clear();
+                    cur = sl;
+                    seg_first = false;
+                }
+#pragma unroll
+                for (int i = 0; i < (VEC ? 4 * CPL : CPL); ++i) acc.v[i] = fmaf(wj, rowv[jj].v[i], acc.v[i]);
+            }
         }
+        tcur = __shfl_sync(0xffffffffu, tmine, n - 1);
     }
     const bool open_start = seg_first && prev == cur;
     const bool open_end = next == cur;

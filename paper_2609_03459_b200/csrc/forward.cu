@@ -971,10 +971,12 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
     return cudaGetLastError();
 }
 
-// any D (scalar path): lane handles elements lane, lane+32, ...
+// any D (scalar path): lane handles elements lane, lane + 32, ... (NC of them per pass over the bag); 32 / NC rows in flight
+template <int NC>
 __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict__ out)
 {
     tt_pdl_enter();
+    constexpr int RF = 32 / NC;     // rows in flight
     const int lane = threadIdx.x & 31;
     const int D = w.D;
     const int64_t nb = (int64_t)w.T * w.B;
@@ -988,26 +990,40 @@ __global__ void __launch_bounds__(256) k_pool_scalar(WsView w, float* __restrict
         lo = lo < 0 ? 0 : (lo > w.L ? w.L : lo);
         hi = hi < lo ? lo : (hi > w.L ? w.L : hi);
         float* o = out + (size_t)b * w.T * D + (size_t)t * D;
-        if (w.upairs)
-            for (int64_t l = lo + lane; l < hi; l += 32) w.upairs[l] = make_uint2(tt_lookup_slot(w, td, l, capK), (uint32_t)b);
-        for (int e0 = 0; e0 < D; e0 += 32 * 8) {
-            float acc[8];
+        for (int e0 = 0; e0 < D; e0 += 32 * NC) {
+            float acc[NC];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-            for (int64_t l = lo; l < hi; ++l) {
-                const uint32_t slot = tt_lookup_slot(w, td, l, capK);
-                if (slot == 0xffffffffu) continue;
-                const float* row = w.E + (size_t)slot * D;
-                const float a = w.psw ? __ldg(w.psw + l) : 1.f;
+            for (int c = 0; c < NC; ++c) acc[c] = 0.f;
+            // 32 lookups at a time: every lane looks one slot up (the two dependent loads of a lookup run 32 wide instead of
+            // one after the other), then the rows are added in lookup order, RF row loads in flight
+            for (int64_t l0 = lo; l0 < hi; l0 += 32) {
+                const int n = (int)min((int64_t)32, hi - l0);
+                const uint32_t slot = lane < n ? tt_lookup_slot(w, td, l0 + lane, capK) : 0xffffffffu;
+                const float a = (w.psw && lane < n) ? __ldg(w.psw + l0 + lane) : 1.f;
+                if (w.upairs && e0 == 0 && lane < n) w.upairs[l0 + lane] = make_uint2(slot, (uint32_t)b);
+                for (int j0 = 0; j0 < n; j0 += RF) {
+                    float v[RF][NC], aj[RF];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int idx = e0 + lane + c * 32;
-                    if (idx < D) acc[c] = fmaf(a, __ldg(row + idx), acc[c]);
+                    for (int jj = 0; jj < RF; ++jj) {
+                        const uint32_t sj = __shfl_sync(0xffffffffu, slot, (j0 + jj) & 31);
+                        aj[jj] = __shfl_sync(0xffffffffu, a, (j0 + jj) & 31);
+                        const bool ok = j0 + jj < n && sj != 0xffffffffu;
+                        const float* row = w.E + (size_t)(ok ? sj : 0u) * D;
+#pragma unroll
+                        for (int c = 0; c < NC; ++c) {
+                            const int idx = e0 + lane + c * 32;
+                            v[jj][c] = (ok && idx < D) ? __ldg(row + idx) : 0.f;
+                        }
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < RF; ++jj)
+#pragma unroll
+                        for (int c = 0; c < NC; ++c) acc[c] = fmaf(aj[jj], v[jj][c], acc[c]);
                 }
             }
             const float inv = (w.pool_mean && hi > lo) ? 1.f / (float)(hi - lo) : 1.f;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
+            for (int c = 0; c < NC; ++c) {
                 const int idx = e0 + lane + c * 32;
                 if (idx < D) o[idx] = acc[c] * inv;
             }
@@ -1040,7 +1056,11 @@ cudaError_t tt_launch_pooling(tt_emb* h, float* out, cudaStream_t s)
     const bool vec_ok = (D % 4 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0);
     if (!vec_ok) {
         int pgrid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
-        cudaError_t e0 = tt_launch_pdl(k_pool_scalar, dim3(pgrid < 1 ? 1 : pgrid), dim3(256), 0, s, w, out);
+        const dim3 pg(pgrid < 1 ? 1 : pgrid);
+        cudaError_t e0 = D <= 32 ? tt_launch_pdl(k_pool_scalar<1>, pg, dim3(256), 0, s, w, out)
+                       : D <= 64 ? tt_launch_pdl(k_pool_scalar<2>, pg, dim3(256), 0, s, w, out)
+                       : D <= 128 ? tt_launch_pdl(k_pool_scalar<4>, pg, dim3(256), 0, s, w, out)
+                                  : tt_launch_pdl(k_pool_scalar<8>, pg, dim3(256), 0, s, w, out);
         if (e0 != cudaSuccess) return e0;
         tt_note_launch();
         return cudaGetLastError();
