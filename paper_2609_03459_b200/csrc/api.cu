@@ -308,7 +308,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         h->off_val[k] = TAKE("val", (size_t)v.cap[k] * sizeof(uint32_t));
         h->off_tb[k] = TAKE("tb", (size_t)(T + 1) * sizeof(uint32_t));
         if (k < K) h->off_cstart[k] = TAKE("cstart", ((size_t)v.cap[k] + 1) * sizeof(uint32_t));
-        if (k >= 2) h->off_parent[k] = TAKE("parent", (size_t)v.cap[k] * sizeof(uint32_t));
+        if (k >= 3 && k <= K - 1) h->off_parent[k] = TAKE("parent", (size_t)v.cap[k] * sizeof(uint32_t));   // read by tt_left_operand only
     }
     h->off_cost = TAKE("cost", ((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
     h->off_unit_rng = TAKE("unit_rng", (size_t)T * h->units_per_table * sizeof(uint2));
@@ -405,7 +405,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
         v.val[k] = (uint32_t*)(base + h->off_val[k]);
         v.tb[k] = (uint32_t*)(base + h->off_tb[k]);
         v.cstart[k] = k < K ? (uint32_t*)(base + h->off_cstart[k]) : nullptr;
-        v.parent[k] = k >= 2 ? (uint32_t*)(base + h->off_parent[k]) : nullptr;
+        v.parent[k] = (k >= 3 && k <= K - 1) ? (uint32_t*)(base + h->off_parent[k]) : nullptr;
     }
     v.cost = (uint32_t*)(base + h->off_cost);
     v.unit_rng = (uint2*)(base + h->off_unit_rng);

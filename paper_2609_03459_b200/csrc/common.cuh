@@ -62,7 +62,7 @@ struct WsView {
     uint32_t* scan_tmp;
     uint32_t* val[TT_MAXK + 1];         // level k: prefix value within the table (k = K: row id)
     uint32_t* cstart[TT_MAXK + 1];      // level k < K: first child (level k+1 node); [count] = sentinel
-    uint32_t* parent[TT_MAXK + 1];      // level k >= 2: parent node at level k-1
+    uint32_t* parent[TT_MAXK + 1];      // levels 3..K-1: parent node at level k-1 (null elsewhere: nothing reads it)
     uint32_t* tb[TT_MAXK + 1];          // [T+1] node range of each table at level k
     uint32_t* cost;                     // [cap_{K-1}+1] exclusive scan of per-group cost (+ total)
     uint2* unit_rng;                    // [T * units per table] group range of every work unit (k_unit_ranges)

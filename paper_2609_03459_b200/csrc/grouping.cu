@@ -135,7 +135,7 @@ struct LevelUp {
     {
         const uint32_t* tbc = w.tb[k + 1];
         const int t = tt_find_table_from(tbc, w.T, v, hint);
-        w.parent[k + 1][v] = excl + flag - 1u;
+        if (w.parent[k + 1]) w.parent[k + 1][v] = excl + flag - 1u;   // kept only where a later stage reads it (levels 3..K-1)
         if (flag) {
             w.val[k][excl] = w.val[k + 1][v] / (uint32_t)w.tdesc[t].n[k];
             w.cstart[k][excl] = v;
@@ -191,7 +191,7 @@ __global__ void __launch_bounds__(256) k_nodedup_levels(WsView w)
         for (int k = K; k >= 1; --k) {
             w.val[k][l] = v;
             if (k < K) w.cstart[k][l] = (uint32_t)l;
-            if (k >= 2) w.parent[k][l] = (uint32_t)l;
+            if (w.parent[k]) w.parent[k][l] = (uint32_t)l;
             v /= (uint32_t)td.n[k - 1];
         }
     }
