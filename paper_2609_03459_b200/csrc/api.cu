@@ -92,6 +92,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     int64_t sumN = 0;
     uint64_t words = 0;
     uint64_t twords[TT_MAXK] = {0, 0, 0, 0};
+    uint64_t lwords[TT_MAXK] = {0, 0, 0, 0};
     uint64_t level_space[TT_MAXK + 1] = {0, 0, 0, 0, 0};
     int stride[TT_MAXK + 1] = {0, 0, 0, 0, 0};
     uint64_t c_mid_max = 0, c_last_max = 0;
@@ -139,6 +140,16 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         words += nw;
         if (words >= (1ULL << 32)) return fail(TT_EMB_ERR_ARG);
         for (int k = 1; k <= K; ++k) level_space[k] += td.prefix_space[k];
+        {   // presence bitmaps of the prefix levels: every table starts on a scan-tile boundary, like the row bitmap
+            uint32_t suf = 1;
+            for (int k = K - 1; k >= 1; --k) {
+                suf *= (uint32_t)td.n[k];
+                td.suffix[k] = suf;
+                td.lword_base[k] = (uint32_t)lwords[k];
+                lwords[k] += align_up((size_t)(td.prefix_space[k] / 32 + 1), TT_LSCAN_TILE);
+                if (lwords[k] >= (1ULL << 32)) return fail(TT_EMB_ERR_ARG);
+            }
+        }
         for (int k = 2; k <= K - 1; ++k) {
             td.tword_base[k] = (uint32_t)twords[k];
             td.tnum_words[k] = td.prefix_space[k] / 32 + 1;
@@ -266,6 +277,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     v.cap[K] = (uint32_t)h->capU;
     v.total_words = (uint32_t)words;
     for (int k = 2; k <= K - 1; ++k) v.ttotal_words[k] = (uint32_t)twords[k];
+    for (int k = 1; k <= K - 1; ++k) v.total_words_l[k] = (uint32_t)lwords[k];
 
     // cost unit 2^shift FMAs such that the largest possible total stays below 2^31
     int shift = 0;
@@ -299,10 +311,12 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     h->off_tlstart = TAKE("tlstart", (size_t)(T + 1) * sizeof(int64_t));
     h->off_vlist = TAKE("vlist", (size_t)(2 + TT_MAXK + 1) * T * sizeof(int32_t));
     h->off_bm = TAKE("bm", (size_t)words * sizeof(uint2));
+    for (int k = 1; k <= K - 1; ++k) h->off_bml[k] = TAKE("bml", (size_t)lwords[k] * sizeof(uint2));
     uint64_t scan_max = words;
+    for (int k = 1; k <= K - 1; ++k) if (lwords[k] > scan_max) scan_max = lwords[k];
     for (int k = 1; k <= K; ++k) if (v.cap[k] > scan_max) scan_max = v.cap[k];
     for (int k = 2; k <= K - 1; ++k) if (twords[k] > scan_max) scan_max = twords[k];
-    h->scan_tmp_elems = (size_t)(scan_max / TT_SCAN_TILE + 4);
+    h->scan_tmp_elems = (size_t)(scan_max / TT_LSCAN_TILE + 4);
     h->off_scan = TAKE("scan", h->scan_tmp_elems * sizeof(uint32_t));
     for (int k = 1; k <= K; ++k) {
         h->off_val[k] = TAKE("val", (size_t)v.cap[k] * sizeof(uint32_t));
@@ -400,6 +414,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     v.tl_start = (int64_t*)(base + h->off_tlstart);
     v.vlist = (int32_t*)(base + h->off_vlist);
     v.bm = (uint2*)(base + h->off_bm);
+    for (int k = 1; k <= K - 1; ++k) v.bml[k] = (uint2*)(base + h->off_bml[k]);
     v.scan_tmp = (uint32_t*)(base + h->off_scan);
     for (int k = 1; k <= K; ++k) {
         v.val[k] = (uint32_t*)(base + h->off_val[k]);

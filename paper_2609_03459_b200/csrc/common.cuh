@@ -10,6 +10,8 @@
 #define TT_SCAN_THREADS 256
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
+#define TT_LSCAN_ITEMS 2                                // the short scans of the prefix-level bitmaps
+#define TT_LSCAN_TILE (TT_SCAN_THREADS * TT_LSCAN_ITEMS)
 #define TT_DE_CHUNK 1024                                  // sorted lookups per warp in the dE segment reduction
 #define TT_NUM_STAGES 33                                // 0..8 pipeline stages, 9..20 forward sweep variants -1..10, 21..32 backward sweep variants
 #define TT_STRIPES 8                                     // L2-resident partial copies of the last core's gradient
@@ -29,6 +31,8 @@ struct TableDesc {
     float* grad[TT_MAXK];
     uint32_t word_base;                 // first 32-row word of this table in the presence bitmap
     uint32_t num_words;
+    uint32_t lword_base[TT_MAXK];       // the same for the presence bitmaps of the length-k prefixes, k = 1..K-1
+    uint32_t suffix[TT_MAXK];           // n_{k+1} * .. * n_K: row id / suffix[k] = length-k prefix value, k = 1..K-1
     uint32_t tword_base[TT_MAXK];       // same for the digit-major ("transposed") node bitmaps, levels 2..K-1
     uint32_t tnum_words[TT_MAXK];
     uint32_t prefix_space[TT_MAXK + 1]; // n_1 * .. * n_k (number of possible length-k prefixes), k = 1..K-1
@@ -59,6 +63,8 @@ struct WsView {
                                         // largest tables first inside each list
     int64_t* tl_start;                  // [T+1] first lookup of each table
     uint2* bm;                          // {32 presence bits, number of set bits before this word (global)}
+    uint2* bml[TT_MAXK];                // the same for the length-k prefixes, k = 1..K-1 (one bit per possible prefix)
+    uint32_t total_words_l[TT_MAXK];
     uint32_t* scan_tmp;
     uint32_t* val[TT_MAXK + 1];         // level k: prefix value within the table (k = K: row id)
     uint32_t* cstart[TT_MAXK + 1];      // level k < K: first child (level k+1 node); [count] = sentinel
@@ -123,6 +129,7 @@ struct tt_emb {
     TableDesc* tab;       // host copy [T]
     size_t ws_bytes;
     size_t off_status, off_counters, off_tdesc, off_tlstart, off_bm, off_scan, off_cost, off_E;
+    size_t off_bml[TT_MAXK];
     size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
     size_t off_Y[TT_MAXK + 1];

@@ -4,9 +4,13 @@
 // domain with one presence bit per row.  The bitmaps of all tables (N_t / 8 bytes each) stay resident in
 // the 126 MB L2, so marking costs one L2 access per lookup, and an exclusive scan of the word popcounts
 // yields (a) the ascending list of distinct rows, (b) a rank structure {bits, base} that maps any row id
-// to its slot with one 8-byte load, so no per-lookup inverse map is ever written.  Prefix levels follow
-// by comparing neighbouring entries of the sorted lists (run-length encoding) and compacting with the
-// same scan.  No kernel waits on another CTA.
+// to its slot with one 8-byte load, so no per-lookup inverse map is ever written.  The prefix levels are
+// built the same way: the marking pass also sets one bit per length-k prefix (k < K) in a small bitmap over
+// the prefix space, and a scan of its word popcounts yields the ascending distinct prefixes; the first child of
+// a prefix is a rank look-up in the next level's bitmap, so the run-length encoding of the sorted rows is never
+// walked.  The bits of level k-1 are set while level k is emitted, one word of 32 values at a time (their
+// prefixes are one or two neighbouring values unless the radix is below 32), so the cost of a prefix level is
+// proportional to the words of the level below, not to the lookups.  No kernel waits on another CTA.
 #include "common.cuh"
 #include "scan.cuh"
 
@@ -72,6 +76,39 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
     if (bad) atomicOr(w.status, TT_EMB_STATUS_INDEX);
 }
 
+// ---------------------------------------------------------------------------------------------- marking one level up
+
+// ORs `m` into word `wi` of a presence bitmap for every lane with `on`; lanes of a warp that aim at the same word
+// combine first, and the word is left alone when it already holds the bits
+__device__ __forceinline__ void tt_mark_word(uint2* bitmap, bool on, uint32_t wi, unsigned m)
+{
+    const unsigned act = __activemask();
+    const unsigned peers = __match_any_sync(act, on ? wi : 0xffffffffu);
+    const unsigned all = __reduce_or_sync(peers, on ? m : 0u);
+    if (on && (int)(threadIdx.x & 31) == __ffs(peers) - 1) {
+        unsigned* pw = &bitmap[wi].x;
+        if ((__ldcg(pw) & all) != all) atomicOr(pw, all);
+    }
+}
+
+// `bits` = presence of the level-k values v0 .. v0+31 of table td: sets the bits of their length-(k-1) prefixes
+// (value / radix) in the bitmap of level k-1.  Called by all lanes that emit a word, also with bits == 0.
+__device__ __forceinline__ void tt_mark_parents(const WsView& w, const TableDesc& td, int k, unsigned bits, uint32_t v0, uint32_t radix)
+{
+    uint2* up = w.bml[k - 1];
+    const uint32_t wb = td.lword_base[k - 1];
+    const bool any = bits != 0u;
+    const uint32_t pf = any ? (v0 + (uint32_t)__ffs(bits) - 1u) / radix : 0u;
+    const uint32_t pl = any ? (v0 + 31u - (uint32_t)__clz(bits)) / radix : 0u;
+    tt_mark_word(up, any, wb + (pf >> 5), 1u << (pf & 31));
+    tt_mark_word(up, any && pl != pf, wb + (pl >> 5), 1u << (pl & 31));
+    if (any && pl > pf + 1u)                                   // radix below 32: prefixes that lie wholly inside the word
+        for (uint32_t p = pf + 1u; p < pl; ++p) {
+            const uint32_t lo = p * radix - v0;                // 0 < lo, lo + radix <= 31
+            if (bits & (((1u << radix) - 1u) << lo)) atomicOr(&up[wb + (p >> 5)].x, 1u << (p & 31));
+        }
+}
+
 // ---------------------------------------------------------------------------------------------- level K: rows
 
 struct PopScan {
@@ -90,14 +127,15 @@ struct PopScan {
     __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bm[i].x); }
     __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
     {
-        w.bm[i].y = excl;
+        unsigned bits = w.bm[i].x;
+        w.bm[i] = make_uint2(bits, excl);   // whole 8-byte words: full sectors for the memory system
         const int K = w.K;
         const uint32_t wb = w.tdesc[t].word_base;
         if (i == wb) w.tb[K][t] = excl < w.cap[K] ? excl : w.cap[K];
+        const uint32_t row0 = (i - wb) << 5;
+        tt_mark_parents(w, w.tdesc[t], K, bits, row0, (uint32_t)w.tdesc[t].n[K - 1]);
         if (v) {
-            unsigned bits = w.bm[i].x;
             uint32_t slot = excl;
-            const uint32_t row0 = (i - wb) << 5;
             while (bits) {
                 const int b = __ffs(bits) - 1;
                 bits &= bits - 1;
@@ -115,48 +153,103 @@ struct PopScan {
     }
 };
 
-// ---------------------------------------------------------------------------------------------- level k from level k+1
+// ---------------------------------------------------------------------------------------------- prefix levels
 
-struct LevelUp {
+// number of level-c nodes before the first one whose value is >= pos (c = K: rows; c < K: length-c prefixes)
+__device__ __forceinline__ uint32_t tt_rank_at(const WsView& w, const TableDesc& td, int c, uint32_t pos)
+{
+    const uint2 e = c == w.K ? w.bm[td.word_base + (pos >> 5)] : w.bml[c][td.lword_base[c] + (pos >> 5)];
+    const uint32_t r = e.y + __popc(e.x & ((1u << (pos & 31)) - 1u));
+    const uint32_t lim = w.counters[CTR_LEVEL0 + c];
+    return r < lim ? r : lim;
+}
+
+// Level k < K from its own presence bitmap: the ascending distinct prefixes of every table.  Runs after the scan of
+// level k + 1, which set this level's bits, and sets those of level k - 1.
+struct LevelScan {
     WsView w;
-    int k;  // level being produced (1..K-1); reads level k+1
-    __device__ uint32_t size() const { return w.counters[CTR_LEVEL0 + k + 1]; }
-    __device__ int locate(uint32_t v0) const { return tt_find_table(w.tb[k + 1], w.T, v0); }
-    __device__ uint32_t value(uint32_t v, int hint) const
+    int k;
+    __device__ uint32_t size() const { return w.total_words_l[k]; }
+    __device__ int locate(uint32_t i0) const
     {
-        const uint32_t* tbc = w.tb[k + 1];
-        const int t = tt_find_table_from(tbc, w.T, v, hint);
-        const uint32_t nk = (uint32_t)w.tdesc[t].n[k];  // radix of digit k+1 (0-based core index k)
-        if (v == tbc[t]) return 1u;
-        if ((w.ablation & 1) && k == w.K - 1) return 1u;   // study switch: no prefix reuse, every row opens a group
-        return (w.val[k + 1][v] / nk != w.val[k + 1][v - 1] / nk) ? 1u : 0u;
+        int lo = 0, hi = w.T;
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (w.tdesc[mid].lword_base[k] <= i0) lo = mid; else hi = mid;
+        }
+        return lo;
     }
-    __device__ void emit(uint32_t v, uint32_t excl, uint32_t flag, int hint) const
+    __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bml[k][i].x); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
     {
-        const uint32_t* tbc = w.tb[k + 1];
-        const int t = tt_find_table_from(tbc, w.T, v, hint);
-        if (w.parent[k + 1]) w.parent[k + 1][v] = excl + flag - 1u;   // kept only where a later stage reads it (levels 3..K-1)
-        if (flag) {
-            w.val[k][excl] = w.val[k + 1][v] / (uint32_t)w.tdesc[t].n[k];
-            w.cstart[k][excl] = v;
-            if (v == tbc[t]) w.tb[k][t] = excl;
+        unsigned bits = w.bml[k][i].x;
+        w.bml[k][i] = make_uint2(bits, excl);
+        const TableDesc& td = w.tdesc[t];
+        const uint32_t wb = td.lword_base[k];
+        if (i == wb) w.tb[k][t] = excl < w.cap[k] ? excl : w.cap[k];
+        const uint32_t p0 = (i - wb) << 5;
+        if (k >= 2) tt_mark_parents(w, td, k, bits, p0, (uint32_t)td.n[k - 1]);
+        if (v) {
+            uint32_t slot = excl;
+            while (bits) {
+                const int b = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (slot < w.cap[k]) w.val[k][slot] = p0 + b;
+                ++slot;
+            }
         }
     }
     __device__ void total(uint32_t tot) const
     {
+        if (tot > w.cap[k]) { atomicOr(w.status, TT_EMB_STATUS_OVERFLOW); tot = w.cap[k]; }
         w.counters[CTR_LEVEL0 + k] = tot;
-        w.cstart[k][tot] = size();
         w.tb[k][w.T] = tot;
     }
 };
 
-// tables without any node at level k+1 never had tb[k][t] written: inherit from the next table
-__global__ void k_fix_tb(WsView w, int k)
+// Links of every level-k node, one thread each (the rank look-ups are random 8-byte loads: kept out of the scan, where
+// one thread would walk them one after the other): first child at the level below (k + 1; with the "no prefix reuse"
+// study switch the groups of level K-1 are the rows themselves, so level K-2 points at rows), and, for the levels
+// whose left operand is looked up through it (3..K-1), the parent at level k-1.
+__global__ void __launch_bounds__(256) k_links(WsView w, int k)
 {
     tt_pdl_enter();
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (int t = w.T - 1; t >= 0; --t)
-            if (w.tb[k + 1][t] == w.tb[k + 1][t + 1]) w.tb[k][t] = w.tb[k][t + 1];
+    const int K = w.K;
+    const uint32_t count = w.counters[CTR_LEVEL0 + k];
+    const bool rows = (w.ablation & 1) && k == K - 1;          // level k holds one node per row, not per prefix
+    const int c = ((w.ablation & 1) && k + 1 == K - 1) ? K : k + 1;
+    const uint32_t first = blockIdx.x * blockDim.x + threadIdx.x;
+    if (first == 0 && !rows) w.cstart[k][count] = w.counters[CTR_LEVEL0 + c];
+    for (uint32_t v = first; v < count; v += gridDim.x * blockDim.x) {
+        const int t = tt_find_table(w.tb[k], w.T, v);
+        const TableDesc& td = w.tdesc[t];
+        if (!rows) {
+            const uint32_t mult = c == k + 1 ? (uint32_t)td.n[k] : td.suffix[k];   // value of the first possible child
+            w.cstart[k][v] = tt_rank_at(w, td, c, w.val[k][v] * mult);
+        }
+        if (w.parent[k]) {
+            const uint32_t up = rows ? w.val[K][v] / td.suffix[k - 1] : w.val[k][v] / (uint32_t)td.n[k - 1];
+            w.parent[k][v] = tt_rank_at(w, td, k - 1, up);
+        }
+    }
+}
+
+// Study switch "no prefix reuse": every distinct row is a group of its own at level K-1
+__global__ void __launch_bounds__(256) k_unique_groups(WsView w)
+{
+    tt_pdl_enter();
+    const int K = w.K, k = K - 1;
+    const uint32_t count = w.counters[CTR_LEVEL0 + K] < w.cap[k] ? w.counters[CTR_LEVEL0 + K] : w.cap[k];
+    const uint32_t first = blockIdx.x * blockDim.x + threadIdx.x;
+    if (first == 0) {
+        w.counters[CTR_LEVEL0 + k] = count;
+        w.cstart[k][count] = count;
+    }
+    if (first <= (uint32_t)w.T) w.tb[k][first] = w.tb[K][first] < count ? w.tb[K][first] : count;
+    for (uint32_t v = first; v < count; v += gridDim.x * blockDim.x) {
+        const int t = tt_find_table(w.tb[K], w.T, v);
+        w.val[k][v] = w.val[K][v] / (uint32_t)w.tdesc[t].n[K - 1];
+        w.cstart[k][v] = v;
     }
 }
 
@@ -214,6 +307,8 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
         return cudaGetLastError();
     }
     if ((e = cudaMemsetAsync(w.bm, 0, (size_t)w.total_words * sizeof(uint2), s)) != cudaSuccess) return e;
+    for (int k = 1; k <= w.K - 1; ++k)
+        if ((e = cudaMemsetAsync(w.bml[k], 0, (size_t)w.total_words_l[k] * sizeof(uint2), s)) != cudaSuccess) return e;
     if ((e = tt_launch_pdl(k_check_offsets, dim3(g0), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     if (w.L > 0) {
@@ -225,9 +320,15 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
     PopScan ps{w};
     if ((e = tt_scan(ps, w.total_words, w.scan_tmp, s)) != cudaSuccess) return e;
     for (int k = w.K - 1; k >= 1; --k) {
-        LevelUp lu{w, k};
-        if ((e = tt_scan(lu, w.cap[k + 1], w.scan_tmp, s)) != cudaSuccess) return e;
-        if ((e = tt_launch_pdl(k_fix_tb, dim3(1), dim3(32), 0, s, w, k)) != cudaSuccess) return e;
+        LevelScan ls{w, k};
+        if ((e = tt_scan<LevelScan, TT_LSCAN_ITEMS>(ls, w.total_words_l[k], w.scan_tmp, s)) != cudaSuccess) return e;
+        if ((w.ablation & 1) && k == w.K - 1) {   // the scan still sets the bits of level K-2; its nodes are replaced
+            if ((e = tt_launch_pdl(k_unique_groups, dim3(h->sm_count * 8), dim3(256), 0, s, w)) != cudaSuccess) return e;
+            tt_note_launch();
+        }
+    }
+    for (int k = w.K - 1; k >= 1; --k) {   // after all the scans: a node's links look into the levels on both sides
+        if ((e = tt_launch_pdl(k_links, dim3(h->sm_count * 8), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
         tt_note_launch();
     }
     return cudaGetLastError();

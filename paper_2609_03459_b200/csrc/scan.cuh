@@ -9,6 +9,8 @@
 //   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int hint) const;   called once per element in the apply pass
 //   __device__ void total(uint32_t tot) const;              called by one thread with the grand total
 //   WsView w;                                               w.counters[CTR_SCAN_TICKET] is the ticket (zero between scans)
+// ITEMS = elements per thread (tile = TT_SCAN_THREADS * ITEMS): the default for long inputs, fewer for short ones whose
+// tiles should still spread over the SMs.
 #pragma once
 #include "common.cuh"
 
@@ -56,25 +58,26 @@ __device__ __forceinline__ void tt_scan_spine_cta(const F& f, uint32_t* tile_sum
     if (threadIdx.x == 0) f.total(carry);
 }
 
-template <class F>
+template <class F, int ITEMS>
 __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t* tile_sums)
 {
     tt_pdl_enter();
+    constexpr int TILE = TT_SCAN_THREADS * ITEMS;
     __shared__ uint32_t sm[34];
     __shared__ uint32_t ticket;
     const uint32_t n = f.size();
-    const uint32_t ntiles = (uint32_t)(((uint64_t)n + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
+    const uint32_t ntiles = (uint32_t)(((uint64_t)n + TILE - 1) / TILE);
     if (ntiles == 0) {   // nothing to scan: the first CTA still reports the total
         if (blockIdx.x == 0 && threadIdx.x == 0) f.total(0u);
         return;
     }
     if (blockIdx.x >= ntiles) return;
-    const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
+    const uint64_t base = (uint64_t)blockIdx.x * TILE;
     uint32_t s = 0;
     const int hint = f.locate((uint32_t)base);
     // a sum has no order: neighbouring threads take neighbouring elements (coalesced)
 #pragma unroll 4
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
         if (i < n) s += f.value((uint32_t)i, hint);
     }
@@ -94,60 +97,62 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
 }
 
 // Elements are read and emitted striped (thread t takes elements t, t + 256, ...: coalesced for the functor's loads and
-// stores), scanned blocked (thread t owns elements 16 t .. 16 t + 15); the two orders meet in shared memory, padded by
+// stores), scanned blocked (thread t owns elements ITEMS t .. ITEMS t + ITEMS - 1); the two orders meet in shared memory, padded by
 // one word per 32 so that both access patterns are free of bank conflicts.
 __device__ __forceinline__ int tt_scan_pad(int i) { return i + (i >> 5); }
 
-template <class F>
+template <class F, int ITEMS>
 __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
 {
     tt_pdl_enter();
+    constexpr int TILE = TT_SCAN_THREADS * ITEMS;
     __shared__ uint32_t sm[34];
-    __shared__ uint32_t sv[TT_SCAN_TILE + TT_SCAN_TILE / 32];
+    __shared__ uint32_t sv[TILE + TILE / 32];
     const uint32_t n = f.size();
-    const uint64_t base = (uint64_t)blockIdx.x * TT_SCAN_TILE;
+    const uint64_t base = (uint64_t)blockIdx.x * TILE;
     if (base >= n) return;
-    uint32_t v[TT_SCAN_ITEMS];
+    uint32_t v[ITEMS];
     const int hint = f.locate((uint32_t)base);
 #pragma unroll
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
         v[j] = i < n ? f.value((uint32_t)i, hint) : 0u;
         sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)] = v[j];
     }
     __syncthreads();
     uint32_t s = 0;
-    uint32_t mine[TT_SCAN_ITEMS];
+    uint32_t mine[ITEMS];
 #pragma unroll
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
-        mine[j] = sv[tt_scan_pad(threadIdx.x * TT_SCAN_ITEMS + j)];
+    for (int j = 0; j < ITEMS; ++j) {
+        mine[j] = sv[tt_scan_pad(threadIdx.x * ITEMS + j)];
         s += mine[j];
     }
     uint32_t tot;
     uint32_t ex = tile_sums[blockIdx.x] + tt_block_excl_scan(s, sm, tot);
 #pragma unroll
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
-        sv[tt_scan_pad(threadIdx.x * TT_SCAN_ITEMS + j)] = ex;   // exclusive prefix of element 16 t + j
+    for (int j = 0; j < ITEMS; ++j) {
+        sv[tt_scan_pad(threadIdx.x * ITEMS + j)] = ex;   // exclusive prefix of element ITEMS t + j
         ex += mine[j];
     }
     __syncthreads();
 #pragma unroll
-    for (int j = 0; j < TT_SCAN_ITEMS; ++j) {
+    for (int j = 0; j < ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
         if (i < n) f.emit((uint32_t)i, sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)], v[j], hint);
     }
 }
 
-// capacity = host-known upper bound of f.size(); tmp must hold ceil(capacity / TT_SCAN_TILE) + 1 words
-template <class F>
+// capacity = host-known upper bound of f.size(); tmp must hold ceil(capacity / tile) + 1 words
+template <class F, int ITEMS = TT_SCAN_ITEMS>
 static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, cudaStream_t s)
 {
-    unsigned tiles = (unsigned)((capacity + TT_SCAN_TILE - 1) / TT_SCAN_TILE);
+    constexpr int TILE = TT_SCAN_THREADS * ITEMS;
+    unsigned tiles = (unsigned)((capacity + TILE - 1) / TILE);
     if (tiles == 0) tiles = 1;
-    cudaError_t e = tt_launch_pdl(tt_scan_reduce<F>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, tmp);
+    cudaError_t e = tt_launch_pdl(tt_scan_reduce<F, ITEMS>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, tmp);
     if (e != cudaSuccess) return e;
     tt_note_launch();
-    if ((e = tt_launch_pdl(tt_scan_apply<F>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, (const uint32_t*)tmp)) != cudaSuccess) return e;
+    if ((e = tt_launch_pdl(tt_scan_apply<F, ITEMS>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, (const uint32_t*)tmp)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
