@@ -127,11 +127,11 @@ struct PopScan {
     __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bm[i].x); }
     __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
     {
-        unsigned bits = w.bm[i].x;
-        w.bm[i] = make_uint2(bits, excl);   // whole 8-byte words: full sectors for the memory system
+        w.bm[i].y = excl;
         const int K = w.K;
         const uint32_t wb = w.tdesc[t].word_base;
         if (i == wb) w.tb[K][t] = excl < w.cap[K] ? excl : w.cap[K];
+        unsigned bits = w.bm[i].x;
         const uint32_t row0 = (i - wb) << 5;
         tt_mark_parents(w, w.tdesc[t], K, bits, row0, (uint32_t)w.tdesc[t].n[K - 1]);
         if (v) {
@@ -182,11 +182,11 @@ struct LevelScan {
     __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bml[k][i].x); }
     __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
     {
-        unsigned bits = w.bml[k][i].x;
-        w.bml[k][i] = make_uint2(bits, excl);
+        w.bml[k][i].y = excl;
         const TableDesc& td = w.tdesc[t];
         const uint32_t wb = td.lword_base[k];
         if (i == wb) w.tb[k][t] = excl < w.cap[k] ? excl : w.cap[k];
+        unsigned bits = w.bml[k][i].x;
         const uint32_t p0 = (i - wb) << 5;
         if (k >= 2) tt_mark_parents(w, td, k, bits, p0, (uint32_t)td.n[k - 1]);
         if (v) {
