@@ -336,10 +336,12 @@ def test_forward_only_handle_and_repeat_calls(binding):
     assert_close(out3, oracle.forward_workload(wl2), "second batch out")
 
 
+@pytest.mark.parametrize("case", ["tiled-r16-r32", "tiled-k4-r64", "k2", "k4"])
 @pytest.mark.parametrize("flags", [1, 2, 3, 4, 6])
-def test_ablation_switches_keep_the_result(binding, flags):
-    # the study switches (no prefix reuse / static schedule / no de-duplication) change cost, never values
-    name, tables, B, pooling = MEDIUM[1]
+def test_ablation_switches_keep_the_result(binding, flags, case):
+    # the study switches (no prefix reuse / static schedule / no de-duplication) change cost, never values;
+    # with two, three and four cores (the prefix levels above a level of per-row groups link to rows, not to prefixes)
+    name, tables, B, pooling = next(c for c in MEDIUM if c[0] == case)
     wl = workloads.custom(tables, B, pooling, seed=21)
     emb = binding.from_workload(wl, ablation=flags)
     out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
@@ -347,7 +349,16 @@ def test_ablation_switches_keep_the_result(binding, flags):
     assert_close(out, oracle.forward_workload(wl), f"ablation {flags} out")
     counts = emb.grouping_counts()
     if flags & 1:   # every distinct row is its own group
-        assert np.array_equal(counts[:, 1], counts[:, 2])
+        assert np.array_equal(counts[:, -2], counts[:, -1])
+    if flags == 1:  # ... and the prefix levels above it are the ordinary ones, counting rows under each prefix
+        for t, s in enumerate(wl.tables):
+            g = oracle.grouping(s.n, wl.table_slice(t)[0])
+            for k in range(1, s.K - 1):
+                lev = g["levels"][k - 1]
+                assert counts[t, k - 1] == lev["vals"].shape[0]
+                vals, rc, _ = emb.export_level(t, k, int(counts[t, k - 1]), with_lookup_counts=False)
+                np.testing.assert_array_equal(vals, lev["vals"])
+                np.testing.assert_array_equal(rc, lev["row_counts"])
     if flags & 4:   # every lookup is a row, a group and a first-level node of its own
         per_table = wl.offsets[np.arange(1, wl.T + 1) * wl.B] - wl.offsets[np.arange(wl.T) * wl.B]
         for k in range(counts.shape[1]):
