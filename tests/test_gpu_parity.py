@@ -471,12 +471,27 @@ def test_guard_check_medium_shapes_and_detection(binding):
     assert emb.check_guards() == "guard_list"
 
 
-def test_unique_row_capacity_overflow_is_flagged(binding):
-    spec = TableSpec(5000, (18, 18, 18), (4, 4, 4), (1, 4, 4, 1), 0.5, "normal", 0.1)
-    wl = workloads.custom([spec], 50, 20, seed=4)
-    emb = binding.from_workload(wl, max_unique_rows=100)
-    emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+@pytest.mark.parametrize("spec", [
+    TableSpec(5000, (18, 18, 18), (4, 4, 4), (1, 4, 4, 1), 0.5, "normal", 0.1),
+    TableSpec(30_000, (14, 13, 13, 13), (2, 4, 4, 4), (1, 6, 9, 5, 1), 0.5, "normal", 0.1),
+    TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 0.5, "uniform", 0.1),
+], ids=["k3", "k4", "k2"])
+def test_unique_row_capacity_overflow_is_flagged(binding, spec):
+    # more distinct rows than the handle was sized for: flagged, and every kernel of the forward and of the backward
+    # still stays inside its workspace region (the rows past the capacity are dropped, prefix levels are clipped to them)
+    wl = workloads.custom([spec, spec], 50, 20, seed=4, with_grad=True)
+    emb = binding.from_workload(wl, max_unique_rows=100, enable_backward=True)
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
     assert emb.status() & binding.STATUS_OVERFLOW
+    assert np.isfinite(out.cpu().numpy()).all()
+    emb.backward(dev(wl.grad_out))
+    assert emb.check_guards() is None
+    # the same handle is fine again with a batch that fits
+    small = workloads.custom([spec, spec], 4, 5, seed=5)
+    small.cores = wl.cores
+    out2 = emb.forward(dev(small.indices), dev(small.offsets), small.B).cpu().numpy()
+    assert emb.status() == 0
+    assert_close(out2, oracle.forward_workload(small), "after overflow")
 
 
 def test_pack_unpack_round_trip(binding):
