@@ -212,6 +212,15 @@ static inline cudaError_t tt_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// a += v as two packed fp32 additions (add.rn.f32x2 of sm_100: two IEEE additions per instruction and lane, the same
+// results as four scalar additions; the row sums of the gathers are bound by issue slots)
+__device__ __forceinline__ void tt_add4(float4& a, const float4& v)
+{
+    const float2 lo = __fadd2_rn(make_float2(a.x, a.y), make_float2(v.x, v.y));
+    const float2 hi = __fadd2_rn(make_float2(a.z, a.w), make_float2(v.z, v.w));
+    a = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+
 // ---- small device helpers ----
 __device__ __forceinline__ int tt_find_table(const uint32_t* __restrict__ tb, int T, uint32_t v)
 {

@@ -899,7 +899,7 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
 #pragma unroll
                     for (int jj = jq; jj < jq + PGRP; ++jj) {
                         const float4 v = buf[(RPI * jj + sub) * R4 + lr];
-                        part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w;
+                        tt_add4(part, v);
                     }
                 } else {
 #pragma unroll
@@ -909,7 +909,7 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
                         if (((valid >> j) & 1u) && lane_on) {
                             const float4 v = buf[j * R4 + lr];
                             if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
-                            else { part.x += v.x; part.y += v.y; part.z += v.z; part.w += v.w; }
+                            else tt_add4(part, v);
                         }
                     }
                 }
