@@ -92,6 +92,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     int64_t sumN = 0;
     uint64_t words = 0;
     uint64_t twords[TT_MAXK] = {0, 0, 0, 0};
+    uint64_t rest_tiles = 0;
     uint64_t lwords[TT_MAXK] = {0, 0, 0, 0};
     uint64_t level_space[TT_MAXK + 1] = {0, 0, 0, 0, 0};
     int stride[TT_MAXK + 1] = {0, 0, 0, 0, 0};
@@ -138,6 +139,8 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
         uint64_t nw = align_up((size_t)((td.N + 31) / 32), TT_SCAN_TILE);
         td.num_words = (uint32_t)nw;
         words += nw;
+        td.rest_base = (uint32_t)rest_tiles;
+        if (nw / TT_SCAN_TILE > TT_HEAD_TILES) rest_tiles += nw / TT_SCAN_TILE - TT_HEAD_TILES;
         if (words >= (1ULL << 32)) return fail(TT_EMB_ERR_ARG);
         for (int k = 1; k <= K; ++k) level_space[k] += td.prefix_space[k];
         {   // presence bitmaps of the prefix levels: every table starts on a scan-tile boundary, like the row bitmap
@@ -278,6 +281,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     v.total_words = (uint32_t)words;
     for (int k = 2; k <= K - 1; ++k) v.ttotal_words[k] = (uint32_t)twords[k];
     for (int k = 1; k <= K - 1; ++k) v.total_words_l[k] = (uint32_t)lwords[k];
+    v.rest_tiles = (uint32_t)rest_tiles;
 
     // cost unit 2^shift FMAs such that the largest possible total stays below 2^31
     int shift = 0;

@@ -10,6 +10,7 @@
 #define TT_SCAN_THREADS 256
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
+#define TT_HEAD_TILES 4                                 // leading scan tiles of a table that are emitted first (see PopScan)
 #define TT_LSCAN_ITEMS 2                                // the short scans of the prefix-level bitmaps
 #define TT_LSCAN_TILE (TT_SCAN_THREADS * TT_LSCAN_ITEMS)
 #define TT_DE_CHUNK 1024                                  // sorted lookups per warp in the dE segment reduction
@@ -31,6 +32,7 @@ struct TableDesc {
     float* grad[TT_MAXK];
     uint32_t word_base;                 // first 32-row word of this table in the presence bitmap
     uint32_t num_words;
+    uint32_t rest_base;                 // scan tiles of the tables before this one, their first TT_HEAD_TILES each left out
     uint32_t lword_base[TT_MAXK];       // the same for the presence bitmaps of the length-k prefixes, k = 1..K-1
     uint32_t suffix[TT_MAXK];           // n_{k+1} * .. * n_K: row id / suffix[k] = length-k prefix value, k = 1..K-1
     uint32_t tword_base[TT_MAXK];       // same for the digit-major ("transposed") node bitmaps, levels 2..K-1
@@ -65,6 +67,7 @@ struct WsView {
     uint2* bm;                          // {32 presence bits, number of set bits before this word (global)}
     uint2* bml[TT_MAXK];                // the same for the length-k prefixes, k = 1..K-1 (one bit per possible prefix)
     uint32_t total_words_l[TT_MAXK];
+    uint32_t rest_tiles;                // scan tiles of the row bitmap beyond the first TT_HEAD_TILES of every table
     uint32_t* scan_tmp;
     uint32_t* val[TT_MAXK + 1];         // level k: prefix value within the table (k = K: row id)
     uint32_t* cstart[TT_MAXK + 1];      // level k < K: first child (level k+1 node); [count] = sentinel

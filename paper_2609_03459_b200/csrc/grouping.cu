@@ -8,9 +8,9 @@
 // built the same way: the marking pass also sets one bit per length-k prefix (k < K) in a small bitmap over
 // the prefix space, and a scan of its word popcounts yields the ascending distinct prefixes; the first child of
 // a prefix is a rank look-up in the next level's bitmap, so the run-length encoding of the sorted rows is never
-// walked.  The bits of level k-1 are set while level k is emitted, one word of 32 values at a time (their
-// prefixes are one or two neighbouring values unless the radix is below 32), so the cost of a prefix level is
-// proportional to the words of the level below, not to the lookups.  No kernel waits on another CTA.
+// walked.  A prefix is present when the scanned bitmap of the level below counts at least one node in its range of
+// children (two rank look-ups per possible prefix, k_prefix_bits), so the cost of a prefix level is proportional
+// to the size of its prefix space, not to the lookups or the rows.  No kernel waits on another CTA.
 #include "common.cuh"
 #include "scan.cuh"
 
@@ -76,37 +76,39 @@ __global__ void __launch_bounds__(256) k_mark(WsView w)
     if (bad) atomicOr(w.status, TT_EMB_STATUS_INDEX);
 }
 
-// ---------------------------------------------------------------------------------------------- marking one level up
-
-// ORs `m` into word `wi` of a presence bitmap for every lane with `on`; lanes of a warp that aim at the same word
-// combine first, and the word is left alone when it already holds the bits
-__device__ __forceinline__ void tt_mark_word(uint2* bitmap, bool on, uint32_t wi, unsigned m)
+// val[excl ..] = v0 + (positions of the set bits of `bits`), clipped at `cap`.  Called by all lanes that emit a word
+// (also with bits == 0).  A lane writes the first bits of its own word; a word with more is handed to the whole warp,
+// one lane per bit: a densely set word then is one coalesced store instead of 32 stores that each touch another
+// sector (a tile of the popular first rows of a table took 80 us against 20 us for a sparse one).
+#define EMIT_OWN 8
+__device__ __forceinline__ void tt_emit_set_bits(uint32_t* __restrict__ val, uint32_t cap, unsigned bits, uint32_t excl, uint32_t v0)
 {
     const unsigned act = __activemask();
-    const unsigned peers = __match_any_sync(act, on ? wi : 0xffffffffu);
-    const unsigned all = __reduce_or_sync(peers, on ? m : 0u);
-    if (on && (int)(threadIdx.x & 31) == __ffs(peers) - 1) {
-        unsigned* pw = &bitmap[wi].x;
-        if ((__ldcg(pw) & all) != all) atomicOr(pw, all);
+    const int lane = threadIdx.x & 31;
+    const bool dense = __popc(bits) > EMIT_OWN;
+    if (!dense) {
+        uint32_t slot = excl;
+#pragma unroll
+        for (int it = 0; it < EMIT_OWN; ++it)
+            if (bits) {
+                const int b = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (slot < cap) val[slot] = v0 + b;
+                ++slot;
+            }
     }
-}
-
-// `bits` = presence of the level-k values v0 .. v0+31 of table td: sets the bits of their length-(k-1) prefixes
-// (value / radix) in the bitmap of level k-1.  Called by all lanes that emit a word, also with bits == 0.
-__device__ __forceinline__ void tt_mark_parents(const WsView& w, const TableDesc& td, int k, unsigned bits, uint32_t v0, uint32_t radix)
-{
-    uint2* up = w.bml[k - 1];
-    const uint32_t wb = td.lword_base[k - 1];
-    const bool any = bits != 0u;
-    const uint32_t pf = any ? (v0 + (uint32_t)__ffs(bits) - 1u) / radix : 0u;
-    const uint32_t pl = any ? (v0 + 31u - (uint32_t)__clz(bits)) / radix : 0u;
-    tt_mark_word(up, any, wb + (pf >> 5), 1u << (pf & 31));
-    tt_mark_word(up, any && pl != pf, wb + (pl >> 5), 1u << (pl & 31));
-    if (any && pl > pf + 1u)                                   // radix below 32: prefixes that lie wholly inside the word
-        for (uint32_t p = pf + 1u; p < pl; ++p) {
-            const uint32_t lo = p * radix - v0;                // 0 < lo, lo + radix <= 31
-            if (bits & (((1u << radix) - 1u) << lo)) atomicOr(&up[wb + (p >> 5)].x, 1u << (p & 31));
+    unsigned todo = __ballot_sync(act, dense);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const unsigned wb = __shfl_sync(act, bits, src);
+        const uint32_t we = __shfl_sync(act, excl, src);
+        const uint32_t wv = __shfl_sync(act, v0, src);
+        if ((wb >> lane) & 1u) {
+            const uint32_t sl = we + __popc(wb & ((1u << lane) - 1u));
+            if (sl < cap) val[sl] = wv + lane;
         }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------- level K: rows
@@ -124,25 +126,37 @@ struct PopScan {
         }
         return lo;
     }
-    __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bm[i].x); }
-    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
+    __device__ uint32_t value(uint32_t i, int) const { return w.bm[i].x; }
+    __device__ uint32_t weight(uint32_t bits) const { return __popc(bits); }
+    // The first TT_HEAD_TILES tiles of every table go first (CTAs 0 .. HEAD * T - 1, tile position major), the others
+    // follow in ascending order.  With the identity rank-to-row mapping the popular rows are the first rows of a table:
+    // those tiles are densely set and emit a hundred times the rows of a tile further down (70 us against 6), and in
+    // ascending order the dense tiles of the last tables ran alone at the end of the kernel.
+    __device__ uint32_t tile_of(uint32_t cta) const
+    {
+        const uint32_t head = (uint32_t)TT_HEAD_TILES * (uint32_t)w.T;
+        if (cta < head) {
+            const uint32_t p = cta / (uint32_t)w.T, t = cta % (uint32_t)w.T;
+            const TableDesc& td = w.tdesc[t];
+            return p < td.num_words / TT_SCAN_TILE ? td.word_base / TT_SCAN_TILE + p : 0xffffffffu;
+        }
+        const uint32_t m = cta - head;
+        if (m >= w.rest_tiles) return 0xffffffffu;
+        int lo = 0, hi = w.T;                    // the table whose remaining tiles hold number m
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (w.tdesc[mid].rest_base <= m) lo = mid; else hi = mid;
+        }
+        return w.tdesc[lo].word_base / TT_SCAN_TILE + TT_HEAD_TILES + (m - w.tdesc[lo].rest_base);
+    }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t bits, int t) const
     {
         w.bm[i].y = excl;
         const int K = w.K;
         const uint32_t wb = w.tdesc[t].word_base;
         if (i == wb) w.tb[K][t] = excl < w.cap[K] ? excl : w.cap[K];
-        unsigned bits = w.bm[i].x;
         const uint32_t row0 = (i - wb) << 5;
-        tt_mark_parents(w, w.tdesc[t], K, bits, row0, (uint32_t)w.tdesc[t].n[K - 1]);
-        if (v) {
-            uint32_t slot = excl;
-            while (bits) {
-                const int b = __ffs(bits) - 1;
-                bits &= bits - 1;
-                if (slot < w.cap[K]) w.val[K][slot] = row0 + b;
-                ++slot;
-            }
-        }
+        tt_emit_set_bits(w.val[K], w.cap[K], bits, excl, row0);
     }
     __device__ void total(uint32_t tot) const
     {
@@ -164,8 +178,54 @@ __device__ __forceinline__ uint32_t tt_rank_at(const WsView& w, const TableDesc&
     return r < lim ? r : lim;
 }
 
+// number of level-c nodes of all tables before position x of table td (x inside the table's space), from the scanned bitmap
+__device__ __forceinline__ uint32_t tt_rank_excl(const WsView& w, const TableDesc& td, int c, uint32_t x)
+{
+    const uint2 e = c == w.K ? w.bm[td.word_base + (x >> 5)] : w.bml[c][td.lword_base[c] + (x >> 5)];
+    return e.y + __popc(e.x & ((1u << (x & 31)) - 1u));
+}
+// ... up to and including position x
+__device__ __forceinline__ uint32_t tt_rank_incl(const WsView& w, const TableDesc& td, int c, uint32_t x)
+{
+    const uint2 e = c == w.K ? w.bm[td.word_base + (x >> 5)] : w.bml[c][td.lword_base[c] + (x >> 5)];
+    return e.y + __popc(e.x & (0xffffffffu >> (31 - (x & 31))));
+}
+
+// Presence bitmap of level k < K (one bit per possible length-k prefix of every table) from the scanned bitmap of level
+// k + 1: prefix p is present when some node of level k + 1 lies in [p n_{k+1}, (p + 1) n_{k+1}).  One warp per word, one
+// lane per prefix (the two rank look-ups of a prefix are dependent loads: 32 of them one after the other per thread
+// took 25 us even for the few words of level 1); the words are written whole (no memset, no atomics).
+__global__ void __launch_bounds__(256) k_prefix_bits(WsView w, int k)
+{
+    tt_pdl_enter();
+    const int c = k + 1;
+    const int lane = threadIdx.x & 31;
+    const uint32_t nwords = w.total_words_l[k];
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < nwords; i += nwarps) {
+        int lo_t = 0, hi_t = w.T;
+        while (hi_t - lo_t > 1) {
+            const int mid = (lo_t + hi_t) >> 1;
+            if (w.tdesc[mid].lword_base[k] <= i) lo_t = mid; else hi_t = mid;
+        }
+        const TableDesc& td = w.tdesc[lo_t];
+        const uint32_t p = ((i - td.lword_base[k]) << 5) + lane;
+        const uint32_t radix = (uint32_t)td.n[k];                       // radix of digit k + 1
+        const uint32_t space_c = c == w.K ? (uint32_t)td.N : td.prefix_space[c];
+        const uint64_t lo = (uint64_t)p * radix;
+        bool present = false;
+        if (p < td.prefix_space[k] && lo < space_c) {                    // rows past N do not exist
+            uint64_t hi = lo + radix;
+            if (hi > space_c) hi = space_c;
+            present = tt_rank_incl(w, td, c, (uint32_t)hi - 1u) != tt_rank_excl(w, td, c, (uint32_t)lo);
+        }
+        const unsigned bits = __ballot_sync(0xffffffffu, present);
+        if (lane == 0) w.bml[k][i] = make_uint2(bits, 0u);
+    }
+}
+
 // Level k < K from its own presence bitmap: the ascending distinct prefixes of every table.  Runs after the scan of
-// level k + 1, which set this level's bits, and sets those of level k - 1.
+// level k + 1 and k_prefix_bits, which sets this level's bits.
 struct LevelScan {
     WsView w;
     int k;
@@ -179,25 +239,16 @@ struct LevelScan {
         }
         return lo;
     }
-    __device__ uint32_t value(uint32_t i, int) const { return __popc(w.bml[k][i].x); }
-    __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int t) const
+    __device__ uint32_t value(uint32_t i, int) const { return w.bml[k][i].x; }
+    __device__ uint32_t weight(uint32_t bits) const { return __popc(bits); }
+    __device__ void emit(uint32_t i, uint32_t excl, uint32_t bits, int t) const
     {
         w.bml[k][i].y = excl;
         const TableDesc& td = w.tdesc[t];
         const uint32_t wb = td.lword_base[k];
         if (i == wb) w.tb[k][t] = excl < w.cap[k] ? excl : w.cap[k];
-        unsigned bits = w.bml[k][i].x;
         const uint32_t p0 = (i - wb) << 5;
-        if (k >= 2) tt_mark_parents(w, td, k, bits, p0, (uint32_t)td.n[k - 1]);
-        if (v) {
-            uint32_t slot = excl;
-            while (bits) {
-                const int b = __ffs(bits) - 1;
-                bits &= bits - 1;
-                if (slot < w.cap[k]) w.val[k][slot] = p0 + b;
-                ++slot;
-            }
-        }
+        tt_emit_set_bits(w.val[k], w.cap[k], bits, excl, p0);
     }
     __device__ void total(uint32_t tot) const
     {
@@ -307,8 +358,6 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
         return cudaGetLastError();
     }
     if ((e = cudaMemsetAsync(w.bm, 0, (size_t)w.total_words * sizeof(uint2), s)) != cudaSuccess) return e;
-    for (int k = 1; k <= w.K - 1; ++k)
-        if ((e = cudaMemsetAsync(w.bml[k], 0, (size_t)w.total_words_l[k] * sizeof(uint2), s)) != cudaSuccess) return e;
     if ((e = tt_launch_pdl(k_check_offsets, dim3(g0), dim3(256), 0, s, w)) != cudaSuccess) return e;
     tt_note_launch();
     if (w.L > 0) {
@@ -318,8 +367,14 @@ cudaError_t tt_launch_grouping(tt_emb* h, cudaStream_t s)
         tt_note_launch();
     }
     PopScan ps{w};
-    if ((e = tt_scan(ps, w.total_words, w.scan_tmp, s)) != cudaSuccess) return e;
+    if ((e = tt_scan(ps, w.total_words, w.scan_tmp, s, (unsigned)(TT_HEAD_TILES * w.T) + w.rest_tiles)) != cudaSuccess) return e;
     for (int k = w.K - 1; k >= 1; --k) {
+        {
+            const uint32_t want = (w.total_words_l[k] + 7u) / 8u;   // a warp per word
+            const uint32_t g = want < (uint32_t)h->sm_count * 8u ? (want ? want : 1u) : (uint32_t)h->sm_count * 8u;
+            if ((e = tt_launch_pdl(k_prefix_bits, dim3(g), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
+            tt_note_launch();
+        }
         LevelScan ls{w, k};
         if ((e = tt_scan<LevelScan, TT_LSCAN_ITEMS>(ls, w.total_words_l[k], w.scan_tmp, s)) != cudaSuccess) return e;
         if ((w.ablation & 1) && k == w.K - 1) {   // the scan still sets the bits of level K-2; its nodes are replaced

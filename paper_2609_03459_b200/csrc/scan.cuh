@@ -6,13 +6,28 @@
 //   __device__ int locate(uint32_t i0) const;               once per tile, for its first element: a hint handed to value / emit
 //                                                           (e.g. the table the tile starts in, so that elements need no search)
 //   __device__ uint32_t value(uint32_t i, int hint) const;  input i
+//   __device__ uint32_t weight(uint32_t v) const;           optional: the amount that input v adds to the scan (default: v
+//                                                           itself); emit is handed v, so that a functor whose input is a
+//                                                           word of flags does not have to load it a second time
 //   __device__ void emit(uint32_t i, uint32_t excl, uint32_t v, int hint) const;   called once per element in the apply pass
 //   __device__ void total(uint32_t tot) const;              called by one thread with the grand total
+//   __device__ uint32_t tile_of(uint32_t cta) const;        optional: the tile that CTA `cta` of the apply pass takes
+//                                                           (0xffffffff: none), for an order other than ascending,
+//                                                           e.g. the tiles with the most output first
 //   WsView w;                                               w.counters[CTR_SCAN_TICKET] is the ticket (zero between scans)
 // ITEMS = elements per thread (tile = TT_SCAN_THREADS * ITEMS): the default for long inputs, fewer for short ones whose
 // tiles should still spread over the SMs.
 #pragma once
 #include "common.cuh"
+
+template <class F>
+__device__ __forceinline__ auto tt_scan_amount(const F& f, uint32_t v, int) -> decltype(f.weight(v)) { return f.weight(v); }
+template <class F>
+__device__ __forceinline__ uint32_t tt_scan_amount(const F&, uint32_t v, long) { return v; }
+template <class F>
+__device__ __forceinline__ auto tt_scan_tile(const F& f, uint32_t cta, int) -> decltype(f.tile_of(cta)) { return f.tile_of(cta); }
+template <class F>
+__device__ __forceinline__ uint32_t tt_scan_tile(const F&, uint32_t cta, long) { return cta; }
 
 __device__ __forceinline__ uint32_t tt_block_excl_scan(uint32_t x, uint32_t* sm /* [34] */, uint32_t& block_total)
 {
@@ -79,7 +94,7 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
 #pragma unroll 4
     for (int j = 0; j < ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
-        if (i < n) s += f.value((uint32_t)i, hint);
+        if (i < n) s += tt_scan_amount(f, f.value((uint32_t)i, hint), 0);
     }
     uint32_t tot;
     tt_block_excl_scan(s, sm, tot);
@@ -102,14 +117,16 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_reduce(F f, uint32_t*
 __device__ __forceinline__ int tt_scan_pad(int i) { return i + (i >> 5); }
 
 template <class F, int ITEMS>
-__global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
+__global__ void __launch_bounds__(TT_SCAN_THREADS, 4) tt_scan_apply(F f, const uint32_t* __restrict__ tile_sums)
 {
     tt_pdl_enter();
     constexpr int TILE = TT_SCAN_THREADS * ITEMS;
     __shared__ uint32_t sm[34];
     __shared__ uint32_t sv[TILE + TILE / 32];
     const uint32_t n = f.size();
-    const uint64_t base = (uint64_t)blockIdx.x * TILE;
+    const uint32_t tile = tt_scan_tile(f, blockIdx.x, 0);
+    if (tile == 0xffffffffu) return;
+    const uint64_t base = (uint64_t)tile * TILE;
     if (base >= n) return;
     uint32_t v[ITEMS];
     const int hint = f.locate((uint32_t)base);
@@ -117,7 +134,7 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint
     for (int j = 0; j < ITEMS; ++j) {
         const uint64_t i = base + (uint64_t)j * TT_SCAN_THREADS + threadIdx.x;
         v[j] = i < n ? f.value((uint32_t)i, hint) : 0u;
-        sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)] = v[j];
+        sv[tt_scan_pad(j * TT_SCAN_THREADS + threadIdx.x)] = i < n ? tt_scan_amount(f, v[j], 0) : 0u;
     }
     __syncthreads();
     uint32_t s = 0;
@@ -128,7 +145,7 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint
         s += mine[j];
     }
     uint32_t tot;
-    uint32_t ex = tile_sums[blockIdx.x] + tt_block_excl_scan(s, sm, tot);
+    uint32_t ex = tile_sums[tile] + tt_block_excl_scan(s, sm, tot);
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) {
         sv[tt_scan_pad(threadIdx.x * ITEMS + j)] = ex;   // exclusive prefix of element ITEMS t + j
@@ -142,9 +159,10 @@ __global__ void __launch_bounds__(TT_SCAN_THREADS) tt_scan_apply(F f, const uint
     }
 }
 
-// capacity = host-known upper bound of f.size(); tmp must hold ceil(capacity / tile) + 1 words
+// capacity = host-known upper bound of f.size(); tmp must hold ceil(capacity / tile) + 1 words; apply_ctas: size of the
+// apply grid for a functor with tile_of (default: one CTA per tile)
 template <class F, int ITEMS = TT_SCAN_ITEMS>
-static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, cudaStream_t s)
+static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, cudaStream_t s, unsigned apply_ctas = 0)
 {
     constexpr int TILE = TT_SCAN_THREADS * ITEMS;
     unsigned tiles = (unsigned)((capacity + TILE - 1) / TILE);
@@ -152,7 +170,7 @@ static inline cudaError_t tt_scan(const F& f, uint64_t capacity, uint32_t* tmp, 
     cudaError_t e = tt_launch_pdl(tt_scan_reduce<F, ITEMS>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, tmp);
     if (e != cudaSuccess) return e;
     tt_note_launch();
-    if ((e = tt_launch_pdl(tt_scan_apply<F, ITEMS>, dim3(tiles), dim3(TT_SCAN_THREADS), 0, s, f, (const uint32_t*)tmp)) != cudaSuccess) return e;
+    if ((e = tt_launch_pdl(tt_scan_apply<F, ITEMS>, dim3(apply_ctas ? apply_ctas : tiles), dim3(TT_SCAN_THREADS), 0, s, f, (const uint32_t*)tmp)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
 }
