@@ -1478,17 +1478,18 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 // up to N * 2^-24 of the sum; the dG accumulators are therefore folded into running sums (a rounded fp32
 // add into the CTA's own gradient slice, which stays in L2) every eighth pass, which keeps every chain at 48 or 96
 // products whatever the length of the node list.
-template <int M, int RA, int COLS>   // M = P_{k-1}: 4 or 2 rows per node
+template <int M, int RA, int COLS, int NQF = 1>   // M = P_{k-1}: 4 or 2 rows per node; NQF: 2 = twice the nodes per pass
 __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, int lbase)
 {
     tt_pdl_enter();
     static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && (COLS % 32 == 0 || COLS == 16), "rows per node; r_{k-1}; columns per warp");
-    constexpr int NQ = 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16, 32 or 64 stacked rows per pass
+    static_assert(NQF == 1 || NQF == 2, "one or two Y row tiles per warp");
+    constexpr int NQ = NQF * 512 / (RA * M), AP = RA + 8, CP = COLS + 8;   // NQ * M = 16, 32 or 64 stacked rows per pass (x NQF)
     constexpr bool AHALF = RA == 8;          // dG: a = 8..15 of the one m-tile do not exist: zero operands, not stored
     constexpr int MT = AHALF ? 1 : RA / 16;  // dG: m-tiles over a
     constexpr int CW = COLS >= 32 ? COLS / 4 : 8;   // dG: columns per warp (16 columns: warps 0 and 1 only)
     constexpr int NTW = CW / 8;              // dG: n-tiles per warp
-    constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ / 4 row tiles of four nodes; NTY * NQ / 4 = 4 warps
+    constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ * M / 16 row tiles; NTY * NQ * M / 16 = 4 NQF tasks, NQF per warp
     constexpr int KTY = COLS / 8;            // Y: k steps over c
     __shared__ __align__(16) float sA[2][NQ * M * AP];
     __shared__ __align__(16) float sD[2][NQ * M * CP];
@@ -1500,7 +1501,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, g = lane >> 2, t = lane & 3;
     const float* __restrict__ Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
     // Y: this warp's n-tile of a and its four nodes
-    const int ynt = wid % NTY, yrt = wid / NTY;
+    const int ynt = wid % NTY, yrt0 = wid / NTY;   // task wid + 4 yi: the same n-tile, row tile yrt0 + yi * 4 / NTY
     Tf32Pair bY[KTY][2];
 #pragma unroll
     for (int kt = 0; kt < KTY; ++kt) {
@@ -1633,8 +1634,10 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
                 for (int mt = 0; mt < MT; ++mt) tt_mma_3xtf32(acc[mt][nt], a[mt], b);
             }
         }
-        // ---- Y of this warp's sixteen stacked rows and eight values of a
-        {
+        // ---- Y of this warp's sixteen stacked rows (NQF times) and eight values of a
+#pragma unroll
+        for (int yi = 0; yi < NQF; ++yi) {
+            const int yrt = yrt0 + yi * (4 / NTY);
             float y[4] = {0.f, 0.f, 0.f, 0.f};
             const float* Ra = D_ + (16 * yrt + g) * CP;       // row g of the tile: stacked row 16 yrt + g
             const float* Rb = D_ + (16 * yrt + g + 8) * CP;   // row g + 8
@@ -1658,7 +1661,7 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
                 *reinterpret_cast<float2*>(&w.Y[k][(size_t)v * strideY + ma * RA + 8 * ynt + 2 * t]) = make_float2(y[2], y[3]);
             }
         }
-        if ((r & 7u) == 7u) fold(false);   // rounded running sums every eighth pass
+        if ((r & (8u / NQF - 1u)) == 8u / NQF - 1u) fold(false);   // rounded running sums every eighth pass (fourth with twice the nodes)
         publish_ids(r + 2);   // its ring slot held pass r - 1
         __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
     }
@@ -1745,9 +1748,9 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // grid of variant v: its own tables only, slices up to the largest n_k among them
         auto mgrid = [&](int v) { return dim3(h->mmaxn[k][v + 1], h->mcount[k][v + 1]); };
         auto mlist = [&](int v) { return (2 + k) * h->T + h->mbase[k][v + 1]; };
-        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128>, mgrid(0), dim3(128), 0, st(), w, k, 0, mlist(0))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128, 2>, mgrid(0), dim3(128), 0, st(), w, k, 0, mlist(0))) != cudaSuccess) return e; tt_note_launch(); }
         if (any_fast[1]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 128>, mgrid(1), dim3(128), 0, st(), w, k, 1, mlist(1))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64>, mgrid(2), dim3(128), 0, st(), w, k, 2, mlist(2))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64, 2>, mgrid(2), dim3(128), 0, st(), w, k, 2, mlist(2))) != cudaSuccess) return e; tt_note_launch(); }
         if (any_fast[3]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 64>, mgrid(3), dim3(128), 0, st(), w, k, 3, mlist(3))) != cudaSuccess) return e; tt_note_launch(); }
         if (any_fast[4]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 128>, mgrid(4), dim3(128), 0, st(), w, k, 4, mlist(4))) != cudaSuccess) return e; tt_note_launch(); }
         if (any_fast[5]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 64>, mgrid(5), dim3(128), 0, st(), w, k, 5, mlist(5))) != cudaSuccess) return e; tt_note_launch(); }
