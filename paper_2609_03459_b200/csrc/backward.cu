@@ -1470,7 +1470,8 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 //   dG_k[a][c] += sum_{node, m} P_{k-1}[node][m][a] * dP_k[node][m][c]   M = a, N = c, K = 8 stacked rows (node, m);
 //                 a warp owns COLS/4 columns c of the slice, accumulators stay in registers over the whole list
 //   Y[node][m][a] = sum_c dP_k[node][m][c] * G_k[a][c]                   M = 16 stacked rows, N = 8 values of a,
-//                 K = c; the slice fragments (split into TF32 head and tail once) stay in registers;
+//                 K = c; the slice sits unsplit in shared memory (its 64 registers of split fragments per thread
+//                 held the kernel at three CTAs per SM; at ~95 registers five are resident);
 //                 warp -> (n-tile of a, tile of sixteen stacked rows)
 // k_mid_sum then adds the Y rows of each parent's (contiguous) children.
 // Row strides RA + 8 and COLS + 8 floats make every fragment load from shared memory conflict-free or 2-way.
@@ -1478,8 +1479,15 @@ __global__ void __launch_bounds__(256) k_mid_slice(WsView w, int k)
 // up to N * 2^-24 of the sum; the dG accumulators are therefore folded into running sums (a rounded fp32
 // add into the CTA's own gradient slice, which stays in L2) every eighth pass, which keeps every chain at 48 or 96
 // products whatever the length of the node list.
+template <int M, int RA, int COLS, int NQF = 1>
+constexpr size_t tt_mid_smem_bytes()
+{
+    constexpr int NQ = NQF * 512 / (RA * M);
+    return sizeof(float) * (size_t)(2 * NQ * M * (RA + 8) + 2 * NQ * M * (COLS + 8) + RA * (COLS + 4));
+}
+
 template <int M, int RA, int COLS, int NQF = 1>   // M = P_{k-1}: 4 or 2 rows per node; NQF: 2 = twice the nodes per pass
-__global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, int lbase)
+__global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant, int lbase)
 {
     tt_pdl_enter();
     static_assert((M == 4 || M == 2) && (RA == 8 || RA % 16 == 0) && (COLS % 32 == 0 || COLS == 16), "rows per node; r_{k-1}; columns per warp");
@@ -1491,8 +1499,9 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
     constexpr int NTW = CW / 8;              // dG: n-tiles per warp
     constexpr int NTY = RA / 8;              // Y: n-tiles over a (4 or 2); NQ * M / 16 row tiles; NTY * NQ * M / 16 = 4 NQF tasks, NQF per warp
     constexpr int KTY = COLS / 8;            // Y: k steps over c
-    __shared__ __align__(16) float sA[2][NQ * M * AP];
-    __shared__ __align__(16) float sD[2][NQ * M * CP];
+    extern __shared__ __align__(16) float mid_sm[];   // [2][NQ M AP] P rows, [2][NQ M CP] dP rows, [RA][COLS + 4] slice (tt_mid_smem_bytes)
+    float* const sA = mid_sm;
+    float* const sD = sA + 2 * NQ * M * AP;
     const int t_ = w.vlist[lbase + blockIdx.y];   // the tables of this variant, largest first: their long node lists start early
     const TableDesc& td = w.tdesc[t_];
     const int kc = k - 1;
@@ -1502,12 +1511,17 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
     const float* __restrict__ Bsl = td.core[kc] + (size_t)ik * td.slice_floats[kc];
     // Y: this warp's n-tile of a and its four nodes
     const int ynt = wid % NTY, yrt0 = wid / NTY;   // task wid + 4 yi: the same n-tile, row tile yrt0 + yi * 4 / NTY
-    Tf32Pair bY[KTY][2];
-#pragma unroll
-    for (int kt = 0; kt < KTY; ++kt) {
-        bY[kt][0] = tt_split_tf32(__ldg(Bsl + (size_t)(8 * ynt + g) * COLS + 8 * kt + t));
-        bY[kt][1] = tt_split_tf32(__ldg(Bsl + (size_t)(8 * ynt + g) * COLS + 8 * kt + t + 4));
+    // the slice G_k[i_k] for the Y product: unsplit in shared memory (row pitch COLS + 4: the fragment loads of a warp hit
+    // 32 different banks), split at every use: registers for a fifth CTA per SM count for more than the 2 x 3 integer
+    // operations per fragment
+    constexpr int BP = COLS + 4;
+    float* const sB = sD + 2 * NQ * M * CP;
+    for (int i = tid; i < RA * (COLS / 4); i += 128) {
+        const int a_ = i / (COLS / 4), c4 = i - a_ * (COLS / 4);
+        *reinterpret_cast<float4*>(&sB[a_ * BP + 4 * c4]) = __ldg(reinterpret_cast<const float4*>(Bsl + (size_t)a_ * COLS) + c4);
     }
+    // (the first barrier of the pass loop, or the one after the ring is primed, orders these stores before their use)
+    const float* const sBw = sB + (8 * ynt + g) * BP + t;
     float acc[MT][NTW][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -1579,14 +1593,14 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
         const float* const* lefts = s_left[r % 3u];
         for (int i = tid; i < NQ * M * (COLS / 4); i += 128) {   // dP_k rows: M * COLS / 4 float4 per node
             const int q = i / (M * (COLS / 4)), rem = i - q * (M * (COLS / 4)), m = rem / (COLS / 4), c4 = rem - m * (COLS / 4);
-            float4* dst = reinterpret_cast<float4*>(&sD[st][(q * M + m) * CP + 4 * c4]);
+            float4* dst = reinterpret_cast<float4*>(&sD[st * NQ * M * CP + (q * M + m) * CP + 4 * c4]);
             const uint32_t v = ids[q];
             if (v != 0xffffffffu) tt_cp_async16(dst, reinterpret_cast<const float4*>(w.dP[k] + (size_t)v * w.stride[k] + m * COLS) + c4);
             else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         for (int i = tid; i < NQ * M * (RA / 4); i += 128) {     // P_{k-1} of the parent: M * RA / 4 float4 per node
             const int q = i / (M * (RA / 4)), rem = i - q * (M * (RA / 4)), m = rem / (RA / 4), a4 = rem - m * (RA / 4);
-            float4* dst = reinterpret_cast<float4*>(&sA[st][(q * M + m) * AP + 4 * a4]);
+            float4* dst = reinterpret_cast<float4*>(&sA[st * NQ * M * AP + (q * M + m) * AP + 4 * a4]);
             if (ids[q] != 0xffffffffu) tt_cp_async16(dst, reinterpret_cast<const float4*>(lefts[q] + m * RA) + a4);
             else *dst = make_float4(0.f, 0.f, 0.f, 0.f);
         }
@@ -1607,8 +1621,8 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         __syncthreads();
-        const float* A_ = sA[r & 1u];
-        const float* D_ = sD[r & 1u];
+        const float* A_ = sA + (r & 1u) * (NQ * M * AP);
+        const float* D_ = sD + (r & 1u) * (NQ * M * CP);
         // ---- dG: eight stacked rows (node, m) give k = 8
 #pragma unroll
         for (int p = 0; p < NQ * M / 8; ++p) {
@@ -1648,7 +1662,10 @@ __global__ void __launch_bounds__(128) k_mid_mma(WsView w, int k, int variant, i
                 a[1] = tt_split_tf32(Rb[8 * kt + t]);
                 a[2] = tt_split_tf32(Ra[8 * kt + t + 4]);
                 a[3] = tt_split_tf32(Rb[8 * kt + t + 4]);
-                tt_mma_3xtf32(y, a, bY[kt]);
+                Tf32Pair by[2];
+                by[0] = tt_split_tf32(sBw[8 * kt]);
+                by[1] = tt_split_tf32(sBw[8 * kt + 4]);
+                tt_mma_3xtf32(y, a, by);
             }
             const uint32_t ja = j0 + r * NQ + (16 * yrt + g) / M, jb2 = j0 + r * NQ + (16 * yrt + g + 8) / M;
             const int ma = (16 * yrt + g) % M;   // the same row of P for g and g + 8 (M divides 8)
@@ -1718,6 +1735,15 @@ cudaError_t tt_launch_tlist(tt_emb* h, int k, cudaStream_t s)
     return cudaGetLastError();
 }
 
+template <int M, int RA, int COLS>
+static cudaError_t tt_launch_mid(dim3 grid, cudaStream_t st, const WsView& w, int k, int variant, int lbase)
+{
+    constexpr size_t smem = tt_mid_smem_bytes<M, RA, COLS>();
+    cudaError_t e = cudaFuncSetAttribute(k_mid_mma<M, RA, COLS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return tt_launch_pdl(k_mid_mma<M, RA, COLS>, grid, dim3(128), smem, st, w, k, variant, lbase);
+}
+
 cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
 {
     WsView& w = h->v;
@@ -1748,17 +1774,17 @@ cudaError_t tt_launch_bwd_middle(tt_emb* h, cudaStream_t s)
         // grid of variant v: its own tables only, slices up to the largest n_k among them
         auto mgrid = [&](int v) { return dim3(h->mmaxn[k][v + 1], h->mcount[k][v + 1]); };
         auto mlist = [&](int v) { return (2 + k) * h->T + h->mbase[k][v + 1]; };
-        if (any_fast[0]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 128, 2>, mgrid(0), dim3(128), 0, st(), w, k, 0, mlist(0))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[1]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 128>, mgrid(1), dim3(128), 0, st(), w, k, 1, mlist(1))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[2]) { if ((e = tt_launch_pdl(k_mid_mma<4, 32, 64, 2>, mgrid(2), dim3(128), 0, st(), w, k, 2, mlist(2))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[3]) { if ((e = tt_launch_pdl(k_mid_mma<4, 16, 64>, mgrid(3), dim3(128), 0, st(), w, k, 3, mlist(3))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[4]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 128>, mgrid(4), dim3(128), 0, st(), w, k, 4, mlist(4))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[5]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 64>, mgrid(5), dim3(128), 0, st(), w, k, 5, mlist(5))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[6]) { if ((e = tt_launch_pdl(k_mid_mma<2, 32, 64>, mgrid(6), dim3(128), 0, st(), w, k, 6, mlist(6))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[7]) { if ((e = tt_launch_pdl(k_mid_mma<2, 16, 32>, mgrid(7), dim3(128), 0, st(), w, k, 7, mlist(7))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[8]) { if ((e = tt_launch_pdl(k_mid_mma<4, 8, 32>, mgrid(8), dim3(128), 0, st(), w, k, 8, mlist(8))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[9]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 32>, mgrid(9), dim3(128), 0, st(), w, k, 9, mlist(9))) != cudaSuccess) return e; tt_note_launch(); }
-        if (any_fast[10]) { if ((e = tt_launch_pdl(k_mid_mma<2, 8, 16>, mgrid(10), dim3(128), 0, st(), w, k, 10, mlist(10))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[0]) { if ((e = tt_launch_mid<4, 32, 128>(mgrid(0), st(), w, k, 0, mlist(0))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[1]) { if ((e = tt_launch_mid<4, 16, 128>(mgrid(1), st(), w, k, 1, mlist(1))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[2]) { if ((e = tt_launch_mid<4, 32, 64>(mgrid(2), st(), w, k, 2, mlist(2))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[3]) { if ((e = tt_launch_mid<4, 16, 64>(mgrid(3), st(), w, k, 3, mlist(3))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[4]) { if ((e = tt_launch_mid<2, 32, 128>(mgrid(4), st(), w, k, 4, mlist(4))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[5]) { if ((e = tt_launch_mid<2, 16, 64>(mgrid(5), st(), w, k, 5, mlist(5))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[6]) { if ((e = tt_launch_mid<2, 32, 64>(mgrid(6), st(), w, k, 6, mlist(6))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[7]) { if ((e = tt_launch_mid<2, 16, 32>(mgrid(7), st(), w, k, 7, mlist(7))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[8]) { if ((e = tt_launch_mid<4, 8, 32>(mgrid(8), st(), w, k, 8, mlist(8))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[9]) { if ((e = tt_launch_mid<2, 8, 32>(mgrid(9), st(), w, k, 9, mlist(9))) != cudaSuccess) return e; tt_note_launch(); }
+        if (any_fast[10]) { if ((e = tt_launch_mid<2, 8, 16>(mgrid(10), st(), w, k, 10, mlist(10))) != cudaSuccess) return e; tt_note_launch(); }
         if (fork && (e = tt_join(h, s, 4)) != cudaSuccess) return e;
         if (nfast > 0) {
             if ((e = tt_launch_pdl(k_mid_sum, dim3(h->sm_count * 8), dim3(256), 0, s, w, k)) != cudaSuccess) return e;
