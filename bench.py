@@ -390,6 +390,7 @@ def main():
 
     # ---- roofline denominators measured in this run
     fp32_peak = binding.probe_fp32()
+    mma_peak = binding.probe_mma()   # warp-level mma.sync m16n8k8 TF32 instructions per second
     l2_gather = binding.probe_gather(32 << 20, device=device)
     hbm_gather = binding.probe_gather(2 << 30, device=device)
     hbm_gbs, peak_src = measured_peaks()
@@ -594,8 +595,14 @@ def main():
             slots = variant_slots(v, bwd)
             ach = slots / (ms * 1e-3) / 1e12
             share = variant_rows.get(v, 0) / max(work["U_rows"], 1)
+            # the same work in the unit of the tensor path: three m16n8k8 instructions per 1024 slots if every product
+            # ran there (the forward sweeps do; the backward sweeps rebuild the intermediate product on the FP32 pipe);
+            # padding of the small shape variants is not counted
+            mma_min = 3.0 * slots / 1024.0
             kernels[name] = (ms, {"kernel": name, "bound": "alu", "achieved": ach, "peak": fp32_peak / 1e12,
                                   "unit": "T FP32 lane-ops/s", "frac": ach / (fp32_peak / 1e12),
+                                  "mma_sync": {"instructions_equiv": mma_min, "per_s": mma_min / (ms * 1e-3), "peak_per_s": mma_peak,
+                                               "frac_equiv": mma_min / (ms * 1e-3) / mma_peak},
                                   "traffic": traffic_of("k_sweep_bwd" if bwd else "k_sweep_fwd", share),
                                   "peak_source": "independent-FMA-chain probe in this run",
                                   "note": "FMA-equivalent slots of the contractions this kernel performs; the row stages "
@@ -607,7 +614,9 @@ def main():
         roofline = dict(kernels[dominant][1], ms_per_launch=kernels[dominant][0])
     else:
         roofline = None
-    kernel_rooflines = {k: {"ms": v[0], "frac": v[1]["frac"], "bound": v[1]["bound"]} for k, v in kernels.items()}
+    kernel_rooflines = {k: dict({"ms": v[0], "frac": v[1]["frac"], "bound": v[1]["bound"]},
+                                **({"mma_sync_frac_equiv": v[1]["mma_sync"]["frac_equiv"]} if "mma_sync" in v[1] else {}))
+                        for k, v in kernels.items()}
     tot_slots = work["fwd_slots"] + (work["bwd_slots"] if train else 0)
     tot_bytes = work["fwd_hbm_bytes"] + (work["bwd_hbm_bytes"] if train else 0)
     tot_l2 = work["fwd_l2_bytes"] + (work["bwd_l2_bytes"] if train else 0)
@@ -633,6 +642,7 @@ def main():
                          "cuda_graph_ms_per_step": fwd_graph_ms},
         "stage_ms": stage_ms, "solo_kernel_ms": solo_ms, "roofline": roofline, "kernel_rooflines": kernel_rooflines, "step_roofline": step_roof,
         "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
+                  "mma_sync_tf32_m16n8k8_per_s": mma_peak,
                   "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},
         "work": work, "device_status": status, "clocks": clocks, "e2e": e2e,
         "gpu_launches": int(round(launches_per_step)),

@@ -255,6 +255,12 @@ int tt_emb_stage_ms(tt_emb_t h, int32_t stage, float* ms);
 /* Independent-FMA-chain micro-benchmark: FP32 lane-instructions per second of the current device. SYNCHRONISES. */
 int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t stream);
 /*
+ * Independent-chain micro-benchmark of the tensor path the contraction kernels use: warp-level
+ * mma.sync.m16n8k8 TF32 instructions (1024 multiply-adds each) per second of the current device.  A product of the
+ * path (Sec. 3.2: C = A.B, E = C.D) costs three of them per 1024 multiply-adds (3xTF32).  SYNCHRONISES.
+ */
+int tt_emb_probe_mma(double* mma_per_second, tt_emb_stream_t stream);
+/*
  * Random 256-byte-row gather bandwidth (bytes/s) from a caller-provided DEVICE buffer of `bytes`
  * bytes (<= L2 size measures L2, >> L2 measures HBM).  scratch_idx: DEVICE int32[num_rows_read].  SYNCHRONISES.
  */

@@ -81,6 +81,7 @@ _SIGS = {
     "tt_emb_enable_timing": (ctypes.c_int, [_vp, _i32]),
     "tt_emb_stage_ms": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_f32)]),
     "tt_emb_probe_fp32": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
+    "tt_emb_probe_mma": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_probe_gather": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp, _i64, ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_launch_count": (ctypes.c_int, [ctypes.POINTER(_i64), _i32]),
     "tt_emb_table_variant": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i32)]),
@@ -390,6 +391,12 @@ def launch_count(reset: bool = False) -> int:
 def probe_fp32() -> float:
     v = ctypes.c_double()
     _check(lib.tt_emb_probe_fp32(ctypes.byref(v), _stream_ptr()), "tt_emb_probe_fp32")
+    return float(v.value)
+
+
+def probe_mma() -> float:
+    v = ctypes.c_double()
+    _check(lib.tt_emb_probe_mma(ctypes.byref(v), _stream_ptr()), "tt_emb_probe_mma")
     return float(v.value)
 
 

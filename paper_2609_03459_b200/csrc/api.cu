@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include "common.cuh"
+#include "mma.cuh"
 
 static thread_local int g_last_cuda_error = 0;
 static thread_local long long g_launches = 0;
@@ -786,6 +787,55 @@ extern "C" int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t strea
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     *slots_per_second = best;
+    return TT_EMB_OK;
+}
+
+// eight independent accumulator chains of mma.sync.m16n8k8 (TF32) per warp: the issue rate of the tensor path that the
+// contraction kernels use
+__global__ void __launch_bounds__(256) k_probe_mma(float* out, int iters)
+{
+    float d[8][4];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) { d[c][0] = 0.f; d[c][1] = 0.f; d[c][2] = 0.f; d[c][3] = 0.f; }
+    const uint32_t a0 = threadIdx.x, a1 = threadIdx.x * 3u, a2 = 7u, a3 = 9u, b0 = threadIdx.x ^ 5u, b1 = 11u;
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) tt_mma_tf32(d[c], a0, a1, a2, a3, b0, b1);
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) sum += d[c][0] + d[c][1] + d[c][2] + d[c][3];
+    if (sum == 123.456f) out[0] = sum;  // never true; keeps the chains alive
+}
+
+extern "C" int tt_emb_probe_mma(double* mma_per_second, tt_emb_stream_t stream)
+{
+    if (!mma_per_second) return TT_EMB_ERR_ARG;
+    int sms = 0;
+    if (!tt_device_ok(&sms)) return TT_EMB_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    float* dsink = nullptr;
+    TT_CUDA(cudaGetSymbolAddress((void**)&dsink, g_probe_sink));
+    cudaEvent_t e0, e1;
+    TT_CUDA(cudaEventCreate(&e0));
+    TT_CUDA(cudaEventCreate(&e1));
+    const int iters = 10000;
+    double best = 0.0;
+    for (int rep = 0; rep < 4; ++rep) {
+        cudaEventRecord(e0, s);
+        k_probe_mma<<<sms * 2, 256, 0, s>>>(dsink, iters);
+        tt_note_launch();
+        cudaEventRecord(e1, s);
+        cudaError_t e = cudaEventSynchronize(e1);
+        if (e != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); g_last_cuda_error = (int)e; return TT_EMB_ERR_CUDA; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double rate = (double)sms * 2 * 8 * 8 * iters / (ms * 1e-3);   // CTAs x warps x chains x iterations
+        if (rep > 0 && rate > best) best = rate;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *mma_per_second = best;
     return TT_EMB_OK;
 }
 

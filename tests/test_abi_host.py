@@ -89,6 +89,7 @@ def test_call_order_and_missing_device_errors(b):
         assert b.lib.tt_emb_bind(h, ptrs, 256 * 1000, 1 << 40, None) == b.TT_EMB_ERR_ARCH
         v = ctypes.c_double()
         assert b.lib.tt_emb_probe_fp32(ctypes.byref(v), None) == b.TT_EMB_ERR_ARCH
+        assert b.lib.tt_emb_probe_mma(ctypes.byref(v), None) == b.TT_EMB_ERR_ARCH
     assert b.lib.tt_emb_backward(h, out.ctypes.data, ptrs, None) == b.TT_EMB_ERR_STATE
     assert b.lib.tt_emb_destroy(h) == 0
     assert b.lib.tt_emb_strerror(b.TT_EMB_ERR_ARCH).decode().startswith("no CUDA device")
