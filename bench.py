@@ -391,6 +391,12 @@ def main():
     # ---- roofline denominators measured in this run
     fp32_peak = binding.probe_fp32()
     mma_peak = binding.probe_mma()   # warp-level mma.sync m16n8k8 TF32 instructions per second
+    # the same products as tcgen05 instructions (M 128, k 8), for the two output widths the path has: TFLOP/s-equivalent
+    tc5 = {}
+    for n_cols in (128, 32):
+        rate5, err5 = binding.probe_tcgen05(n_cols)
+        tc5["n%d_tflops" % n_cols] = rate5 * 2.0 * 128 * n_cols * 8 / 1e12
+        tc5["n%d_max_abs_err" % n_cols] = err5
     l2_gather = binding.probe_gather(32 << 20, device=device)
     hbm_gather = binding.probe_gather(2 << 30, device=device)
     hbm_gbs, peak_src = measured_peaks()
@@ -642,7 +648,8 @@ def main():
                          "cuda_graph_ms_per_step": fwd_graph_ms},
         "stage_ms": stage_ms, "solo_kernel_ms": solo_ms, "roofline": roofline, "kernel_rooflines": kernel_rooflines, "step_roofline": step_roof,
         "peaks": {"hbm_GBs": hbm_gbs, "hbm_source": peak_src, "fp32_lane_ops_per_s": fp32_peak,
-                  "mma_sync_tf32_m16n8k8_per_s": mma_peak,
+                  "mma_sync_tf32_m16n8k8_per_s": mma_peak, "mma_sync_tf32_tflops": mma_peak * 2048 / 1e12,
+                  "tcgen05_tf32": tc5,
                   "l2_row_gather_GBs": l2_gather / 1e9, "hbm_row_gather_GBs": hbm_gather / 1e9},
         "work": work, "device_status": status, "clocks": clocks, "e2e": e2e,
         "gpu_launches": int(round(launches_per_step)),

@@ -261,6 +261,16 @@ int tt_emb_probe_fp32(double* slots_per_second, tt_emb_stream_t stream);
  */
 int tt_emb_probe_mma(double* mma_per_second, tt_emb_stream_t stream);
 /*
+ * The same question for the fifth-generation tensor cores: D[128 x n_cols] = A[128 x 32] . B[32 x n_cols] as
+ * tcgen05.mma kind::tf32 instructions (M 128, N n_cols, k 8; operands in shared memory, accumulator in tensor
+ * memory).  One product is checked against a plain FP32 loop on operands that are exact in TF32 (*max_abs_err, 0
+ * when the instruction does what this file says), then one CTA per SM issues a long run of them
+ * (*mma_per_second: M128.N.k8 instructions per second of the device = 128 * n_cols * 8 multiply-adds each).
+ * n_cols must be 32 or 128 (TT_EMB_ERR_ARG otherwise): the widths of the middle-core products (Sec. 3.2, dB) and of
+ * the stacked intermediate product (C = A.B).  Allocates two floats of device memory for its result.  SYNCHRONISES.
+ */
+int tt_emb_probe_tcgen05(int32_t n_cols, double* mma_per_second, double* max_abs_err, tt_emb_stream_t stream);
+/*
  * Random 256-byte-row gather bandwidth (bytes/s) from a caller-provided DEVICE buffer of `bytes`
  * bytes (<= L2 size measures L2, >> L2 measures HBM).  scratch_idx: DEVICE int32[num_rows_read].  SYNCHRONISES.
  */

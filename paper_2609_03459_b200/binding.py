@@ -82,6 +82,7 @@ _SIGS = {
     "tt_emb_stage_ms": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_f32)]),
     "tt_emb_probe_fp32": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_probe_mma": (ctypes.c_int, [ctypes.POINTER(ctypes.c_double), _vp]),
+    "tt_emb_probe_tcgen05": (ctypes.c_int, [ctypes.c_int32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_probe_gather": (ctypes.c_int, [_vp, ctypes.c_size_t, _vp, _i64, ctypes.POINTER(ctypes.c_double), _vp]),
     "tt_emb_launch_count": (ctypes.c_int, [ctypes.POINTER(_i64), _i32]),
     "tt_emb_table_variant": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i32)]),
@@ -398,6 +399,13 @@ def probe_mma() -> float:
     v = ctypes.c_double()
     _check(lib.tt_emb_probe_mma(ctypes.byref(v), _stream_ptr()), "tt_emb_probe_mma")
     return float(v.value)
+
+
+def probe_tcgen05(n_cols: int):
+    """(M128.N.k8 tcgen05 TF32 instructions per second, max |error| of the checked product)."""
+    rate, err = ctypes.c_double(), ctypes.c_double()
+    _check(lib.tt_emb_probe_tcgen05(int(n_cols), ctypes.byref(rate), ctypes.byref(err), _stream_ptr()), "tt_emb_probe_tcgen05")
+    return float(rate.value), float(err.value)
 
 
 def probe_gather(nbytes: int, rows_read: int = 1 << 22, device="cuda:0") -> float:

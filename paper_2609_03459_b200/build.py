@@ -7,7 +7,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SRC = [os.path.join(HERE, "csrc", f) for f in ("api.cu", "grouping.cu", "forward.cu", "backward.cu", "noalloc.cu")]
+SRC = [os.path.join(HERE, "csrc", f) for f in ("api.cu", "grouping.cu", "forward.cu", "backward.cu", "noalloc.cu", "probe_tcgen05.cu")]
 HDR = [os.path.join(HERE, "csrc", f) for f in ("common.cuh", "scan.cuh", "mma.cuh", "quad_mid.cuh")] + [os.path.join(ROOT, "include", "tt_emb.h")]
 SO = os.path.join(HERE, "libtt_emb.so")
 

@@ -90,6 +90,9 @@ def test_call_order_and_missing_device_errors(b):
         v = ctypes.c_double()
         assert b.lib.tt_emb_probe_fp32(ctypes.byref(v), None) == b.TT_EMB_ERR_ARCH
         assert b.lib.tt_emb_probe_mma(ctypes.byref(v), None) == b.TT_EMB_ERR_ARCH
+        v2 = ctypes.c_double()
+        assert b.lib.tt_emb_probe_tcgen05(128, ctypes.byref(v), ctypes.byref(v2), None) == b.TT_EMB_ERR_ARCH
+    assert b.lib.tt_emb_probe_tcgen05(64, ctypes.byref(ctypes.c_double()), ctypes.byref(ctypes.c_double()), None) == b.TT_EMB_ERR_ARG
     assert b.lib.tt_emb_backward(h, out.ctypes.data, ptrs, None) == b.TT_EMB_ERR_STATE
     assert b.lib.tt_emb_destroy(h) == 0
     assert b.lib.tt_emb_strerror(b.TT_EMB_ERR_ARCH).decode().startswith("no CUDA device")

@@ -545,3 +545,12 @@ def test_forward_and_grouping_are_bit_reproducible(binding):
         for k in range(wl.tables[t].K):
             scale = max(np.abs(a[4][t][k]).max(), 1e-30)
             assert np.abs(a[4][t][k] - b[4][t][k]).max() <= 2e-6 * scale
+
+
+@pytest.mark.parametrize("n_cols", [32, 128])
+def test_tcgen05_probe_product_is_exact(binding, n_cols):
+    # the measurement helper's tile product D[128 x N] = A[128 x 32] . B[32 x N] on the fifth-generation tensor cores
+    # against a plain FP32 loop over the same operands (multiples of 1/4: exact in TF32, sums exact in fp32)
+    rate, err = binding.probe_tcgen05(n_cols)
+    assert err == 0.0
+    assert rate > 1e9    # M128.N.k8 instructions per second of the whole device
