@@ -331,6 +331,7 @@ extern "C" int tt_emb_create(const tt_emb_config_t* cfg, tt_emb_t* out_handle)
     }
     h->off_cost = TAKE("cost", ((size_t)v.cap[K - 1] + 1) * sizeof(uint32_t));
     h->off_unit_rng = TAKE("unit_rng", (size_t)T * h->units_per_table * sizeof(uint2));
+    h->off_pool_bounds = TAKE("pool_bounds", ((size_t)TT_POOL_MAX_SHARES + 1) * sizeof(int64_t));
     v.units_per_table = h->units_per_table;
     for (int k = 2; k <= K - 2; ++k) h->off_pbuf[k] = TAKE("pbuf", (size_t)v.cap[k] * stride[k] * sizeof(float));
     h->off_E = TAKE("E", (size_t)h->capU * D * sizeof(float));
@@ -429,6 +430,7 @@ extern "C" int tt_emb_bind(tt_emb_t h, float* const* core_ptrs, void* workspace,
     }
     v.cost = (uint32_t*)(base + h->off_cost);
     v.unit_rng = (uint2*)(base + h->off_unit_rng);
+    v.pool_bounds = (int64_t*)(base + h->off_pool_bounds);
     for (int k = 2; k <= K - 2; ++k) v.pbuf[k] = (float*)(base + h->off_pbuf[k]);
     v.E = (float*)(base + h->off_E);
     v.upairs = nullptr;

@@ -10,6 +10,7 @@
 #define TT_SCAN_THREADS 256
 #define TT_SCAN_ITEMS 16
 #define TT_SCAN_TILE (TT_SCAN_THREADS * TT_SCAN_ITEMS)  // elements per scan tile
+#define TT_POOL_MAX_SHARES 262144                       // shares of the lookups that the pooling warps take in order
 #define TT_HEAD_TILES 4                                 // leading scan tiles of a table that are emitted first (see PopScan)
 #define TT_LSCAN_ITEMS 2                                // the short scans of the prefix-level bitmaps
 #define TT_LSCAN_TILE (TT_SCAN_THREADS * TT_LSCAN_ITEMS)
@@ -74,6 +75,7 @@ struct WsView {
     uint32_t* parent[TT_MAXK + 1];      // levels 3..K-1: parent node at level k-1 (null elsewhere: nothing reads it)
     uint32_t* tb[TT_MAXK + 1];          // [T+1] node range of each table at level k
     uint32_t* cost;                     // [cap_{K-1}+1] exclusive scan of per-group cost (+ total)
+    int64_t* pool_bounds;               // [shares + 1] first bag of every share of the pooling pass (k_pool_bounds)
     uint2* unit_rng;                    // [T * units per table] group range of every work unit (k_unit_ranges)
     int32_t units_per_table;
     float* pbuf[TT_MAXK + 1];           // partial products P_k of level-k nodes, 2 <= k <= K-2
@@ -110,7 +112,8 @@ __device__ __forceinline__ int64_t tt_index(const WsView& w, int64_t l)
     return STREAM ? __ldcs(w.indices + l) : __ldg(w.indices + l);
 }
 
-enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16, CTR_SCAN_TICKET = 32 /* tiles of the running scan that have reported */ };
+enum { CTR_LEVEL0 = 0 /* +k */, CTR_TLEVEL0 = 8 /* +k */, CTR_COST_TOTAL = 16, CTR_SCAN_TICKET = 32 /* tiles of the running scan that have reported */,
+       CTR_POOL_NEXT = 34 /* next share of the lookups to be pooled (shares are handed out in order) */ };
 
 struct tt_emb {
     int T, K, D;
@@ -136,7 +139,7 @@ struct tt_emb {
     size_t off_val[TT_MAXK + 1], off_cstart[TT_MAXK + 1], off_parent[TT_MAXK + 1], off_tb[TT_MAXK + 1];
     size_t off_pbuf[TT_MAXK + 1], off_dP[TT_MAXK + 1], off_tbm[TT_MAXK + 1], off_tnode[TT_MAXK + 1];
     size_t off_Y[TT_MAXK + 1];
-    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted, off_unit_rng;
+    size_t off_cnt, off_cursor, off_pairs, off_carry, off_gpart, off_wsorted, off_unit_rng, off_pool_bounds;
     // guard bytes after every workspace region (tt_emb_check_guards): [guard_off[i], guard_off[i] + guard_len[i])
     int num_regions;
     size_t guard_off[96], guard_len[96];

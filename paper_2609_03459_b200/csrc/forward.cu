@@ -649,14 +649,48 @@ __device__ __forceinline__ uint32_t tt_lookup_slot(const WsView& w, const TableD
     return slot;
 }
 
-// Pooling partition: the lookups are cut into C = W * chunks equal shares and warp wi takes shares wi, wi + W, ...
-// (whole bags, found by bisection on offsets).  All resident warps therefore work inside one moving window of
+// Pooling partition: the lookups are cut into C = W * chunks equal shares of whole bags (k_pool_bounds), and the
+// warps take the shares in order from a counter.  All resident warps therefore work inside one moving window of
 // about W shares at a time - a few tables - so the rows that several bags share are still in L2 when the next
-// bag asks for them; one contiguous share per warp would spread the warps over all tables at once.
-__device__ __forceinline__ int64_t tt_pool_chunks(int64_t L, int64_t W)
+// bag asks for them; one contiguous share per warp would spread the warps over all tables at once.  Equal lookups are
+// not equal time (a share of popular rows is served by L2, one of unpopular rows by HBM): with a fixed assignment the
+// first warp finished at 84 % of the kernel, the median one at 90 %.  Eight shares per warp: more of them cost more
+// in pipeline fill and drain per share than they give in balance (4 / 8 / 16 / 32: 2.62 / 2.39 / 2.50 / 2.76 ms).
+#define TT_POOL_MAX_CHUNKS 8
+__host__ __device__ __forceinline__ int64_t tt_pool_chunks(int64_t L, int64_t W)
 {
-    const int64_t c = L / (W * 512);                    // at least 512 lookups per share
-    return c < 1 ? 1 : (c > 8 ? 8 : c);
+    int64_t c = L / (W * 512);                          // at least 512 lookups per share
+    c = c < 1 ? 1 : (c > TT_POOL_MAX_CHUNKS ? TT_POOL_MAX_CHUNKS : c);
+    while (W * c > TT_POOL_MAX_SHARES && c > 1) --c;
+    return c;
+}
+
+// first bag of every share: share ci starts at the first bag whose offset is >= L ci / C (the same search for both
+// neighbours of a boundary, whatever the offsets hold).  One thread per boundary: the bisections (21 dependent loads for
+// two million bags) run side by side here instead of at the start of every share in the pooling warps.
+__global__ void __launch_bounds__(256) k_pool_bounds(WsView w, int64_t C)
+{
+    tt_pdl_enter();
+    const int64_t nb = (int64_t)w.T * w.B;
+    for (int64_t ci = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; ci <= C; ci += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t target = (w.L * ci) / C;
+        int64_t lo = 0, hi = nb;
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (__ldg(w.offsets + mid) < target) lo = mid + 1; else hi = mid;
+        }
+        w.pool_bounds[ci] = ci == 0 ? 0 : (ci == C ? nb : lo);
+    }
+}
+
+static cudaError_t launch_pool_bounds(tt_emb* h, int64_t W, cudaStream_t s)
+{
+    const int64_t C = W * tt_pool_chunks(h->v.L, W);
+    const int64_t want = (C + 1 + 255) / 256;
+    const int grid = (int)(want < (int64_t)h->sm_count * 8 ? want : (int64_t)h->sm_count * 8);
+    cudaError_t e = tt_launch_pdl(k_pool_bounds, dim3(grid), dim3(256), 0, s, h->v, C);
+    if (e == cudaSuccess) tt_note_launch();
+    return e;
 }
 
 template <int LPR, int CPL, bool WT>  // lanes per row, float4 chunks per lane, weighted / mean pooling
@@ -669,31 +703,20 @@ __global__ void __launch_bounds__(256, (CPL == 1 ? 6 : (CPL == 2 ? 2 : 1))) k_po
     constexpr int NIT = 32 / RPI;                       // load instructions per 32 lookups
     constexpr int NF = NIT < 4 ? NIT : 4;               // load instructions in flight
     const int D4 = w.D >> 2;
-    const int64_t nb = (int64_t)w.T * w.B;
     const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
     const uint32_t capK = w.cap[w.K];
     // Skew-aware split: the grid is exactly resident (persistent warps); a share holds the bags whose first
     // lookup falls into it (offsets is the cost prefix sum).
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
     auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
-    for (int64_t ci = wi; ci < C; ci += W) {
-    int64_t b0, b1;
-    {
-        const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
-        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target; the same search for
-                                                        // both neighbours of a boundary, whatever the offsets hold
-        if (lane < 2)
-            while (lo < hi) {
-                const int64_t mid = (lo + hi) >> 1;
-                if (__ldg(w.offsets + mid) < target) lo = mid + 1; else hi = mid;
-            }
-        b0 = __shfl_sync(0xffffffffu, lo, 0);
-        b1 = __shfl_sync(0xffffffffu, lo, 1);
-        if (ci == 0) b0 = 0;
-        if (ci == C - 1) b1 = nb;
-    }
+    for (;;) {
+    // shares are handed out in order through a counter: a warp whose shares hold popular (L2-resident) rows takes more of them
+    int64_t ci = 0;
+    if (lane == 0) ci = (int64_t)atomicAdd(&w.counters[CTR_POOL_NEXT], 1u);
+    ci = __shfl_sync(0xffffffffu, ci, 0);
+    if (ci >= C) break;
+    const int64_t b0 = __ldg(w.pool_bounds + ci), b1 = __ldg(w.pool_bounds + ci + 1);
     if (b0 >= b1) continue;
     // every bag is summed over its own (offsets[bag], offsets[bag + 1]) pair, clamped to [0, L]; an inverted pair (malformed
     // offsets) is an empty bag.  o_next: start of the next bag = this bag's end as stored, before the inversion fix
@@ -809,29 +832,18 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     float4* buf = pool_buf + (size_t)wid * 32 * R4;
     const int D4 = w.D >> 2;
     const bool lane_on = lr < D4;
-    const int64_t nb = (int64_t)w.T * w.B;
     const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
     const uint32_t capK = w.cap[w.K];
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t wi = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
     auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
-    for (int64_t ci = wi; ci < C; ci += W) {
-    int64_t b0, b1;
-    {
-        const int64_t target = lane == 0 ? (w.L * ci) / C : (w.L * (ci + 1)) / C;
-        int64_t lo = 0, hi = nb;                        // first bag with offsets[bag] >= target; the same search for
-                                                        // both neighbours of a boundary, whatever the offsets hold
-        if (lane < 2)
-            while (lo < hi) {
-                const int64_t mid = (lo + hi) >> 1;
-                if (__ldg(w.offsets + mid) < target) lo = mid + 1; else hi = mid;
-            }
-        b0 = __shfl_sync(0xffffffffu, lo, 0);
-        b1 = __shfl_sync(0xffffffffu, lo, 1);
-        if (ci == 0) b0 = 0;
-        if (ci == C - 1) b1 = nb;
-    }
+    for (;;) {
+    // shares are handed out in order through a counter: a warp whose shares hold popular (L2-resident) rows takes more of them
+    int64_t ci = 0;
+    if (lane == 0) ci = (int64_t)atomicAdd(&w.counters[CTR_POOL_NEXT], 1u);
+    ci = __shfl_sync(0xffffffffu, ci, 0);
+    if (ci >= C) break;
+    const int64_t b0 = __ldg(w.pool_bounds + ci), b1 = __ldg(w.pool_bounds + ci + 1);
     if (b0 >= b1) continue;
     // every bag is summed over its own (offsets[bag], offsets[bag + 1]) pair, clamped to [0, L]; an inverted pair (malformed
     // offsets) is an empty bag.  o_next: start of the next bag = this bag's end as stored, before the inversion fix
@@ -949,6 +961,7 @@ static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
     const int64_t need = (nb + POOL_WARPS - 1) / POOL_WARPS;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
+    if ((e = launch_pool_bounds(h, grid * POOL_WARPS, s)) != cudaSuccess) return e;
     if ((e = tt_launch_pdl(k_pool_async<R4, WT>, dim3((int)grid), dim3(32 * POOL_WARPS), smem, s, h->v, out)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
@@ -966,6 +979,7 @@ static cudaError_t launch_pool_vec(tt_emb* h, float* out, cudaStream_t s)
     const int64_t need = (nb + 7) / 8;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
+    if ((e = launch_pool_bounds(h, grid * 8, s)) != cudaSuccess) return e;
     if ((e = tt_launch_pdl(k_pool_vec<LPR, CPL, WT>, dim3((int)grid), dim3(256), 0, s, h->v, out)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();
