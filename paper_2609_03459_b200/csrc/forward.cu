@@ -367,15 +367,16 @@ __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& 
 template <int COLS>
 __device__ __forceinline__ void tt_pair_mid_staged(const float* __restrict__ B, int ra, const float* __restrict__ srcA,
                                                    const float* __restrict__ srcB, bool selA, bool selB, float* Cs2, float* stg,
-                                                   int lane, int wid)
+                                                   int lane, int wid, bool stage)
 {
     constexpr int RS = 68;
     const int g = lane >> 2, t = lane & 3;
     const int c0 = 64 * wid;   // first column of this warp's block
-    for (int i = lane; i < 64 * 16; i += 32) {
-        const int k = i >> 4, f = i & 15;
-        if (k < ra) tt_cp_async16(stg + k * RS + 4 * f, B + (size_t)k * COLS + c0 + 4 * f);
-    }
+    if (stage)                 // (the block of the previous pair is still there when the pair shares its slice)
+        for (int i = lane; i < 64 * 16; i += 32) {
+            const int k = i >> 4, f = i & 15;
+            if (k < ra) tt_cp_async16(stg + k * RS + 4 * f, B + (size_t)k * COLS + c0 + 4 * f);
+        }
     asm volatile("cp.async.commit_group;" ::: "memory");
     float araw[8][4];   // rows g (first group) and g + 8 (second group) of the stacked operand, unsplit
 #pragma unroll
@@ -443,6 +444,7 @@ __device__ __forceinline__ void tt_sweep_pair_cta(const WsView& w, const TableDe
     const int K = w.K, km = K - 2;
     const int ra = td.r[km];
     const uint32_t nK = (uint32_t)td.n[K - 1];
+    uint32_t staged = 0xffffffffu;   // slice whose blocks the warps hold in shared memory (the same for all four warps)
     for (uint32_t base = g0; base < g1; base += 2) {
         const int cnt = (int)min(2u, g1 - base);
         if (threadIdx.x < 2) {
@@ -463,13 +465,18 @@ __device__ __forceinline__ void tt_sweep_pair_cta(const WsView& w, const TableDe
         __syncthreads();
         const float* B0 = td.core[km] + (size_t)m_im[0] * td.slice_floats[km];
         float* stg = Cs2 + 2 * PM * RB + (size_t)wid * (64 * 68);   // this warp's staged 64 x 64 block of the slice
+        // neighbouring pairs of the digit-major order share the slice: its 64 KB are fetched again only when it changes
         if (cnt == 2 && m_im[1] == m_im[0]) {
-            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, true, Cs2, stg, lane, wid);
+            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, true, Cs2, stg, lane, wid, staged != m_im[0]);
+            staged = m_im[0];
         } else {
-            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, false, Cs2, stg, lane, wid);
-            if (cnt == 2)
+            tt_pair_mid_staged<COLS>(B0, ra, m_src[0], m_src[1], true, false, Cs2, stg, lane, wid, staged != m_im[0]);
+            staged = m_im[0];
+            if (cnt == 2) {
                 tt_pair_mid_staged<COLS>(td.core[km] + (size_t)m_im[1] * td.slice_floats[km], ra, m_src[0], m_src[1], false, true, Cs2,
-                                         stg, lane, wid);
+                                         stg, lane, wid, true);
+                staged = m_im[1];
+            }
         }
         __syncthreads();
         {
