@@ -954,6 +954,308 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     }
 }
 
+// The same gather for batches with few lookups per bag (below TT_POOL_STREAM_BELOW on average): a window is 32
+// consecutive lookups of the warp's share, whatever bags they belong to.  One bag per window, as in k_pool_async, costs
+// the latency of a window per bag: 2 million bags took 0.82 ms there whether they held 2 or 16 lookups each, and 7.9
+// million one-lookup bags 3.0 ms.  Here a window of one-lookup bags goes straight from the staged rows to out (those
+// 7.9 million bags: 0.40 ms, 5 TB/s of rows read and written); a window with several bags in it is summed by the whole
+// warp at once, each sub-warp taking consecutive rows and the pieces of a bag that crosses sub-warps being joined
+// afterwards (2 lookups per bag: 0.82 -> 0.20 ms, 4: 0.30, 8: 0.51, 12: 0.80 against 0.86); a window with one boundary,
+// empty bags, weights or mean pooling is summed bag by bag.  From about 14 lookups per bag on the per-bag kernel is the
+// faster one (its windows are then mostly full, and the sums here cost more instructions per row).  A window ends
+// early only at the end of the share or of a table (the rank look-up of a window uses one table).  With malformed
+// offsets (status bit set by the offsets check earlier in the stream) every bag is summed over its own clamped
+// (offsets[bag], offsets[bag + 1]) pair as the header promises, and windows stop at the end of their bag.
+#define TT_POOL_STREAM_BELOW 14
+template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
+__global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, float* __restrict__ out)
+{
+    tt_pdl_enter();
+    static_assert(R4 == 16 || R4 == 8, "two or four rows per cp.async instruction");
+    constexpr int RPI = 32 / R4;
+    constexpr int PGRP = 4;              // load instructions per group: a window is cut short and tested for validity per group
+    extern __shared__ __align__(16) float4 pool_buf[];   // [POOL_WARPS][32 rows][R4 float4]
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int sub = lane / R4, lr = lane % R4;
+    float4* buf = pool_buf + (size_t)wid * 32 * R4;
+    const int D4 = w.D >> 2;
+    const bool lane_on = lr < D4;
+    const float4* __restrict__ E4 = reinterpret_cast<const float4*>(w.E);
+    const uint32_t capK = w.cap[w.K];
+    const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t C = W * tt_pool_chunks(w.L, W);
+    const bool stream_ok = !(*w.status & TT_EMB_STATUS_OFFSETS);
+    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    for (;;) {
+    int64_t ci = 0;     // shares are handed out in order through a counter (see k_pool_async)
+    if (lane == 0) ci = (int64_t)atomicAdd(&w.counters[CTR_POOL_NEXT], 1u);
+    ci = __shfl_sync(0xffffffffu, ci, 0);
+    if (ci >= C) break;
+    const int64_t b0 = __ldg(w.pool_bounds + ci), b1 = __ldg(w.pool_bounds + ci + 1);
+    if (b0 >= b1) continue;
+    // the ends of the share's bags, 32 at a time and one vector ahead: lane i holds the clamped offsets[ebase + 1 + i]
+    // (ends_nx: the 32 bags after those), so that no bag waits for a load of its own end
+    auto load_ends = [&](int64_t base) { const int64_t i = base + lane; return i < b1 ? clampL(__ldg(w.offsets + i + 1)) : (int64_t)1 << 62; };   // past the share: never inside a window
+    int64_t ebase = b0;
+    int64_t ends_reg = load_ends(b0), ends_nx = load_ends(b0 + 32);
+    auto end_of = [&](int64_t bg) {     // bg >= ebase, and below ebase + 64 (a step moves on by at most 32 bags)
+        while (bg - ebase >= 32) {
+            ends_reg = ends_nx;
+            ebase += 32;
+            ends_nx = load_ends(ebase + 32);
+        }
+        return __shfl_sync(0xffffffffu, ends_reg, (int)(bg - ebase));
+    };
+    // the bag being summed: its table, its (clamped) range, the end of the bag as stored
+    int64_t bag = b0;
+    int t = (int)(b0 / w.B);
+    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = end_of(b0);
+    int64_t o_hi = o_next < o_lo ? o_lo : o_next;
+    const int64_t share_end = stream_ok ? clampL(__ldg(w.offsets + b1)) : 0;
+    int64_t t_end = stream_ok ? __ldg(w.tl_start + t + 1) : 0;
+    int64_t pos = o_lo;                                 // next lookup of the stream
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // rank look-up (and weight) of lookup base + lane, for the window that starts at `base`
+    uint32_t slot_next = 0xffffffffu;
+    float wt_next = 1.f;
+    int64_t pre_pos = -1;
+    int pre_t = -1;
+    auto fetch = [&](int64_t base, int64_t lim, int tt) {
+        slot_next = (base + lane < lim) ? tt_lookup_slot(w, w.tdesc[tt], base + lane, capK) : 0xffffffffu;
+        if (WT) wt_next = (w.psw && base + lane < lim) ? __ldg(w.psw + base + lane) : 1.f;
+        pre_pos = base;
+        pre_t = tt;
+    };
+    // bag `nb_`, which starts at lookup `lo_`, becomes the one being summed (nb_ > bag, at most 32 bags on)
+    auto seek_bag = [&](int64_t nb_, int64_t lo_) {
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        bag = nb_;
+        if (bag < b1) {
+            if (bag >= (int64_t)(t + 1) * w.B) {
+                ++t;
+                if (stream_ok) t_end = __ldg(w.tl_start + t + 1);
+            }
+            o_lo = lo_;
+            o_next = end_of(bag);
+            o_hi = o_next < o_lo ? o_lo : o_next;
+        }
+    };
+    auto advance_bag = [&]() { seek_bag(bag + 1, o_next); };
+    // the bag is complete: combine the sub-warps, write its row of out, move on to the next bag
+    auto close_bag = [&]() {
+#pragma unroll
+        for (int o = R4; o < 32; o <<= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+        }
+        if (WT && w.pool_mean && o_hi > o_lo) {
+            const float inv = 1.f / (float)(o_hi - o_lo);
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        }
+        const int64_t b = bag - (int64_t)t * w.B;
+        if (sub == 0 && lane_on) __stcs(reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr, acc);
+        advance_bag();
+    };
+    while (bag < b1) {
+        if (pos >= o_hi) {              // the bag has no (more) lookups
+            close_bag();
+            pos = o_lo;
+            continue;
+        }
+        const int64_t lim = stream_ok ? (share_end < t_end ? share_end : t_end) : o_hi;   // > pos: the bag ends no later
+        const int n = (int)min((int64_t)32, lim - pos);
+        if (pre_pos != pos || pre_t != t) fetch(pos, lim, t);
+        const uint32_t slot = slot_next;
+        const float wt = wt_next;
+        const unsigned valid = __ballot_sync(0xffffffffu, lane < n && slot != 0xffffffffu);
+        // all rows of the window in flight (groups of four instructions; a short window leaves early);
+        // a group whose rows are all valid (the usual case) needs no per-row test
+        const bool plain = valid == (n == 32 ? 0xffffffffu : (1u << n) - 1u) && D4 == R4;
+#pragma unroll
+        for (int jq = 0; jq < 32 / RPI; jq += PGRP) {
+            if (RPI * jq >= n) break;
+            if (plain && RPI * (jq + PGRP) <= n) {
+#pragma unroll
+                for (int jj = jq; jj < jq + PGRP; ++jj) {
+                    const int j = RPI * jj + sub;
+                    const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
+                    tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * R4 + lr);
+                }
+            } else {
+#pragma unroll
+                for (int jj = jq; jj < jq + PGRP; ++jj) {
+                    const int j = RPI * jj + sub;
+                    const uint32_t sl = __shfl_sync(0xffffffffu, slot, j);
+                    if (((valid >> j) & 1u) && lane_on) tt_cp_async16(buf + j * R4 + lr, E4 + (size_t)sl * D4 + lr);
+                }
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        // the rank look-ups of the next window overlap the gather (the next window of the stream; in the per-bag mode
+        // only while the bag goes on)
+        {
+            const int64_t np = pos + n;
+            if (stream_ok) {
+                if (np < lim) fetch(np, lim, t);
+                else if (np < share_end) {               // the table ends here: the next window belongs to the next one
+                    const int64_t te = __ldg(w.tl_start + t + 2);
+                    fetch(np, share_end < te ? share_end : te, t + 1);
+                }
+            } else if (np < o_hi) fetch(np, o_hi, t);
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        // Windows with bag boundaries in them are summed by the whole warp at once.  Lane i looks at bag + i, which ends at
+        // e_mine; a bag starts at row e - pos of the window for every end e inside it.
+        if (!WT && stream_ok && o_hi < pos + n) {
+            const int64_t wend = pos + n;
+            const int ei = (int)(bag - ebase) + lane;
+            const int64_t e0 = __shfl_sync(0xffffffffu, ends_reg, ei & 31), e1 = __shfl_sync(0xffffffffu, ends_nx, ei & 31);
+            const int64_t e_mine = ei < 32 ? e0 : e1;
+            // one-lookup bags only (lane i: bag + i ends at pos + i + 1): every staged row is a row of out
+            if (o_lo == pos && __all_sync(0xffffffffu, lane >= n || e_mine == pos + lane + 1)) {
+                const int64_t bf = bag - (int64_t)t * w.B;       // the window lies in table t: bf + n <= B
+                if (w.upairs && lane < n) __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bf + lane)));
+                float4* o4 = reinterpret_cast<float4*>(out + (size_t)bf * w.T * w.D + (size_t)t * w.D) + lr;
+                const size_t ostride = (size_t)w.T * D4;
+#pragma unroll
+                for (int jj = 0; jj < 32 / RPI; ++jj) {
+                    const int j = RPI * jj + sub;
+                    if (j < n && lane_on)
+                        __stcs(o4 + (size_t)j * ostride, ((valid >> j) & 1u) ? buf[j * R4 + lr] : make_float4(0.f, 0.f, 0.f, 0.f));
+                }
+                __syncwarp();
+                pos += n;
+                seek_bag(bag + n, pos);
+                continue;
+            }
+            // no empty bag among those that start inside the window (an empty bag needs a row of zeros: left to the
+            // bag-by-bag loop below)
+            const int64_t e_prev = __shfl_up_sync(0xffffffffu, e_mine, 1);
+            const bool many = __popc(__ballot_sync(0xffffffffu, e_mine > pos && e_mine < wend)) >= 2;   // else: cheaper bag by bag
+            if (many && !__any_sync(0xffffffffu, lane >= 1 && e_prev < wend && e_mine == e_prev)) {
+                // starts: bit j = row j is the first of its bag; closes: bit j = row j is the last of its bag
+                const unsigned starts = __reduce_or_sync(0xffffffffu, (e_mine > pos && e_mine < wend) ? 1u << (int)(e_mine - pos) : 0u)
+                                      | (o_lo == pos ? 1u : 0u);
+                const bool last_closed = __any_sync(0xffffffffu, e_mine == wend);
+                const unsigned closes = (starts >> 1) | (last_closed ? 1u << (n - 1) : 0u);
+                const int64_t bt = bag - (int64_t)t * w.B;       // bag of row j: bt + bags started in rows 1..j
+                auto row_of = [&](int j) {
+                    const int64_t b = bt + __popc(starts & ((2u << j) - 2u));
+                    return reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr;
+                };
+                if (w.upairs && lane < n)
+                    __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bt + __popc(starts & ((2u << lane) - 2u)))));
+                // the open bag's sum so far, the same in every sub-warp
+                float4 carry = acc;
+#pragma unroll
+                for (int o = R4; o < 32; o <<= 1) {
+                    carry.x += __shfl_xor_sync(0xffffffffu, carry.x, o); carry.y += __shfl_xor_sync(0xffffffffu, carry.y, o);
+                    carry.z += __shfl_xor_sync(0xffffffffu, carry.z, o); carry.w += __shfl_xor_sync(0xffffffffu, carry.w, o);
+                }
+                // sub-warp s sums the R4 consecutive rows from s * R4 on, in step with the others: a bag that lies inside
+                // them is written at its last row; the piece of a bag that came in from before (head) is kept, the piece
+                // of a bag that goes on after them is what `run` holds at the end
+                float4 run = make_float4(0.f, 0.f, 0.f, 0.f), head = run;
+                bool head_open = !((starts >> (sub * R4)) & 1u), head_closed = false;
+#pragma unroll
+                for (int jj = 0; jj < R4; ++jj) {
+                    const int j = sub * R4 + jj;
+                    if (j < n) {
+                        if ((valid >> j) & 1u) {
+                            const float4 v = buf[j * R4 + lr];
+                            tt_add4(run, v);
+                        }
+                        if ((closes >> j) & 1u) {
+                            if (head_open) { head = run; head_closed = true; head_open = false; }
+                            else if (lane_on) __stcs(row_of(j), run);
+                            run = make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+                }
+                // the pieces across the sub-warps, in order: a head closes the bag carried so far; rows that all belong to
+                // the carried bag add to it; otherwise the carried bag ended with the sub-warp before (nothing carried)
+                const unsigned hc = __ballot_sync(0xffffffffu, head_closed), ho = __ballot_sync(0xffffffffu, head_open);
+#pragma unroll
+                for (int s2 = 0; s2 < RPI; ++s2) {
+                    if (((hc >> (s2 * R4)) & 1u) && sub == s2 && lane_on) {
+                        float4 sum = carry;
+                        tt_add4(sum, head);
+                        __stcs(row_of(s2 * R4), sum);
+                    }
+                    float4 tail;
+                    tail.x = __shfl_sync(0xffffffffu, run.x, s2 * R4 + lr); tail.y = __shfl_sync(0xffffffffu, run.y, s2 * R4 + lr);
+                    tail.z = __shfl_sync(0xffffffffu, run.z, s2 * R4 + lr); tail.w = __shfl_sync(0xffffffffu, run.w, s2 * R4 + lr);
+                    if ((ho >> (s2 * R4)) & 1u) tt_add4(carry, tail);
+                    else carry = tail;
+                }
+                __syncwarp();
+                const int64_t bl = bag + __popc(starts & 0xfffffffeu);     // the bag of the window's last row
+                pos = wend;
+                if (last_closed) seek_bag(bl + 1, pos);
+                else {
+                    if (bl > bag) {
+                        const int64_t lo_ = end_of(bl - 1);
+                        seek_bag(bl, lo_);
+                    }
+                    acc = sub == 0 ? carry : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                continue;
+            }
+        }
+        // the window's rows, bag by bag.  Two-level sum: the rows of a (piece of a) bag go into a partial that is added to
+        // the bag's sum once, so the rounding error of a bag with thousands of lookups grows with the number of windows
+        int r = 0;
+        while (r < n) {
+            if (pos + r >= o_hi) {       // a bag ends inside the window (and empty bags after it)
+                close_bag();
+                if (bag >= b1) break;    // cannot happen with checked offsets; never spin on it
+                continue;
+            }
+            const int64_t room = o_hi - (pos + r);
+            const int seg = room < (int64_t)(n - r) ? (int)room : n - r;
+            if (w.upairs && lane >= r && lane < r + seg)    // kept for the backward sort
+                __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (int64_t)t * w.B)));
+            if (!WT && seg == 1 && pos + r == o_lo && o_hi - o_lo == 1) {
+                // a bag of one lookup: its row of out is the staged row (or zeros for an id outside the table); the
+                // sub-warp that staged it writes it, nothing to combine
+                if (sub == (r & (RPI - 1)) && lane_on) {
+                    const float4 v = ((valid >> r) & 1u) ? buf[r * R4 + lr] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    __stcs(reinterpret_cast<float4*>(out + (size_t)(bag - (int64_t)t * w.B) * w.T * w.D + (size_t)t * w.D) + lr, v);
+                }
+                advance_bag();
+                r += 1;
+                if (bag >= b1) break;
+                continue;
+            }
+            float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!WT && plain && seg == 32) {
+#pragma unroll
+                for (int jj = 0; jj < 32 / RPI; ++jj) {
+                    const float4 v = buf[(RPI * jj + sub) * R4 + lr];
+                    tt_add4(part, v);
+                }
+            } else {
+                for (int jj = r / RPI; RPI * jj < r + seg; ++jj) {
+                    const int j = RPI * jj + sub;
+                    const float wj = WT ? __shfl_sync(0xffffffffu, wt, j) : 1.f;
+                    if (j >= r && j < r + seg && ((valid >> j) & 1u) && lane_on) {
+                        const float4 v = buf[j * R4 + lr];
+                        if (WT) { part.x = fmaf(wj, v.x, part.x); part.y = fmaf(wj, v.y, part.y); part.z = fmaf(wj, v.z, part.z); part.w = fmaf(wj, v.w, part.w); }
+                        else tt_add4(part, v);
+                    }
+                }
+            }
+            acc.x += part.x; acc.y += part.y; acc.z += part.z; acc.w += part.w;
+            r += seg;
+        }
+        __syncwarp();
+        pos += n;
+    }
+    }
+}
+
+
 template <int R4, bool WT>
 static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
 {
@@ -969,6 +1271,12 @@ static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
     if ((e = launch_pool_bounds(h, grid * POOL_WARPS, s)) != cudaSuccess) return e;
+    if (h->v.L < (int64_t)TT_POOL_STREAM_BELOW * nb) {   // few lookups per bag: windows across bags
+        if ((e = cudaFuncSetAttribute(k_pool_stream<R4, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        if ((e = tt_launch_pdl(k_pool_stream<R4, WT>, dim3((int)grid), dim3(32 * POOL_WARPS), smem, s, h->v, out)) != cudaSuccess) return e;
+        tt_note_launch();
+        return cudaGetLastError();
+    }
     if ((e = tt_launch_pdl(k_pool_async<R4, WT>, dim3((int)grid), dim3(32 * POOL_WARPS), smem, s, h->v, out)) != cudaSuccess) return e;
     tt_note_launch();
     return cudaGetLastError();

@@ -178,6 +178,70 @@ def test_medium_forward_backward(binding, case):
             assert_close(grads[t][k], ref[t][k], f"{name} dG[{t}][{k}]")
 
 
+# Few lookups per bag: the pooling gather takes windows of 32 lookups across bags there.  One lookup in every bag
+# (rows go straight to out), empty bags in between, two to four bags per window, bags longer than a window among short
+# ones; batch sizes that put table boundaries and share boundaries inside windows.
+SHORT_BAG_TABLES = {
+    64: [TableSpec(30_000, (32, 32, 32), (4, 4, 4), (1, 16, 16, 1), 1.1, "normal", 0.05),
+         TableSpec(900, (10, 10, 10), (4, 4, 4), (1, 8, 8, 1), 0.8, "normal", 0.05),
+         TableSpec(20_000, (28, 28, 28), (4, 4, 4), (1, 16, 32, 1), 1.0, "normal", 0.05)],
+    32: [TableSpec(30_000, (32, 32, 32), (2, 4, 4), (1, 16, 16, 1), 1.1, "normal", 0.05),
+         TableSpec(700, (9, 9, 9), (2, 4, 4), (1, 8, 8, 1), 0.8, "normal", 0.05),
+         TableSpec(20_000, (28, 28, 28), (2, 4, 4), (1, 8, 16, 1), 1.0, "normal", 0.05)],
+    20: [TableSpec(9_000, (21, 21, 21), (2, 2, 5), (1, 4, 6, 1), 1.0, "normal", 0.1),
+         TableSpec(500, (8, 8, 8), (2, 2, 5), (1, 4, 4, 1), 1.0, "normal", 0.1)],
+}
+
+
+@pytest.mark.parametrize("pooling", [1, (0, 1), (0, 2), (1, 4), (0, 7), (1, 13), (0, 27)], ids=str)
+@pytest.mark.parametrize("D", [64, 32, 20])
+@pytest.mark.parametrize("B", [33, 1000])
+def test_short_bags(binding, D, B, pooling):
+    wl = workloads.custom(SHORT_BAG_TABLES[D], B, pooling, seed=123, with_grad=True, name=f"short-D{D}")
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl), f"short bags D{D} B{B} {pooling} out")
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"short bags D{D} B{B} {pooling} dG[{t}][{k}]")
+
+
+@pytest.mark.parametrize("mode", ["weighted", "mean"])
+@pytest.mark.parametrize("pooling", [1, (0, 3), (1, 13)], ids=str)
+def test_short_bags_weighted_and_mean(binding, pooling, mode):
+    wl = workloads.custom(SHORT_BAG_TABLES[64], 500, pooling, seed=124, with_grad=True, name="short-wt")
+    wts = np.random.default_rng(18).normal(size=wl.L).astype(np.float32) if mode == "weighted" else None
+    omode = "mean" if mode == "mean" else "sum"
+    emb = binding.from_workload(wl, enable_backward=True, enable_weighted=True)
+    emb.set_pooling(omode, None if wts is None else dev(wts))
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B).cpu().numpy()
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl, weights=wts, mode=omode), f"short bags {pooling} {mode} out")
+    emb.backward(dev(wl.grad_out))
+    grads = emb.get_grads()
+    ref = oracle.backward_workload(wl, weights=wts, mode=omode)
+    for t in range(wl.T):
+        for k in range(wl.tables[t].K):
+            assert_close(grads[t][k], ref[t][k], f"short bags {pooling} {mode} dG[{t}][{k}]")
+
+
+def test_short_bags_with_rows_outside_the_table(binding):
+    # ids outside the table among one- and two-lookup bags: flagged, and they add nothing to their bag
+    wl = workloads.custom(SHORT_BAG_TABLES[32], 777, (0, 3), seed=125, name="short-oor")
+    idx = wl.indices.copy()
+    rng = np.random.default_rng(5)
+    bad = rng.choice(wl.L, size=wl.L // 7, replace=False)
+    t_of = np.searchsorted(wl.offsets[:: wl.B][1:], bad, side="right")
+    idx[bad] = np.array([wl.tables[t].N for t in t_of]) + rng.integers(0, 5, size=bad.size)
+    wl_bad = workloads.Workload(wl.name, wl.tables, wl.B, idx, wl.offsets, wl.cores, wl.grad_out)
+    emb, out = run_forward(binding, wl_bad)
+    assert emb.status() & binding.STATUS_INDEX
+    assert_close(out, oracle.forward_workload(wl_bad), "short bags with bad ids out")   # the oracle skips them as well
+
+
 @pytest.mark.parametrize("D,rank", [(16, 8), (16, 16), (16, 32), (32, 8), (32, 16), (32, 32), (64, 8), (64, 16), (64, 32)])
 def test_sweep_point_shapes(binding, D, rank):
     # the shapes of the dimension / rank sweep (dim factors 2x2x4, 2x4x4, 4x4x4) at a batch the oracle finishes fast
