@@ -954,19 +954,23 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     }
 }
 
-// The same gather for batches with few lookups per bag (below TT_POOL_STREAM_BELOW on average): a window is 32
-// consecutive lookups of the warp's share, whatever bags they belong to.  One bag per window, as in k_pool_async, costs
-// the latency of a window per bag: 2 million bags took 0.82 ms there whether they held 2 or 16 lookups each, and 7.9
-// million one-lookup bags 3.0 ms.  Here a window of one-lookup bags goes straight from the staged rows to out (those
-// 7.9 million bags: 0.40 ms, 5 TB/s of rows read and written); a window with several bags in it is summed by the whole
-// warp at once, each sub-warp taking consecutive rows and the pieces of a bag that crosses sub-warps being joined
-// afterwards (2 lookups per bag: 0.82 -> 0.20 ms, 4: 0.30, 8: 0.51, 12: 0.80 against 0.86); a window with one boundary,
-// empty bags, weights or mean pooling is summed bag by bag.  From about 14 lookups per bag on the per-bag kernel is the
-// faster one (its windows are then mostly full, and the sums here cost more instructions per row).  A window ends
-// early only at the end of the share or of a table (the rank look-up of a window uses one table).  With malformed
-// offsets (status bit set by the offsets check earlier in the stream) every bag is summed over its own clamped
-// (offsets[bag], offsets[bag + 1]) pair as the header promises, and windows stop at the end of their bag.
-#define TT_POOL_STREAM_BELOW 14
+// The same gather for batches with few lookups per bag (on average below TT_POOL_STREAM_BELOW, or ..._WIDE for rows
+// of more than 128 bytes): a window is 32 consecutive lookups of the warp's share, whatever bags they belong to.  One
+// bag per window, as in k_pool_async, costs the latency of a window per bag: 2 million bags took 0.82 ms there whether
+// they held 2 or 16 lookups each, and 7.9 million one-lookup bags 3.0 ms.  Here a window of one-lookup bags goes
+// straight from the staged rows to out (those 7.9 million bags: 0.40 ms, 5 TB/s of rows read and written); a full
+// window with one boundary is summed into two partial sums in one unrolled pass; a window with several bags in it is
+// summed by the whole warp at once, each sub-warp taking consecutive rows and the pieces of a bag that crosses
+// sub-warps being joined afterwards; a window with empty bags, weights or mean pooling is summed bag by bag.  2 million
+// bags of 128-byte rows with 2 / 4 / 8 / 16 / 24 lookups each: 0.20 / 0.30 / 0.51 / 0.70 / 0.92 ms against 0.82 / 0.82 /
+// 0.84 / 0.84 / 0.97 with one bag per window, at 32 lookups 1.16 against 1.04; 256-byte rows: 2 lookups 0.33 against
+// 0.92 ms, 8 lookups 0.87 against 0.88, 12 lookups 1.28 against 1.01 (the warp-wide sum runs 16 rows per sub-warp there
+// and spills registers).  Hence the two thresholds.  A window ends early only at the end of the share or of a table
+// (the rank look-up of a window uses one table).  With malformed offsets (status bit set by the offsets check earlier in
+// the stream) every bag is summed over its own clamped (offsets[bag], offsets[bag + 1]) pair as the header promises,
+// and windows stop at the end of their bag.
+#define TT_POOL_STREAM_BELOW 24        // rows of up to 128 bytes
+#define TT_POOL_STREAM_BELOW_WIDE 8    // rows of up to 256 bytes
 template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, float* __restrict__ out)
 {
@@ -1132,7 +1136,26 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
             // no empty bag among those that start inside the window (an empty bag needs a row of zeros: left to the
             // bag-by-bag loop below)
             const int64_t e_prev = __shfl_up_sync(0xffffffffu, e_mine, 1);
-            const bool many = __popc(__ballot_sync(0xffffffffu, e_mine > pos && e_mine < wend)) >= 2;   // else: cheaper bag by bag
+            const int inside = __popc(__ballot_sync(0xffffffffu, e_mine > pos && e_mine < wend));   // bag ends inside the window
+            if (inside == 1 && plain && n == 32) {
+                // one boundary, at row c: the rows before it complete the open bag, the others start the next one
+                const int c = (int)(o_hi - pos);
+                if (w.upairs) __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (int64_t)t * w.B) + (lane >= c ? 1u : 0u)));
+                float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
+#pragma unroll
+                for (int jj = 0; jj < 32 / RPI; ++jj) {
+                    const int j = RPI * jj + sub;
+                    const float4 v = buf[j * R4 + lr];
+                    if (j < c) tt_add4(pa, v); else tt_add4(pb, v);
+                }
+                acc.x += pa.x; acc.y += pa.y; acc.z += pa.z; acc.w += pa.w;
+                close_bag();
+                acc = pb;
+                __syncwarp();
+                pos = wend;
+                continue;
+            }
+            const bool many = inside >= 2;   // else: cheaper bag by bag
             if (many && !__any_sync(0xffffffffu, lane >= 1 && e_prev < wend && e_mine == e_prev)) {
                 // starts: bit j = row j is the first of its bag; closes: bit j = row j is the last of its bag
                 const unsigned starts = __reduce_or_sync(0xffffffffu, (e_mine > pos && e_mine < wend) ? 1u << (int)(e_mine - pos) : 0u)
@@ -1271,7 +1294,7 @@ static cudaError_t launch_pool_async(tt_emb* h, float* out, cudaStream_t s)
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
     if ((e = launch_pool_bounds(h, grid * POOL_WARPS, s)) != cudaSuccess) return e;
-    if (h->v.L < (int64_t)TT_POOL_STREAM_BELOW * nb) {   // few lookups per bag: windows across bags
+    if (h->v.L < (int64_t)(R4 == 16 ? TT_POOL_STREAM_BELOW_WIDE : TT_POOL_STREAM_BELOW) * nb) {   // few lookups per bag: windows across bags
         if ((e = cudaFuncSetAttribute(k_pool_stream<R4, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
         if ((e = tt_launch_pdl(k_pool_stream<R4, WT>, dim3((int)grid), dim3(32 * POOL_WARPS), smem, s, h->v, out)) != cudaSuccess) return e;
         tt_note_launch();
