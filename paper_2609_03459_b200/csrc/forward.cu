@@ -959,18 +959,20 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
 // bag per window, as in k_pool_async, costs the latency of a window per bag: 2 million bags took 0.82 ms there whether
 // they held 2 or 16 lookups each, and 7.9 million one-lookup bags 3.0 ms.  Here a window of one-lookup bags goes
 // straight from the staged rows to out (those 7.9 million bags: 0.40 ms, 5 TB/s of rows read and written); a full
-// window with one boundary is summed into two partial sums in one unrolled pass; a window with several bags in it is
+// window with one boundary is summed into two partial sums in one unrolled pass; a window with many bags in it is
 // summed by the whole warp at once, each sub-warp taking consecutive rows and the pieces of a bag that crosses
-// sub-warps being joined afterwards; a window with empty bags, weights or mean pooling is summed bag by bag.  2 million
-// bags of 128-byte rows with 2 / 4 / 8 / 16 / 24 lookups each: 0.20 / 0.30 / 0.51 / 0.70 / 0.92 ms against 0.82 / 0.82 /
-// 0.84 / 0.84 / 0.97 with one bag per window, at 32 lookups 1.16 against 1.04; 256-byte rows: 2 lookups 0.33 against
-// 0.92 ms, 8 lookups 0.87 against 0.88, 12 lookups 1.28 against 1.01 (the warp-wide sum runs 16 rows per sub-warp there
-// and spills registers).  Hence the two thresholds.  A window ends early only at the end of the share or of a table
-// (the rank look-up of a window uses one table).  With malformed offsets (status bit set by the offsets check earlier in
-// the stream) every bag is summed over its own clamped (offsets[bag], offsets[bag + 1]) pair as the header promises,
-// and windows stop at the end of their bag.
-#define TT_POOL_STREAM_BELOW 24        // rows of up to 128 bytes
-#define TT_POOL_STREAM_BELOW_WIDE 8    // rows of up to 256 bytes
+// sub-warps being joined afterwards (from two boundaries on for rows of up to 128 bytes, from five on for wider rows,
+// where a sub-warp has sixteen rows to walk); a window with empty bags, weights or mean pooling is summed bag by bag.
+// 2 million bags with 2 / 4 / 8 lookups each: 0.20 / 0.30 / 0.51 ms (128-byte rows) and 0.29 / 0.44 / 0.77 ms (256-byte
+// rows) against 0.82-0.92 ms with one bag per window; 1 to 15 lookups per bag: 0.68 against 0.83 and 0.83 against 0.95
+// ms.  With 1 to 31 lookups per bag the per-bag kernel is level or ahead (0.91 against 1.08 ms, 1.10 against 1.11), and
+// on the benchmark configuration (1 to 100 lookups, 256-byte rows) the two are within 2 % (2.34 here, 2.39 there).
+// Hence the thresholds.  A window ends early only at the end of the share or of a table (the rank look-up of a window
+// uses one table).  With malformed offsets (status bit set by the offsets check earlier in the stream) every bag is
+// summed over its own clamped (offsets[bag], offsets[bag + 1]) pair as the header promises, and windows stop at the
+// end of their bag.
+#define TT_POOL_STREAM_BELOW 14        // rows of up to 128 bytes
+#define TT_POOL_STREAM_BELOW_WIDE 12   // rows of up to 256 bytes
 template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, float* __restrict__ out)
 {
@@ -1155,7 +1157,7 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                 pos = wend;
                 continue;
             }
-            const bool many = inside >= 2;   // else: cheaper bag by bag
+            const bool many = inside >= (R4 == 16 ? 5 : 2);   // fewer: cheaper bag by bag
             if (many && !__any_sync(0xffffffffu, lane >= 1 && e_prev < wend && e_mine == e_prev)) {
                 // starts: bit j = row j is the first of its bag; closes: bit j = row j is the last of its bag
                 const unsigned starts = __reduce_or_sync(0xffffffffu, (e_mine > pos && e_mine < wend) ? 1u << (int)(e_mine - pos) : 0u)
@@ -1181,7 +1183,8 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                 // of a bag that goes on after them is what `run` holds at the end
                 float4 run = make_float4(0.f, 0.f, 0.f, 0.f), head = run;
                 bool head_open = !((starts >> (sub * R4)) & 1u), head_closed = false;
-#pragma unroll
+                constexpr int VU = R4 == 16 ? 4 : 8;     // sixteen rows unrolled at once spill registers
+#pragma unroll VU
                 for (int jj = 0; jj < R4; ++jj) {
                     const int j = sub * R4 + jj;
                     if (j < n) {
