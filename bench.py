@@ -47,10 +47,17 @@ WORKLOADS = {
     # a shape outside the register-tiled kernel variants: what a user of the any-shape path gets
     "generic": (0, True, "generic path: 8 tables of the config-3 recipe with dim factors 3x3x5 (D=45), ranks [1,6,4,1], "
                          "batch 32768, pooling U[1,100], forward + backward + SGD"),
+    # the operating point of the paper's evaluation (Sec. 4.1) on stand-in inputs
+    "many-tables": (6, True, "many tables: 240 tables of the config-3 recipe, D=32 (2x4x4), ranks [1,32,32,1], batch 32768, "
+                             "bag lengths U[1,P_t] with P_t logU[1,64] per table, forward + backward + SGD"),
 }
 
 
 def make_workload(cfg_id, mapping, num_tables=None, batch=None, batch_seed=None):
+    if cfg_id == 6:
+        if batch_seed is not None:
+            raise SystemExit("the many-tables workload is a single-GPU measurement")
+        return workloads.many_tables_point(batch or 32768, num_tables=num_tables or 240, mapping=mapping)
     if cfg_id == 0:
         if batch_seed is not None:
             raise SystemExit("the generic workload is a single-GPU measurement")
@@ -349,7 +356,8 @@ def main():
     # Room for distinct rows: the safe bound min(L, sum N) would size the row buffer for 99 M rows (25 GB) on the 60-table
     # workload, whose batches hold about 0.2 L distinct rows.  Large batches get L / 4 rows; a batch with more would set the
     # overflow status bit, which is checked below.
-    mur = 0 if (abl & 4) else max(L // 4, min(L, 1 << 22))
+    # (the many-tables workload, with its short bags, holds 0.25 L: it gets L / 2)
+    mur = 0 if (abl & 4) else max(L // (2 if cfg_id == 6 else 4), min(L, 1 << 22))
     emb = binding.from_workload(wl, enable_backward=train, ablation=abl, max_unique_rows=mur, device=device)
     h_idx = torch.from_numpy(wl.indices).pin_memory()
     h_off = torch.from_numpy(wl.offsets).pin_memory()

@@ -228,6 +228,24 @@ def test_short_bags_weighted_and_mean(binding, pooling, mode):
             assert_close(grads[t][k], ref[t][k], f"short bags {pooling} {mode} dG[{t}][{k}]")
 
 
+def test_many_tables_point_reduced(binding):
+    # the many-tables bench workload (D = 32, ranks 32, every table with its own bag-length law) at a size the oracle
+    # finishes in seconds: both pooling kernels' territory in one batch, fused update
+    wl = workloads.many_tables_point(700, num_tables=16, with_grad=True)
+    emb, out = run_forward(binding, wl, enable_backward=True)
+    assert emb.status() == 0
+    assert_close(out, oracle.forward_workload(wl, memo=True), "many-tables out")
+    emb.backward_sgd(dev(wl.grad_out), 0.01)
+    grads = emb.get_grads()
+    cores = emb.get_cores()
+    ref = oracle.backward_workload(wl, memo=True)
+    for t in range(wl.T):
+        want = oracle.sgd(wl.cores[t], ref[t], 0.01)
+        for k in range(3):
+            assert_close(grads[t][k], ref[t][k], f"many-tables dG[{t}][{k}]")
+            assert_close(cores[t][k], want[k], f"many-tables core[{t}][{k}]")
+
+
 def test_short_bags_with_rows_outside_the_table(binding):
     # ids outside the table among one- and two-lookup bags: flagged, and they add nothing to their bag
     wl = workloads.custom(SHORT_BAG_TABLES[32], 777, (0, 3), seed=125, name="short-oor")

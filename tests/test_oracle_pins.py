@@ -340,3 +340,20 @@ def test_forward_bags_sampling_agrees_with_full():
     got = oracle.forward_bags(wl, pairs)
     for i, (t, b) in enumerate(pairs):
         np.testing.assert_array_equal(got[i], full[b, t * wl.D:(t + 1) * wl.D])
+
+
+def test_per_table_bag_lengths_and_the_many_tables_point():
+    # a list gives every table its own bag-length law; the many-tables point (the paper's operating shape, Sec. 4.1:
+    # D = 32, ranks 32, three cores) draws one per table and records it
+    spec = workloads.TableSpec(500, (8, 8, 8), (2, 4, 4), (1, 4, 4, 1), 1.0, "normal", 0.1)
+    wl = workloads.custom([spec, spec, spec], 50, [1, (0, 3), (5, 9)], seed=3)
+    lens = np.diff(wl.offsets).reshape(3, 50)
+    assert (lens[0] == 1).all() and lens[1].min() >= 0 and lens[1].max() <= 3 and lens[2].min() >= 5 and lens[2].max() <= 9
+    assert wl.L == int(lens.sum()) and wl.indices.min() >= 0 and wl.indices.max() < 500
+    mt = workloads.many_tables_point(16, num_tables=6, with_grad=True)
+    assert mt.T == 6 and mt.D == 32 and all(s.r == (1, 32, 32, 1) and s.d == (2, 4, 4) for s in mt.tables)
+    lens = np.diff(mt.offsets).reshape(6, 16)
+    for t, cap in enumerate(mt.meta["max_bag"]):
+        assert 1 <= cap <= 64 and lens[t].min() >= 1 and lens[t].max() <= cap
+    again = workloads.many_tables_point(16, num_tables=6, with_grad=True)
+    assert np.array_equal(mt.indices, again.indices) and np.array_equal(mt.grad_out, again.grad_out)

@@ -131,7 +131,7 @@ def near_equal_factors3(N: int) -> Tuple[int, int, int]:
 
 
 def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None, batch_seed0=None) -> Workload:
-    """pooling: int (fixed) or (lo, hi) inclusive uniform per (table, bag).
+    """pooling: int (fixed) or (lo, hi) inclusive uniform per (table, bag); a list gives one of these per table.
     batch_seed0: draw the batch (bag lengths, indices, grad_out) from another stream while the cores stay
     those of seed0 (used for the per-rank batches of a multi-GPU run)."""
     T = len(tables)
@@ -143,10 +143,11 @@ def _assemble(name, tables, B, pooling, seed0, mapping, with_grad, meta=None, ba
         tc = make_cores(rng, spec)
         if batch_seed0 is not None:
             rng = np.random.default_rng(batch_seed0 + t)
-        if isinstance(pooling, tuple):
-            lens = rng.integers(pooling[0], pooling[1] + 1, size=B, dtype=np.int64)
+        pool_t = pooling[t] if isinstance(pooling, list) else pooling
+        if isinstance(pool_t, tuple):
+            lens = rng.integers(pool_t[0], pool_t[1] + 1, size=B, dtype=np.int64)
         else:
-            lens = np.full(B, int(pooling), dtype=np.int64)
+            lens = np.full(B, int(pool_t), dtype=np.int64)
         return tc, lens, zipf_rows(rng, spec.N, spec.alpha, int(lens.sum()), mapping)
 
     if T > 1 and sum(s.N for s in tables) > 1_000_000:
@@ -271,3 +272,21 @@ def generic_point(batch: int = 32768, *, num_tables: int = 8, with_grad: bool = 
     tables = [TableSpec(N=s.N, n=s.n, d=(3, 3, 5), r=(1, 6, 4, 1), alpha=s.alpha, core_dist="normal", core_scale=0.05)
               for s in base]
     return _assemble(f"generic-d3x3x5-r6x4-B{batch}", tables, batch, (1, 100), seed3 + 4500, mapping, with_grad=with_grad)
+
+
+def many_tables_point(batch: int = 32768, *, num_tables: int = 240, with_grad: bool = True, mapping: str = "identity",
+                      seed: Optional[int] = None) -> Workload:
+    """The operating point of the paper's evaluation (Sec. 4.1): hundreds of tables, three cores, D = 32 (dim factors
+    2 x 4 x 4), ranks (1, 32, 32, 1), batch 32768.  The paper's tables and index streams are a public benchmark that
+    is not available here and whose pooling factors the paper does not state, so this is a stand-in: row counts and
+    Zipf exponents from the config-3 recipe (log-uniform in [1e4, 4e7], exponent uniform in [0.8, 1.2]); every table
+    has its own largest bag length P_t, log-uniform in [1, 64] (a quarter of the tables come out with at most three
+    lookups per bag, a fifth with up to 32 or more), bag lengths uniform in [1, P_t]."""
+    seed6 = (BASE_SEED if seed is None else seed) + 1000 * 6
+    trng = np.random.default_rng(seed6 + 500)
+    base = _cfg3_tables(trng, num_tables)
+    tables = [TableSpec(N=s.N, n=s.n, d=(2, 4, 4), r=(1, 32, 32, 1), alpha=s.alpha, core_dist="normal", core_scale=0.05)
+              for s in base]
+    pooling = [(1, int(round(64.0 ** trng.uniform(0.0, 1.0)))) for _ in range(num_tables)]
+    return _assemble(f"many-tables-T{num_tables}-D32-r32-B{batch}", tables, batch, pooling, seed6, mapping,
+                     with_grad=with_grad, meta={"max_bag": [p[1] for p in pooling]})
