@@ -1058,11 +1058,17 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
             ct[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
             ct[mt][kt][3] = tt_split_tf32(KHALF || BHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
         }
-    float dc[MT][NT][4], dct[MT][NT][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
+    // C of 8 or 4 rows would fill half or a quarter of the row tiles of dC: there the product runs transposed,
+    // dC^T[b][p] += sum_{(row, j)} D_row[b][j] * dE_row[p][j], M = b, N = 8 columns p (PM = 4: four of them zero), K = 8 =
+    // two rows x 4 columns j: RB_/16 tiles per pair instead of RB_/8
+    constexpr bool TR = HALF && RB_ >= 16;
+    constexpr int MTT = RB_ / 16;
+    constexpr int DM = TR ? MTT : MT, DN = TR ? 1 : NT;
+    float dc[DM][DN][4], dct[DM][DN][4];   // tensor-core accumulators and their rounded running sums (see tt_warp_rows_dC_mma)
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int mt = 0; mt < DM; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < DN; ++nt)
 #pragma unroll
             for (int x = 0; x < 4; ++x) { dc[mt][nt][x] = 0.f; dct[mt][nt][x] = 0.f; }
     const int rb_ = g >> 2, jb = g & 3;       // dG B fragment: row rb_ of the pair, column jb of dE
@@ -1079,6 +1085,7 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
         float av[MT][4], bv[NT][2], ev[KT2][2];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
+            // (transposed: av[0][0], av[0][2] are the B fragment dE_a[p = g][j = t], dE_c[g][t])
             av[mt][0] = rowok ? __ldg(Ea + (16 * mt + g) * 4 + t) : 0.f;
             av[mt][1] = HALF ? 0.f : __ldg(Ea + (16 * mt + g + 8) * 4 + t);
             av[mt][2] = two && rowok ? __ldg(Ec + (16 * mt + g) * 4 + t) : 0.f;
@@ -1088,8 +1095,9 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
         const float* __restrict__ Dc = GK + (size_t)iKc * (RB_ * 4) + t;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
+            // (transposed: bv[2 mt][.], bv[2 mt + 1][.] are the A fragment rows b = 16 mt + g and + 8 of D_a, D_c)
             bv[nt][0] = __ldg(Da + (8 * nt + g) * 4);
-            bv[nt][1] = __ldg(Dc + (8 * nt + g) * 4);
+            bv[nt][1] = two || !TR ? __ldg(Dc + (8 * nt + g) * 4) : 0.f;
         }
         const bool valid = rb_ == 0 || two;
         const float* __restrict__ El = (rb_ == 0 ? Ea : Ec) + jb;
@@ -1099,7 +1107,20 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
             ev[kt][1] = valid && !KHALF ? __ldg(El + (8 * kt + t + 4) * 4) : 0.f;
         }
         // ---- dC += dE . D^T
-        {
+        if constexpr (TR) {
+            Tf32Pair b[2];
+            b[0] = tt_split_tf32(av[0][0]);
+            b[1] = tt_split_tf32(av[0][2]);
+#pragma unroll
+            for (int mt = 0; mt < MTT; ++mt) {
+                Tf32Pair a[4];
+                a[0] = tt_split_tf32(bv[2 * mt][0]);
+                a[1] = tt_split_tf32(bv[2 * mt + 1][0]);
+                a[2] = tt_split_tf32(bv[2 * mt][1]);
+                a[3] = tt_split_tf32(bv[2 * mt + 1][1]);
+                tt_mma_3xtf32(dc[mt][0], a, b);
+            }
+        } else {
             Tf32Pair a[MT][4];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
@@ -1138,11 +1159,24 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
         }
     }
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int mt = 0; mt < DM; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < DN; ++nt)
 #pragma unroll
             for (int x = 0; x < 4; ++x) { dct[mt][nt][x] += dc[mt][nt][x]; dc[mt][nt][x] = 0.f; }
+    }
+    if constexpr (TR) {
+        // the lane holds dC[p = 2t][b], dC[2t + 1][b] for b = 16 mt + g and b + 8
+        if (2 * t < PM) {
+#pragma unroll
+            for (int mt = 0; mt < MTT; ++mt) {
+                dPdst[(2 * t) * RB_ + 16 * mt + g] = dct[mt][0][0];
+                dPdst[(2 * t + 1) * RB_ + 16 * mt + g] = dct[mt][0][1];
+                dPdst[(2 * t) * RB_ + 16 * mt + g + 8] = dct[mt][0][2];
+                dPdst[(2 * t + 1) * RB_ + 16 * mt + g + 8] = dct[mt][0][3];
+            }
+        }
+        return;
     }
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)

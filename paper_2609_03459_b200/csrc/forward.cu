@@ -290,6 +290,81 @@ __device__ __forceinline__ void tt_warp_rows_mma(const float* Cs, const WsView& 
     }
 }
 
+// The same product for C of 8 or 4 rows (d_1 d_2 = 8 or 4), where the form above fills half or a quarter of its row
+// tile: transposed, E_u[p][j] = sum_b D_u[b][j] * C[p][b] as m16n8k8 tiles with M = 16 = four child rows x 4 columns
+// j, K = 8 values of b, N = 8 rows p of C (PM = 4: columns 4..7 are zero operands).  Half the tensor-core
+// instructions per row (a quarter for PM = 4); the split fragments of C^T take RB/2 registers.  A lane ends up with
+// single floats of four rows of E (p = 2t, 2t+1; column j = g % 4) and stores them as such.
+template <int PM, int RB, int CS = RB>
+__device__ __forceinline__ void tt_warp_rows_mma_t(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
+                                                   uint32_t row_base, int lane)
+{
+    static_assert(PM == 8 || PM == 4, "C of 8 or 4 rows");
+    constexpr int KT = RB / 8;
+    const int g = lane >> 2, t = lane & 3;
+    const bool pok = g < PM;                // this lane's column p of C^T exists
+    Tf32Pair cb[KT][2];                     // B[k = b][n = p] = C[p][b]
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+        cb[kt][0] = tt_split_tf32(pok ? Cs[g * CS + 8 * kt + t] : 0.f);
+        cb[kt][1] = tt_split_tf32(pok ? Cs[g * CS + 8 * kt + t + 4] : 0.f);
+    }
+    const int K = w.K;
+    const float* __restrict__ GK = td.core[K - 1];
+    const uint32_t* __restrict__ rows = w.val[K];
+    const int q0 = g >> 2, j = g & 3;       // A-fragment rows g and g + 8: child rows q0 and q0 + 2 of the four, column j
+    constexpr int NQ = 2;                   // fours of rows in flight
+    constexpr uint32_t IDC = 32;            // rows per id chunk: a multiple of the rows per iteration
+    uint32_t ids = 0, cbase = u0;           // last digits of IDC rows at a time, one per lane (the loop takes them by shuffle)
+    for (uint32_t ub = u0; ub < u1; ub += 4 * NQ) {
+        if (ub == cbase + IDC || ub == u0) {
+            cbase = ub;
+            ids = (ub + lane < u1) ? rows[ub + lane] - row_base : 0u;
+        }
+        float av[NQ][KT][4];
+#pragma unroll
+        for (int nq = 0; nq < NQ; ++nq) {
+            // a short tail repeats the last row; it is computed but not stored
+            const uint32_t ula = min(ub + 4 * nq + (uint32_t)q0, u1 - 1), ulc = min(ub + 4 * nq + (uint32_t)q0 + 2, u1 - 1);
+            const uint32_t iKa = __shfl_sync(0xffffffffu, ids, ula - cbase), iKc = __shfl_sync(0xffffffffu, ids, ulc - cbase);
+            const float* __restrict__ Da = GK + (size_t)iKa * (RB * 4) + j;
+            const float* __restrict__ Dc = GK + (size_t)iKc * (RB * 4) + j;
+#pragma unroll
+            for (int kt = 0; kt < KT; ++kt) {
+                av[nq][kt][0] = __ldg(Da + (8 * kt + t) * 4);
+                av[nq][kt][1] = __ldg(Dc + (8 * kt + t) * 4);
+                av[nq][kt][2] = __ldg(Da + (8 * kt + t + 4) * 4);
+                av[nq][kt][3] = __ldg(Dc + (8 * kt + t + 4) * 4);
+            }
+        }
+#pragma unroll
+        for (int nq = 0; nq < NQ; ++nq) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kt = 0; kt < KT; ++kt) {
+                Tf32Pair a[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) a[x] = tt_split_tf32(av[nq][kt][x]);
+                tt_mma_3xtf32(acc, a, cb[kt]);
+            }
+            // acc: E[p = 2t][j], E[2t + 1][j] of child row q0, then of child row q0 + 2
+            const uint32_t usa = ub + 4 * nq + (uint32_t)q0, usc = usa + 2;
+            if (2 * t < PM) {
+                if (usa < u1) {
+                    float* e = w.E + (size_t)usa * (PM * 4) + (2 * t) * 4 + j;
+                    __stcs(e, acc[0]);
+                    __stcs(e + 4, acc[1]);
+                }
+                if (usc < u1) {
+                    float* e = w.E + (size_t)usc * (PM * 4) + (2 * t) * 4 + j;
+                    __stcs(e, acc[2]);
+                    __stcs(e + 4, acc[3]);
+                }
+            }
+        }
+    }
+}
+
 // one warp: groups fetched dynamically from the CTA's range through a shared counter
 template <int PM, int RB, int TP, int M, int CPL, bool MMA>
 __device__ __forceinline__ void tt_sweep_fast(const WsView& w, const TableDesc& td, uint32_t g1, float* As, float* Cs,
@@ -354,7 +429,8 @@ __device__ __forceinline__ void tt_sweep_quad(const WsView& w, const TableDesc& 
         for (int q = 0; q < cnt; ++q) {
             const uint32_t val = __shfl_sync(0xffffffffu, valq, q);
             const uint32_t u0 = __shfl_sync(0xffffffffu, u0q, q), u1 = __shfl_sync(0xffffffffu, u1q, q);
-            if constexpr (TP == 0) tt_warp_rows_mma<PM, RB, RB + 4>(Cs4 + (size_t)q * (PM * (RB + 4)), w, td, u0, u1, val * nK, lane);
+            if constexpr (TP == 0 && PM < 16) tt_warp_rows_mma_t<PM, RB, RB + 4>(Cs4 + (size_t)q * (PM * (RB + 4)), w, td, u0, u1, val * nK, lane);
+            else if constexpr (TP == 0) tt_warp_rows_mma<PM, RB, RB + 4>(Cs4 + (size_t)q * (PM * (RB + 4)), w, td, u0, u1, val * nK, lane);
             else tt_warp_rows<PM, RB, TP>(Cs4 + (size_t)q * (PM * RB), w, td, u0, u1, val * nK, lane);
         }
         __syncwarp();
