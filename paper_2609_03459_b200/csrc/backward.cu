@@ -1176,15 +1176,15 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
                 dPdst[(2 * t + 1) * RB_ + 16 * mt + g + 8] = dct[mt][0][3];
             }
         }
-        return;
+    } else {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (rowok) *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
+                if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
+            }
     }
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            if (rowok) *reinterpret_cast<float2*>(dPdst + (16 * mt + g) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][0], dct[mt][nt][1]);
-            if (!HALF) *reinterpret_cast<float2*>(dPdst + (16 * mt + g + 8) * RB_ + 8 * nt + 2 * t) = make_float2(dct[mt][nt][2], dct[mt][nt][3]);
-        }
 }
 
 template <int PM, int RB_, int TP, int M, int CPL, bool MMA>
