@@ -1580,32 +1580,45 @@ __global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant
     float* const cdst = td.core[kc] + (size_t)ik * td.slice_floats[kc];
     auto fold = [&](bool last) {
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
+        for (int mt = 0; mt < MT; ++mt) {
+            // all loads of a row tile first, then the sums and stores: one round trip per tile instead of one per
+            // column block (the compiler cannot move a load above a store it cannot tell apart)
+            float2 v0[NTW], v1[NTW], u0[NTW], u1[NTW];
+            const bool upd = last && w.fused_lr != 0.f;
 #pragma unroll
             for (int nt = 0; nt < NTW; ++nt) {
                 const int c = wid * CW + 8 * nt + 2 * t;
+                v0[nt] = make_float2(0.f, 0.f); v1[nt] = v0[nt]; u0[nt] = v0[nt]; u1[nt] = v0[nt];
                 if (c >= COLS) continue;     // this warp owns no columns of the slice gradient
-                float2* p0 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g) * COLS + c);
-                float2* p1 = reinterpret_cast<float2*>(gdst + (size_t)(16 * mt + g + 8) * COLS + c);
-                float2 v0 = first_fold ? make_float2(0.f, 0.f) : *p0;
-                float2 v1 = (first_fold || AHALF) ? make_float2(0.f, 0.f) : *p1;
-                v0.x += acc[mt][nt][0]; v0.y += acc[mt][nt][1]; v1.x += acc[mt][nt][2]; v1.y += acc[mt][nt][3];
-                *p0 = v0;
-                if (!AHALF) *p1 = v1;
-                if (last && w.fused_lr != 0.f) {
-                    float2* c0 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g) * COLS + c);
-                    float2 u0 = *c0;
-                    u0.x = u0.x - w.fused_lr * v0.x; u0.y = u0.y - w.fused_lr * v0.y;
-                    *c0 = u0;
+                const size_t o0 = (size_t)(16 * mt + g) * COLS + c, o1 = (size_t)(16 * mt + g + 8) * COLS + c;
+                if (!first_fold) {
+                    v0[nt] = *reinterpret_cast<const float2*>(gdst + o0);
+                    if (!AHALF) v1[nt] = *reinterpret_cast<const float2*>(gdst + o1);
+                }
+                if (upd) {
+                    u0[nt] = *reinterpret_cast<const float2*>(cdst + o0);
+                    if (!AHALF) u1[nt] = *reinterpret_cast<const float2*>(cdst + o1);
+                }
+            }
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) {
+                const int c = wid * CW + 8 * nt + 2 * t;
+                if (c >= COLS) continue;
+                const size_t o0 = (size_t)(16 * mt + g) * COLS + c, o1 = (size_t)(16 * mt + g + 8) * COLS + c;
+                v0[nt].x += acc[mt][nt][0]; v0[nt].y += acc[mt][nt][1]; v1[nt].x += acc[mt][nt][2]; v1[nt].y += acc[mt][nt][3];
+                *reinterpret_cast<float2*>(gdst + o0) = v0[nt];
+                if (!AHALF) *reinterpret_cast<float2*>(gdst + o1) = v1[nt];
+                if (upd) {
+                    u0[nt].x = u0[nt].x - w.fused_lr * v0[nt].x; u0[nt].y = u0[nt].y - w.fused_lr * v0[nt].y;
+                    *reinterpret_cast<float2*>(cdst + o0) = u0[nt];
                     if (!AHALF) {
-                        float2* c1 = reinterpret_cast<float2*>(cdst + (size_t)(16 * mt + g + 8) * COLS + c);
-                        float2 u1 = *c1;
-                        u1.x = u1.x - w.fused_lr * v1.x; u1.y = u1.y - w.fused_lr * v1.y;
-                        *c1 = u1;
+                        u1[nt].x = u1[nt].x - w.fused_lr * v1[nt].x; u1[nt].y = u1[nt].y - w.fused_lr * v1[nt].y;
+                        *reinterpret_cast<float2*>(cdst + o1) = u1[nt];
                     }
                 }
                 acc[mt][nt][0] = 0.f; acc[mt][nt][1] = 0.f; acc[mt][nt][2] = 0.f; acc[mt][nt][3] = 0.f;
             }
+        }
         first_fold = false;
     };
     const uint32_t space = td.prefix_space[k - 1];
@@ -1650,10 +1663,18 @@ __global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    lookup_ids(0);
-    publish_ids(0);
-    lookup_ids(1);
-    publish_ids(1);
+    // passes 0 and 1 are looked up side by side (threads 0..NQ-1 and NQ..2NQ-1): one chain of round trips, not two
+    if (tid < 2 * NQ) {
+        const uint32_t r = (uint32_t)tid / NQ, q = (uint32_t)tid % NQ;
+        uint32_t nd = 0xffffffffu;
+        const float* lf = nullptr;
+        if (j0 + r * NQ + q < j1) {
+            nd = w.tnode[k][j0 + r * NQ + q];
+            lf = tt_left_operand(w, td, k, nd);
+        }
+        s_node[r][q] = nd;
+        s_left[r][q] = lf;
+    }
     __syncthreads();
     if (passes > 0) issue(0);
     for (uint32_t r = 0; r < passes; ++r) {
