@@ -555,7 +555,7 @@ def main():
     # and is scaled by the units this launch processes; it is reported only for the shape the capture was taken on.
     ncu_traffic, capture = dram_traffic_per_unit()
     pool_kernel = "k_pool_async" if 16 < D <= 64 and D % 4 == 0 else ("k_pool_vec" if D % 4 == 0 else "k_pool_scalar")
-    if pool_kernel == "k_pool_async" and L < (12 if D > 32 else 14) * T * B:
+    if pool_kernel == "k_pool_async" and L < (12 if D > 32 else 33) * T * B:
         pool_kernel = "k_pool_stream"   # the library's choice for short bags (windows of lookups across bags)
     same_shape = capture.get("capture_D") == str(D) and capture.get("capture_recipe") in ("cfg3", "cfg5") and cfg_id in (3, 5)
 

@@ -1035,19 +1035,19 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
 // bag per window, as in k_pool_async, costs the latency of a window per bag: 2 million bags took 0.82 ms there whether
 // they held 2 or 16 lookups each, and 7.9 million one-lookup bags 3.0 ms.  Here a window of one-lookup bags goes
 // straight from the staged rows to out (those 7.9 million bags: 0.40 ms, 5 TB/s of rows read and written); a full
-// window with one boundary is summed into two partial sums in one unrolled pass; a window with many bags in it is
+// window with one boundary is summed into two partial sums in one unrolled pass; a window with several bags in it is
 // summed by the whole warp at once, each sub-warp taking consecutive rows and the pieces of a bag that crosses
 // sub-warps being joined afterwards (from two boundaries on for rows of up to 128 bytes, from five on for wider rows,
 // where a sub-warp has sixteen rows to walk); a window with empty bags, weights or mean pooling is summed bag by bag.
-// 2 million bags with 2 / 4 / 8 lookups each: 0.20 / 0.30 / 0.51 ms (128-byte rows) and 0.29 / 0.44 / 0.77 ms (256-byte
-// rows) against 0.82-0.92 ms with one bag per window; 1 to 15 lookups per bag: 0.68 against 0.83 and 0.83 against 0.95
-// ms.  With 1 to 31 lookups per bag the per-bag kernel is level or ahead (0.91 against 1.08 ms, 1.10 against 1.11), and
-// on the benchmark configuration (1 to 100 lookups, 256-byte rows) the two are within 2 % (2.34 here, 2.39 there).
-// Hence the thresholds.  A window ends early only at the end of the share or of a table (the rank look-up of a window
-// uses one table).  With malformed offsets (status bit set by the offsets check earlier in the stream) every bag is
-// summed over its own clamped (offsets[bag], offsets[bag + 1]) pair as the header promises, and windows stop at the
-// end of their bag.
-#define TT_POOL_STREAM_BELOW 14        // rows of up to 128 bytes
+// 2 million bags of 128-byte rows, stream against one bag per window: 2 / 4 / 8 lookups each 0.20 / 0.28 / 0.51 ms
+// against 0.82; 1 to 15 lookups 0.54 against 0.83, 1 to 31 0.83 against 0.91, 1 to 63 1.22 against 1.27, 1 to 100 1.69
+// against 1.72, 1 to 200 3.09 against 3.00 ms.  256-byte rows: 2 / 4 / 8 lookups 0.29 / 0.44 / 0.74 ms against 0.88-0.92;
+// 1 to 15 lookups 0.78 against 0.95; 1 to 31 1.11-1.19 against 1.10; on the benchmark configuration (1 to 100 lookups)
+// 2.34-2.36 against 2.39 ms.  Hence the thresholds (the benchmark configuration stays with the per-bag kernel).  A
+// window ends early only at the end of the share or of a table (the rank look-up of a window uses one table).  With
+// malformed offsets (status bit set by the offsets check earlier in the stream) every bag is summed over its own
+// clamped (offsets[bag], offsets[bag + 1]) pair as the header promises, and windows stop at the end of their bag.
+#define TT_POOL_STREAM_BELOW 33        // rows of up to 128 bytes
 #define TT_POOL_STREAM_BELOW_WIDE 12   // rows of up to 256 bytes
 template <int R4, bool WT>   // R4: float4 pieces per staged row, 16 (D <= 64) or 8 (D <= 32)
 __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, float* __restrict__ out)
@@ -1259,8 +1259,9 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                 // of a bag that goes on after them is what `run` holds at the end
                 float4 run = make_float4(0.f, 0.f, 0.f, 0.f), head = run;
                 bool head_open = !((starts >> (sub * R4)) & 1u), head_closed = false;
-                constexpr int VU = R4 == 16 ? 4 : 8;     // sixteen rows unrolled at once spill registers
-#pragma unroll VU
+                // (not unrolled: the kernel's warps are spread over its four summing paths, and with this loop unrolled
+                // they waited for instructions: 2.39 -> 1.90 ms on the 240-table workload, ncu `no_instruction` stalls)
+#pragma unroll 1
                 for (int jj = 0; jj < R4; ++jj) {
                     const int j = sub * R4 + jj;
                     if (j < n) {
