@@ -19,6 +19,7 @@
 #include "common.cuh"
 #include "scan.cuh"
 #include "mma.cuh"
+#include "quad_mid.cuh"
 
 #define HT_SIZE 4096
 #define HT_TILE 2048
@@ -1033,7 +1034,7 @@ __device__ __forceinline__ void tt_warp_rows_dG_mma(const float* Cs, const WsVie
 
 // Both row passes in one loop over the group's row pairs: the row ids and the dE rows come from memory once (the
 // second fragment layout of dE is served by L1), dC accumulates across the loop, dG_K tiles leave per pair.
-template <int PM, int RB_>
+template <int PM, int RB_, int CS = RB_ + 8>   // CS: row stride of C in shared memory
 __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsView& w, const TableDesc& td, uint32_t u0, uint32_t u1,
                                                      uint32_t row_base, float* dPdst, float* gk, int lane)
 {
@@ -1053,10 +1054,10 @@ __device__ __forceinline__ void tt_warp_rows_bwd_mma(const float* Cs, const WsVi
     for (int mt = 0; mt < MT2; ++mt)
 #pragma unroll
         for (int kt = 0; kt < KT2; ++kt) {
-            ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g]);
-            ct[mt][kt][1] = tt_split_tf32(BHALF ? 0.f : Cs[(8 * kt + t) * (RB_ + 8) + 16 * mt + g + 8]);
-            ct[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g]);
-            ct[mt][kt][3] = tt_split_tf32(KHALF || BHALF ? 0.f : Cs[(8 * kt + t + 4) * (RB_ + 8) + 16 * mt + g + 8]);
+            ct[mt][kt][0] = tt_split_tf32(Cs[(8 * kt + t) * CS + 16 * mt + g]);
+            ct[mt][kt][1] = tt_split_tf32(BHALF ? 0.f : Cs[(8 * kt + t) * CS + 16 * mt + g + 8]);
+            ct[mt][kt][2] = tt_split_tf32(KHALF ? 0.f : Cs[(8 * kt + t + 4) * CS + 16 * mt + g]);
+            ct[mt][kt][3] = tt_split_tf32(KHALF || BHALF ? 0.f : Cs[(8 * kt + t + 4) * CS + 16 * mt + g + 8]);
         }
     // C of 8 or 4 rows would fill half or a quarter of the row tiles of dC: there the product runs transposed,
     // dC^T[b][p] += sum_{(row, j)} D_row[b][j] * dE_row[p][j], M = b, N = 8 columns p (PM = 4: four of them zero), K = 8 =
@@ -1228,10 +1229,50 @@ __device__ __forceinline__ void tt_sweep_bwd_fast(const WsView& w, const TableDe
     }
 }
 
+// The fused-loop shapes with the intermediate products of NG = 16 / MROWS neighbouring groups formed together on the
+// tensor cores, as in the forward sweep (quad_mid.cuh): one group at a time, every group read its whole slice of core
+// K-1 (16 KB at rank 32) for a product of MROWS rows, which made the L1/L2 path the limit where groups hold few rows.
+template <int PM, int RB_, int MROWS, int KTMAX>
+__device__ __forceinline__ void tt_sweep_bwd_quad(const WsView& w, const TableDesc& td, uint32_t g1, float* gk, float* Cs4,
+                                                  uint32_t* next, int lane)
+{
+    constexpr int COLS = PM / MROWS * RB_;   // d_{K-1} * r_{K-1}
+    constexpr int NG = 16 / MROWS;
+    const int K = w.K, km = K - 2;
+    const int ra = td.r[km];
+    const uint32_t nK = (uint32_t)td.n[K - 1];
+    for (;;) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(next, (uint32_t)NG);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (base >= g1) break;
+        const int cnt = (int)min((uint32_t)NG, g1 - base);
+        uint32_t gq = 0, valq = 0, imq = 0, u0q = 0, u1q = 0;
+        const float* srcq = nullptr;
+        if (lane < cnt) {
+            gq = w.tnode[K - 1][base + lane];   // position in the digit-major order -> group
+            valq = w.val[K - 1][gq];
+            imq = valq % (uint32_t)td.n[km];
+            srcq = tt_left_operand(w, td, K - 1, gq);
+            u0q = w.cstart[K - 1][gq];
+            u1q = w.cstart[K - 1][gq + 1];
+        }
+        tt_quad_mid<COLS, MROWS, KTMAX, RB_>(td.core[km], td.slice_floats[km], ra, cnt, imq, srcq, Cs4, lane);
+        __syncwarp();
+        for (int q = 0; q < cnt; ++q) {
+            const uint32_t g = __shfl_sync(0xffffffffu, gq, q), val = __shfl_sync(0xffffffffu, valq, q);
+            const uint32_t u0 = __shfl_sync(0xffffffffu, u0q, q), u1 = __shfl_sync(0xffffffffu, u1q, q);
+            tt_warp_rows_bwd_mma<PM, RB_, RB_ + 4>(Cs4 + (size_t)q * (PM * (RB_ + 4)), w, td, u0, u1, val * nK,
+                                                   w.dP[K - 1] + (size_t)g * w.stride[K - 1], gk, lane);
+        }
+        __syncwarp();
+    }
+}
+
 // One CTA (4 warps) per work unit (table, q); last-core gradients go to one of TT_STRIPES L2-resident partial
 // copies with vector reductions, added up in fixed stripe order by k_reduce_gpart.
 template <int V>
-__global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int c_floats, int vbase)
+__global__ void __launch_bounds__(128, (V == 5 || V == 6 || V == 8 || V == 9 || V == 1) ? 6 : 0) k_sweep_bwd(WsView w, int pl_floats, int c_floats, int vbase)
 {
     tt_pdl_enter();
     extern __shared__ __align__(16) float sm[];
@@ -1256,15 +1297,15 @@ __global__ void __launch_bounds__(128) k_sweep_bwd(WsView w, int pl_floats, int 
     float* As = sm + (size_t)wid * (pl_floats + c_floats);
     float* Cs = As + pl_floats;
     if (V == 0) tt_sweep_bwd_fast<16, 32, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 1) tt_sweep_bwd_fast<16, 16, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 1) tt_sweep_bwd_quad<16, 16, 4, 4>(w, td, g1, gk, sm + (size_t)wid * (4 * 16 * 20), &next, lane);
     if (V == 2) tt_sweep_bwd_fast<16, 8, 4, 4, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 3) tt_sweep_bwd_fast<32, 32, 4, 4, 2, true>(w, td, g1, gk, As, Cs, &next, lane);
     if (V == 4) tt_sweep_bwd_fast<32, 64, 2, 8, 2, false>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 5) tt_sweep_bwd_fast<8, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 6) tt_sweep_bwd_fast<8, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 5) tt_sweep_bwd_quad<8, 32, 2, 4>(w, td, g1, gk, sm + (size_t)wid * (8 * 8 * 36), &next, lane);
+    if (V == 6) tt_sweep_bwd_quad<8, 16, 2, 4>(w, td, g1, gk, sm + (size_t)wid * (8 * 8 * 20), &next, lane);
     if (V == 7) tt_sweep_bwd_fast<8, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);   // 8 x 8: the FP32 pipe wins (0.39 against 0.41 ms)
-    if (V == 8) tt_sweep_bwd_fast<4, 32, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
-    if (V == 9) tt_sweep_bwd_fast<4, 16, 2, 2, 1, true>(w, td, g1, gk, As, Cs, &next, lane);
+    if (V == 8) tt_sweep_bwd_quad<4, 32, 2, 4>(w, td, g1, gk, sm + (size_t)wid * (8 * 4 * 36), &next, lane);
+    if (V == 9) tt_sweep_bwd_quad<4, 16, 2, 4>(w, td, g1, gk, sm + (size_t)wid * (8 * 4 * 20), &next, lane);
     if (V == 10) tt_sweep_bwd_fast<4, 8, 2, 2, 1, false>(w, td, g1, gk, As, Cs, &next, lane);
 }
 
@@ -1300,8 +1341,13 @@ static cudaError_t launch_sweep_bwd(tt_emb* h, int max_pl, int max_c, cudaStream
     if (V == 6) max_c = 8 * (16 + 8);
     if (V == 8) max_c = 4 * (32 + 8);
     if (V == 9) max_c = 4 * (16 + 8);
-    const size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
-                              : (size_t)4 * (max_pl + max_c) * sizeof(float);
+    size_t smem = V < 0 ? (size_t)(max_pl + 2 * max_c + RB * h->D) * sizeof(float)
+                        : (size_t)4 * (max_pl + max_c) * sizeof(float);
+    if (V == 5) smem = (size_t)4 * 8 * 8 * 36 * sizeof(float);    // eight C tiles per warp, rows padded by four floats
+    if (V == 6) smem = (size_t)4 * 8 * 8 * 20 * sizeof(float);
+    if (V == 8) smem = (size_t)4 * 8 * 4 * 36 * sizeof(float);
+    if (V == 9) smem = (size_t)4 * 8 * 4 * 20 * sizeof(float);
+    if (V == 1) smem = (size_t)4 * 4 * 16 * 20 * sizeof(float);   // four C tiles per warp
     cudaError_t e = cudaFuncSetAttribute(k_sweep_bwd<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if ((e = tt_stage_begin(h, 9 + TT_NUM_VARIANTS + 1 + V + 1, s)) != cudaSuccess) return e;
