@@ -1641,9 +1641,9 @@ __global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant
                     v0[nt] = *reinterpret_cast<const float2*>(gdst + o0);
                     if (!AHALF) v1[nt] = *reinterpret_cast<const float2*>(gdst + o1);
                 }
-                if (upd) {
-                    u0[nt] = *reinterpret_cast<const float2*>(cdst + o0);
-                    if (!AHALF) u1[nt] = *reinterpret_cast<const float2*>(cdst + o1);
+                if (upd) {   // the slice as it was read at the start (nobody else writes it): from its shared-memory copy
+                    u0[nt] = *reinterpret_cast<const float2*>(sB + (16 * mt + g) * BP + c);
+                    if (!AHALF) u1[nt] = *reinterpret_cast<const float2*>(sB + (16 * mt + g + 8) * BP + c);
                 }
             }
 #pragma unroll
