@@ -1608,9 +1608,11 @@ __global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant
     float* const sB = sD + 2 * NQ * M * CP;
     for (int i = tid; i < RA * (COLS / 4); i += 128) {
         const int a_ = i / (COLS / 4), c4 = i - a_ * (COLS / 4);
-        *reinterpret_cast<float4*>(&sB[a_ * BP + 4 * c4]) = __ldg(reinterpret_cast<const float4*>(Bsl + (size_t)a_ * COLS) + c4);
+        tt_cp_async16(&sB[a_ * BP + 4 * c4], reinterpret_cast<const float4*>(Bsl + (size_t)a_ * COLS) + c4);
     }
-    // (the first barrier of the pass loop, or the one after the ring is primed, orders these stores before their use)
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    // (asynchronous, so that the look-ups below do not queue behind it; it is the oldest copy group, so the wait for the
+    // first pass's rows covers it, and the barrier after that wait orders it before its first use)
     const float* const sBw = sB + (8 * ynt + g) * BP + t;
     float acc[MT][NTW][4];
 #pragma unroll
@@ -1792,6 +1794,10 @@ __global__ void __launch_bounds__(128, 5) k_mid_mma(WsView w, int k, int variant
         if ((r & (8u / NQF - 1u)) == 8u / NQF - 1u) fold(false);   // rounded running sums every eighth pass (fourth with twice the nodes)
         publish_ids(r + 2);   // its ring slot held pass r - 1
         __syncthreads();   // everyone is done with this stage before pass r + 2 overwrites it
+    }
+    if (passes == 0) {   // no pass has waited for the slice copy
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
     }
     fold(true);   // also writes the zeros of a slice without nodes
 }
