@@ -1261,18 +1261,24 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                 bool head_open = !((starts >> (sub * R4)) & 1u), head_closed = false;
                 // (not unrolled: the kernel's warps are spread over its four summing paths, and with this loop unrolled
                 // they waited for instructions: 2.39 -> 1.90 ms on the 240-table workload, ncu `no_instruction` stalls)
+                // (the row of out of the bag being summed moves on by one bag per segment end; masks shifted to the sub-warp)
+                {
+                    const int j0 = sub * R4, ns = min(R4, n - j0);
+                    unsigned vs = valid >> j0, cs = closes >> j0;
+                    float4* orow = row_of(j0);
+                    const size_t ostride = (size_t)w.T * D4;
+                    const float4* src = buf + j0 * R4 + lr;
 #pragma unroll 1
-                for (int jj = 0; jj < R4; ++jj) {
-                    const int j = sub * R4 + jj;
-                    if (j < n) {
-                        if ((valid >> j) & 1u) {
-                            const float4 v = buf[j * R4 + lr];
+                    for (int jj = 0; jj < ns; ++jj, vs >>= 1, cs >>= 1, src += R4) {
+                        if (vs & 1u) {
+                            const float4 v = *src;
                             tt_add4(run, v);
                         }
-                        if ((closes >> j) & 1u) {
+                        if (cs & 1u) {
                             if (head_open) { head = run; head_closed = true; head_open = false; }
-                            else if (lane_on) __stcs(row_of(j), run);
+                            else if (lane_on) __stcs(orow, run);
                             run = make_float4(0.f, 0.f, 0.f, 0.f);
+                            orow += ostride;
                         }
                     }
                 }
