@@ -228,6 +228,25 @@ def test_short_bags_weighted_and_mean(binding, pooling, mode):
             assert_close(grads[t][k], ref[t][k], f"short bags {pooling} {mode} dG[{t}][{k}]")
 
 
+@pytest.mark.parametrize("B", [1, 2, 97])
+@pytest.mark.parametrize("D", [64, 32])
+def test_short_bags_with_whole_tables_empty(binding, D, B):
+    # tables without a single lookup between, before and after tables with short bags; one-bag batches
+    tabs = SHORT_BAG_TABLES[D]
+    tables = [tabs[0], tabs[1], tabs[2], tabs[0], tabs[1]]
+    for pooling in ([0, (0, 3), 0, (1, 5), 0], [(1, 2), 0, 0, 1, (0, 40)], [1, 1, 0, 1, 1]):
+        wl = workloads.custom(tables, B, pooling, seed=131, with_grad=True, name="short-empty-tables")
+        emb, out = run_forward(binding, wl, enable_backward=True)
+        assert emb.status() == 0
+        assert_close(out, oracle.forward_workload(wl), f"empty tables D{D} B{B} {pooling} out")
+        emb.backward(dev(wl.grad_out))
+        grads = emb.get_grads()
+        ref = oracle.backward_workload(wl)
+        for t in range(wl.T):
+            for k in range(wl.tables[t].K):
+                assert_close(grads[t][k], ref[t][k], f"empty tables D{D} B{B} {pooling} dG[{t}][{k}]")
+
+
 def test_many_tables_point_reduced(binding):
     # the many-tables bench workload (D = 32, ranks 32, every table with its own bag-length law) at a size the oracle
     # finishes in seconds: both pooling kernels' territory in one batch, fused update
