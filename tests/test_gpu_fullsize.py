@@ -167,3 +167,20 @@ def test_config5_separate_backward_and_update_every_gradient_and_core(binding, f
     assert emb.status() == 0
     check_training_all(wl, emb, full.ref_grads, "cfg5 unfused")
     del emb
+
+
+def test_many_tables_training_step_every_output_gradient_and_core(binding):
+    # the many-tables bench workload at full size (240 tables, D = 32, ranks 32, every table with its own bag lengths:
+    # the short-bag pooling kernel, the transposed row products and the stacked backward products), in the launch
+    # configuration bench.py times, against the memoised oracle
+    wl = workloads.many_tables_point(32768)
+    ref_out = oracle.forward_workload(wl, memo=True)
+    ref_grads = oracle.backward_workload(wl, memo=True)
+    emb = binding.from_workload(wl, enable_backward=True, max_unique_rows=wl.L // 2)
+    out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
+    emb.backward_sgd(dev(wl.grad_out), wl.lr)
+    assert emb.status() == 0
+    check_out_all(wl, out.cpu().numpy(), ref_out, "many-tables")
+    del out
+    check_training_all(wl, emb, ref_grads, "many-tables")
+    del emb
