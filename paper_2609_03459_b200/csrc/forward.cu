@@ -1067,20 +1067,22 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
     const bool stream_ok = !(*w.status & TT_EMB_STATUS_OFFSETS);
-    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    // lookup positions and bag indices fit in 32 bits (L and T * B are below 2^31, checked when the handle is made)
+    typedef int32_t pos_t;
+    auto clampL = [&](int64_t x) { return x < 0 ? (pos_t)0 : (x > w.L ? (pos_t)w.L : (pos_t)x); };
     for (;;) {
     int64_t ci = 0;     // shares are handed out in order through a counter (see k_pool_async)
     if (lane == 0) ci = (int64_t)atomicAdd(&w.counters[CTR_POOL_NEXT], 1u);
     ci = __shfl_sync(0xffffffffu, ci, 0);
     if (ci >= C) break;
-    const int64_t b0 = __ldg(w.pool_bounds + ci), b1 = __ldg(w.pool_bounds + ci + 1);
+    const pos_t b0 = (pos_t)__ldg(w.pool_bounds + ci), b1 = (pos_t)__ldg(w.pool_bounds + ci + 1);
     if (b0 >= b1) continue;
     // the ends of the share's bags, 32 at a time and one vector ahead: lane i holds the clamped offsets[ebase + 1 + i]
     // (ends_nx: the 32 bags after those), so that no bag waits for a load of its own end
-    auto load_ends = [&](int64_t base) { const int64_t i = base + lane; return i < b1 ? clampL(__ldg(w.offsets + i + 1)) : (int64_t)1 << 62; };   // past the share: never inside a window
-    int64_t ebase = b0;
-    int64_t ends_reg = load_ends(b0), ends_nx = load_ends(b0 + 32);
-    auto end_of = [&](int64_t bg) {     // bg >= ebase, and below ebase + 64 (a step moves on by at most 32 bags)
+    auto load_ends = [&](pos_t base) { const pos_t i = base + lane; return i < b1 ? clampL(__ldg(w.offsets + i + 1)) : (pos_t)0x7fffffff; };   // past the share: never inside a window
+    pos_t ebase = b0;
+    pos_t ends_reg = load_ends(b0), ends_nx = load_ends(b0 + 32);
+    auto end_of = [&](pos_t bg) {     // bg >= ebase, and below ebase + 64 (a step moves on by at most 32 bags)
         while (bg - ebase >= 32) {
             ends_reg = ends_nx;
             ebase += 32;
@@ -1089,33 +1091,33 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
         return __shfl_sync(0xffffffffu, ends_reg, (int)(bg - ebase));
     };
     // the bag being summed: its table, its (clamped) range, the end of the bag as stored
-    int64_t bag = b0;
+    pos_t bag = b0;
     int t = (int)(b0 / w.B);
-    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = end_of(b0);
-    int64_t o_hi = o_next < o_lo ? o_lo : o_next;
-    const int64_t share_end = stream_ok ? clampL(__ldg(w.offsets + b1)) : 0;
-    int64_t t_end = stream_ok ? __ldg(w.tl_start + t + 1) : 0;
-    int64_t pos = o_lo;                                 // next lookup of the stream
+    pos_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = end_of(b0);
+    pos_t o_hi = o_next < o_lo ? o_lo : o_next;
+    const pos_t share_end = stream_ok ? clampL(__ldg(w.offsets + b1)) : 0;
+    pos_t t_end = stream_ok ? (pos_t)__ldg(w.tl_start + t + 1) : 0;
+    pos_t pos = o_lo;                                 // next lookup of the stream
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     // rank look-up (and weight) of lookup base + lane, for the window that starts at `base`
     uint32_t slot_next = 0xffffffffu;
     float wt_next = 1.f;
-    int64_t pre_pos = -1;
+    pos_t pre_pos = -1;
     int pre_t = -1;
-    auto fetch = [&](int64_t base, int64_t lim, int tt) {
+    auto fetch = [&](pos_t base, pos_t lim, int tt) {
         slot_next = (base + lane < lim) ? tt_lookup_slot(w, w.tdesc[tt], base + lane, capK) : 0xffffffffu;
         if (WT) wt_next = (w.psw && base + lane < lim) ? __ldg(w.psw + base + lane) : 1.f;
         pre_pos = base;
         pre_t = tt;
     };
     // bag `nb_`, which starts at lookup `lo_`, becomes the one being summed (nb_ > bag, at most 32 bags on)
-    auto seek_bag = [&](int64_t nb_, int64_t lo_) {
+    auto seek_bag = [&](pos_t nb_, pos_t lo_) {
         acc = make_float4(0.f, 0.f, 0.f, 0.f);
         bag = nb_;
         if (bag < b1) {
-            if (bag >= (int64_t)(t + 1) * w.B) {
+            if (bag >= (pos_t)(t + 1) * w.B) {
                 ++t;
-                if (stream_ok) t_end = __ldg(w.tl_start + t + 1);
+                if (stream_ok) t_end = (pos_t)__ldg(w.tl_start + t + 1);
             }
             o_lo = lo_;
             o_next = end_of(bag);
@@ -1134,7 +1136,7 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
             const float inv = 1.f / (float)(o_hi - o_lo);
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
-        const int64_t b = bag - (int64_t)t * w.B;
+        const pos_t b = bag - (pos_t)t * w.B;
         if (sub == 0 && lane_on) __stcs(reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr, acc);
         advance_bag();
     };
@@ -1144,8 +1146,8 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
             pos = o_lo;
             continue;
         }
-        const int64_t lim = stream_ok ? (share_end < t_end ? share_end : t_end) : o_hi;   // > pos: the bag ends no later
-        const int n = (int)min((int64_t)32, lim - pos);
+        const pos_t lim = stream_ok ? (share_end < t_end ? share_end : t_end) : o_hi;   // > pos: the bag ends no later
+        const int n = (int)min((pos_t)32, lim - pos);
         if (pre_pos != pos || pre_t != t) fetch(pos, lim, t);
         const uint32_t slot = slot_next;
         const float wt = wt_next;
@@ -1176,11 +1178,11 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
         // the rank look-ups of the next window overlap the gather (the next window of the stream; in the per-bag mode
         // only while the bag goes on)
         {
-            const int64_t np = pos + n;
+            const pos_t np = pos + n;
             if (stream_ok) {
                 if (np < lim) fetch(np, lim, t);
                 else if (np < share_end) {               // the table ends here: the next window belongs to the next one
-                    const int64_t te = __ldg(w.tl_start + t + 2);
+                    const pos_t te = (pos_t)__ldg(w.tl_start + t + 2);
                     fetch(np, share_end < te ? share_end : te, t + 1);
                 }
             } else if (np < o_hi) fetch(np, o_hi, t);
@@ -1190,13 +1192,13 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
         // Windows with bag boundaries in them are summed by the whole warp at once.  Lane i looks at bag + i, which ends at
         // e_mine; a bag starts at row e - pos of the window for every end e inside it.
         if (!WT && stream_ok && o_hi < pos + n) {
-            const int64_t wend = pos + n;
+            const pos_t wend = pos + n;
             const int ei = (int)(bag - ebase) + lane;
-            const int64_t e0 = __shfl_sync(0xffffffffu, ends_reg, ei & 31), e1 = __shfl_sync(0xffffffffu, ends_nx, ei & 31);
-            const int64_t e_mine = ei < 32 ? e0 : e1;
+            const pos_t e0 = __shfl_sync(0xffffffffu, ends_reg, ei & 31), e1 = __shfl_sync(0xffffffffu, ends_nx, ei & 31);
+            const pos_t e_mine = ei < 32 ? e0 : e1;
             // one-lookup bags only (lane i: bag + i ends at pos + i + 1): every staged row is a row of out
             if (o_lo == pos && __all_sync(0xffffffffu, lane >= n || e_mine == pos + lane + 1)) {
-                const int64_t bf = bag - (int64_t)t * w.B;       // the window lies in table t: bf + n <= B
+                const pos_t bf = bag - (pos_t)t * w.B;       // the window lies in table t: bf + n <= B
                 if (w.upairs && lane < n) __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bf + lane)));
                 float4* o4 = reinterpret_cast<float4*>(out + (size_t)bf * w.T * w.D + (size_t)t * w.D) + lr;
                 const size_t ostride = (size_t)w.T * D4;
@@ -1213,12 +1215,12 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
             }
             // no empty bag among those that start inside the window (an empty bag needs a row of zeros: left to the
             // bag-by-bag loop below)
-            const int64_t e_prev = __shfl_up_sync(0xffffffffu, e_mine, 1);
+            const pos_t e_prev = __shfl_up_sync(0xffffffffu, e_mine, 1);
             const int inside = __popc(__ballot_sync(0xffffffffu, e_mine > pos && e_mine < wend));   // bag ends inside the window
             if (inside == 1 && plain && n == 32) {
                 // one boundary, at row c: the rows before it complete the open bag, the others start the next one
                 const int c = (int)(o_hi - pos);
-                if (w.upairs) __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (int64_t)t * w.B) + (lane >= c ? 1u : 0u)));
+                if (w.upairs) __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (pos_t)t * w.B) + (lane >= c ? 1u : 0u)));
                 float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
 #pragma unroll
                 for (int jj = 0; jj < 32 / RPI; ++jj) {
@@ -1240,9 +1242,9 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                                       | (o_lo == pos ? 1u : 0u);
                 const bool last_closed = __any_sync(0xffffffffu, e_mine == wend);
                 const unsigned closes = (starts >> 1) | (last_closed ? 1u << (n - 1) : 0u);
-                const int64_t bt = bag - (int64_t)t * w.B;       // bag of row j: bt + bags started in rows 1..j
+                const pos_t bt = bag - (pos_t)t * w.B;       // bag of row j: bt + bags started in rows 1..j
                 auto row_of = [&](int j) {
-                    const int64_t b = bt + __popc(starts & ((2u << j) - 2u));
+                    const pos_t b = bt + __popc(starts & ((2u << j) - 2u));
                     return reinterpret_cast<float4*>(out + (size_t)b * w.T * w.D + (size_t)t * w.D) + lr;
                 };
                 if (w.upairs && lane < n)
@@ -1299,12 +1301,12 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                     else carry = tail;
                 }
                 __syncwarp();
-                const int64_t bl = bag + __popc(starts & 0xfffffffeu);     // the bag of the window's last row
+                const pos_t bl = bag + __popc(starts & 0xfffffffeu);     // the bag of the window's last row
                 pos = wend;
                 if (last_closed) seek_bag(bl + 1, pos);
                 else {
                     if (bl > bag) {
-                        const int64_t lo_ = end_of(bl - 1);
+                        const pos_t lo_ = end_of(bl - 1);
                         seek_bag(bl, lo_);
                     }
                     acc = sub == 0 ? carry : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1321,16 +1323,16 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_stream(WsView w, fl
                 if (bag >= b1) break;    // cannot happen with checked offsets; never spin on it
                 continue;
             }
-            const int64_t room = o_hi - (pos + r);
-            const int seg = room < (int64_t)(n - r) ? (int)room : n - r;
+            const pos_t room = o_hi - (pos + r);
+            const int seg = room < (pos_t)(n - r) ? (int)room : n - r;
             if (w.upairs && lane >= r && lane < r + seg)    // kept for the backward sort
-                __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (int64_t)t * w.B)));
+                __stcs(&w.upairs[pos + lane], make_uint2(slot, (uint32_t)(bag - (pos_t)t * w.B)));
             if (!WT && seg == 1 && pos + r == o_lo && o_hi - o_lo == 1) {
                 // a bag of one lookup: its row of out is the staged row (or zeros for an id outside the table); the
                 // sub-warp that staged it writes it, nothing to combine
                 if (sub == (r & (RPI - 1)) && lane_on) {
                     const float4 v = ((valid >> r) & 1u) ? buf[r * R4 + lr] : make_float4(0.f, 0.f, 0.f, 0.f);
-                    __stcs(reinterpret_cast<float4*>(out + (size_t)(bag - (int64_t)t * w.B) * w.T * w.D + (size_t)t * w.D) + lr, v);
+                    __stcs(reinterpret_cast<float4*>(out + (size_t)(bag - (pos_t)t * w.B) * w.T * w.D + (size_t)t * w.D) + lr, v);
                 }
                 advance_bag();
                 r += 1;
