@@ -919,41 +919,43 @@ __global__ void __launch_bounds__(32 * POOL_WARPS, 4) k_pool_async(WsView w, flo
     const uint32_t capK = w.cap[w.K];
     const int64_t W = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t C = W * tt_pool_chunks(w.L, W);
-    auto clampL = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > w.L ? w.L : x); };
+    // lookup positions and bag indices fit in 32 bits (L and T * B are below 2^31, checked when the handle is made)
+    typedef int32_t pos_t;
+    auto clampL = [&](int64_t x) { return x < 0 ? (pos_t)0 : (x > w.L ? (pos_t)w.L : (pos_t)x); };
     for (;;) {
     // shares are handed out in order through a counter: a warp whose shares hold popular (L2-resident) rows takes more of them
     int64_t ci = 0;
     if (lane == 0) ci = (int64_t)atomicAdd(&w.counters[CTR_POOL_NEXT], 1u);
     ci = __shfl_sync(0xffffffffu, ci, 0);
     if (ci >= C) break;
-    const int64_t b0 = __ldg(w.pool_bounds + ci), b1 = __ldg(w.pool_bounds + ci + 1);
+    const pos_t b0 = (pos_t)__ldg(w.pool_bounds + ci), b1 = (pos_t)__ldg(w.pool_bounds + ci + 1);
     if (b0 >= b1) continue;
     // every bag is summed over its own (offsets[bag], offsets[bag + 1]) pair, clamped to [0, L]; an inverted pair (malformed
     // offsets) is an empty bag.  o_next: start of the next bag = this bag's end as stored, before the inversion fix
-    int64_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = clampL(__ldg(w.offsets + b0 + 1));
-    int64_t o_hi = o_next < o_lo ? o_lo : o_next;
+    pos_t o_lo = clampL(__ldg(w.offsets + b0)), o_next = clampL(__ldg(w.offsets + b0 + 1));
+    pos_t o_hi = o_next < o_lo ? o_lo : o_next;
     int t = (int)(b0 / w.B);
     uint32_t slot_next;
     float wt_next = 1.f;
-    auto fetch = [&](int64_t base, int64_t lim, int tt) {   // rank look-up (and weight) of lookup base + lane
+    auto fetch = [&](pos_t base, pos_t lim, int tt) {   // rank look-up (and weight) of lookup base + lane
         slot_next = (base + lane < lim) ? tt_lookup_slot(w, w.tdesc[tt], base + lane, capK) : 0xffffffffu;
         if (WT) wt_next = (w.psw && base + lane < lim) ? __ldg(w.psw + base + lane) : 1.f;
     };
     fetch(o_lo, o_hi, t);
-    for (int64_t bag = b0; bag < b1; ++bag) {
-        const int64_t b = bag - (int64_t)t * w.B;
+    for (pos_t bag = b0; bag < b1; ++bag) {
+        const pos_t b = bag - (pos_t)t * w.B;
         const bool has_next = bag + 1 < b1;
-        const int64_t n_lo = o_next;
-        const int64_t n_next = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_next;
-        const int64_t n_hi = n_next < n_lo ? n_lo : n_next;
+        const pos_t n_lo = o_next;
+        const pos_t n_next = has_next ? clampL(__ldg(w.offsets + bag + 2)) : o_next;
+        const pos_t n_hi = n_next < n_lo ? n_lo : n_next;
         const int tn = (has_next && b + 1 == w.B) ? t + 1 : t;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (o_lo >= o_hi && has_next) fetch(n_lo, n_hi, tn);
-        for (int64_t l0 = o_lo; l0 < o_hi; l0 += 32) {
+        for (pos_t l0 = o_lo; l0 < o_hi; l0 += 32) {
             const uint32_t slot = slot_next;
             const float wt = wt_next;
             if (w.upairs && l0 + lane < o_hi) __stcs(&w.upairs[l0 + lane], make_uint2(slot, (uint32_t)b));
-            const int n = (int)min((int64_t)32, o_hi - l0);
+            const int n = (int)min((pos_t)32, o_hi - l0);
             const unsigned valid = __ballot_sync(0xffffffffu, lane < n && slot != 0xffffffffu);
             // two-level sum: the batch's rows go into a partial that is added to the bag's sum once per batch, so the
             // rounding error of a bag with thousands of lookups grows with the number of batches, not of rows
