@@ -577,10 +577,12 @@ def test_guard_check_medium_shapes_and_detection(binding):
     TableSpec(30_000, (14, 13, 13, 13), (2, 4, 4, 4), (1, 6, 9, 5, 1), 0.5, "normal", 0.1),
     TableSpec(9_999, (100, 100), (8, 8), (1, 12, 1), 0.5, "uniform", 0.1),
 ], ids=["k3", "k4", "k2"])
-def test_unique_row_capacity_overflow_is_flagged(binding, spec):
+@pytest.mark.parametrize("pooling,B", [(20, 50), ((0, 3), 600)], ids=["long-bags", "short-bags"])
+def test_unique_row_capacity_overflow_is_flagged(binding, spec, pooling, B):
     # more distinct rows than the handle was sized for: flagged, and every kernel of the forward and of the backward
-    # still stays inside its workspace region (the rows past the capacity are dropped, prefix levels are clipped to them)
-    wl = workloads.custom([spec, spec], 50, 20, seed=4, with_grad=True)
+    # still stays inside its workspace region (the rows past the capacity are dropped, prefix levels are clipped to them);
+    # with long bags (one bag per pooling window) and with short ones (windows across bags)
+    wl = workloads.custom([spec, spec], B, pooling, seed=4, with_grad=True)
     emb = binding.from_workload(wl, max_unique_rows=100, enable_backward=True)
     out = emb.forward(dev(wl.indices), dev(wl.offsets), wl.B)
     assert emb.status() & binding.STATUS_OVERFLOW
