@@ -207,6 +207,7 @@ def test_short_bags(binding, D, B, pooling):
     for t in range(wl.T):
         for k in range(wl.tables[t].K):
             assert_close(grads[t][k], ref[t][k], f"short bags D{D} B{B} {pooling} dG[{t}][{k}]")
+    assert emb.check_guards() is None
 
 
 @pytest.mark.parametrize("mode", ["weighted", "mean"])
@@ -263,6 +264,7 @@ def test_many_tables_point_reduced(binding):
         for k in range(3):
             assert_close(grads[t][k], ref[t][k], f"many-tables dG[{t}][{k}]")
             assert_close(cores[t][k], want[k], f"many-tables core[{t}][{k}]")
+    assert emb.check_guards() is None
 
 
 def test_short_bags_with_rows_outside_the_table(binding):
@@ -293,6 +295,7 @@ def test_sweep_point_shapes(binding, D, rank):
     for t in range(wl.T):
         for k in range(3):
             assert_close(grads[t][k], ref[t][k], f"sweep D{D} r{rank} dG[{t}][{k}]")
+    assert emb.check_guards() is None      # no kernel of these shape variants wrote past its workspace region
 
 
 @pytest.mark.parametrize("D,rank", [(16, 16), (16, 32), (32, 8), (32, 32), (64, 8)])
